@@ -1,0 +1,257 @@
+"""CPU oracle for the SparSP single-device hot path -- TEST INFRASTRUCTURE, not product code.
+
+Only ``tests/``, ``__graft_entry__.smoke()`` and the CPU-baseline legs of ``bench.py`` may import
+this package.  It shares nothing with the CUDA path: the arithmetic lives in ``sparsp_oracle.c``
+(plain C, compiled by gcc) and in the few pure-Python definitions below.
+
+Pins (see tests/test_oracle_*.py): every function here is checked against closed forms, brute
+force, textbook special cases or library routines.  The one example of the paper that cannot be
+pinned is the re-placement figure (23 -> 16 transferred blocks, Section 4.3): its mask exists only
+as a picture, so nothing here reproduces it -- "parity unpinned" for that example alone.
+
+Layouts are canonical and dense: Q/K/V ``[H][N][d]`` bf16, masks ``[H][NB][Wd]`` uint32 with KV
+block ``j`` at bit ``j & 31`` of word ``j >> 5``.
+"""
+from __future__ import annotations
+
+import ctypes
+import math
+import os
+import subprocess
+
+import numpy as np
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+_SRC = os.path.join(_HERE, "sparsp_oracle.c")
+_LIB = os.path.join(_HERE, "libsparsp_oracle.so")
+_lib = None
+
+
+def build(force: bool = False) -> str:
+    """Compile the C oracle with gcc (no fast-math, no FMA contraction)."""
+    if force or not os.path.exists(_LIB) or os.path.getmtime(_LIB) < os.path.getmtime(_SRC):
+        cmd = ["gcc", "-O2", "-std=c11", "-ffp-contract=off", "-fno-fast-math", "-fopenmp",
+               "-shared", "-fPIC", "-o", _LIB, _SRC, "-lm"]
+        subprocess.run(cmd, check=True)
+    return _LIB
+
+
+def lib() -> ctypes.CDLL:
+    global _lib
+    if _lib is None:
+        _lib = ctypes.CDLL(build())
+        _lib.oracle_num_threads.restype = ctypes.c_int
+    return _lib
+
+
+def num_threads() -> int:
+    return int(lib().oracle_num_threads())
+
+
+# ---------------------------------------------------------------------------------------------
+# marshalling helpers
+# ---------------------------------------------------------------------------------------------
+def _u16(x) -> np.ndarray:
+    """bf16 torch tensor (CPU) or uint16 array -> contiguous uint16 numpy array."""
+    if isinstance(x, np.ndarray):
+        assert x.dtype == np.uint16
+        return np.ascontiguousarray(x)
+    import torch
+    assert x.dtype == torch.bfloat16 and x.device.type == "cpu"
+    return np.ascontiguousarray(x.contiguous().view(torch.int16).numpy().view(np.uint16))
+
+
+def _p(a: np.ndarray):
+    return a.ctypes.data_as(ctypes.c_void_p)
+
+
+def _i64(v) -> ctypes.c_int64:
+    return ctypes.c_int64(int(v))
+
+
+def n_blocks(N: int, b: int) -> int:
+    return (N + b - 1) // b
+
+
+def n_words(NB: int) -> int:
+    return (NB + 31) // 32
+
+
+# ---------------------------------------------------------------------------------------------
+# pure-Python definitions (host-side readings)
+# ---------------------------------------------------------------------------------------------
+def text_block_flags(n_video: int, n_text: int, b: int) -> np.ndarray:
+    """is_text[j] = 1 iff block j holds at least one text token; tokens are ordered video first,
+    then text, and blocks are flat runs of ``b`` tokens."""
+    N = n_video + n_text
+    NB = n_blocks(N, b)
+    flags = np.zeros(NB, dtype=np.uint8)
+    for j in range(NB):
+        last = min((j + 1) * b, N) - 1
+        if n_text > 0 and last >= n_video:
+            flags[j] = 1
+    return flags
+
+
+def resolve_topk(pct: int, nb_video: int) -> int:
+    """"top-k = pct % of blocks": integer ceiling of pct*nb_video/100, clamped to [1, nb_video]."""
+    k = -(-pct * nb_video // 100)
+    return max(1, min(nb_video, k))
+
+
+def placement_contiguous(NB: int, P: int) -> np.ndarray:
+    """Naive contiguous sequence partition: rank(j) = floor(j*P/NB)."""
+    return np.array([(j * P) // NB for j in range(NB)], dtype=np.int32)
+
+
+def placement_periodic(NB: int, P: int, b: int, frame_tokens: int, n_video: int) -> np.ndarray:
+    """Interval-periodic layout (Eq. "periodic-placement"): each frame is cut into P contiguous
+    spatial intervals and interval g belongs to rank g in every frame.  With B = frame_tokens/b
+    blocks per frame and s the in-frame block index this is floor(P*s/B); for frames that are not a
+    whole number of blocks the block's first token decides: floor(P*((j*b) mod F)/F).  Blocks that
+    start in the text tail are dealt round-robin (j mod P)."""
+    out = np.zeros(NB, dtype=np.int32)
+    for j in range(NB):
+        first = j * b
+        if first >= n_video:
+            out[j] = j % P
+        else:
+            out[j] = (P * (first % frame_tokens)) // frame_tokens
+    return out
+
+
+# ---------------------------------------------------------------------------------------------
+# step 1
+# ---------------------------------------------------------------------------------------------
+def pool(x, b: int) -> np.ndarray:
+    xs = _u16(x)
+    H, N, d = xs.shape
+    NB = n_blocks(N, b)
+    out = np.empty((H, NB, d), dtype=np.float32)
+    lib().oracle_pool(_p(xs), _i64(H), _i64(N), _i64(d), _i64(b), _p(out))
+    return out
+
+
+def scores(pq: np.ndarray, pk: np.ndarray) -> np.ndarray:
+    pq = np.ascontiguousarray(pq, dtype=np.float32)
+    pk = np.ascontiguousarray(pk, dtype=np.float32)
+    H, NB, d = pq.shape
+    out = np.empty((H, NB, NB), dtype=np.float32)
+    lib().oracle_scores(_p(pq), _p(pk), _i64(H), _i64(NB), _i64(d), _p(out))
+    return out
+
+
+def scores_f64(pq: np.ndarray, pk: np.ndarray) -> np.ndarray:
+    pq = np.ascontiguousarray(pq, dtype=np.float32)
+    pk = np.ascontiguousarray(pk, dtype=np.float32)
+    H, NB, d = pq.shape
+    out = np.empty((H, NB, NB), dtype=np.float64)
+    lib().oracle_scores_f64(_p(pq), _p(pk), _i64(H), _i64(NB), _i64(d), _p(out))
+    return out
+
+
+def topk_mask(sc: np.ndarray, is_text: np.ndarray, k: int):
+    """-> (mask [H][NB][Wd] uint32, kv_list [H][NB][kept] int32 ascending, kv_count [H][NB])."""
+    sc = np.ascontiguousarray(sc, dtype=np.float32)
+    is_text = np.ascontiguousarray(is_text, dtype=np.uint8)
+    H, NB, _ = sc.shape
+    Wd = n_words(NB)
+    kept_cap = min(k, int((is_text == 0).sum())) + int(is_text.sum())
+    mask = np.empty((H, NB, Wd), dtype=np.uint32)
+    kv_list = np.empty((H, NB, kept_cap), dtype=np.int32)
+    kv_count = np.empty((H, NB), dtype=np.int32)
+    lib().oracle_topk_mask(_p(sc), _p(is_text), _i64(H), _i64(NB), _i64(k), _p(mask), _p(kv_list),
+                           _i64(kept_cap), _p(kv_count))
+    return mask, kv_list, kv_count
+
+
+def block_mask(Q, K, b: int, k: int, n_text: int = 0):
+    """Whole step 1: pool -> scores -> top-k.  Returns dict with mask, kv_list, kv_count, pq, pk."""
+    H, N, d = Q.shape
+    pq, pk = pool(Q, b), pool(K, b)
+    sc = scores(pq, pk)
+    is_text = text_block_flags(N - n_text, n_text, b)
+    mask, kv_list, kv_count = topk_mask(sc, is_text, k)
+    return dict(mask=mask, kv_list=kv_list, kv_count=kv_count, pq=pq, pk=pk, scores=sc,
+                is_text=is_text)
+
+
+# ---------------------------------------------------------------------------------------------
+# step 2
+# ---------------------------------------------------------------------------------------------
+def demand(mask: np.ndarray, rank_of_block: np.ndarray, P: int, b: int, d: int,
+           include_local: bool = False, w_bytes: int = 2):
+    mask = np.ascontiguousarray(mask, dtype=np.uint32)
+    rank_of_block = np.ascontiguousarray(rank_of_block, dtype=np.int32)
+    H, NB, Wd = mask.shape
+    U = np.empty((P, H, Wd), dtype=np.uint32)
+    cnt = np.empty((P, P, H), dtype=np.int32)
+    seg_off = np.empty((P, P, H), dtype=np.int64)
+    total = np.empty((P,), dtype=np.int64)
+    volume = np.empty((P,), dtype=np.int64)
+    lib().oracle_demand(_p(mask), _p(rank_of_block), _i64(H), _i64(NB), _i64(P), _i64(b), _i64(d),
+                        _i64(w_bytes), ctypes.c_int(int(include_local)), _p(U), _p(cnt),
+                        _p(seg_off), _p(total), _p(volume))
+    return dict(U=U, cnt=cnt, seg_off=seg_off, total=total, volume=volume)
+
+
+def pack(K, V, U: np.ndarray, rank_of_block: np.ndarray, b: int, P: int, total: np.ndarray,
+         include_local: bool = False, dst_base: np.ndarray | None = None) -> np.ndarray:
+    """-> packed bytes (uint8).  Default destination bases are the dense prefix of ``total``."""
+    Ks, Vs = _u16(K), _u16(V)
+    H, N, d = Ks.shape
+    entry = 2 * b * d * 2
+    if dst_base is None:
+        dst_base = np.concatenate([[0], np.cumsum(total)[:-1]]).astype(np.int64) * entry
+    dst_base = np.ascontiguousarray(dst_base, dtype=np.int64)
+    size = int(max(dst_base[r] + total[r] * entry for r in range(P))) if P else 0
+    out = np.zeros(size, dtype=np.uint8)
+    U = np.ascontiguousarray(U, dtype=np.uint32)
+    rank_of_block = np.ascontiguousarray(rank_of_block, dtype=np.int32)
+    lib().oracle_pack(_p(Ks), _p(Vs), _p(U), _p(rank_of_block), _i64(H), _i64(N), _i64(d), _i64(b),
+                      _i64(P), ctypes.c_int(int(include_local)), _p(dst_base), _p(out))
+    return out
+
+
+# ---------------------------------------------------------------------------------------------
+# step 3
+# ---------------------------------------------------------------------------------------------
+def attn_rows(Q, K, V, mask: np.ndarray, b: int, units, scale: float | None = None):
+    """Attention for the listed (head, query block) units.  -> (out [U][b][d] fp32, lse [U][b])."""
+    Qs, Ks, Vs = _u16(Q), _u16(K), _u16(V)
+    H, N, d = Qs.shape
+    units = np.asarray(units, dtype=np.int32).reshape(-1, 2)
+    uh = np.ascontiguousarray(units[:, 0])
+    ub = np.ascontiguousarray(units[:, 1])
+    n = len(uh)
+    out = np.zeros((n, b, d), dtype=np.float32)
+    lse = np.zeros((n, b), dtype=np.float32)
+    sc = (1.0 / math.sqrt(d)) if scale is None else float(scale)
+    mask = np.ascontiguousarray(mask, dtype=np.uint32)
+    lib().oracle_attn_rows(_p(Qs), _p(Ks), _p(Vs), _p(mask), _i64(H), _i64(N), _i64(d), _i64(b),
+                           ctypes.c_double(sc), _p(uh), _p(ub), _i64(n), _p(out), _p(lse))
+    return out, lse
+
+
+def attn_all(Q, K, V, mask: np.ndarray, b: int, scale: float | None = None):
+    """Attention for every (head, query block); -> out [H][N][d] fp32, lse [H][N]."""
+    H, N, d = Q.shape
+    NB = n_blocks(N, b)
+    units = [(h, i) for h in range(H) for i in range(NB)]
+    out, lse = attn_rows(Q, K, V, mask, b, units, scale)
+    out = out.reshape(H, NB * b, d)[:, :N]
+    lse = lse.reshape(H, NB * b)[:, :N]
+    return np.ascontiguousarray(out), np.ascontiguousarray(lse)
+
+
+def attn_dense_masked(Q, K, V, mask: np.ndarray, b: int, scale: float | None = None):
+    """Textbook masked-row form (tiny inputs).  -> (out [H][N][d] fp32, rowsum [H][N] fp64)."""
+    Qs, Ks, Vs = _u16(Q), _u16(K), _u16(V)
+    H, N, d = Qs.shape
+    out = np.zeros((H, N, d), dtype=np.float32)
+    rowsum = np.zeros((H, N), dtype=np.float64)
+    sc = (1.0 / math.sqrt(d)) if scale is None else float(scale)
+    mask = np.ascontiguousarray(mask, dtype=np.uint32)
+    lib().oracle_attn_dense_masked(_p(Qs), _p(Ks), _p(Vs), _p(mask), _i64(H), _i64(N), _i64(d),
+                                   _i64(b), ctypes.c_double(sc), _p(out), _p(rowsum))
+    return out, rowsum

@@ -1,0 +1,112 @@
+"""Pins for the oracle's step 3 (block-sparse attention): library SDPA in fp64 (dense and with a
+token-level Boolean mask), special cases with closed forms, and agreement of the two oracle forms."""
+import numpy as np
+import torch
+import torch.nn.functional as F
+
+
+def _rand_qkv(rng, H, N, d, scale=1.0):
+    mk = lambda: torch.tensor(rng.standard_normal((H, N, d)) * scale, dtype=torch.float32).to(torch.bfloat16)
+    return mk(), mk(), mk()
+
+
+def _mask_words(M):
+    H, NB, _ = M.shape
+    Wd = (NB + 31) // 32
+    out = np.zeros((H, NB, Wd), np.uint32)
+    for h in range(H):
+        for i in range(NB):
+            for j in range(NB):
+                if M[h, i, j]:
+                    out[h, i, j >> 5] |= np.uint32(1 << (j & 31))
+    return out
+
+
+def _sdpa64(Q, K, V, token_mask=None):
+    q, k, v = (x.to(torch.float64).unsqueeze(0) for x in (Q, K, V))
+    am = None if token_mask is None else torch.tensor(token_mask).unsqueeze(0)
+    return F.scaled_dot_product_attention(q, k, v, attn_mask=am)[0].numpy()
+
+
+def test_all_ones_mask_equals_dense_attention(oracle_mod):
+    rng = np.random.default_rng(0)
+    H, b, d = 2, 64, 32
+    N = 3 * b + 17
+    NB = 4
+    Q, K, V = _rand_qkv(rng, H, N, d)
+    M = np.ones((H, NB, NB), bool)
+    out, lse = oracle_mod.attn_all(Q, K, V, _mask_words(M), b)
+    ref = _sdpa64(Q, K, V)
+    assert np.abs(out - ref).max() < 1e-6
+    # log-sum-exp against an independent fp64 computation
+    s = torch.einsum("hqc,hkc->hqk", Q.double(), K.double()) / np.sqrt(d)
+    assert np.abs(lse - torch.logsumexp(s, dim=-1).numpy()).max() < 1e-5
+
+
+def test_block_mask_equals_sdpa_with_token_mask(oracle_mod):
+    rng = np.random.default_rng(1)
+    H, b, d = 3, 64, 16
+    N = 4 * b + 5
+    NB = 5
+    Q, K, V = _rand_qkv(rng, H, N, d, 1.5)
+    M = rng.random((H, NB, NB)) < 0.4
+    for i in range(NB):
+        M[:, i, i] = True
+    blk = np.arange(N) // b
+    tok = M[:, blk][:, :, blk]  # [H][N][N]
+    out, _ = oracle_mod.attn_all(Q, K, V, _mask_words(M), b)
+    ref = _sdpa64(Q, K, V, tok)
+    assert np.abs(out - ref).max() < 1e-6
+
+
+def test_dense_masked_form_agrees_and_rows_sum_to_one(oracle_mod):
+    rng = np.random.default_rng(2)
+    H, b, d = 2, 64, 64
+    N = 2 * b + 40
+    NB = 3
+    Q, K, V = _rand_qkv(rng, H, N, d)
+    M = rng.random((H, NB, NB)) < 0.5
+    M[:, :, 0] = True
+    words = _mask_words(M)
+    a, _ = oracle_mod.attn_all(Q, K, V, words, b)
+    bb, rowsum = oracle_mod.attn_dense_masked(Q, K, V, words, b)
+    assert np.abs(a - bb).max() < 1e-6
+    assert np.abs(rowsum - 1.0).max() < 1e-12
+
+
+def test_single_kept_block_constant_v_and_zero_q(oracle_mod):
+    rng = np.random.default_rng(3)
+    H, b, d, NB = 1, 64, 8, 4
+    N = NB * b - 9
+    Q, K, V = _rand_qkv(rng, H, N, d)
+    # (a) only block 2 kept, V constant on block 2 -> output equals that constant
+    V2 = V.clone()
+    V2[0, 2 * b:3 * b] = 0.75
+    M = np.zeros((H, NB, NB), bool)
+    M[:, :, 2] = True
+    out, _ = oracle_mod.attn_all(Q, K, V2, _mask_words(M), b)
+    assert np.abs(out - 0.75).max() < 1e-7
+    # (b) Q = 0 -> uniform weights -> mean of V over the kept valid tokens (ragged block included)
+    M = np.zeros((H, NB, NB), bool)
+    M[:, :, 1] = True
+    M[:, :, 3] = True
+    out, lse = oracle_mod.attn_all(torch.zeros_like(Q), K, V, _mask_words(M), b)
+    kept = torch.cat([V[0, b:2 * b], V[0, 3 * b:N]]).double()
+    assert np.abs(out[0] - kept.mean(0).numpy()).max() < 1e-6
+    assert np.abs(lse - np.log(len(kept))).max() < 1e-6
+
+
+def test_explicit_scale_and_sampled_units(oracle_mod):
+    rng = np.random.default_rng(4)
+    H, b, d, NB = 2, 64, 16, 3
+    N = NB * b
+    Q, K, V = _rand_qkv(rng, H, N, d)
+    M = np.ones((H, NB, NB), bool)
+    words = _mask_words(M)
+    full, _ = oracle_mod.attn_all(Q, K, V, words, b, scale=0.3)
+    q = Q.double() * (0.3 * np.sqrt(d))  # SDPA divides by sqrt(d)
+    ref = F.scaled_dot_product_attention(q.unsqueeze(0), K.double().unsqueeze(0), V.double().unsqueeze(0))[0].numpy()
+    assert np.abs(full - ref).max() < 1e-6
+    part, _ = oracle_mod.attn_rows(Q, K, V, words, b, [(1, 2), (0, 0)], scale=0.3)
+    assert np.array_equal(part[0], full[1, 2 * b:3 * b])
+    assert np.array_equal(part[1], full[0, 0:b])
