@@ -1,0 +1,169 @@
+/*
+ * sparsp.h -- C ABI of the SparSP single-device hot path on B200 (sm_100a).
+ *
+ * Three calls make one sparse sequence-parallel attention layer for P *virtual* ranks that all live
+ * on one GPU (nothing crosses devices):
+ *
+ *   sparsp_block_mask       block mask M[h,i,j] from mean-pooled query / key tiles
+ *   sparsp_demand_pack      receiver demand D[r,h,p], exchange volume V_r, row-major packing
+ *   sparsp_sparse_attn_fwd  block-sparse softmax(QK^T/sqrt(d))V over M
+ *
+ * Conventions shared by every call
+ *   - Return value: SPARSP_OK (0) or a negative SPARSP_ERR_* code.  Argument errors are detected
+ *     on the host before anything is launched; sparsp_last_error() returns a text for the calling
+ *     thread's most recent failure.
+ *   - Unless a parameter says "host", every data pointer is a DEVICE pointer owned by the caller.
+ *     The library never allocates, frees or keeps caller memory; scratch lives in a caller-provided
+ *     device workspace of sparsp_workspace_bytes() bytes (256-byte aligned).  Calls that share a
+ *     workspace must be ordered on one stream.
+ *   - `stream` is a cudaStream_t passed as void*; all work is enqueued on it asynchronously.
+ *     Conditions only the device can detect (packed buffer too small, a bounded wait inside a
+ *     kernel running out) are written to a status word in the workspace; sparsp_status()
+ *     synchronises the stream and returns it.  No kernel traps or asserts.
+ *   - Q, K, V, O are bf16 with the head_dim axis contiguous; element strides for batch, head and
+ *     token are given in sparsp_shape, so both [B][H][N][d] and [B][N][H][d] work.  Base pointers
+ *     and strides must be multiples of 8 elements (16 bytes).
+ *   - Tokens: the grid_t*grid_h*grid_w video tokens in row-major (t, h, w) order, then n_text text
+ *     tokens.  N = their sum.  Blocks are flat runs of `block` tokens, NB = ceil(N/block); the last
+ *     block may be ragged.  A block is a *text block* iff it holds at least one text token.
+ *   - Masks are uint32 words: KV block j of row (b, h, i) is bit (j & 31) of word (j >> 5);
+ *     Wd = ceil(NB/32) words per row; bits at and beyond NB are zero.
+ *   - Supported: head_dim in {64, 128}, block in {64, 128}, NB <= 1024, n_ranks <= 64.
+ */
+#ifndef SPARSP_H_
+#define SPARSP_H_
+
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#if defined(__GNUC__)
+#define SPARSP_API __attribute__((visibility("default")))
+#else
+#define SPARSP_API
+#endif
+
+#define SPARSP_OK 0
+#define SPARSP_ERR_INVALID_ARG (-1)
+#define SPARSP_ERR_UNSUPPORTED (-2)
+#define SPARSP_ERR_CAPACITY (-3)
+#define SPARSP_ERR_CUDA (-4)
+#define SPARSP_ERR_TIMEOUT (-5)
+
+/* flags of sparsp_demand_pack */
+#define SPARSP_PLAN_ONLY 1     /* compute union/cnt/offsets/volume, copy nothing */
+#define SPARSP_INCLUDE_LOCAL 2 /* also pack the p == r segment (in its ascending-p position) */
+
+typedef struct sparsp_shape {
+  int32_t batch, heads, head_dim;         /* B, H, d */
+  int32_t grid_t, grid_h, grid_w, n_text; /* latent grid T x H x W, text tokens appended */
+  int32_t block;                          /* b: tokens per query / KV block */
+  int64_t stride_batch, stride_head, stride_token; /* in elements, for Q, K, V and O alike */
+} sparsp_shape;
+
+/* Host helpers (no GPU work). ---------------------------------------------------------------- */
+
+/* N, NB, Wd and the number of candidate (text-free) blocks for a shape.  Any out pointer may be
+ * NULL.  Returns SPARSP_ERR_INVALID_ARG for non-positive dimensions. */
+SPARSP_API int sparsp_geometry(const sparsp_shape* shape, int64_t* n_tokens, int32_t* n_blocks,
+                    int32_t* n_words, int32_t* n_video_blocks);
+
+/* "top-k = pct % of the blocks": ceil(pct * n_video_blocks / 100) clamped to [1, n_video_blocks]. */
+SPARSP_API int32_t sparsp_resolve_topk(int32_t pct, int32_t n_video_blocks);
+
+/* Naive contiguous partition of the sequence (Section 3.1): rank(j) = floor(j * n_ranks / NB).
+ * rank_of_block: HOST array of NB int32. */
+SPARSP_API int sparsp_placement_contiguous(const sparsp_shape* shape, int32_t n_ranks, int32_t* rank_of_block);
+
+/* Interval-periodic layout (Section 4.3, Eq. "periodic-placement"): each frame is cut into
+ * n_ranks contiguous spatial intervals and the same interval goes to the same rank in every frame.
+ * For block j whose first token lies in the video part, rank = floor(G * ((j*b) mod F) / F) with
+ * F = grid_h * grid_w tokens per frame, which is floor(G*s/B) when frames are whole blocks; blocks
+ * starting in the text tail get j mod G.  rank_of_block: HOST array of NB int32. */
+SPARSP_API int sparsp_placement_periodic(const sparsp_shape* shape, int32_t n_ranks, int32_t* rank_of_block);
+
+/* Bytes of device workspace the three calls need for this shape and rank count. */
+SPARSP_API int sparsp_workspace_bytes(const sparsp_shape* shape, int32_t n_ranks, int64_t* bytes);
+
+/* Step 1 -- block-importance estimation (Section 4.2: masks are materialised from pooled query
+ * and key tiles; selection rule: top-k per query block).
+ *   pooled[b,h,i,:] = mean over the valid tokens of block i (fp32, ascending-token sum, one division)
+ *   S[b,h,i,j]      = sum_c pooledQ[i,c] * pooledK[j,c]   (fp32 fused multiply-add chain, c ascending)
+ *   per row keep the topk_video highest-scoring text-free blocks (equal scores: lower j first,
+ *   -0 == +0), then every text block.
+ * Q, K        in   bf16, strided as in `shape`
+ * topk_video  in   1 .. n_video_blocks
+ * mask        out  uint32 [B][H][NB][Wd]
+ * kv_list     out  int32 [B][H][NB][kept] ascending kept blocks, kept = topk_video + #text blocks; may be NULL
+ * kv_count    out  int32 [B][H][NB]; may be NULL
+ * pooled_q/k  out  fp32 [B][H][NB][d]; may be NULL (kept in the workspace then)
+ */
+SPARSP_API int sparsp_block_mask(const sparsp_shape* shape, const void* Q, const void* K, int32_t topk_video,
+                      uint32_t* mask, int32_t* kv_list, int32_t* kv_count, float* pooled_q,
+                      float* pooled_k, void* workspace, void* stream);
+
+/* Step 2 -- demand and packing for n_ranks virtual ranks (Section 4.2, Eq. "receiver-demand" and
+ * Eq. "sparse-exchange-volume"; Section 5.2: head-preserving demand, row-major packing with
+ * locally derived offsets; Section 6: one slot per (producer, consumer) pair).
+ *   Q_r = { i : rank_of_block[i] = r },  P(j) = rank_of_block[j]
+ *   union_mask[b,r,h]  = OR_{i in Q_r} M[b,h,i]
+ *   cnt[b,r,p,h]       = | { j in union_mask[b,r,h] : P(j) = p } |         (p == r: local reuse)
+ *   volume_bytes[b,r]  = 2*block*d*2 * sum_h sum_{p != r} cnt[b,r,p,h]
+ *   seg_offset[b,r,p,h]= entry index in consumer r's buffer of the first block of (producer p, head h):
+ *                        exclusive scan of cnt over p ascending (p == r skipped unless
+ *                        SPARSP_INCLUDE_LOCAL) then h ascending
+ *   seg_total[b,r]     = number of entries in consumer r's buffer
+ *   packed             = for every (b, r): at byte dst_base_bytes[b,r], the entries in that order, each
+ *                        entry = K tile (block x d bf16) then V tile of (h, j), j ascending inside a head;
+ *                        rows at or beyond N are zero.
+ * mask            in   uint32 [B][H][NB][Wd]
+ * rank_of_block   in   DEVICE int32 [NB], values 0 .. n_ranks-1
+ * K, V            in   bf16 (ignored with SPARSP_PLAN_ONLY)
+ * union_mask      out  uint32 [B][P][H][Wd]
+ * cnt             out  int32 [B][P][P][H]
+ * seg_offset      out  int64 [B][P][P][H]
+ * seg_total       out  int64 [B][P]
+ * volume_bytes    out  int64 [B][P]
+ * packed          out  bytes; 16-byte aligned (ignored with SPARSP_PLAN_ONLY)
+ * packed_capacity_bytes  size of `packed`
+ * dst_base_bytes  in   DEVICE int64 [B][P], multiples of 16, or NULL = consumers back to back in
+ *                      (b, r) order starting at byte 0
+ * If an entry would end beyond packed_capacity_bytes it is not written and the status word becomes
+ * SPARSP_ERR_CAPACITY.
+ */
+SPARSP_API int sparsp_demand_pack(const sparsp_shape* shape, const uint32_t* mask, const int32_t* rank_of_block,
+                       int32_t n_ranks, int32_t flags, const void* K, const void* V,
+                       uint32_t* union_mask, int32_t* cnt, int64_t* seg_offset, int64_t* seg_total,
+                       int64_t* volume_bytes, void* packed, int64_t packed_capacity_bytes,
+                       const int64_t* dst_base_bytes, void* workspace, void* stream);
+
+/* Step 3 -- block-sparse attention forward (Section 2.2, Eq. "attention", restricted to the kept
+ * blocks of M): for every valid query token q of block i,
+ *   O[q,:] = sum_t p_t V[t,:] / sum_t p_t,   p_t = exp(s_t - max s),   s_t = scale * Q[q,:].K[t,:]
+ * over the tokens t < N of the KV blocks kept in row (b,h,i).  bf16 tensor-core products, fp32
+ * accumulation and fp32 online softmax.  Every row must keep at least one block.
+ *   mask           in   uint32 [B][H][NB][Wd]
+ *   softmax_scale  in   0 means 1/sqrt(d)
+ *   O              out  bf16, strided like Q; rows of tokens >= N are not written
+ *   lse            out  fp32 [B][H][N], natural-log sum-exp of the scaled logits; may be NULL
+ */
+SPARSP_API int sparsp_sparse_attn_fwd(const sparsp_shape* shape, const void* Q, const void* K, const void* V,
+                           const uint32_t* mask, float softmax_scale, void* O, float* lse,
+                           void* workspace, void* stream);
+
+/* Synchronises `stream` and returns the workspace's status word in *code (SPARSP_OK if no kernel
+ * reported a problem since the last reset), then resets it. */
+SPARSP_API int sparsp_status(void* workspace, void* stream, int32_t* code);
+
+/* Text of the calling thread's most recent error ("" if none). */
+SPARSP_API const char* sparsp_last_error(void);
+
+/* Number of kernels this library has launched in the calling process (for benchmarks). */
+SPARSP_API int64_t sparsp_launch_count(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* SPARSP_H_ */

@@ -1,0 +1,202 @@
+"""ctypes binding of libsparsp.so: argument marshalling only.
+
+Every function here has the name of the C entry point it forwards to (include/sparsp.h).  Tensors
+are torch CUDA tensors used purely as device buffers; the current torch CUDA stream is passed down.
+There is no fallback: if the library is missing or fails to load, importing a function works but the
+first call raises.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+from dataclasses import dataclass
+
+import torch
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libsparsp.so")
+
+SPARSP_OK = 0
+SPARSP_ERR_INVALID_ARG = -1
+SPARSP_ERR_UNSUPPORTED = -2
+SPARSP_ERR_CAPACITY = -3
+SPARSP_ERR_CUDA = -4
+SPARSP_ERR_TIMEOUT = -5
+SPARSP_PLAN_ONLY = 1
+SPARSP_INCLUDE_LOCAL = 2
+
+EXPORTS = [
+    "sparsp_geometry", "sparsp_resolve_topk", "sparsp_placement_contiguous", "sparsp_placement_periodic",
+    "sparsp_workspace_bytes", "sparsp_block_mask", "sparsp_demand_pack", "sparsp_sparse_attn_fwd",
+    "sparsp_status", "sparsp_last_error", "sparsp_launch_count",
+]
+
+
+class SparspError(RuntimeError):
+    def __init__(self, code: int, text: str):
+        super().__init__(f"sparsp error {code}: {text}")
+        self.code = code
+
+
+class sparsp_shape(ctypes.Structure):
+    _fields_ = [("batch", ctypes.c_int32), ("heads", ctypes.c_int32), ("head_dim", ctypes.c_int32),
+                ("grid_t", ctypes.c_int32), ("grid_h", ctypes.c_int32), ("grid_w", ctypes.c_int32),
+                ("n_text", ctypes.c_int32), ("block", ctypes.c_int32),
+                ("stride_batch", ctypes.c_int64), ("stride_head", ctypes.c_int64),
+                ("stride_token", ctypes.c_int64)]
+
+
+_lib = None
+
+
+def lib() -> ctypes.CDLL:
+    """Loads the CUDA library; raises if it has not been built."""
+    global _lib
+    if _lib is None:
+        if not os.path.exists(LIB_PATH):
+            raise RuntimeError(f"{LIB_PATH} is missing: build it with `python -m paper_2609_32197_b200.build` "
+                               "(there is no CPU fallback)")
+        L = ctypes.CDLL(LIB_PATH)
+        L.sparsp_last_error.restype = ctypes.c_char_p
+        L.sparsp_launch_count.restype = ctypes.c_int64
+        L.sparsp_resolve_topk.restype = ctypes.c_int32
+        for name in EXPORTS:
+            getattr(L, name)  # AttributeError if a declared symbol is not exported
+        _lib = L
+    return _lib
+
+
+def _check(rc: int):
+    if rc != SPARSP_OK:
+        raise SparspError(rc, lib().sparsp_last_error().decode())
+
+
+def _ptr(t):
+    if t is None:
+        return ctypes.c_void_p(0)
+    return ctypes.c_void_p(t.data_ptr())
+
+
+def _stream():
+    return ctypes.c_void_p(torch.cuda.current_stream().cuda_stream)
+
+
+@dataclass
+class Geometry:
+    n_tokens: int
+    n_blocks: int
+    n_words: int
+    n_video_blocks: int
+
+
+def make_shape(heads: int, head_dim: int, grid, n_text: int, block: int, batch: int = 1,
+               layout: str = "HND") -> sparsp_shape:
+    """Shape for dense tensors laid out [B][H][N][d] ("HND") or [B][N][H][d] ("NHD")."""
+    N = grid[0] * grid[1] * grid[2] + n_text
+    if layout == "HND":
+        sh, st = N * head_dim, head_dim
+    elif layout == "NHD":
+        sh, st = head_dim, heads * head_dim
+    else:
+        raise ValueError(layout)
+    return sparsp_shape(batch, heads, head_dim, grid[0], grid[1], grid[2], n_text, block,
+                        heads * N * head_dim, sh, st)
+
+
+def sparsp_geometry(shape: sparsp_shape) -> Geometry:
+    n, nb, wd, nv = ctypes.c_int64(), ctypes.c_int32(), ctypes.c_int32(), ctypes.c_int32()
+    _check(lib().sparsp_geometry(ctypes.byref(shape), ctypes.byref(n), ctypes.byref(nb), ctypes.byref(wd),
+                                 ctypes.byref(nv)))
+    return Geometry(n.value, nb.value, wd.value, nv.value)
+
+
+def sparsp_resolve_topk(pct: int, n_video_blocks: int) -> int:
+    return int(lib().sparsp_resolve_topk(ctypes.c_int32(pct), ctypes.c_int32(n_video_blocks)))
+
+
+def _placement(fn, shape, n_ranks):
+    g = sparsp_geometry(shape)
+    out = torch.empty(g.n_blocks, dtype=torch.int32)
+    _check(fn(ctypes.byref(shape), ctypes.c_int32(n_ranks), ctypes.c_void_p(out.data_ptr())))
+    return out
+
+
+def sparsp_placement_contiguous(shape: sparsp_shape, n_ranks: int) -> torch.Tensor:
+    return _placement(lib().sparsp_placement_contiguous, shape, n_ranks)
+
+
+def sparsp_placement_periodic(shape: sparsp_shape, n_ranks: int) -> torch.Tensor:
+    return _placement(lib().sparsp_placement_periodic, shape, n_ranks)
+
+
+def sparsp_workspace_bytes(shape: sparsp_shape, n_ranks: int) -> int:
+    out = ctypes.c_int64()
+    _check(lib().sparsp_workspace_bytes(ctypes.byref(shape), ctypes.c_int32(n_ranks), ctypes.byref(out)))
+    return out.value
+
+
+def make_workspace(shape: sparsp_shape, n_ranks: int, device="cuda") -> torch.Tensor:
+    """Allocates a workspace (torch owns the memory) with its header zero-filled."""
+    ws = torch.empty(sparsp_workspace_bytes(shape, n_ranks), dtype=torch.uint8, device=device)
+    ws[:256].zero_()
+    return ws
+
+
+def sparsp_block_mask(shape, Q, K, topk_video, mask, kv_list, kv_count, pooled_q, pooled_k, workspace):
+    _check(lib().sparsp_block_mask(ctypes.byref(shape), _ptr(Q), _ptr(K), ctypes.c_int32(topk_video),
+                                   _ptr(mask), _ptr(kv_list), _ptr(kv_count), _ptr(pooled_q),
+                                   _ptr(pooled_k), _ptr(workspace), _stream()))
+
+
+def sparsp_demand_pack(shape, mask, rank_of_block, n_ranks, flags, K, V, union_mask, cnt, seg_offset,
+                       seg_total, volume_bytes, packed, packed_capacity_bytes, dst_base_bytes, workspace):
+    _check(lib().sparsp_demand_pack(ctypes.byref(shape), _ptr(mask), _ptr(rank_of_block),
+                                    ctypes.c_int32(n_ranks), ctypes.c_int32(flags), _ptr(K), _ptr(V),
+                                    _ptr(union_mask), _ptr(cnt), _ptr(seg_offset), _ptr(seg_total),
+                                    _ptr(volume_bytes), _ptr(packed), ctypes.c_int64(packed_capacity_bytes),
+                                    _ptr(dst_base_bytes), _ptr(workspace), _stream()))
+
+
+def sparsp_sparse_attn_fwd(shape, Q, K, V, mask, softmax_scale, O, lse, workspace):
+    _check(lib().sparsp_sparse_attn_fwd(ctypes.byref(shape), _ptr(Q), _ptr(K), _ptr(V), _ptr(mask),
+                                        ctypes.c_float(softmax_scale), _ptr(O), _ptr(lse), _ptr(workspace),
+                                        _stream()))
+
+
+def sparsp_status(workspace) -> int:
+    code = ctypes.c_int32()
+    _check(lib().sparsp_status(_ptr(workspace), _stream(), ctypes.byref(code)))
+    return code.value
+
+
+def sparsp_last_error() -> str:
+    return lib().sparsp_last_error().decode()
+
+
+def sparsp_launch_count() -> int:
+    return int(lib().sparsp_launch_count())
+
+
+# ---------------------------------------------------------------------------------------------
+# allocation helpers (device buffers for the outputs; no arithmetic)
+# ---------------------------------------------------------------------------------------------
+def alloc_mask_outputs(shape: sparsp_shape, topk_video: int, device="cuda", with_list=True, with_pooled=False):
+    g = sparsp_geometry(shape)
+    B, H, d = shape.batch, shape.heads, shape.head_dim
+    kept = topk_video + (g.n_blocks - g.n_video_blocks)
+    out = dict(mask=torch.empty(B, H, g.n_blocks, g.n_words, dtype=torch.int32, device=device))
+    out["kv_list"] = torch.full((B, H, g.n_blocks, kept), -1, dtype=torch.int32, device=device) if with_list else None
+    out["kv_count"] = torch.empty(B, H, g.n_blocks, dtype=torch.int32, device=device) if with_list else None
+    out["pooled_q"] = torch.empty(B, H, g.n_blocks, d, dtype=torch.float32, device=device) if with_pooled else None
+    out["pooled_k"] = torch.empty(B, H, g.n_blocks, d, dtype=torch.float32, device=device) if with_pooled else None
+    return out
+
+
+def alloc_demand_outputs(shape: sparsp_shape, n_ranks: int, device="cuda"):
+    g = sparsp_geometry(shape)
+    B, H, P = shape.batch, shape.heads, n_ranks
+    return dict(union_mask=torch.empty(B, P, H, g.n_words, dtype=torch.int32, device=device),
+                cnt=torch.empty(B, P, P, H, dtype=torch.int32, device=device),
+                seg_offset=torch.empty(B, P, P, H, dtype=torch.int64, device=device),
+                seg_total=torch.empty(B, P, dtype=torch.int64, device=device),
+                volume_bytes=torch.empty(B, P, dtype=torch.int64, device=device))

@@ -1,0 +1,291 @@
+// extern "C" entry points of the SparSP library: argument checking, workspace carving, launch order.
+#include <cstring>
+
+#include "common.cuh"
+
+namespace sparsp {
+
+static thread_local char tl_error[512] = "";
+std::atomic<int64_t> g_launches{0};
+
+void set_error(const char* fmt, ...) {
+  va_list ap;
+  va_start(ap, fmt);
+  vsnprintf(tl_error, sizeof tl_error, fmt, ap);
+  va_end(ap);
+}
+
+int cuda_fail(cudaError_t e, const char* what) {
+  set_error("CUDA error %d (%s) in %s", (int)e, cudaGetErrorString(e), what);
+  return SPARSP_ERR_CUDA;
+}
+
+int make_geometry(const sparsp_shape* s, Geometry* g) {
+  if (!s) {
+    set_error("shape is NULL");
+    return SPARSP_ERR_INVALID_ARG;
+  }
+  if (s->batch < 1 || s->heads < 1 || s->head_dim < 1 || s->grid_t < 1 || s->grid_h < 1 ||
+      s->grid_w < 1 || s->n_text < 0 || s->block < 1) {
+    set_error("shape has a non-positive dimension");
+    return SPARSP_ERR_INVALID_ARG;
+  }
+  g->B = s->batch;
+  g->H = s->heads;
+  g->d = s->head_dim;
+  g->b = s->block;
+  g->n_video = (int64_t)s->grid_t * s->grid_h * s->grid_w;
+  g->N = g->n_video + s->n_text;
+  int64_t nb = (g->N + s->block - 1) / s->block;
+  if (nb > kMaxBlocks) {
+    set_error("NB = %lld exceeds the supported %d blocks", (long long)nb, kMaxBlocks);
+    return SPARSP_ERR_UNSUPPORTED;
+  }
+  g->NB = (int32_t)nb;
+  g->Wd = (g->NB + 31) / 32;
+  g->nb_cand = s->n_text > 0 ? (int32_t)(g->n_video / s->block) : g->NB;
+  return SPARSP_OK;
+}
+
+static int check_supported(const Geometry& g) {
+  if (g.d != 64 && g.d != 128) {
+    set_error("head_dim %d unsupported (64 or 128)", g.d);
+    return SPARSP_ERR_UNSUPPORTED;
+  }
+  if (g.b != 64 && g.b != 128) {
+    set_error("block %d unsupported (64 or 128)", g.b);
+    return SPARSP_ERR_UNSUPPORTED;
+  }
+  return SPARSP_OK;
+}
+
+int check_strides(const sparsp_shape* s, const Geometry& g) {
+  if (s->stride_token < g.d || s->stride_token % 8 || s->stride_head % 8 || s->stride_batch % 8 ||
+      s->stride_head < 1 || (g.B > 1 && s->stride_batch < 1)) {
+    set_error("strides must be positive multiples of 8 elements with stride_token >= head_dim");
+    return SPARSP_ERR_INVALID_ARG;
+  }
+  return SPARSP_OK;
+}
+
+static int check_ptr(const void* p, const char* name, size_t align = 16) {
+  if (!p) {
+    set_error("%s is NULL", name);
+    return SPARSP_ERR_INVALID_ARG;
+  }
+  if ((uintptr_t)p % align) {
+    set_error("%s must be %zu-byte aligned", name, align);
+    return SPARSP_ERR_INVALID_ARG;
+  }
+  return SPARSP_OK;
+}
+
+WsLayout make_layout(const Geometry& g, int P) {
+  WsLayout L;
+  int64_t off = 0;
+  L.status = off;
+  off += align_up(kStatusWords * 4, 256);
+  const int64_t pooled = (int64_t)g.B * g.H * g.NB * g.d * 4;
+  L.pooled_q = off;
+  off += align_up(pooled, 256);
+  L.pooled_k = off;
+  off += align_up(pooled, 256);
+  L.own = off;
+  off += align_up((int64_t)P * g.Wd * 4, 256);
+  L.ent_base = off;
+  off += align_up((int64_t)g.B * P * 8, 256);
+  L.n_entries = off;
+  off += 256;
+  L.entries = off;
+  off += align_up((int64_t)g.B * P * g.H * g.NB * (int64_t)sizeof(PackEntry), 256);
+  L.total = off;
+  return L;
+}
+
+}  // namespace sparsp
+
+using namespace sparsp;
+
+#define SPARSP_TRY(x)             \
+  do {                            \
+    int rc__ = (x);               \
+    if (rc__ != SPARSP_OK) return rc__; \
+  } while (0)
+
+extern "C" {
+
+const char* sparsp_last_error(void) { return tl_error; }
+
+int64_t sparsp_launch_count(void) { return g_launches.load(); }
+
+int sparsp_geometry(const sparsp_shape* shape, int64_t* n_tokens, int32_t* n_blocks, int32_t* n_words,
+                    int32_t* n_video_blocks) {
+  Geometry g;
+  SPARSP_TRY(make_geometry(shape, &g));
+  if (n_tokens) *n_tokens = g.N;
+  if (n_blocks) *n_blocks = g.NB;
+  if (n_words) *n_words = g.Wd;
+  if (n_video_blocks) *n_video_blocks = g.nb_cand;
+  return SPARSP_OK;
+}
+
+int32_t sparsp_resolve_topk(int32_t pct, int32_t n_video_blocks) {
+  int64_t k = ((int64_t)pct * n_video_blocks + 99) / 100;
+  if (k < 1) k = 1;
+  if (k > n_video_blocks) k = n_video_blocks;
+  return (int32_t)k;
+}
+
+int sparsp_placement_contiguous(const sparsp_shape* shape, int32_t n_ranks, int32_t* rank_of_block) {
+  Geometry g;
+  SPARSP_TRY(make_geometry(shape, &g));
+  if (n_ranks < 1 || n_ranks > kMaxRanks || !rank_of_block) {
+    set_error("bad n_ranks or NULL output");
+    return SPARSP_ERR_INVALID_ARG;
+  }
+  for (int32_t j = 0; j < g.NB; ++j) rank_of_block[j] = (int32_t)(((int64_t)j * n_ranks) / g.NB);
+  return SPARSP_OK;
+}
+
+int sparsp_placement_periodic(const sparsp_shape* shape, int32_t n_ranks, int32_t* rank_of_block) {
+  Geometry g;
+  SPARSP_TRY(make_geometry(shape, &g));
+  if (n_ranks < 1 || n_ranks > kMaxRanks || !rank_of_block) {
+    set_error("bad n_ranks or NULL output");
+    return SPARSP_ERR_INVALID_ARG;
+  }
+  const int64_t F = (int64_t)shape->grid_h * shape->grid_w;
+  for (int32_t j = 0; j < g.NB; ++j) {
+    const int64_t first = (int64_t)j * g.b;
+    rank_of_block[j] = first >= g.n_video ? j % n_ranks : (int32_t)((n_ranks * (first % F)) / F);
+  }
+  return SPARSP_OK;
+}
+
+int sparsp_workspace_bytes(const sparsp_shape* shape, int32_t n_ranks, int64_t* bytes) {
+  Geometry g;
+  SPARSP_TRY(make_geometry(shape, &g));
+  if (n_ranks < 1 || n_ranks > kMaxRanks || !bytes) {
+    set_error("bad n_ranks or NULL output");
+    return SPARSP_ERR_INVALID_ARG;
+  }
+  *bytes = make_layout(g, n_ranks).total;
+  return SPARSP_OK;
+}
+
+int sparsp_block_mask(const sparsp_shape* shape, const void* Q, const void* K, int32_t topk_video,
+                      uint32_t* mask, int32_t* kv_list, int32_t* kv_count, float* pooled_q,
+                      float* pooled_k, void* workspace, void* stream) {
+  Geometry g;
+  SPARSP_TRY(make_geometry(shape, &g));
+  SPARSP_TRY(check_supported(g));
+  SPARSP_TRY(check_strides(shape, g));
+  SPARSP_TRY(check_ptr(Q, "Q"));
+  SPARSP_TRY(check_ptr(K, "K"));
+  SPARSP_TRY(check_ptr(mask, "mask", 4));
+  SPARSP_TRY(check_ptr(workspace, "workspace", 256));
+  if (topk_video < 1 || topk_video > g.nb_cand) {
+    set_error("topk_video %d outside 1..%d", topk_video, g.nb_cand);
+    return SPARSP_ERR_INVALID_ARG;
+  }
+  if (pooled_q && (uintptr_t)pooled_q % 16) return check_ptr((void*)1, "pooled_q");
+  if (pooled_k && (uintptr_t)pooled_k % 16) return check_ptr((void*)1, "pooled_k");
+  char* ws = (char*)workspace;
+  const WsLayout L = make_layout(g, 1);
+  float* pq = pooled_q ? pooled_q : (float*)(ws + L.pooled_q);
+  float* pk = pooled_k ? pooled_k : (float*)(ws + L.pooled_k);
+  cudaStream_t st = (cudaStream_t)stream;
+  SPARSP_TRY(launch_pool(*shape, g, Q, K, pq, pk, st));
+  SPARSP_TRY(launch_score_topk(g, pq, pk, topk_video, mask, kv_list, kv_count, st));
+  return SPARSP_OK;
+}
+
+int sparsp_demand_pack(const sparsp_shape* shape, const uint32_t* mask, const int32_t* rank_of_block,
+                       int32_t n_ranks, int32_t flags, const void* K, const void* V,
+                       uint32_t* union_mask, int32_t* cnt, int64_t* seg_offset, int64_t* seg_total,
+                       int64_t* volume_bytes, void* packed, int64_t packed_capacity_bytes,
+                       const int64_t* dst_base_bytes, void* workspace, void* stream) {
+  Geometry g;
+  SPARSP_TRY(make_geometry(shape, &g));
+  SPARSP_TRY(check_supported(g));
+  if (n_ranks < 1 || n_ranks > kMaxRanks) {
+    set_error("n_ranks %d outside 1..%d", n_ranks, kMaxRanks);
+    return SPARSP_ERR_INVALID_ARG;
+  }
+  if (flags & ~(SPARSP_PLAN_ONLY | SPARSP_INCLUDE_LOCAL)) {
+    set_error("unknown flag bits 0x%x", flags);
+    return SPARSP_ERR_INVALID_ARG;
+  }
+  SPARSP_TRY(check_ptr(mask, "mask", 4));
+  SPARSP_TRY(check_ptr(rank_of_block, "rank_of_block", 4));
+  SPARSP_TRY(check_ptr(union_mask, "union_mask", 4));
+  SPARSP_TRY(check_ptr(cnt, "cnt", 4));
+  SPARSP_TRY(check_ptr(seg_offset, "seg_offset", 8));
+  SPARSP_TRY(check_ptr(seg_total, "seg_total", 8));
+  SPARSP_TRY(check_ptr(volume_bytes, "volume_bytes", 8));
+  SPARSP_TRY(check_ptr(workspace, "workspace", 256));
+  const bool plan_only = flags & SPARSP_PLAN_ONLY;
+  if (!plan_only) {
+    SPARSP_TRY(check_strides(shape, g));
+    SPARSP_TRY(check_ptr(K, "K"));
+    SPARSP_TRY(check_ptr(V, "V"));
+    SPARSP_TRY(check_ptr(packed, "packed"));
+    if (packed_capacity_bytes < 0) {
+      set_error("negative packed_capacity_bytes");
+      return SPARSP_ERR_INVALID_ARG;
+    }
+  }
+  if (dst_base_bytes && (uintptr_t)dst_base_bytes % 8) return check_ptr((void*)1, "dst_base_bytes", 8);
+  char* ws = (char*)workspace;
+  const WsLayout L = make_layout(g, n_ranks);
+  cudaStream_t st = (cudaStream_t)stream;
+  SPARSP_TRY(launch_demand(g, mask, rank_of_block, n_ranks, flags, union_mask, cnt, seg_offset,
+                           seg_total, volume_bytes, dst_base_bytes,
+                           plan_only ? (int64_t)-1 : packed_capacity_bytes, ws, L, st));
+  if (!plan_only) SPARSP_TRY(launch_pack(*shape, g, K, V, packed, packed_capacity_bytes, n_ranks, ws, L, st));
+  return SPARSP_OK;
+}
+
+int sparsp_sparse_attn_fwd(const sparsp_shape* shape, const void* Q, const void* K, const void* V,
+                           const uint32_t* mask, float softmax_scale, void* O, float* lse,
+                           void* workspace, void* stream) {
+  Geometry g;
+  SPARSP_TRY(make_geometry(shape, &g));
+  SPARSP_TRY(check_supported(g));
+  SPARSP_TRY(check_strides(shape, g));
+  SPARSP_TRY(check_ptr(Q, "Q"));
+  SPARSP_TRY(check_ptr(K, "K"));
+  SPARSP_TRY(check_ptr(V, "V"));
+  SPARSP_TRY(check_ptr(O, "O"));
+  SPARSP_TRY(check_ptr(mask, "mask", 4));
+  SPARSP_TRY(check_ptr(workspace, "workspace", 256));
+  if (lse && (uintptr_t)lse % 4) return check_ptr((void*)1, "lse", 4);
+  if (!(softmax_scale >= 0.0f)) {
+    set_error("softmax_scale must be >= 0");
+    return SPARSP_ERR_INVALID_ARG;
+  }
+  const WsLayout L = make_layout(g, 1);
+  return launch_attn(*shape, g, Q, K, V, mask, softmax_scale, O, lse, (char*)workspace, L,
+                     (cudaStream_t)stream);
+}
+
+int sparsp_status(void* workspace, void* stream, int32_t* code) {
+  SPARSP_TRY(check_ptr(workspace, "workspace", 256));
+  if (!code) {
+    set_error("code is NULL");
+    return SPARSP_ERR_INVALID_ARG;
+  }
+  cudaStream_t st = (cudaStream_t)stream;
+  int32_t words[4] = {0, 0, 0, 0};
+  SPARSP_CUDA_OK(cudaMemcpyAsync(words, workspace, sizeof words, cudaMemcpyDeviceToHost, st));
+  SPARSP_CUDA_OK(cudaStreamSynchronize(st));
+  *code = words[0];
+  if (words[0] != SPARSP_OK) {
+    set_error("device status %d (detail %d %d %d)", words[0], words[1], words[2], words[3]);
+    SPARSP_CUDA_OK(cudaMemsetAsync(workspace, 0, kStatusWords * 4, st));
+    SPARSP_CUDA_OK(cudaStreamSynchronize(st));
+  }
+  return SPARSP_OK;
+}
+
+}  // extern "C"

@@ -1,0 +1,243 @@
+// Step 2: per-rank per-head unions of required KV blocks, demand counts, exchange volume,
+// pack-order offsets, the entry table, and the gather of K/V tiles into per-consumer buffers.
+// Everything before the gather is small integer work on bit words; the gather is the HBM-bound part.
+#include "common.cuh"
+
+namespace sparsp {
+
+// own[p][w]: bit j set iff rank_of_block[j] == p.  One thread per (p, w).
+__global__ void own_kernel(const int32_t* __restrict__ rank, int NB, int Wd, int P,
+                           uint32_t* __restrict__ own) {
+  const int idx = blockIdx.x * blockDim.x + threadIdx.x;
+  if (idx >= P * Wd) return;
+  const int p = idx / Wd, w = idx % Wd;
+  uint32_t bits = 0;
+  for (int t = 0; t < 32; ++t) {
+    const int j = w * 32 + t;
+    if (j < NB && rank[j] == p) bits |= 1u << t;
+  }
+  own[idx] = bits;
+}
+
+// U[b][r][h][w] = OR over the query blocks i of rank r of M[b][h][i][w].  One thread per output word.
+__global__ void union_kernel(const uint32_t* __restrict__ mask, const int32_t* __restrict__ rank,
+                             int B, int H, int NB, int Wd, int P, uint32_t* __restrict__ U) {
+  const int64_t idx = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+  const int64_t total = (int64_t)B * P * H * Wd;
+  if (idx >= total) return;
+  const int w = (int)(idx % Wd);
+  const int h = (int)((idx / Wd) % H);
+  const int r = (int)((idx / ((int64_t)Wd * H)) % P);
+  const int bb = (int)(idx / ((int64_t)Wd * H * P));
+  const uint32_t* m = mask + ((int64_t)(bb * H + h) * NB) * Wd + w;
+  uint32_t acc = 0;
+  for (int i = 0; i < NB; ++i)
+    if (rank[i] == r) acc |= m[(int64_t)i * Wd];
+  U[idx] = acc;
+}
+
+// cnt[b][r][p][h] = popcount(U[b][r][h] & own[p]).  One thread per output.
+__global__ void count_kernel(const uint32_t* __restrict__ U, const uint32_t* __restrict__ own, int B,
+                             int H, int Wd, int P, int32_t* __restrict__ cnt) {
+  const int64_t idx = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+  const int64_t total = (int64_t)B * P * P * H;
+  if (idx >= total) return;
+  const int h = (int)(idx % H);
+  const int p = (int)((idx / H) % P);
+  const int r = (int)((idx / ((int64_t)H * P)) % P);
+  const int bb = (int)(idx / ((int64_t)H * P * P));
+  const uint32_t* u = U + ((int64_t)(bb * P + r) * H + h) * Wd;
+  const uint32_t* o = own + (int64_t)p * Wd;
+  int c = 0;
+  for (int w = 0; w < Wd; ++w) c += __popc(u[w] & o[w]);
+  cnt[idx] = c;
+}
+
+// One thread per (b, r): exclusive scan of cnt over (p, h) in pack order, totals and volume; then
+// thread 0 turns the totals into table bases.  Sizes are tiny (P*H values per thread).
+__global__ void scan_kernel(const int32_t* __restrict__ cnt, int B, int H, int P, int include_local,
+                            int64_t entry_bytes, int64_t* __restrict__ seg_off,
+                            int64_t* __restrict__ seg_total, int64_t* __restrict__ volume,
+                            int64_t* __restrict__ ent_base, int64_t* __restrict__ n_entries) {
+  const int idx = threadIdx.x;
+  if (idx < B * P) {
+    const int r = idx % P;
+    int64_t cursor = 0, remote = 0;
+    for (int p = 0; p < P; ++p) {
+      for (int h = 0; h < H; ++h) {
+        const int64_t o = ((int64_t)idx * P + p) * H + h;
+        const int c = cnt[o];
+        seg_off[o] = cursor;
+        if (p != r) remote += c;
+        if (p != r || include_local) cursor += c;
+      }
+    }
+    seg_total[idx] = cursor;
+    volume[idx] = entry_bytes * remote;
+  }
+  __syncthreads();
+  if (idx == 0) {
+    int64_t base = 0;
+    for (int t = 0; t < B * P; ++t) {
+      ent_base[t] = base;
+      base += seg_total[t];
+    }
+    *n_entries = base;
+  }
+}
+
+// Entry table: one warp per (b, r, p, h) segment enumerates the set bits of U & own[p] in ascending
+// order and writes entry records at table index ent_base[b,r] + seg_off + t.
+__global__ void entries_kernel(const uint32_t* __restrict__ U, const uint32_t* __restrict__ own, int B,
+                               int H, int Wd, int P, int include_local, int64_t entry_bytes,
+                               const int64_t* __restrict__ seg_off, const int64_t* __restrict__ ent_base,
+                               const int64_t* __restrict__ dst_base, int64_t capacity,
+                               PackEntry* __restrict__ entries, int32_t* __restrict__ status) {
+  const int64_t seg = ((int64_t)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
+  const int lane = threadIdx.x & 31;
+  const int64_t n_seg = (int64_t)B * P * P * H;
+  if (seg >= n_seg) return;
+  const int h = (int)(seg % H);
+  const int p = (int)((seg / H) % P);
+  const int r = (int)((seg / ((int64_t)H * P)) % P);
+  const int bb = (int)(seg / ((int64_t)H * P * P));
+  if (p == r && !include_local) return;
+  const uint32_t* u = U + ((int64_t)(bb * P + r) * H + h) * Wd;
+  const uint32_t* o = own + (int64_t)p * Wd;
+  const int64_t br = (int64_t)bb * P + r;
+  const int64_t first = seg_off[seg];
+  const int64_t base_byte = dst_base ? dst_base[br] : ent_base[br] * entry_bytes;
+  PackEntry* out = entries + ent_base[br] + first;
+  int running = 0;
+  for (int w0 = 0; w0 < Wd; w0 += 32) {
+    const int w = w0 + lane;
+    uint32_t bits = w < Wd ? (u[w] & o[w]) : 0u;
+    const int mine = __popc(bits);
+    int incl = mine;
+#pragma unroll
+    for (int s = 1; s < 32; s <<= 1) {
+      const int v = __shfl_up_sync(0xffffffffu, incl, s);
+      if (lane >= s) incl += v;
+    }
+    int pos = running + incl - mine;
+    while (bits) {
+      const int t = __ffs(bits) - 1;
+      bits &= bits - 1;
+      PackEntry e;
+      e.dst_byte = base_byte + (first + pos) * entry_bytes;
+      e.bh = bb * H + h;
+      e.j = w * 32 + t;
+      if (capacity >= 0 && e.dst_byte + entry_bytes > capacity) {
+        e.j = -1;  // would overflow: skipped by the gather
+        atomicExch(status, SPARSP_ERR_CAPACITY);
+      }
+      out[pos] = e;
+      ++pos;
+    }
+    running += __shfl_sync(0xffffffffu, incl, 31);
+  }
+}
+
+int launch_demand(const Geometry& g, const uint32_t* mask, const int32_t* rank_of_block, int P,
+                  int flags, uint32_t* U, int32_t* cnt, int64_t* seg_off, int64_t* seg_total,
+                  int64_t* volume, const int64_t* dst_base, int64_t capacity, char* ws,
+                  const WsLayout& L, cudaStream_t st) {
+  uint32_t* own = (uint32_t*)(ws + L.own);
+  int64_t* ent_base = (int64_t*)(ws + L.ent_base);
+  int64_t* n_entries = (int64_t*)(ws + L.n_entries);
+  PackEntry* entries = (PackEntry*)(ws + L.entries);
+  int32_t* status = (int32_t*)(ws + L.status);
+  const int include_local = (flags & SPARSP_INCLUDE_LOCAL) ? 1 : 0;
+  const int64_t entry_bytes = 2LL * g.b * g.d * 2;
+  if (g.B * P > 1024) {
+    set_error("batch * n_ranks = %d exceeds 1024", g.B * P);
+    return SPARSP_ERR_UNSUPPORTED;
+  }
+  own_kernel<<<(P * g.Wd + 127) / 128, 128, 0, st>>>(rank_of_block, g.NB, g.Wd, P, own);
+  const int64_t n_u = (int64_t)g.B * P * g.H * g.Wd;
+  union_kernel<<<(int)((n_u + 127) / 128), 128, 0, st>>>(mask, rank_of_block, g.B, g.H, g.NB, g.Wd, P, U);
+  const int64_t n_c = (int64_t)g.B * P * P * g.H;
+  count_kernel<<<(int)((n_c + 127) / 128), 128, 0, st>>>(U, own, g.B, g.H, g.Wd, P, cnt);
+  scan_kernel<<<1, 1024, 0, st>>>(cnt, g.B, g.H, P, include_local, entry_bytes, seg_off, seg_total,
+                                  volume, ent_base, n_entries);
+  entries_kernel<<<(int)((n_c * 32 + 255) / 256), 256, 0, st>>>(U, own, g.B, g.H, g.Wd, P,
+                                                               include_local, entry_bytes, seg_off,
+                                                               ent_base, dst_base, capacity, entries,
+                                                               status);
+  count_launch(5);
+  SPARSP_CUDA_OK(cudaGetLastError());
+  return SPARSP_OK;
+}
+
+// ------------------------------------------------------------------------------------------------
+// Gather.  Work item = one K or V tile of one entry (block x d bf16 = 8..32 KiB).  Persistent CTAs
+// stride over the items; a CTA moves a tile with 16-byte loads and stores, kUnroll independent loads
+// in flight per thread, fully coalesced when a tile's rows are adjacent in memory.  Rows at or
+// beyond N are written as zeros.
+// ------------------------------------------------------------------------------------------------
+constexpr int kPackThreads = 256;
+constexpr int kPackUnroll = 8;
+
+template <int D>
+__global__ void __launch_bounds__(kPackThreads) pack_kernel(
+    const __nv_bfloat16* __restrict__ K, const __nv_bfloat16* __restrict__ V,
+    const PackEntry* __restrict__ entries, const int64_t* __restrict__ n_entries_p, int H, int b,
+    int64_t N, int64_t sB, int64_t sH, int64_t sT, unsigned char* __restrict__ packed) {
+  constexpr int VPR = D / 8;  // 16-byte vectors per row
+  const int64_t n_items = 2 * (*n_entries_p);
+  const int vec_per_tile = b * VPR;
+  const int64_t tile_bytes = (int64_t)b * D * 2;
+  for (int64_t item = blockIdx.x; item < n_items; item += gridDim.x) {
+    const PackEntry e = entries[item >> 1];
+    if (e.j < 0) continue;
+    const int which = (int)(item & 1);
+    const int64_t batch = e.bh / H, head = e.bh % H;
+    const int64_t tok0 = (int64_t)e.j * b;
+    const int n_valid = (int)min((int64_t)b, N - tok0);
+    const __nv_bfloat16* src = (which ? V : K) + batch * sB + head * sH + tok0 * sT;
+    uint4* dst = reinterpret_cast<uint4*>(packed + e.dst_byte + which * tile_bytes);
+    for (int v0 = threadIdx.x; v0 < vec_per_tile; v0 += kPackThreads * kPackUnroll) {
+      uint4 buf[kPackUnroll];
+#pragma unroll
+      for (int u = 0; u < kPackUnroll; ++u) {
+        const int v = v0 + u * kPackThreads;
+        const int row = v / VPR, col = v % VPR;
+        buf[u] = make_uint4(0u, 0u, 0u, 0u);
+        if (v < vec_per_tile && row < n_valid)
+          buf[u] = __ldcs(reinterpret_cast<const uint4*>(src + (int64_t)row * sT) + col);
+      }
+#pragma unroll
+      for (int u = 0; u < kPackUnroll; ++u) {
+        const int v = v0 + u * kPackThreads;
+        if (v < vec_per_tile) __stcs(dst + v, buf[u]);
+      }
+    }
+  }
+}
+
+int launch_pack(const sparsp_shape& s, const Geometry& g, const void* K, const void* V, void* packed,
+                int64_t capacity, int P, char* ws, const WsLayout& L, cudaStream_t st) {
+  (void)capacity;
+  (void)P;
+  const PackEntry* entries = (const PackEntry*)(ws + L.entries);
+  const int64_t* n_entries = (const int64_t*)(ws + L.n_entries);
+  int dev = 0, sms = 148;
+  SPARSP_CUDA_OK(cudaGetDevice(&dev));
+  SPARSP_CUDA_OK(cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev));
+  const int grid = sms * 8;
+  auto k = (const __nv_bfloat16*)K;
+  auto v = (const __nv_bfloat16*)V;
+  if (g.d == 64)
+    pack_kernel<64><<<grid, kPackThreads, 0, st>>>(k, v, entries, n_entries, g.H, g.b, g.N,
+                                                   s.stride_batch, s.stride_head, s.stride_token,
+                                                   (unsigned char*)packed);
+  else
+    pack_kernel<128><<<grid, kPackThreads, 0, st>>>(k, v, entries, n_entries, g.H, g.b, g.N,
+                                                    s.stride_batch, s.stride_head, s.stride_token,
+                                                    (unsigned char*)packed);
+  count_launch();
+  SPARSP_CUDA_OK(cudaGetLastError());
+  return SPARSP_OK;
+}
+
+}  // namespace sparsp

@@ -1,0 +1,219 @@
+// Step 1: mean-pool Q and K per block, score pooled-Q x pooled-K^T per head, warp-level top-k.
+//
+// Arithmetic contract (the result decides which blocks are kept, so it is fixed to the operation):
+//   pool : fp32 sum of the block's valid tokens in ascending token order starting from 0, then one
+//          IEEE division by the valid count;
+//   score: acc = fmaf(q_c, k_c, acc) from acc = 0, channel c ascending;
+//   top-k: score descending, index ascending on equal scores, -0 == +0.
+#include "common.cuh"
+
+namespace sparsp {
+
+// ------------------------------------------------------------------------------------------------
+// pool: a group of d/8 lanes owns one (tensor, batch*head, block) tile; lane l owns channels
+// 8l..8l+7 and walks the tile's rows with 16-byte loads, so every channel is one sequential chain.
+// ------------------------------------------------------------------------------------------------
+template <int D>
+__global__ void __launch_bounds__(256) pool_kernel(const __nv_bfloat16* __restrict__ Q,
+                                                   const __nv_bfloat16* __restrict__ K,
+                                                   float* __restrict__ pq, float* __restrict__ pk,
+                                                   int H, int NB, int b, int64_t N, int64_t sB,
+                                                   int64_t sH, int64_t sT, int64_t n_tiles) {
+  constexpr int G = D / 8;  // lanes per tile
+  constexpr int U = 8;      // rows in flight per lane
+  const int64_t tile = ((int64_t)blockIdx.x * blockDim.x + threadIdx.x) / G;
+  const int lane = threadIdx.x % G;
+  if (tile >= 2 * n_tiles) return;
+  const bool is_k = tile >= n_tiles;
+  const int64_t t = is_k ? tile - n_tiles : tile;  // (batch*H + head) * NB + block
+  const int blk = (int)(t % NB);
+  const int64_t bh = t / NB;
+  const int64_t batch = bh / H, head = bh % H;
+  const int64_t tok0 = (int64_t)blk * b;
+  const int n = (int)min((int64_t)b, N - tok0);
+  const __nv_bfloat16* src = (is_k ? K : Q) + batch * sB + head * sH + tok0 * sT + lane * 8;
+
+  float acc[8];
+#pragma unroll
+  for (int c = 0; c < 8; ++c) acc[c] = 0.0f;
+
+  int r = 0;
+  for (; r + U <= n; r += U) {
+    uint4 v[U];
+#pragma unroll
+    for (int u = 0; u < U; ++u) v[u] = __ldg(reinterpret_cast<const uint4*>(src + (int64_t)(r + u) * sT));
+#pragma unroll
+    for (int u = 0; u < U; ++u) {
+      const uint32_t w[4] = {v[u].x, v[u].y, v[u].z, v[u].w};
+#pragma unroll
+      for (int p = 0; p < 4; ++p) {
+        acc[2 * p] = __fadd_rn(acc[2 * p], __uint_as_float(w[p] << 16));
+        acc[2 * p + 1] = __fadd_rn(acc[2 * p + 1], __uint_as_float(w[p] & 0xffff0000u));
+      }
+    }
+  }
+  for (; r < n; ++r) {
+    const uint4 v = __ldg(reinterpret_cast<const uint4*>(src + (int64_t)r * sT));
+    const uint32_t w[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+    for (int p = 0; p < 4; ++p) {
+      acc[2 * p] = __fadd_rn(acc[2 * p], __uint_as_float(w[p] << 16));
+      acc[2 * p + 1] = __fadd_rn(acc[2 * p + 1], __uint_as_float(w[p] & 0xffff0000u));
+    }
+  }
+  const float cntf = (float)n;
+  float* dst = (is_k ? pk : pq) + t * D + lane * 8;
+  float4 o0, o1;
+  o0.x = __fdiv_rn(acc[0], cntf);
+  o0.y = __fdiv_rn(acc[1], cntf);
+  o0.z = __fdiv_rn(acc[2], cntf);
+  o0.w = __fdiv_rn(acc[3], cntf);
+  o1.x = __fdiv_rn(acc[4], cntf);
+  o1.y = __fdiv_rn(acc[5], cntf);
+  o1.z = __fdiv_rn(acc[6], cntf);
+  o1.w = __fdiv_rn(acc[7], cntf);
+  reinterpret_cast<float4*>(dst)[0] = o0;
+  reinterpret_cast<float4*>(dst)[1] = o1;
+}
+
+int launch_pool(const sparsp_shape& s, const Geometry& g, const void* Q, const void* K, float* pq,
+                float* pk, cudaStream_t st) {
+  const int64_t n_tiles = (int64_t)g.B * g.H * g.NB;
+  const int G = g.d / 8;
+  const int64_t threads = 2 * n_tiles * G;
+  const int grid = (int)((threads + 255) / 256);
+  auto q = (const __nv_bfloat16*)Q;
+  auto k = (const __nv_bfloat16*)K;
+  if (g.d == 64)
+    pool_kernel<64><<<grid, 256, 0, st>>>(q, k, pq, pk, g.H, g.NB, g.b, g.N, s.stride_batch,
+                                          s.stride_head, s.stride_token, n_tiles);
+  else
+    pool_kernel<128><<<grid, 256, 0, st>>>(q, k, pq, pk, g.H, g.NB, g.b, g.N, s.stride_batch,
+                                           s.stride_head, s.stride_token, n_tiles);
+  count_launch();
+  SPARSP_CUDA_OK(cudaGetLastError());
+  return SPARSP_OK;
+}
+
+// ------------------------------------------------------------------------------------------------
+// score + top-k.  A CTA owns ROWS = WARPS*RPW query blocks of one (batch, head); pooled K streams
+// through shared memory in 32-block tiles; lane l of a warp computes the scores of column l of the
+// tile for the warp's RPW rows.  Scores stay in shared memory as order-preserving uint32 keys and
+// the warp then selects its rows' k largest by a 32-step radix search with ballots.
+// ------------------------------------------------------------------------------------------------
+constexpr int kScoreWarps = 8;
+constexpr int kScoreRPW = 2;
+constexpr int kScoreRows = kScoreWarps * kScoreRPW;
+
+__device__ __forceinline__ uint32_t score_key(float s) {
+  if (s == 0.0f) s = 0.0f;  // -0 -> +0 so that they compare equal
+  const uint32_t u = __float_as_uint(s);
+  return (u & 0x80000000u) ? ~u : (u | 0x80000000u);
+}
+
+template <int D>
+__global__ void __launch_bounds__(kScoreWarps * 32) score_topk_kernel(
+    const float* __restrict__ pq, const float* __restrict__ pk, int NB, int Wd, int nb_cand, int topk,
+    int kept_cap, uint32_t* __restrict__ mask, int32_t* __restrict__ kv_list,
+    int32_t* __restrict__ kv_count) {
+  extern __shared__ __align__(16) unsigned char smem_raw[];
+  float* sQ = reinterpret_cast<float*>(smem_raw);                 // [ROWS][D]
+  float* sK = sQ + kScoreRows * D;                                // [32][D+1]
+  uint32_t* sS = reinterpret_cast<uint32_t*>(sK + 32 * (D + 1));  // [ROWS][NBpad]
+  const int NBpad = Wd * 32;
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int64_t bh = blockIdx.y;
+  const int row0 = blockIdx.x * kScoreRows;
+
+  for (int idx = threadIdx.x; idx < kScoreRows * D; idx += blockDim.x) {
+    const int r = row0 + idx / D;
+    sQ[idx] = r < NB ? pq[(bh * NB + r) * D + idx % D] : 0.0f;
+  }
+
+  for (int t = 0; t < Wd; ++t) {
+    __syncthreads();
+    for (int idx = threadIdx.x; idx < 32 * D; idx += blockDim.x) {
+      const int jj = idx / D, c = idx % D;
+      const int j = t * 32 + jj;
+      sK[jj * (D + 1) + c] = j < NB ? pk[(bh * NB + j) * D + c] : 0.0f;
+    }
+    __syncthreads();
+    float acc[kScoreRPW];
+#pragma unroll
+    for (int r = 0; r < kScoreRPW; ++r) acc[r] = 0.0f;
+    const float* kcol = sK + lane * (D + 1);
+#pragma unroll 8
+    for (int c = 0; c < D; ++c) {
+      const float kv = kcol[c];
+#pragma unroll
+      for (int r = 0; r < kScoreRPW; ++r)
+        acc[r] = __fmaf_rn(sQ[(warp * kScoreRPW + r) * D + c], kv, acc[r]);
+    }
+#pragma unroll
+    for (int r = 0; r < kScoreRPW; ++r)
+      sS[(warp * kScoreRPW + r) * NBpad + t * 32 + lane] = score_key(acc[r]);
+  }
+  __syncwarp();
+
+  const uint32_t lt_mask = (1u << lane) - 1u;
+  for (int r = 0; r < kScoreRPW; ++r) {
+    const int i = row0 + warp * kScoreRPW + r;
+    if (i >= NB) break;  // warp-uniform
+    const uint32_t* keys = sS + (warp * kScoreRPW + r) * NBpad;
+    // largest T with |{ candidates : key >= T }| >= topk  ==> T is the topk-th largest key
+    uint32_t T = 0;
+    for (int bit = 31; bit >= 0; --bit) {
+      const uint32_t trial = T | (1u << bit);
+      int c = 0;
+      for (int t = 0; t < Wd; ++t) {
+        const int j = t * 32 + lane;
+        c += (j < nb_cand && keys[j] >= trial) ? 1 : 0;
+      }
+      c = __reduce_add_sync(0xffffffffu, c);
+      if (c >= topk) T = trial;
+    }
+    int gt = 0;
+    for (int t = 0; t < Wd; ++t) {
+      const int j = t * 32 + lane;
+      gt += (j < nb_cand && keys[j] > T) ? 1 : 0;
+    }
+    gt = __reduce_add_sync(0xffffffffu, gt);
+    const int need_eq = topk - gt;  // ties at T taken in ascending index order
+    int eq_seen = 0, out_pos = 0;
+    const int64_t row = bh * NB + i;
+    for (int t = 0; t < Wd; ++t) {
+      const int j = t * 32 + lane;
+      const bool cand = j < nb_cand;
+      const uint32_t key = keys[j];
+      const bool is_eq = cand && key == T;
+      const uint32_t eq_ballot = __ballot_sync(0xffffffffu, is_eq);
+      const bool take_eq = is_eq && (eq_seen + __popc(eq_ballot & lt_mask) < need_eq);
+      eq_seen += __popc(eq_ballot);
+      const bool keep = (cand && key > T) || take_eq || (j >= nb_cand && j < NB);
+      const uint32_t word = __ballot_sync(0xffffffffu, keep);
+      if (lane == 0) mask[row * Wd + t] = word;
+      if (kv_list && keep) {
+        const int pos = out_pos + __popc(word & lt_mask);
+        if (pos < kept_cap) kv_list[row * kept_cap + pos] = j;
+      }
+      out_pos += __popc(word);
+    }
+    if (kv_count && lane == 0) kv_count[row] = out_pos;
+  }
+}
+
+int launch_score_topk(const Geometry& g, const float* pq, const float* pk, int topk, uint32_t* mask,
+                      int32_t* kv_list, int32_t* kv_count, cudaStream_t st) {
+  const int kept_cap = topk + (g.NB - g.nb_cand);
+  const size_t smem = (size_t)(kScoreRows * g.d + 32 * (g.d + 1) + kScoreRows * g.Wd * 32) * 4;
+  dim3 grid((g.NB + kScoreRows - 1) / kScoreRows, g.B * g.H);
+  auto kern = g.d == 64 ? score_topk_kernel<64> : score_topk_kernel<128>;
+  SPARSP_CUDA_OK(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+  kern<<<grid, kScoreWarps * 32, smem, st>>>(pq, pk, g.NB, g.Wd, g.nb_cand, topk, kept_cap, mask,
+                                            kv_list, kv_count);
+  count_launch();
+  SPARSP_CUDA_OK(cudaGetLastError());
+  return SPARSP_OK;
+}
+
+}  // namespace sparsp

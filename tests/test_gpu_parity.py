@@ -1,0 +1,215 @@
+"""GPU parity tests (small sizes): the three C-ABI calls against the CPU oracle, element by element.
+Sizes are chosen so that the oracle finishes in seconds yet every kernel runs several tiles and a
+ragged tail; both memory layouts and every supported (head_dim, block) pair are covered."""
+import numpy as np
+import pytest
+import torch
+
+import parity_util as pu
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def binding():
+    from paper_2609_32197_b200 import binding as b
+    b.lib()  # raises if the CUDA library is missing: there is no fallback
+    assert torch.cuda.is_available()
+    return b
+
+
+def _gen(wl):
+    from paper_2609_32197_b200 import synth
+    return synth.make_qkv(wl, "cpu")
+
+
+def _workload(name, heads, d, grid, n_text, b, k, ranks, seed=0):
+    from paper_2609_32197_b200 import synth
+    return synth.Workload(name, heads, d, grid, n_text, b, k, None, ranks, seed=seed)
+
+
+def _run_all(oracle, binding, wl, rank_np, layout="HND", include_local=False, full_attn=True, lse=True):
+    Q, K, V = _gen(wl)
+    H, N, d = Q.shape
+    b, P, k = wl.block, wl.ranks, wl.topk_abs
+    shape = binding.make_shape(H, d, wl.grid, wl.n_text, b, layout=layout)
+    Qd, Kd, Vd = (pu.to_layout(x.cuda(), layout) for x in (Q, K, V))
+    ws = binding.make_workspace(shape, P)
+    # step 1
+    ref, got = pu.check_mask(oracle, binding, shape, Q, K, Qd, Kd, k, wl.n_text, ws)
+    # step 2
+    rank_d = torch.as_tensor(rank_np, dtype=torch.int32).cuda()
+    flags = binding.SPARSP_INCLUDE_LOCAL if include_local else 0
+    dg = pu.gpu_demand_pack(binding, shape, got["mask"], rank_d, P, flags, Kd, Vd, ws)
+    dref = pu.check_demand(oracle, binding, shape, ref["mask"], rank_np, P, include_local, dg)
+    packed_ref = oracle.pack(K, V, dref["U"], rank_np, b, P, dref["total"], include_local=include_local)
+    packed = dg["packed"].cpu().numpy()
+    assert np.array_equal(packed[:packed_ref.size], packed_ref), "packed bytes"
+    assert (packed[packed_ref.size:] == 0xAB).all(), "wrote past the end"
+    # step 3
+    Od = torch.zeros_like(Qd)
+    lse_d = torch.zeros(1, H, N, dtype=torch.float32, device="cuda") if lse else None
+    binding.sparsp_sparse_attn_fwd(shape, Qd, Kd, Vd, got["mask"], 0.0, Od, lse_d, ws)
+    torch.cuda.synchronize()
+    assert binding.sparsp_status(ws) == binding.SPARSP_OK
+    NB = wl.n_blocks
+    units = [(h, i) for h in range(H) for i in range(NB)] if full_attn else pu.sample_units(H, NB, rank_np, 8, 0)
+    return pu.check_attn_units(oracle, Q, K, V, ref["mask"], b, pu.from_layout(Od, layout), units,
+                               lse_gpu=None if lse_d is None else lse_d[0])
+
+
+def test_tiny_config_full(oracle_mod, binding):
+    from paper_2609_32197_b200 import synth
+    wl = synth.WORKLOADS["tiny"]
+    rank = oracle_mod.placement_contiguous(wl.n_blocks, wl.ranks)
+    mx, mean = _run_all(oracle_mod, binding, wl, rank)
+    print(f"tiny: attn max abs {mx:.3e} mean abs {mean:.3e}")
+
+
+@pytest.mark.parametrize("d,b", [(64, 64), (128, 64), (64, 128), (128, 128)])
+@pytest.mark.parametrize("layout", ["HND", "NHD"])
+def test_ragged_text_all_shapes(oracle_mod, binding, d, b, layout):
+    # 5*11*13 = 715 video + 70 text = 785 tokens: ragged last block for both block sizes, text tail
+    wl = _workload("ragged", 3, d, (5, 11, 13), 70, b, 3 if b == 128 else 5, 3, seed=3)
+    rank = np.array([(j * 5) % 3 for j in range(wl.n_blocks)], np.int32)  # scattered placement
+    _run_all(oracle_mod, binding, wl, rank, layout=layout, include_local=(layout == "NHD"))
+
+
+def test_multi_word_masks_and_periodic_placement(oracle_mod, binding):
+    # 4*24*32 = 3072 tokens, block 64 -> 48 blocks (2 mask words), frames aligned to blocks
+    wl = _workload("multiword", 4, 64, (4, 24, 32), 0, 64, 7, 4, seed=5)
+    rank = oracle_mod.placement_periodic(wl.n_blocks, 4, 64, wl.frame_tokens, wl.n_video)
+    shape = binding.make_shape(4, 64, wl.grid, 0, 64)
+    assert np.array_equal(binding.sparsp_placement_periodic(shape, 4).numpy(), rank)
+    assert np.array_equal(binding.sparsp_placement_contiguous(shape, 4).numpy(),
+                          oracle_mod.placement_contiguous(wl.n_blocks, 4))
+    _run_all(oracle_mod, binding, wl, rank)
+
+
+def test_exact_ties_lowest_index_wins(oracle_mod, binding):
+    """Integer construction with S[i][j] = i^2 - (i-j)^2: every row has exact score ties."""
+    NB, b, d, H = 40, 64, 64, 2
+    N = NB * b
+    q = np.zeros((H, N, d), np.float32)
+    k = np.zeros((H, N, d), np.float32)
+    for j in range(NB):
+        sq = j * j
+        q[:, j * b:(j + 1) * b, :4] = [2 * j, -1, -16, -256]
+        k[:, j * b:(j + 1) * b, :4] = [j, sq % 16, (sq // 16) % 16, sq // 256]
+    Q, K = torch.tensor(q).to(torch.bfloat16), torch.tensor(k).to(torch.bfloat16)
+    shape = binding.make_shape(H, d, (1, NB, b), 0, b)
+    ws = binding.make_workspace(shape, 1)
+    for kk in (1, 2, 6, 39, 40):
+        ref, got = pu.check_mask(oracle_mod, binding, shape, Q, K, Q.cuda(), K.cuda(), kk, 0, ws)
+        row = pu.u32(got["mask"][0])[0, 20]
+        bits = [j for j in range(NB) if (int(row[j >> 5]) >> (j & 31)) & 1]
+        assert bits == sorted(sorted(range(NB), key=lambda j: (abs(20 - j), j))[:kk])
+
+
+def test_signed_zero_scores_tie(oracle_mod, binding):
+    """Q block 0 is all zeros with K mixing signs: scores are +0 and -0, which must compare equal."""
+    NB, b, d, H = 8, 64, 64, 1
+    N = NB * b
+    rng = np.random.default_rng(0)
+    k = rng.standard_normal((H, N, d)).astype(np.float32)
+    q = rng.standard_normal((H, N, d)).astype(np.float32)
+    q[:, :b] = 0.0
+    q[:, :b:2, 0] = -0.0
+    Q, K = torch.tensor(q).to(torch.bfloat16), torch.tensor(k).to(torch.bfloat16)
+    shape = binding.make_shape(H, d, (1, NB, b), 0, b)
+    ws = binding.make_workspace(shape, 1)
+    ref, got = pu.check_mask(oracle_mod, binding, shape, Q, K, Q.cuda(), K.cuda(), 3, 0, ws)
+    assert list(ref["kv_list"][0, 0]) == [0, 1, 2]
+
+
+def test_dense_mask_matches_library_sdpa(oracle_mod, binding):
+    """top-k = NB keeps everything: the kernel must reproduce dense attention (library fp32 SDPA)."""
+    wl = _workload("dense", 2, 128, (2, 12, 20), 0, 128, 4, 2, seed=9)  # 480 tokens -> 4 blocks (last: 96)
+    Q, K, V = _gen(wl)
+    shape = binding.make_shape(2, 128, wl.grid, 0, 128)
+    ws = binding.make_workspace(shape, 2)
+    Qd, Kd, Vd = Q.cuda(), K.cuda(), V.cuda()
+    got = pu.gpu_block_mask(binding, shape, Qd, Kd, wl.n_blocks, ws)
+    assert int(torch.bitwise_and(got["mask"], 0xF).eq(0xF).all())
+    Od = torch.zeros_like(Qd)
+    binding.sparsp_sparse_attn_fwd(shape, Qd, Kd, Vd, got["mask"], 0.0, Od, None, ws)
+    ref = torch.nn.functional.scaled_dot_product_attention(Qd.float()[None], Kd.float()[None], Vd.float()[None])[0]
+    err = (Od.float() - ref).abs()
+    assert err.max().item() <= pu.ATTN_MAX_ABS and err.mean().item() <= pu.ATTN_MEAN_ABS
+
+
+def test_explicit_scale_single_rank_and_capacity_overflow(oracle_mod, binding):
+    wl = _workload("cap", 2, 64, (2, 16, 16), 0, 64, 3, 2, seed=11)  # 512 tokens, 8 blocks
+    Q, K, V = _gen(wl)
+    shape = binding.make_shape(2, 64, wl.grid, 0, 64)
+    ws = binding.make_workspace(shape, 2)
+    Qd, Kd, Vd = Q.cuda(), K.cuda(), V.cuda()
+    ref, got = pu.check_mask(oracle_mod, binding, shape, Q, K, Qd, Kd, 3, 0, ws)
+    # explicit softmax scale
+    Od = torch.zeros_like(Qd)
+    binding.sparsp_sparse_attn_fwd(shape, Qd, Kd, Vd, got["mask"], 0.05, Od, None, ws)
+    units = [(h, i) for h in range(2) for i in range(8)]
+    pu.check_attn_units(oracle_mod, Q, K, V, ref["mask"], 64, Od, units, scale=0.05)
+    # one rank: nothing is remote
+    rank1 = torch.zeros(8, dtype=torch.int32, device="cuda")
+    d1 = pu.gpu_demand_pack(binding, shape, got["mask"], rank1, 1, 0, Kd, Vd, ws)
+    assert d1["total_entries"] == 0 and int(d1["volume_bytes"].sum()) == 0
+    assert bool((d1["packed"] == 0xAB).all())
+    # capacity one entry short: the last entry is skipped, nothing beyond capacity is touched
+    rank2 = torch.as_tensor(oracle_mod.placement_contiguous(8, 2)).cuda()
+    full = pu.gpu_demand_pack(binding, shape, got["mask"], rank2, 2, 0, Kd, Vd, ws)
+    assert binding.sparsp_status(ws) == binding.SPARSP_OK
+    n = full["total_entries"]
+    short = pu.gpu_demand_pack(binding, shape, got["mask"], rank2, 2, 0, Kd, Vd, ws, capacity_entries=n - 1)
+    assert binding.sparsp_status(ws) == binding.SPARSP_ERR_CAPACITY
+    assert binding.sparsp_status(ws) == binding.SPARSP_OK  # reading resets it
+    entry = 2 * 64 * 64 * 2
+    assert torch.equal(short["packed"][:(n - 1) * entry], full["packed"][:(n - 1) * entry])
+    assert bool((short["packed"][(n - 1) * entry:] == 0xAB).all())
+
+
+def test_destination_bases(oracle_mod, binding):
+    wl = _workload("bases", 2, 64, (2, 16, 16), 0, 64, 3, 2, seed=12)
+    Q, K, V = _gen(wl)
+    shape = binding.make_shape(2, 64, wl.grid, 0, 64)
+    ws = binding.make_workspace(shape, 2)
+    Qd, Kd, Vd = Q.cuda(), K.cuda(), V.cuda()
+    ref, got = pu.check_mask(oracle_mod, binding, shape, Q, K, Qd, Kd, 3, 0, ws)
+    rank = oracle_mod.placement_contiguous(8, 2)
+    dref = oracle_mod.demand(ref["mask"], rank, 2, 64, 64)
+    entry = 2 * 64 * 64 * 2
+    base = np.array([int(dref["total"][1]) * entry + 4096, 0], np.int64)  # swapped, with a gap
+    expect = oracle_mod.pack(K, V, dref["U"], rank, 64, 2, dref["total"], dst_base=base)
+    outs = binding.alloc_demand_outputs(shape, 2)
+    packed = torch.zeros(expect.size, dtype=torch.uint8, device="cuda")
+    binding.sparsp_demand_pack(shape, got["mask"], torch.as_tensor(rank).cuda(), 2, 0, Kd, Vd, outs["union_mask"],
+                               outs["cnt"], outs["seg_offset"], outs["seg_total"], outs["volume_bytes"], packed,
+                               expect.size, torch.as_tensor(base).cuda(), ws)
+    torch.cuda.synchronize()
+    assert np.array_equal(packed.cpu().numpy(), expect)
+
+
+def test_invalid_arguments_are_rejected_on_the_host(binding):
+    shape = binding.make_shape(2, 64, (2, 16, 16), 0, 64)
+    ws = binding.make_workspace(shape, 2)
+    x = torch.zeros(2, 512, 64, dtype=torch.bfloat16, device="cuda")
+    outs = binding.alloc_mask_outputs(shape, 3)
+    with pytest.raises(binding.SparspError) as e:
+        binding.sparsp_block_mask(shape, x, x, 0, outs["mask"], None, None, None, None, ws)
+    assert e.value.code == binding.SPARSP_ERR_INVALID_ARG
+    with pytest.raises(binding.SparspError) as e:
+        binding.sparsp_block_mask(shape, None, x, 3, outs["mask"], None, None, None, None, ws)
+    assert e.value.code == binding.SPARSP_ERR_INVALID_ARG
+    bad = binding.make_shape(2, 96, (2, 16, 16), 0, 64)
+    with pytest.raises(binding.SparspError) as e:
+        binding.sparsp_block_mask(bad, x, x, 3, outs["mask"], None, None, None, None, ws)
+    assert e.value.code == binding.SPARSP_ERR_UNSUPPORTED
+    with pytest.raises(binding.SparspError) as e:
+        binding.sparsp_sparse_attn_fwd(shape, x, x, x, outs["mask"], -1.0, x, None, ws)
+    assert e.value.code == binding.SPARSP_ERR_INVALID_ARG
+    d = binding.alloc_demand_outputs(shape, 2)
+    with pytest.raises(binding.SparspError) as e:
+        binding.sparsp_demand_pack(shape, outs["mask"], torch.zeros(8, dtype=torch.int32, device="cuda"), 0, 0, x, x,
+                                   d["union_mask"], d["cnt"], d["seg_offset"], d["seg_total"], d["volume_bytes"],
+                                   x, 16, None, ws)
+    assert e.value.code == binding.SPARSP_ERR_INVALID_ARG
