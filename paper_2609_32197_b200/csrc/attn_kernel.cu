@@ -1,17 +1,22 @@
-// Step 3: block-sparse FlashAttention forward on tcgen05 tensor cores.
+// Step 3: block-sparse FlashAttention forward on tcgen05 tensor cores (sm_100a).
 //
-// One CTA owns a 128-row query tile of one (batch, head): one query block when block = 128, two
-// adjacent query blocks when block = 64 (the tile then walks the UNION of the two rows' kept KV
-// blocks and each half masks out the blocks its own row does not keep, so the MMAs always run at
-// the full M = 128 rate).  Per kept KV block j:
-//     TMA   K_j, V_j -> shared memory (128-byte swizzle, 2-stage ring)
-//     MMA   S = Q K_j^T            (tcgen05.mma, fp32 accumulator in tensor memory)
-//     all   thread r reads row r of S from tensor memory, online softmax in fp32 (base-2
-//           exponentials, lazy rescale of O only when a row's max grows by more than 2^8),
-//           writes P (bf16) to shared memory in the swizzled K-major operand layout
-//     MMA   O += P V_j             (V consumed in place as an MN-major operand)
-// Epilogue: O / l -> bf16 -> global, optional log-sum-exp.
-// Every mbarrier wait is bounded; a wait that runs out sets SPARSP_ERR_TIMEOUT in the status word.
+// A CTA owns two adjacent query blocks of one (batch, head) and runs two independent softmax
+// "streams" so that one stream's exponentials overlap the other stream's MMAs:
+//   block = 128: the two query blocks are two 128-row Q tiles; stream s = Q tile s.  The CTA walks
+//                the UNION of the two rows' kept KV blocks; a stream skips the blocks its own row
+//                does not keep, K/V tiles that both keep are loaded once.
+//   block = 64 : the two query blocks are stacked into ONE 128-row Q tile (full-rate M = 128 MMAs);
+//                a KV tile is two entries of the union list (128 keys, full-rate N = 128); each
+//                64x64 quadrant the mask does not keep is zeroed in P.  Stream s takes the KV tiles
+//                of parity s into its own accumulator; the two partial results are merged at the end.
+// Warp roles (384 threads): warp 0 = TMA producer (K ring and V ring, polled independently),
+// warp 1 = MMA issuer (one thread), warps 2-3 idle, warps 4-7 / 8-11 = softmax warpgroups of stream
+// 0 / 1, one query row per thread; the first warpgroup gives registers up to the softmax ones.  Tensor memory: S_s (128 fp32 columns, overwritten in place by bf16 P_s, which
+// the P.V MMA reads straight from tensor memory) and O_s (d fp32 columns) per stream.
+// Online softmax is base-2 in fp32; O is rescaled lazily, only when a row's maximum has grown by
+// more than 2^8 since the reference last moved.
+// Every mbarrier wait is bounded; a wait that runs out sets SPARSP_ERR_TIMEOUT in the status word
+// and raises a CTA-wide flag that makes all later waits fall through, so the CTA still drains.
 #include "common.cuh"
 #include "sm100_ptx.cuh"
 
@@ -31,58 +36,71 @@ struct AttnParams {
   long long wait_limit;
 };
 
-constexpr int kAttnThreads = 128;
-constexpr int kTileM = 128;
-constexpr int kStages = 2;
-constexpr int kTmemCols = 256;
+constexpr int kAttnThreads = 384;
+constexpr int kTmemCols = 512;
+constexpr float kGrowThreshold = 8.0f;
 
 template <int D, int BLK>
-struct AttnSmem {
-  static constexpr int kQBytes = kTileM * D * 2;
-  static constexpr int kKVBytes = BLK * D * 2;
-  static constexpr int kPBytes = kTileM * BLK * 2;
+struct AttnCfg {
+  static constexpr bool kSplitKV = (BLK == 64);   // one Q tile, streams split the KV tiles
+  static constexpr int kQTiles = kSplitKV ? 1 : 2;
+  static constexpr int kEPT = 128 / BLK;          // union-list entries per 128-key KV tile
+  static constexpr int kStages = (D == 64) ? 4 : 2;
+  static constexpr int kQBytes = 128 * D * 2;
+  static constexpr int kTileBytes = 128 * D * 2;  // one K or V tile
   static constexpr int kOffQ = 0;
-  static constexpr int kOffK = kOffQ + kQBytes;
-  static constexpr int kOffV = kOffK + kStages * kKVBytes;
-  static constexpr int kOffP = kOffV + kStages * kKVBytes;
-  static constexpr int kOffList = kOffP + kPBytes;            // uint16 [1024] kept KV blocks of the tile
-  static constexpr int kOffFlags = kOffList + 2 * kMaxBlocks;  // uint8 [1024] which tile halves keep it
-  static constexpr int kOffBars = kOffFlags + kMaxBlocks;      // mbarriers
-  static constexpr int kOffMisc = kOffBars + 64;
-  static constexpr int kTotal = kOffMisc + 64;
+  static constexpr int kOffK = kOffQ + kQTiles * kQBytes;
+  static constexpr int kOffV = kOffK + kStages * kTileBytes;
+  static constexpr int kOffEntJ = kOffV + kStages * kTileBytes;  // uint16 [1024] union list
+  static constexpr int kOffEntF = kOffEntJ + 2 * kMaxBlocks;     // uint8 [1024] bit q: kept by query block q
+  static constexpr int kOffStat = kOffEntF + kMaxBlocks;         // float2 [2][128] stream statistics
+  static constexpr int kOffBars = kOffStat + 2 * 128 * 8;
+  static constexpr int kNumBars = 1 + 4 * kStages + 6;
+  static constexpr int kOffMisc = kOffBars + 8 * kNumBars;
+  static constexpr int kTotal = kOffMisc + 32;
   static constexpr int kDynamic = kTotal + 1024;  // slack for the 1024-byte alignment of the base
+  static constexpr int kMergeStride = D / 2 + 4;  // floats per row of the merge buffer
+  static_assert(2 * 128 * kMergeStride * 4 <= 2 * kStages * kTileBytes, "merge buffer must fit the K/V rings");
+  static_assert(kDynamic <= 232448, "shared memory budget");
 };
+
+__device__ __forceinline__ void named_bar_sync(int id, int n) {
+  asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(n) : "memory");
+}
 
 template <int D, int BLK>
 __global__ void __launch_bounds__(kAttnThreads, 1)
     attn_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmK,
                     const __grid_constant__ CUtensorMap tmV, const AttnParams p) {
-  using L = AttnSmem<D, BLK>;
-  constexpr int QB = kTileM / BLK;  // query blocks per tile
+  using C = AttnCfg<D, BLK>;
+  constexpr int S = C::kStages;
   extern __shared__ unsigned char smem_dyn[];
-  unsigned char* smem = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_dyn) + 1023) & ~uintptr_t(1023));
-  unsigned char* sQ = smem + L::kOffQ;
-  unsigned char* sK = smem + L::kOffK;
-  unsigned char* sV = smem + L::kOffV;
-  unsigned char* sP = smem + L::kOffP;
-  uint16_t* sList = reinterpret_cast<uint16_t*>(smem + L::kOffList);
-  uint8_t* sFlags = smem + L::kOffFlags;
-  uint64_t* bars = reinterpret_cast<uint64_t*>(smem + L::kOffBars);
-  uint64_t* bar_q = bars + 0;
-  uint64_t* bar_full = bars + 1;  // [kStages]
-  uint64_t* bar_s = bars + 3;
-  uint64_t* bar_o = bars + 4;
-  uint32_t* s_tmem = reinterpret_cast<uint32_t*>(smem + L::kOffMisc);
-  int* s_ntiles = reinterpret_cast<int*>(smem + L::kOffMisc + 4);
-  volatile int* s_abort = reinterpret_cast<volatile int*>(smem + L::kOffMisc + 8);
+  unsigned char* smem =
+      reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_dyn) + 1023) & ~uintptr_t(1023));
+  unsigned char* sQ = smem + C::kOffQ;
+  unsigned char* sK = smem + C::kOffK;
+  unsigned char* sV = smem + C::kOffV;
+  uint16_t* sEntJ = reinterpret_cast<uint16_t*>(smem + C::kOffEntJ);
+  uint8_t* sEntF = smem + C::kOffEntF;
+  float2* sStat = reinterpret_cast<float2*>(smem + C::kOffStat);
+  uint64_t* bars = reinterpret_cast<uint64_t*>(smem + C::kOffBars);
+  uint64_t* bar_q = bars;
+  uint64_t* k_full = bars + 1;
+  uint64_t* k_empty = k_full + S;
+  uint64_t* v_full = k_empty + S;
+  uint64_t* v_empty = v_full + S;
+  uint64_t* s_full = v_empty + S;  // [2] S_s written by Q K^T
+  uint64_t* p_full = s_full + 2;   // [2] P_s written by the softmax warpgroup (128 arrivals)
+  uint64_t* o_full = p_full + 2;   // [2] a P V of stream s has completed
+  uint32_t* s_tmem = reinterpret_cast<uint32_t*>(smem + C::kOffMisc);
+  int* s_nent = reinterpret_cast<int*>(smem + C::kOffMisc + 4);
+  volatile int* s_abort = reinterpret_cast<volatile int*>(smem + C::kOffMisc + 8);
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-  const int tile = blockIdx.x;
   const int bh = blockIdx.y;
   const int batch = bh / p.H, head = bh % p.H;
-  const int64_t q0 = (int64_t)tile * kTileM;
-  const int my_qb = tid / BLK;  // which of the tile's query blocks this row belongs to
-  const int i0 = tile * QB;
+  const int i0 = blockIdx.x * 2;  // first of the CTA's two query blocks
+  const int64_t q0 = (int64_t)i0 * BLK;
 
   // ---- setup ------------------------------------------------------------------------------
   if (tid == 0) {
@@ -90,25 +108,34 @@ __global__ void __launch_bounds__(kAttnThreads, 1)
     prefetch_tmap(&tmK);
     prefetch_tmap(&tmV);
     mbar_init(bar_q, 1);
-    for (int s = 0; s < kStages; ++s) mbar_init(bar_full + s, 1);
-    mbar_init(bar_s, 1);
-    mbar_init(bar_o, 1);
+    for (int s = 0; s < S; ++s) {
+      mbar_init(k_full + s, 1);
+      mbar_init(k_empty + s, 1);
+      mbar_init(v_full + s, 1);
+      mbar_init(v_empty + s, 1);
+    }
+    for (int s = 0; s < 2; ++s) {
+      mbar_init(s_full + s, 1);
+      mbar_init(p_full + s, 128);
+      mbar_init(o_full + s, 1);
+    }
     mbar_init_fence();
     *s_abort = 0;
   }
+  if (warp == 1) {
+    tmem_alloc(s_tmem, kTmemCols);
+    tmem_relinquish();
+  }
   if (warp == 0) {
-    // union of the tile's mask rows -> ascending list of KV blocks + per-block "kept by half q" flags
+    // union of the two mask rows -> ascending entry list; flag bit q = kept by query block i0 + q
     const uint32_t* mrow = p.mask + ((int64_t)bh * p.NB + i0) * p.Wd;
     int running = 0;
     for (int w0 = 0; w0 < p.Wd; w0 += 32) {
       const int w = w0 + lane;
-      uint32_t rowbits[QB];
-      uint32_t u = 0;
-#pragma unroll
-      for (int q = 0; q < QB; ++q) {
-        rowbits[q] = (w < p.Wd && i0 + q < p.NB) ? mrow[(int64_t)q * p.Wd + w] : 0u;
-        u |= rowbits[q];
-      }
+      uint32_t rb[2];
+      rb[0] = (w < p.Wd) ? mrow[w] : 0u;
+      rb[1] = (w < p.Wd && i0 + 1 < p.NB) ? mrow[p.Wd + w] : 0u;
+      uint32_t u = rb[0] | rb[1];
       const int mine = __popc(u);
       int incl = mine;
 #pragma unroll
@@ -120,202 +147,355 @@ __global__ void __launch_bounds__(kAttnThreads, 1)
       while (u) {
         const int t = __ffs(u) - 1;
         u &= u - 1;
-        const int j = w * 32 + t;
-        if (j < p.NB) {
-          uint8_t f = 0;
-#pragma unroll
-          for (int q = 0; q < QB; ++q) f |= ((rowbits[q] >> t) & 1u) << q;
-          sList[pos] = (uint16_t)j;
-          sFlags[pos] = f;
-          ++pos;
-        }
+        sEntJ[pos] = (uint16_t)(w * 32 + t);
+        sEntF[pos] = (uint8_t)(((rb[0] >> t) & 1u) | (((rb[1] >> t) & 1u) << 1));
+        ++pos;
       }
       running += __shfl_sync(0xffffffffu, incl, 31);
     }
-    if (lane == 0) *s_ntiles = running;
-    tmem_alloc(s_tmem, kTmemCols);
-    tmem_relinquish();
+    if (lane == 0) *s_nent = running;
   }
   tc_fence_before();
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem_base = *s_tmem;
-  const int n_tiles = *s_ntiles;
-  const uint32_t tmem_S = tmem_base;        // columns [0, BLK)
-  const uint32_t tmem_O = tmem_base + BLK;  // columns [BLK, BLK + D)
-  const uint32_t lane_off = (uint32_t)(warp * 32) << 16;
+  const int n_ent = *s_nent;
+  const int n_tiles = (n_ent + C::kEPT - 1) / C::kEPT;
 
-  constexpr uint32_t kIdescQK = make_idesc_bf16(kTileM, BLK, 0, 0);
-  constexpr uint32_t kIdescPV = make_idesc_bf16(kTileM, D, 0, 1);
-  constexpr uint32_t kStageTx = 2u * L::kKVBytes;
+  // which streams work on KV tile n
+  auto stream_mask = [&](int n) -> int { return C::kSplitKV ? (1 << (n & 1)) : (int)sEntF[n]; };
 
-  auto load_kv = [&](int n) {
-    const int s = n % kStages;
-    const int j = sList[n];
-    mbar_expect_tx(bar_full + s, kStageTx);
+  if (warp == 0) {
+    // ================================ TMA producer ========================================
+    if (lane == 0 && n_tiles > 0) {
+      mbar_expect_tx(bar_q, C::kQTiles * C::kQBytes);
 #pragma unroll
-    for (int c = 0; c < D / 64; ++c) {
-      tma_load_4d(sK + s * L::kKVBytes + c * (BLK * 128), &tmK, bar_full + s, c * 64, j * BLK, head, batch);
-      tma_load_4d(sV + s * L::kKVBytes + c * (BLK * 128), &tmV, bar_full + s, c * 64, j * BLK, head, batch);
-    }
-  };
-  auto issue_qk = [&](int n) {
-    const int s = n % kStages;
-    const uint32_t a0 = smem_u32(sQ), b0 = smem_u32(sK + s * L::kKVBytes);
+      for (int t = 0; t < C::kQTiles; ++t)
 #pragma unroll
-    for (int kk = 0; kk < D / 16; ++kk) {
-      const uint64_t da = make_smem_desc(a0 + (kk / 4) * (kTileM * 128) + (kk % 4) * 32, 16, 1024);
-      const uint64_t db = make_smem_desc(b0 + (kk / 4) * (BLK * 128) + (kk % 4) * 32, 16, 1024);
-      mma_ss(tmem_S, da, db, kIdescQK, kk > 0 ? 1u : 0u);
-    }
-    mma_commit(bar_s);
-  };
-  auto issue_pv = [&](int n) {
-    const int s = n % kStages;
-    const uint32_t a0 = smem_u32(sP), b0 = smem_u32(sV + s * L::kKVBytes);
+        for (int c = 0; c < D / 64; ++c)
+          tma_load_4d(sQ + t * C::kQBytes + c * 16384, &tmQ, bar_q, c * 64, (int)q0 + t * 128, head, batch);
+      auto load_tile = [&](unsigned char* dst, const CUtensorMap* tm, uint64_t* bar, int n) {
+        mbar_expect_tx(bar, C::kTileBytes);
 #pragma unroll
-    for (int kk = 0; kk < BLK / 16; ++kk) {
-      const uint64_t da = make_smem_desc(a0 + (kk / 4) * (kTileM * 128) + (kk % 4) * 32, 16, 1024);
-      const uint64_t db = make_smem_desc(b0 + kk * 2048, BLK * 128, 1024);
-      mma_ss(tmem_O, da, db, kIdescPV, (n > 0 || kk > 0) ? 1u : 0u);
+        for (int e = 0; e < C::kEPT; ++e) {
+          const int ent = min(n * C::kEPT + e, n_ent - 1);  // an absent second half re-reads the last entry
+          const int j = sEntJ[ent];
+#pragma unroll
+          for (int c = 0; c < D / 64; ++c)
+            tma_load_4d(dst + c * 16384 + e * (BLK * 128), tm, bar, c * 64, j * BLK, head, batch);
+        }
+      };
+      int kn = 0, vn = 0;
+      const long long t0 = clock64();
+      while ((kn < n_tiles || vn < n_tiles) && !*s_abort) {
+        bool progressed = false;
+        if (kn < n_tiles && mbar_try_wait(k_empty + kn % S, ((kn / S) & 1) ^ 1)) {
+          load_tile(sK + (kn % S) * C::kTileBytes, &tmK, k_full + kn % S, kn);
+          ++kn;
+          progressed = true;
+        }
+        if (vn < n_tiles && mbar_try_wait(v_empty + vn % S, ((vn / S) & 1) ^ 1)) {
+          load_tile(sV + (vn % S) * C::kTileBytes, &tmV, v_full + vn % S, vn);
+          ++vn;
+          progressed = true;
+        }
+        if (!progressed && clock64() - t0 > p.wait_limit * 8) {
+          *s_abort = 1;
+          if (atomicCAS(p.status, 0, SPARSP_ERR_TIMEOUT) == 0) p.status[1] = 10;
+        }
+      }
     }
-    mma_commit(bar_o);
-  };
+  } else if (warp == 1) {
+    // ================================ MMA issuer ==========================================
+    if (lane == 0 && n_tiles > 0) {
+      constexpr uint32_t kIdescQK = make_idesc_bf16(128, 128, 0, 0);
+      constexpr uint32_t kIdescPV = make_idesc_bf16(128, D, 0, 1);
+      int pending[2] = {-1, -1};  // KV tile whose S_s is with the softmax warpgroup
+      int pcnt[2] = {0, 0};       // P tiles consumed per stream
+      bool started[2] = {false, false};
+      int v_users[S];             // P V MMAs still to be issued per V stage
+#pragma unroll
+      for (int s = 0; s < S; ++s) v_users[s] = 0;
 
-  float m_used = -INFINITY;  // running reference max (log2 domain) the row's exponentials use
-  float l_run = 0.0f;
-
-  if (n_tiles > 0) {
-    if (tid == 0) {
-      mbar_expect_tx(bar_q, L::kQBytes);
+      auto flush = [&](int s) {  // issue O_s += P_s V for the stream's pending tile
+        const int m = pending[s];
+        mbar_wait_bounded(p_full + s, pcnt[s] & 1, s_abort, p.status, 20 + s, p.wait_limit);
+        ++pcnt[s];
+        mbar_wait_bounded(v_full + m % S, (m / S) & 1, s_abort, p.status, 22, p.wait_limit);
+        tc_fence_after();
+        const uint32_t b0 = smem_u32(sV + (m % S) * C::kTileBytes);
+        const uint32_t tP = tmem_base + s * 128;
+        const uint32_t tO = tmem_base + 256 + s * D;
 #pragma unroll
-      for (int c = 0; c < D / 64; ++c)
-        tma_load_4d(sQ + c * (kTileM * 128), &tmQ, bar_q, c * 64, (int)q0, head, batch);
-      load_kv(0);
-      mbar_wait_bounded(bar_q, 0, s_abort, p.status, 1, p.wait_limit);
+        for (int kk = 0; kk < 8; ++kk) {
+          const uint64_t db = make_smem_desc(b0 + kk * 2048, 16384, 1024);
+          mma_ts(tO, tP + kk * 8, db, kIdescPV, (started[s] || kk > 0) ? 1u : 0u);
+        }
+        started[s] = true;
+        mma_commit(o_full + s);
+        pending[s] = -1;
+#pragma unroll
+        for (int st = 0; st < S; ++st)
+          if (st == m % S && --v_users[st] == 0) mma_commit(v_empty + st);
+      };
+
+      mbar_wait_bounded(bar_q, 0, s_abort, p.status, 11, p.wait_limit);
+      for (int n = 0; n < n_tiles; ++n) {
+        const int sm = stream_mask(n);
+        // a stream that skipped tile n-1 may still owe the P V of an older tile: issue it first, so
+        // that its V stage is released no later than two steps after it was filled
+#pragma unroll
+        for (int s = 0; s < 2; ++s)
+          if (pending[s] >= 0 && pending[s] < n - 1) flush(s);
+        mbar_wait_bounded(k_full + n % S, (n / S) & 1, s_abort, p.status, 12, p.wait_limit);
+        tc_fence_after();
+#pragma unroll
+        for (int st = 0; st < S; ++st)
+          if (st == n % S) v_users[st] = (sm & 1) + ((sm >> 1) & 1);
+#pragma unroll
+        for (int s = 0; s < 2; ++s) {
+          if (!((sm >> s) & 1)) continue;
+          if (pending[s] >= 0) flush(s);  // tile n-1: frees S_s for the next Q K^T
+          const uint32_t a0 = smem_u32(sQ + (C::kSplitKV ? 0 : s) * C::kQBytes);
+          const uint32_t b0 = smem_u32(sK + (n % S) * C::kTileBytes);
+#pragma unroll
+          for (int kk = 0; kk < D / 16; ++kk) {
+            const uint64_t da = make_smem_desc(a0 + (kk / 4) * 16384 + (kk % 4) * 32, 16, 1024);
+            const uint64_t db = make_smem_desc(b0 + (kk / 4) * 16384 + (kk % 4) * 32, 16, 1024);
+            mma_ss(tmem_base + s * 128, da, db, kIdescQK, kk > 0 ? 1u : 0u);
+          }
+          mma_commit(s_full + s);
+          pending[s] = n;
+        }
+        mma_commit(k_empty + n % S);
+      }
+#pragma unroll
+      for (int s = 0; s < 2; ++s)
+        if (pending[s] >= 0) flush(s);
     }
+  } else if (warp >= 4) {
+    // ================================ softmax warpgroups ==================================
+    const int wg = (warp - 4) >> 2;  // stream
+    const int rgrp = warp & 3;       // tensor-memory lane group this warp may access
+    const int row = rgrp * 32 + lane;
+    const int rh = row >> 6;         // which query block of a stacked Q tile the row belongs to
+    const uint32_t lane_off = (uint32_t)(rgrp * 32) << 16;
+    const uint32_t tS = tmem_base + wg * 128 + lane_off;
+    const uint32_t tO = tmem_base + 256 + wg * D + lane_off;
+    float m_used = -INFINITY;  // reference maximum (log2 domain) of the row's exponentials
+    float l_run = 0.0f;
+    int cnt = 0;
 
     for (int n = 0; n < n_tiles; ++n) {
-      const int s = n % kStages;
-      if (tid == 0) {
-        mbar_wait_bounded(bar_full + s, (n / kStages) & 1, s_abort, p.status, 2, p.wait_limit);
-        tc_fence_after();
-        issue_qk(n);
-        if (n > 0) mbar_wait_bounded(bar_o, (n - 1) & 1, s_abort, p.status, 3, p.wait_limit);
-        if (n + 1 < n_tiles) load_kv(n + 1);  // stage (n+1)%2 was last read by P V of tile n-1
-      }
-      __syncwarp();
-      mbar_wait_bounded(bar_s, n & 1, s_abort, p.status, 4, p.wait_limit);
-      tc_fence_after();
-
-      float sv[BLK];
+      if (!((stream_mask(n) >> wg) & 1)) continue;
+      // valid / kept columns of each 32-column chunk (warp-uniform)
+      int valid[4];
+      if (C::kSplitKV) {
 #pragma unroll
-      for (int c = 0; c < BLK / 32; ++c)
-        tmem_ld32(tmem_S + lane_off + c * 32, reinterpret_cast<uint32_t*>(sv) + c * 32);
-      tmem_ld_wait();
+        for (int ch = 0; ch < 2; ++ch) {
+          const int ent = n * 2 + ch;
+          int nv = 0;
+          if (ent < n_ent && ((sEntF[ent] >> rh) & 1))
+            nv = (int)min((int64_t)64, p.N - (int64_t)sEntJ[ent] * 64);
+          valid[2 * ch] = min(nv, 32);
+          valid[2 * ch + 1] = max(nv - 32, 0);
+        }
+      } else {
+        const int nv = (int)min((int64_t)128, p.N - (int64_t)sEntJ[n] * 128);
+#pragma unroll
+        for (int c = 0; c < 4; ++c) valid[c] = max(0, min(32, nv - 32 * c));
+      }
 
-      const int j = sList[n];
-      const bool kept = (sFlags[n] >> my_qb) & 1;  // warp-uniform (BLK >= 64 rows per half)
-      const int ncols = (int)min((int64_t)BLK, p.N - (int64_t)j * BLK);
+      mbar_wait_bounded(s_full + wg, cnt & 1, s_abort, p.status, 30 + wg, p.wait_limit);
+      tc_fence_after();
+      // pass 1: row maximum over the kept, valid columns (two 64-column halves)
       float mx = -INFINITY;
 #pragma unroll
-      for (int c = 0; c < BLK; ++c) mx = fmaxf(mx, c < ncols ? sv[c] : -INFINITY);
+      for (int h = 0; h < 2; ++h) {
+        float sv[64];
+        tmem_ld32(tS + h * 64, reinterpret_cast<uint32_t*>(sv));
+        tmem_ld32(tS + h * 64 + 32, reinterpret_cast<uint32_t*>(sv) + 32);
+        tmem_ld_wait();
+#pragma unroll
+        for (int cc = 0; cc < 2; ++cc) {
+          const int vc = valid[2 * h + cc];
+          if (vc == 32) {
+#pragma unroll
+            for (int e = 0; e < 32; e += 2) mx = fmaxf(mx, fmaxf(sv[cc * 32 + e], sv[cc * 32 + e + 1]));
+          } else if (vc > 0) {
+#pragma unroll
+            for (int e = 0; e < 32; ++e) mx = fmaxf(mx, e < vc ? sv[cc * 32 + e] : -INFINITY);
+          }
+        }
+      }
       mx *= p.scale_log2;
       const float m_new = fmaxf(m_used, mx);
-      const bool grow = kept && (m_new > m_used + 8.0f || m_used == -INFINITY);
-      const bool any_grow = __any_sync(0xffffffffu, grow);
-
-      // P V of the previous tile must be done before P is overwritten or O is rescaled
-      if (n > 0) mbar_wait_bounded(bar_o, (n - 1) & 1, s_abort, p.status, 5, p.wait_limit);
-      tc_fence_after();
-      if (any_grow) {
+      const bool grow = m_new > m_used + kGrowThreshold || (m_used == -INFINITY && m_new > -INFINITY);
+      if (__any_sync(0xffffffffu, grow)) {
         const float alpha = grow ? ex2(m_used - m_new) : 1.0f;  // m_used = -inf -> 0
-        if (n > 0) {
+        if (cnt > 0) {  // S_s of this tile is complete, hence so is every earlier P V of the stream
 #pragma unroll
           for (int c = 0; c < D / 32; ++c) {
             uint32_t o[32];
-            tmem_ld32(tmem_O + lane_off + c * 32, o);
+            tmem_ld32(tO + c * 32, o);
             tmem_ld_wait();
 #pragma unroll
             for (int e = 0; e < 32; ++e) o[e] = __float_as_uint(__uint_as_float(o[e]) * alpha);
-            tmem_st32(tmem_O + lane_off + c * 32, o);
+            tmem_st32(tO + c * 32, o);
           }
-          tmem_st_wait();
         }
         l_run *= alpha;
         if (grow) m_used = m_new;
       }
 
+      // pass 2: exponentials chunk by chunk; bf16 P overwrites S in place (P chunk c occupies
+      // columns [16c, 16c+16), which lie inside the S columns already consumed)
       float lsum = 0.0f;
-      const int row = tid;
+      const float neg_m = -m_used;
+      float buf[2][32];
+      tmem_ld32(tS, reinterpret_cast<uint32_t*>(buf[0]));
 #pragma unroll
-      for (int c8 = 0; c8 < BLK / 8; ++c8) {
-        uint32_t packed[4];
+      for (int c = 0; c < 4; ++c) {
+        tmem_ld_wait();
+        if (c < 3) tmem_ld32(tS + (c + 1) * 32, reinterpret_cast<uint32_t*>(buf[(c + 1) & 1]));
+        const float* sv = buf[c & 1];
+        uint32_t pk[16];
+        if (valid[c] == 32) {
 #pragma unroll
-        for (int e = 0; e < 4; ++e) {
-          const int c = c8 * 8 + 2 * e;
-          float p0 = 0.0f, p1 = 0.0f;
-          if (kept) {
-            if (c < ncols) p0 = ex2(fmaf(sv[c], p.scale_log2, -m_used));
-            if (c + 1 < ncols) p1 = ex2(fmaf(sv[c + 1], p.scale_log2, -m_used));
+          for (int e = 0; e < 16; ++e) {
+            const float p0 = ex2(fmaf(sv[2 * e], p.scale_log2, neg_m));
+            const float p1 = ex2(fmaf(sv[2 * e + 1], p.scale_log2, neg_m));
+            lsum += p0 + p1;
+            const __nv_bfloat162 h2 = __floats2bfloat162_rn(p0, p1);
+            pk[e] = *reinterpret_cast<const uint32_t*>(&h2);
           }
-          lsum += p0 + p1;
-          const __nv_bfloat162 h2 = __floats2bfloat162_rn(p0, p1);
-          packed[e] = *reinterpret_cast<const uint32_t*>(&h2);
+        } else if (valid[c] > 0) {
+#pragma unroll
+          for (int e = 0; e < 16; ++e) {
+            const float p0 = 2 * e < valid[c] ? ex2(fmaf(sv[2 * e], p.scale_log2, neg_m)) : 0.0f;
+            const float p1 = 2 * e + 1 < valid[c] ? ex2(fmaf(sv[2 * e + 1], p.scale_log2, neg_m)) : 0.0f;
+            lsum += p0 + p1;
+            const __nv_bfloat162 h2 = __floats2bfloat162_rn(p0, p1);
+            pk[e] = *reinterpret_cast<const uint32_t*>(&h2);
+          }
+        } else {
+#pragma unroll
+          for (int e = 0; e < 16; ++e) pk[e] = 0u;
         }
-        // K-major operand, 128-byte swizzle: 16-byte chunk cc of row r sits at chunk (cc ^ (r & 7))
-        const int sub = c8 / 8, cc = c8 % 8;
-        unsigned char* dst = sP + sub * (kTileM * 128) + row * 128 + ((cc ^ (row & 7)) * 16);
-        *reinterpret_cast<uint4*>(dst) = make_uint4(packed[0], packed[1], packed[2], packed[3]);
+        tmem_st16(tS + c * 16, pk);
       }
       l_run += lsum;
-
-      fence_proxy_async_smem();
+      tmem_st_wait();
       tc_fence_before();
-      __syncthreads();
-      if (tid == 0) {
-        tc_fence_after();
-        issue_pv(n);
-      }
+      mbar_arrive(p_full + wg);
+      ++cnt;
     }
-    mbar_wait_bounded(bar_o, (n_tiles - 1) & 1, s_abort, p.status, 6, p.wait_limit);
-    tc_fence_after();
-  }
 
-  // ---- epilogue ---------------------------------------------------------------------------
-  const int64_t tok = q0 + tid;
-  const float inv_l = l_run > 0.0f ? 1.0f / l_run : 0.0f;
-  __nv_bfloat16* orow = p.O + (int64_t)batch * p.sB + (int64_t)head * p.sH + tok * p.sT;
-#pragma unroll
-  for (int c = 0; c < D / 32; ++c) {
-    uint32_t o[32];
-    if (n_tiles > 0) {
-      tmem_ld32(tmem_O + lane_off + c * 32, o);
-      tmem_ld_wait();
-    } else {
-#pragma unroll
-      for (int e = 0; e < 32; ++e) o[e] = 0u;
+    // ---- epilogue -------------------------------------------------------------------------
+    if (cnt > 0) {
+      mbar_wait_bounded(o_full + wg, (cnt - 1) & 1, s_abort, p.status, 40 + wg, p.wait_limit);
+      tc_fence_after();
     }
-    if (tok < p.N) {
+    if (!C::kSplitKV) {
+      const int64_t tok = q0 + wg * 128 + row;
+      const float inv_l = l_run > 0.0f ? 1.0f / l_run : 0.0f;
+      __nv_bfloat16* orow = p.O + (int64_t)batch * p.sB + (int64_t)head * p.sH + tok * p.sT;
 #pragma unroll
-      for (int v = 0; v < 4; ++v) {
-        uint32_t w[4];
+      for (int c = 0; c < D / 32; ++c) {
+        uint32_t o[32];
+        if (cnt > 0) {  // warp-uniform: tensor-memory loads are warp-collective
+          tmem_ld32(tO + c * 32, o);
+          tmem_ld_wait();
+        } else {
 #pragma unroll
-        for (int e = 0; e < 4; ++e) {
-          const __nv_bfloat162 h2 = __floats2bfloat162_rn(__uint_as_float(o[v * 8 + 2 * e]) * inv_l,
-                                                          __uint_as_float(o[v * 8 + 2 * e + 1]) * inv_l);
-          w[e] = *reinterpret_cast<const uint32_t*>(&h2);
+          for (int e = 0; e < 32; ++e) o[e] = 0u;
         }
-        *reinterpret_cast<uint4*>(orow + c * 32 + v * 8) = make_uint4(w[0], w[1], w[2], w[3]);
+        if (tok < p.N) {
+#pragma unroll
+          for (int v = 0; v < 4; ++v) {
+            uint32_t w[4];
+#pragma unroll
+            for (int e = 0; e < 4; ++e) {
+              const __nv_bfloat162 h2 = __floats2bfloat162_rn(__uint_as_float(o[v * 8 + 2 * e]) * inv_l,
+                                                              __uint_as_float(o[v * 8 + 2 * e + 1]) * inv_l);
+              w[e] = *reinterpret_cast<const uint32_t*>(&h2);
+            }
+            *reinterpret_cast<uint4*>(orow + c * 32 + v * 8) = make_uint4(w[0], w[1], w[2], w[3]);
+          }
+        }
       }
+      if (p.lse && tok < p.N)
+        p.lse[(int64_t)bh * p.N + tok] = l_run > 0.0f ? (m_used + log2f(l_run)) * 0.6931471805599453f : -INFINITY;
+    } else {
+      // merge the two streams' partial results: stream s finalises columns [s*D/2, (s+1)*D/2)
+      constexpr int HALF = D / 2;
+      float* mbuf = reinterpret_cast<float*>(sK);  // K/V rings are idle once both streams are done
+      sStat[wg * 128 + row] = make_float2(m_used, l_run);
+      named_bar_sync(1, 256);
+      const float2 other = sStat[(1 - wg) * 128 + row];
+      const float m = fmaxf(m_used, other.x);
+      const float a_me = m_used > -INFINITY ? ex2(m_used - m) : 0.0f;
+      const float a_ot = other.x > -INFINITY ? ex2(other.x - m) : 0.0f;
+      const float l = l_run * a_me + other.y * a_ot;
+      const float inv_l = l > 0.0f ? 1.0f / l : 0.0f;
+      // hand the partner its half of my accumulator, scaled to the common reference
+      float* give = mbuf + ((size_t)wg * 128 + row) * C::kMergeStride;
+#pragma unroll
+      for (int c = 0; c < HALF / 32; ++c) {
+        uint32_t o[32];
+        if (cnt > 0) {
+          tmem_ld32(tO + (1 - wg) * HALF + c * 32, o);
+          tmem_ld_wait();
+        } else {
+#pragma unroll
+          for (int e = 0; e < 32; ++e) o[e] = 0u;
+        }
+#pragma unroll
+        for (int v = 0; v < 8; ++v)
+          *reinterpret_cast<float4*>(give + c * 32 + v * 4) =
+              make_float4(__uint_as_float(o[v * 4]) * a_me, __uint_as_float(o[v * 4 + 1]) * a_me,
+                          __uint_as_float(o[v * 4 + 2]) * a_me, __uint_as_float(o[v * 4 + 3]) * a_me);
+      }
+      named_bar_sync(1, 256);
+      const int64_t tok = q0 + row;
+      const float* take = mbuf + ((size_t)(1 - wg) * 128 + row) * C::kMergeStride;
+      __nv_bfloat16* orow = p.O + (int64_t)batch * p.sB + (int64_t)head * p.sH + tok * p.sT + wg * HALF;
+#pragma unroll
+      for (int c = 0; c < HALF / 32; ++c) {
+        uint32_t o[32];
+        if (cnt > 0) {
+          tmem_ld32(tO + wg * HALF + c * 32, o);
+          tmem_ld_wait();
+        } else {
+#pragma unroll
+          for (int e = 0; e < 32; ++e) o[e] = 0u;
+        }
+        if (tok < p.N) {
+#pragma unroll
+          for (int v = 0; v < 4; ++v) {
+            const float4 t0 = *reinterpret_cast<const float4*>(take + c * 32 + v * 8);
+            const float4 t1 = *reinterpret_cast<const float4*>(take + c * 32 + v * 8 + 4);
+            const float tt[8] = {t0.x, t0.y, t0.z, t0.w, t1.x, t1.y, t1.z, t1.w};
+            uint32_t w[4];
+#pragma unroll
+            for (int e = 0; e < 4; ++e) {
+              const float x0 = (__uint_as_float(o[v * 8 + 2 * e]) * a_me + tt[2 * e]) * inv_l;
+              const float x1 = (__uint_as_float(o[v * 8 + 2 * e + 1]) * a_me + tt[2 * e + 1]) * inv_l;
+              const __nv_bfloat162 h2 = __floats2bfloat162_rn(x0, x1);
+              w[e] = *reinterpret_cast<const uint32_t*>(&h2);
+            }
+            *reinterpret_cast<uint4*>(orow + c * 32 + v * 8) = make_uint4(w[0], w[1], w[2], w[3]);
+          }
+        }
+      }
+      if (p.lse && wg == 0 && tok < p.N)
+        p.lse[(int64_t)bh * p.N + tok] = l > 0.0f ? (m + log2f(l)) * 0.6931471805599453f : -INFINITY;
     }
   }
-  if (p.lse && tok < p.N)
-    p.lse[(int64_t)bh * p.N + tok] = l_run > 0.0f ? (m_used + log2f(l_run)) * 0.6931471805599453f : -INFINITY;
 
   tc_fence_before();
   __syncthreads();
-  if (warp == 0) tmem_dealloc(tmem_base, kTmemCols);
+  if (warp == 1) tmem_dealloc(tmem_base, kTmemCols);
 }
 
 // ------------------------------------------------------------------------------------------------
@@ -365,13 +545,13 @@ static int launch_attn_t(const sparsp_shape& s, const Geometry& g, const void* Q
                          const AttnParams& p, cudaStream_t st) {
   CUtensorMap tq, tk, tv;
   int rc;
-  if ((rc = make_tmap(&tq, Q, s, g, kTileM)) != SPARSP_OK) return rc;
+  if ((rc = make_tmap(&tq, Q, s, g, 128)) != SPARSP_OK) return rc;
   if ((rc = make_tmap(&tk, K, s, g, BLK)) != SPARSP_OK) return rc;
   if ((rc = make_tmap(&tv, V, s, g, BLK)) != SPARSP_OK) return rc;
   auto kern = attn_fwd_kernel<D, BLK>;
-  const int smem = AttnSmem<D, BLK>::kDynamic;
+  const int smem = AttnCfg<D, BLK>::kDynamic;
   SPARSP_CUDA_OK(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
-  dim3 grid((unsigned)((g.N + kTileM - 1) / kTileM), (unsigned)(g.B * g.H));
+  dim3 grid((unsigned)((g.NB + 1) / 2), (unsigned)(g.B * g.H));
   kern<<<grid, kAttnThreads, smem, st>>>(tq, tk, tv, p);
   count_launch();
   SPARSP_CUDA_OK(cudaGetLastError());
@@ -395,7 +575,7 @@ int launch_attn(const sparsp_shape& s, const Geometry& g, const void* Q, const v
   p.Wd = g.Wd;
   const float sc = scale > 0.0f ? scale : 1.0f / sqrtf((float)g.d);
   p.scale_log2 = sc * 1.4426950408889634f;
-  p.wait_limit = 2000000000LL;  // ~1 s of SM clocks
+  p.wait_limit = 200000000LL;  // about 0.1 s of SM clocks
   if (g.d == 64 && g.b == 64) return launch_attn_t<64, 64>(s, g, Q, K, V, p, st);
   if (g.d == 64 && g.b == 128) return launch_attn_t<64, 128>(s, g, Q, K, V, p, st);
   if (g.d == 128 && g.b == 64) return launch_attn_t<128, 64>(s, g, Q, K, V, p, st);
