@@ -9,9 +9,12 @@
 //                a KV tile is two entries of the union list (128 keys, full-rate N = 128); each
 //                64x64 quadrant the mask does not keep is zeroed in P.  Stream s takes the KV tiles
 //                of parity s into its own accumulator; the two partial results are merged at the end.
-// Warp roles (384 threads): warp 0 = TMA producer (K ring and V ring, polled independently),
-// warp 1 = MMA issuer (one thread), warps 2-3 idle, warps 4-7 / 8-11 = softmax warpgroups of stream
-// 0 / 1, one query row per thread; the first warpgroup gives registers up to the softmax ones.  Tensor memory: S_s (128 fp32 columns, overwritten in place by bf16 P_s, which
+// Warp roles (608 threads): warp 0 = TMA producer (K ring and V ring, polled independently),
+// warps 1 and 18 = MMA issuers of stream 0 / 1 (one thread each, so the streams never serialise on
+// one instruction stream), warps 2-9 / 10-17 = softmax warps of stream 0 / 1.  A query row
+// is shared by TWO threads of different warps, each owning 64 of the tile's 128 key columns: a row
+// of S is read from tensor memory once, in 64 registers, and the pair exchanges its two partial row
+// maxima through shared memory behind a 64-thread named barrier.  Tensor memory: S_s (128 fp32 columns, overwritten in place by bf16 P_s, which
 // the P.V MMA reads straight from tensor memory) and O_s (d fp32 columns) per stream.
 // Online softmax is base-2 in fp32; O is rescaled lazily, only when a row's maximum has grown by
 // more than 2^8 since the reference last moved.
@@ -36,7 +39,8 @@ struct AttnParams {
   long long wait_limit;
 };
 
-constexpr int kAttnThreads = 384;
+constexpr int kAttnThreads = 608;
+constexpr int kIssuer1Warp = 18;  // warp 1 issues the MMAs of stream 0, warp 18 those of stream 1
 constexpr int kTmemCols = 512;
 constexpr float kGrowThreshold = 8.0f;
 
@@ -53,23 +57,36 @@ struct AttnCfg {
   static constexpr int kOffV = kOffK + kStages * kTileBytes;
   static constexpr int kOffEntJ = kOffV + kStages * kTileBytes;  // uint16 [1024] union list
   static constexpr int kOffEntF = kOffEntJ + 2 * kMaxBlocks;     // uint8 [1024] bit q: kept by query block q
-  static constexpr int kOffStat = kOffEntF + kMaxBlocks;         // float2 [2][128] stream statistics
-  static constexpr int kOffBars = kOffStat + 2 * 128 * 8;
+  static constexpr int kOffStat = kOffEntF + kMaxBlocks;         // float2 [2 streams][2 halves][128]
+  static constexpr int kOffMax = kOffStat + 2 * 2 * 128 * 8;     // float [2 parities][2][2][128]
+  static constexpr int kOffBars = kOffMax + 2 * 2 * 2 * 128 * 4;
   static constexpr int kNumBars = 1 + 4 * kStages + 6;
   static constexpr int kOffMisc = kOffBars + 8 * kNumBars;
   static constexpr int kTotal = kOffMisc + 32;
   static constexpr int kDynamic = kTotal + 1024;  // slack for the 1024-byte alignment of the base
-  static constexpr int kMergeStride = D / 2 + 4;  // floats per row of the merge buffer
-  static_assert(2 * 128 * kMergeStride * 4 <= 2 * kStages * kTileBytes, "merge buffer must fit the K/V rings");
+  static constexpr int kMergeStride = D / 4 + 4;  // floats per row of the merge buffer
+  static_assert(4 * 128 * kMergeStride * 4 <= 2 * kStages * kTileBytes, "merge buffer must fit the K/V rings");
   static_assert(kDynamic <= 232448, "shared memory budget");
 };
+
+#ifdef SPARSP_ATTN_PROFILE
+// Optional cycle accounting for tuning builds: per-phase SM-clock totals of one softmax lane and of
+// the MMA thread of every CTA.  Off in normal builds.
+__device__ unsigned long long g_attn_prof[16];
+#define PROF_T(var) const long long var = clock64()
+#define PROF_ADD(slot, a, b) \
+  if (lane == 0 && (warp == 2 || warp == 1)) atomicAdd(&g_attn_prof[slot], (unsigned long long)((b) - (a)))
+#else
+#define PROF_T(var)
+#define PROF_ADD(slot, a, b)
+#endif
 
 __device__ __forceinline__ void named_bar_sync(int id, int n) {
   asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(n) : "memory");
 }
 
 template <int D, int BLK>
-__global__ void __launch_bounds__(kAttnThreads, 1)
+__global__ void __maxnreg__(96)
     attn_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmK,
                     const __grid_constant__ CUtensorMap tmV, const AttnParams p) {
   using C = AttnCfg<D, BLK>;
@@ -83,6 +100,7 @@ __global__ void __launch_bounds__(kAttnThreads, 1)
   uint16_t* sEntJ = reinterpret_cast<uint16_t*>(smem + C::kOffEntJ);
   uint8_t* sEntF = smem + C::kOffEntF;
   float2* sStat = reinterpret_cast<float2*>(smem + C::kOffStat);
+  float* sMax = reinterpret_cast<float*>(smem + C::kOffMax);
   uint64_t* bars = reinterpret_cast<uint64_t*>(smem + C::kOffBars);
   uint64_t* bar_q = bars;
   uint64_t* k_full = bars + 1;
@@ -90,13 +108,14 @@ __global__ void __launch_bounds__(kAttnThreads, 1)
   uint64_t* v_full = k_empty + S;
   uint64_t* v_empty = v_full + S;
   uint64_t* s_full = v_empty + S;  // [2] S_s written by Q K^T
-  uint64_t* p_full = s_full + 2;   // [2] P_s written by the softmax warpgroup (128 arrivals)
+  uint64_t* p_full = s_full + 2;   // [2] P_s written by the stream's 8 softmax warps (one arrival each)
   uint64_t* o_full = p_full + 2;   // [2] a P V of stream s has completed
   uint32_t* s_tmem = reinterpret_cast<uint32_t*>(smem + C::kOffMisc);
   int* s_nent = reinterpret_cast<int*>(smem + C::kOffMisc + 4);
   volatile int* s_abort = reinterpret_cast<volatile int*>(smem + C::kOffMisc + 8);
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  PROF_T(t_cta0);
   const int bh = blockIdx.y;
   const int batch = bh / p.H, head = bh % p.H;
   const int i0 = blockIdx.x * 2;  // first of the CTA's two query blocks
@@ -110,13 +129,13 @@ __global__ void __launch_bounds__(kAttnThreads, 1)
     mbar_init(bar_q, 1);
     for (int s = 0; s < S; ++s) {
       mbar_init(k_full + s, 1);
-      mbar_init(k_empty + s, 1);
+      mbar_init(k_empty + s, 2);
       mbar_init(v_full + s, 1);
-      mbar_init(v_empty + s, 1);
+      mbar_init(v_empty + s, 2);
     }
     for (int s = 0; s < 2; ++s) {
       mbar_init(s_full + s, 1);
-      mbar_init(p_full + s, 128);
+      mbar_init(p_full + s, 8);
       mbar_init(o_full + s, 1);
     }
     mbar_init_fence();
@@ -175,6 +194,12 @@ __global__ void __launch_bounds__(kAttnThreads, 1)
         for (int c = 0; c < D / 64; ++c)
           tma_load_4d(sQ + t * C::kQBytes + c * 16384, &tmQ, bar_q, c * 64, (int)q0 + t * 128, head, batch);
       auto load_tile = [&](unsigned char* dst, const CUtensorMap* tm, uint64_t* bar, int n) {
+#ifdef SPARSP_ATTN_NOLOAD  // tuning builds only: reuse stale tiles to take TMA traffic out of the picture
+        if (n >= S) {
+          mbar_arrive(bar);
+          return;
+        }
+#endif
         mbar_expect_tx(bar, C::kTileBytes);
 #pragma unroll
         for (int e = 0; e < C::kEPT; ++e) {
@@ -189,12 +214,12 @@ __global__ void __launch_bounds__(kAttnThreads, 1)
       const long long t0 = clock64();
       while ((kn < n_tiles || vn < n_tiles) && !*s_abort) {
         bool progressed = false;
-        if (kn < n_tiles && mbar_try_wait(k_empty + kn % S, ((kn / S) & 1) ^ 1)) {
+        if (kn < n_tiles && mbar_test_wait(k_empty + kn % S, ((kn / S) & 1) ^ 1)) {
           load_tile(sK + (kn % S) * C::kTileBytes, &tmK, k_full + kn % S, kn);
           ++kn;
           progressed = true;
         }
-        if (vn < n_tiles && mbar_try_wait(v_empty + vn % S, ((vn / S) & 1) ^ 1)) {
+        if (vn < n_tiles && mbar_test_wait(v_empty + vn % S, ((vn / S) & 1) ^ 1)) {
           load_tile(sV + (vn % S) * C::kTileBytes, &tmV, v_full + vn % S, vn);
           ++vn;
           progressed = true;
@@ -205,166 +230,180 @@ __global__ void __launch_bounds__(kAttnThreads, 1)
         }
       }
     }
-  } else if (warp == 1) {
-    // ================================ MMA issuer ==========================================
+  } else if (warp == 1 || warp == kIssuer1Warp) {
+    // ================================ MMA issuers (one thread per stream) =================
+    // Each issuer walks ALL KV tiles in order and, for every tile, first observes the tile's "full"
+    // barrier and then arrives once on its "empty" barrier (count 2: one arrival per issuer) --
+    // through tcgen05.commit after its MMAs if its stream uses the tile, directly otherwise.  The
+    // two streams therefore never wait on each other's softmax, only on the shared K/V rings.
     if (lane == 0 && n_tiles > 0) {
+      const int s = (warp == 1) ? 0 : 1;
       constexpr uint32_t kIdescQK = make_idesc_bf16(128, 128, 0, 0);
       constexpr uint32_t kIdescPV = make_idesc_bf16(128, D, 0, 1);
-      int pending[2] = {-1, -1};  // KV tile whose S_s is with the softmax warpgroup
-      int pcnt[2] = {0, 0};       // P tiles consumed per stream
-      bool started[2] = {false, false};
-      int v_users[S];             // P V MMAs still to be issued per V stage
-#pragma unroll
-      for (int s = 0; s < S; ++s) v_users[s] = 0;
+      const uint32_t tSs = tmem_base + s * 128;
+      const uint32_t tOs = tmem_base + 256 + s * D;
+      const uint64_t descQ = make_smem_desc(smem_u32(sQ + (C::kSplitKV ? 0 : s) * C::kQBytes), 16, 1024);
+      const uint64_t descK = make_smem_desc(smem_u32(sK), 16, 1024);
+      const uint64_t descV = make_smem_desc(smem_u32(sV), 16384, 1024);
+      int vdone = 0;       // tiles whose V obligation (P V or plain release) has been handled
+      int last_kept = -1;  // last tile whose Q K^T this stream has issued
+      int pcnt = 0;        // P tiles consumed
+      uint32_t started = 0;
 
-      auto flush = [&](int s) {  // issue O_s += P_s V for the stream's pending tile
-        const int m = pending[s];
-        mbar_wait_bounded(p_full + s, pcnt[s] & 1, s_abort, p.status, 20 + s, p.wait_limit);
-        ++pcnt[s];
-        mbar_wait_bounded(v_full + m % S, (m / S) & 1, s_abort, p.status, 22, p.wait_limit);
-        tc_fence_after();
-        const uint32_t b0 = smem_u32(sV + (m % S) * C::kTileBytes);
-        const uint32_t tP = tmem_base + s * 128;
-        const uint32_t tO = tmem_base + 256 + s * D;
-#pragma unroll
-        for (int kk = 0; kk < 8; ++kk) {
-          const uint64_t db = make_smem_desc(b0 + kk * 2048, 16384, 1024);
-          mma_ts(tO, tP + kk * 8, db, kIdescPV, (started[s] || kk > 0) ? 1u : 0u);
+      auto handle_v = [&](int m) {
+        const bool keep = (stream_mask(m) >> s) & 1;
+        if (keep) {
+          PROF_T(t_p0);
+          mbar_wait_bounded(p_full + s, pcnt & 1, s_abort, p.status, 20 + s, p.wait_limit);
+          ++pcnt;
+          PROF_T(t_p1);
+          PROF_ADD(8, t_p0, t_p1);  // issuer waiting for P
         }
-        started[s] = true;
-        mma_commit(o_full + s);
-        pending[s] = -1;
+        PROF_T(t_v0);
+        mbar_wait_bounded(v_full + m % S, (m / S) & 1, s_abort, p.status, 22, p.wait_limit);
+        PROF_T(t_v1);
+        PROF_ADD(10, t_v0, t_v1);  // issuer waiting for V
+        if (keep) {
+          tc_fence_after();
+          const uint64_t db0 = descV + (uint64_t)(((m % S) * C::kTileBytes) >> 4);
 #pragma unroll
-        for (int st = 0; st < S; ++st)
-          if (st == m % S && --v_users[st] == 0) mma_commit(v_empty + st);
+          for (int kk = 0; kk < 8; ++kk)
+            mma_ts(tOs, tSs + kk * 8, db0 + (uint64_t)((kk * 2048) >> 4), kIdescPV, (kk > 0) ? 1u : started);
+          started = 1u;
+          mma_commit(o_full + s);
+          mma_commit(v_empty + m % S);
+          PROF_T(t_v2);
+          PROF_ADD(6, t_v1, t_v2);  // issuer issuing P V
+        } else {
+          mbar_arrive(v_empty + m % S);
+        }
       };
 
       mbar_wait_bounded(bar_q, 0, s_abort, p.status, 11, p.wait_limit);
       for (int n = 0; n < n_tiles; ++n) {
-        const int sm = stream_mask(n);
-        // a stream that skipped tile n-1 may still owe the P V of an older tile: issue it first, so
-        // that its V stage is released no later than two steps after it was filled
-#pragma unroll
-        for (int s = 0; s < 2; ++s)
-          if (pending[s] >= 0 && pending[s] < n - 1) flush(s);
+        const bool keep = (stream_mask(n) >> s) & 1;
+        while (vdone < n - 1) handle_v(vdone++);  // a V stage is released at most two steps after its fill
+        PROF_T(t_k0);
         mbar_wait_bounded(k_full + n % S, (n / S) & 1, s_abort, p.status, 12, p.wait_limit);
-        tc_fence_after();
-#pragma unroll
-        for (int st = 0; st < S; ++st)
-          if (st == n % S) v_users[st] = (sm & 1) + ((sm >> 1) & 1);
-#pragma unroll
-        for (int s = 0; s < 2; ++s) {
-          if (!((sm >> s) & 1)) continue;
-          if (pending[s] >= 0) flush(s);  // tile n-1: frees S_s for the next Q K^T
-          const uint32_t a0 = smem_u32(sQ + (C::kSplitKV ? 0 : s) * C::kQBytes);
-          const uint32_t b0 = smem_u32(sK + (n % S) * C::kTileBytes);
+        PROF_T(t_k1);
+        PROF_ADD(9, t_k0, t_k1);  // issuer waiting for K
+        if (keep) {
+          while (vdone <= last_kept) handle_v(vdone++);  // P V of the previous kept tile frees S_s
+          tc_fence_after();
+          const uint64_t db0 = descK + (uint64_t)(((n % S) * C::kTileBytes) >> 4);
 #pragma unroll
           for (int kk = 0; kk < D / 16; ++kk) {
-            const uint64_t da = make_smem_desc(a0 + (kk / 4) * 16384 + (kk % 4) * 32, 16, 1024);
-            const uint64_t db = make_smem_desc(b0 + (kk / 4) * 16384 + (kk % 4) * 32, 16, 1024);
-            mma_ss(tmem_base + s * 128, da, db, kIdescQK, kk > 0 ? 1u : 0u);
+            const uint64_t off = (uint64_t)(((kk / 4) * 16384 + (kk % 4) * 32) >> 4);
+            mma_ss(tSs, descQ + off, db0 + off, kIdescQK, kk > 0 ? 1u : 0u);
           }
           mma_commit(s_full + s);
-          pending[s] = n;
+          mma_commit(k_empty + n % S);
+          last_kept = n;
+          PROF_T(t_k2);
+          PROF_ADD(7, t_k1, t_k2);  // issuer issuing Q K^T
+        } else {
+          mbar_arrive(k_empty + n % S);
         }
-        mma_commit(k_empty + n % S);
       }
-#pragma unroll
-      for (int s = 0; s < 2; ++s)
-        if (pending[s] >= 0) flush(s);
+      while (vdone < n_tiles) handle_v(vdone++);
     }
-  } else if (warp >= 4) {
-    // ================================ softmax warpgroups ==================================
-    const int wg = (warp - 4) >> 2;  // stream
-    const int rgrp = warp & 3;       // tensor-memory lane group this warp may access
+  } else if (warp >= 2 && warp < 18) {
+    // ================================ softmax warps =======================================
+    const int sidx = (warp - 2) >> 3;       // stream
+    const int half = ((warp - 2) >> 2) & 1;  // which 64 key columns of a tile this thread owns
+    const int rgrp = warp & 3;               // tensor-memory lane group this warp may access
     const int row = rgrp * 32 + lane;
-    const int rh = row >> 6;         // which query block of a stacked Q tile the row belongs to
+    const int rh = row >> 6;                 // which query block of a stacked Q tile the row belongs to
+    const int pair_bar = 1 + sidx * 4 + rgrp;  // named barrier shared with the row's other thread
     const uint32_t lane_off = (uint32_t)(rgrp * 32) << 16;
-    const uint32_t tS = tmem_base + wg * 128 + lane_off;
-    const uint32_t tO = tmem_base + 256 + wg * D + lane_off;
+    const uint32_t tS = tmem_base + sidx * 128 + lane_off;
+    const uint32_t tO = tmem_base + 256 + sidx * D + lane_off;
     float m_used = -INFINITY;  // reference maximum (log2 domain) of the row's exponentials
-    float l_run = 0.0f;
+    float l_run = 0.0f;        // this thread's share of the row sum
     int cnt = 0;
 
+    PROF_T(t_loop0);
+    PROF_ADD(11, t_cta0, t_loop0);  // prologue up to the softmax loop
     for (int n = 0; n < n_tiles; ++n) {
-      if (!((stream_mask(n) >> wg) & 1)) continue;
-      // valid / kept columns of each 32-column chunk (warp-uniform)
-      int valid[4];
+      if (!((stream_mask(n) >> sidx) & 1)) continue;
+      // kept / valid columns of my 64-column half (warp-uniform)
+      int nv;
       if (C::kSplitKV) {
-#pragma unroll
-        for (int ch = 0; ch < 2; ++ch) {
-          const int ent = n * 2 + ch;
-          int nv = 0;
-          if (ent < n_ent && ((sEntF[ent] >> rh) & 1))
-            nv = (int)min((int64_t)64, p.N - (int64_t)sEntJ[ent] * 64);
-          valid[2 * ch] = min(nv, 32);
-          valid[2 * ch + 1] = max(nv - 32, 0);
-        }
+        const int ent = n * 2 + half;
+        nv = 0;
+        if (ent < n_ent && ((sEntF[ent] >> rh) & 1)) nv = (int)min((int64_t)64, p.N - (int64_t)sEntJ[ent] * 64);
       } else {
-        const int nv = (int)min((int64_t)128, p.N - (int64_t)sEntJ[n] * 128);
-#pragma unroll
-        for (int c = 0; c < 4; ++c) valid[c] = max(0, min(32, nv - 32 * c));
+        nv = (int)min((int64_t)128, p.N - (int64_t)sEntJ[n] * 128) - 64 * half;
+        nv = max(0, min(64, nv));
       }
+      const int valid[2] = {min(nv, 32), max(nv - 32, 0)};
 
-      mbar_wait_bounded(s_full + wg, cnt & 1, s_abort, p.status, 30 + wg, p.wait_limit);
+      PROF_T(t_a);
+      mbar_wait_bounded(s_full + sidx, cnt & 1, s_abort, p.status, 30 + sidx, p.wait_limit);
       tc_fence_after();
-      // pass 1: row maximum over the kept, valid columns (two 64-column halves)
+      PROF_T(t_b);
+#ifdef SPARSP_ATTN_NOSOFTMAX  // tuning builds only: measure the MMA / TMA pipeline alone
+      tc_fence_before();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(p_full + sidx);
+      ++cnt;
+      continue;
+#endif
+      float sv[64];
+      tmem_ld32(tS + half * 64, reinterpret_cast<uint32_t*>(sv));
+      tmem_ld32(tS + half * 64 + 32, reinterpret_cast<uint32_t*>(sv) + 32);
+      tmem_ld_wait();
       float mx = -INFINITY;
 #pragma unroll
-      for (int h = 0; h < 2; ++h) {
-        float sv[64];
-        tmem_ld32(tS + h * 64, reinterpret_cast<uint32_t*>(sv));
-        tmem_ld32(tS + h * 64 + 32, reinterpret_cast<uint32_t*>(sv) + 32);
-        tmem_ld_wait();
+      for (int c = 0; c < 2; ++c) {
+        if (valid[c] == 32) {
 #pragma unroll
-        for (int cc = 0; cc < 2; ++cc) {
-          const int vc = valid[2 * h + cc];
-          if (vc == 32) {
+          for (int e = 0; e < 32; e += 2) mx = fmaxf(mx, fmaxf(sv[c * 32 + e], sv[c * 32 + e + 1]));
+        } else if (valid[c] > 0) {
 #pragma unroll
-            for (int e = 0; e < 32; e += 2) mx = fmaxf(mx, fmaxf(sv[cc * 32 + e], sv[cc * 32 + e + 1]));
-          } else if (vc > 0) {
-#pragma unroll
-            for (int e = 0; e < 32; ++e) mx = fmaxf(mx, e < vc ? sv[cc * 32 + e] : -INFINITY);
-          }
+          for (int e = 0; e < 32; ++e) mx = fmaxf(mx, e < valid[c] ? sv[c * 32 + e] : -INFINITY);
         }
       }
-      mx *= p.scale_log2;
+      // exchange the two halves' maxima (double-buffered by tile parity); the barrier also orders
+      // my partner's reads of S before my writes of P into the columns it read
+      float* mslot = sMax + (((cnt & 1) * 2 + sidx) * 2) * 128;
+      mslot[half * 128 + row] = mx;
+      named_bar_sync(pair_bar, 64);
+      mx = fmaxf(mx, mslot[(1 - half) * 128 + row]) * p.scale_log2;
+      PROF_T(t_c);
       const float m_new = fmaxf(m_used, mx);
       const bool grow = m_new > m_used + kGrowThreshold || (m_used == -INFINITY && m_new > -INFINITY);
       if (__any_sync(0xffffffffu, grow)) {
         const float alpha = grow ? ex2(m_used - m_new) : 1.0f;  // m_used = -inf -> 0
         if (cnt > 0) {  // S_s of this tile is complete, hence so is every earlier P V of the stream
 #pragma unroll
-          for (int c = 0; c < D / 32; ++c) {
-            uint32_t o[32];
-            tmem_ld32(tO + c * 32, o);
+          for (int c = 0; c < D / 32; ++c) {  // my half of the accumulator's columns, 16 at a time
+            uint32_t o[16];
+            tmem_ld16(tO + half * (D / 2) + c * 16, o);
             tmem_ld_wait();
 #pragma unroll
-            for (int e = 0; e < 32; ++e) o[e] = __float_as_uint(__uint_as_float(o[e]) * alpha);
-            tmem_st32(tO + c * 32, o);
+            for (int e = 0; e < 16; ++e) o[e] = __float_as_uint(__uint_as_float(o[e]) * alpha);
+            tmem_st16(tO + half * (D / 2) + c * 16, o);
           }
         }
         l_run *= alpha;
         if (grow) m_used = m_new;
       }
+      PROF_T(t_d);
 
-      // pass 2: exponentials chunk by chunk; bf16 P overwrites S in place (P chunk c occupies
-      // columns [16c, 16c+16), which lie inside the S columns already consumed)
+      // exponentials; bf16 P overwrites S in place: my keys [64*half, 64*half+64) go to columns
+      // [32*half, 32*half+32)
       float lsum = 0.0f;
       const float neg_m = -m_used;
-      float buf[2][32];
-      tmem_ld32(tS, reinterpret_cast<uint32_t*>(buf[0]));
 #pragma unroll
-      for (int c = 0; c < 4; ++c) {
-        tmem_ld_wait();
-        if (c < 3) tmem_ld32(tS + (c + 1) * 32, reinterpret_cast<uint32_t*>(buf[(c + 1) & 1]));
-        const float* sv = buf[c & 1];
+      for (int c = 0; c < 2; ++c) {
         uint32_t pk[16];
+        const float* svc = sv + c * 32;
         if (valid[c] == 32) {
 #pragma unroll
           for (int e = 0; e < 16; ++e) {
-            const float p0 = ex2(fmaf(sv[2 * e], p.scale_log2, neg_m));
-            const float p1 = ex2(fmaf(sv[2 * e + 1], p.scale_log2, neg_m));
+            const float p0 = ex2(fmaf(svc[2 * e], p.scale_log2, neg_m));
+            const float p1 = ex2(fmaf(svc[2 * e + 1], p.scale_log2, neg_m));
             lsum += p0 + p1;
             const __nv_bfloat162 h2 = __floats2bfloat162_rn(p0, p1);
             pk[e] = *reinterpret_cast<const uint32_t*>(&h2);
@@ -372,8 +411,8 @@ __global__ void __launch_bounds__(kAttnThreads, 1)
         } else if (valid[c] > 0) {
 #pragma unroll
           for (int e = 0; e < 16; ++e) {
-            const float p0 = 2 * e < valid[c] ? ex2(fmaf(sv[2 * e], p.scale_log2, neg_m)) : 0.0f;
-            const float p1 = 2 * e + 1 < valid[c] ? ex2(fmaf(sv[2 * e + 1], p.scale_log2, neg_m)) : 0.0f;
+            const float p0 = 2 * e < valid[c] ? ex2(fmaf(svc[2 * e], p.scale_log2, neg_m)) : 0.0f;
+            const float p1 = 2 * e + 1 < valid[c] ? ex2(fmaf(svc[2 * e + 1], p.scale_log2, neg_m)) : 0.0f;
             lsum += p0 + p1;
             const __nv_bfloat162 h2 = __floats2bfloat162_rn(p0, p1);
             pk[e] = *reinterpret_cast<const uint32_t*>(&h2);
@@ -382,29 +421,45 @@ __global__ void __launch_bounds__(kAttnThreads, 1)
 #pragma unroll
           for (int e = 0; e < 16; ++e) pk[e] = 0u;
         }
-        tmem_st16(tS + c * 16, pk);
+        tmem_st16(tS + half * 32 + c * 16, pk);
       }
       l_run += lsum;
+      PROF_T(t_e);
       tmem_st_wait();
       tc_fence_before();
-      mbar_arrive(p_full + wg);
+      __syncwarp();
+      if (lane == 0) mbar_arrive(p_full + sidx);
       ++cnt;
+      PROF_T(t_f);
+      PROF_ADD(0, t_a, t_b);  // wait for S
+      PROF_ADD(1, t_b, t_c);  // load + max + exchange
+      PROF_ADD(2, t_c, t_d);  // rescale decision
+      PROF_ADD(3, t_d, t_e);  // exponentials + P store
+      PROF_ADD(4, t_e, t_f);  // store wait + arrive
+      PROF_ADD(5, t_a, t_a + 1);  // tile count
     }
 
     // ---- epilogue -------------------------------------------------------------------------
+    PROF_T(t_ep0);
     if (cnt > 0) {
-      mbar_wait_bounded(o_full + wg, (cnt - 1) & 1, s_abort, p.status, 40 + wg, p.wait_limit);
+      mbar_wait_bounded(o_full + sidx, (cnt - 1) & 1, s_abort, p.status, 40 + sidx, p.wait_limit);
       tc_fence_after();
     }
+    PROF_T(t_ep1);
+    PROF_ADD(12, t_ep0, t_ep1);  // wait for the last P V
+    sStat[(sidx * 2 + half) * 128 + row] = make_float2(m_used, l_run);
     if (!C::kSplitKV) {
-      const int64_t tok = q0 + wg * 128 + row;
-      const float inv_l = l_run > 0.0f ? 1.0f / l_run : 0.0f;
-      __nv_bfloat16* orow = p.O + (int64_t)batch * p.sB + (int64_t)head * p.sH + tok * p.sT;
+      // the row's two threads add their partial sums; each writes its half of the columns
+      named_bar_sync(pair_bar, 64);
+      const float l = l_run + sStat[(sidx * 2 + 1 - half) * 128 + row].y;
+      const int64_t tok = q0 + sidx * 128 + row;
+      const float inv_l = l > 0.0f ? 1.0f / l : 0.0f;
+      __nv_bfloat16* orow = p.O + (int64_t)batch * p.sB + (int64_t)head * p.sH + tok * p.sT + half * (D / 2);
 #pragma unroll
-      for (int c = 0; c < D / 32; ++c) {
+      for (int c = 0; c < D / 64; ++c) {
         uint32_t o[32];
         if (cnt > 0) {  // warp-uniform: tensor-memory loads are warp-collective
-          tmem_ld32(tO + c * 32, o);
+          tmem_ld32(tO + half * (D / 2) + c * 32, o);
           tmem_ld_wait();
         } else {
 #pragma unroll
@@ -424,57 +479,59 @@ __global__ void __launch_bounds__(kAttnThreads, 1)
           }
         }
       }
-      if (p.lse && tok < p.N)
-        p.lse[(int64_t)bh * p.N + tok] = l_run > 0.0f ? (m_used + log2f(l_run)) * 0.6931471805599453f : -INFINITY;
+      if (p.lse && half == 0 && tok < p.N)
+        p.lse[(int64_t)bh * p.N + tok] = l > 0.0f ? (m_used + log2f(l)) * 0.6931471805599453f : -INFINITY;
     } else {
-      // merge the two streams' partial results: stream s finalises columns [s*D/2, (s+1)*D/2)
-      constexpr int HALF = D / 2;
+      // merge the two streams' partial results.  Thread (stream s, half h) finalises the column
+      // quarter 2s+h; it hands the other stream's thread of the same half the quarter that one
+      // finalises, scaled to the common reference maximum.
+      constexpr int QW = D / 4;
       float* mbuf = reinterpret_cast<float*>(sK);  // K/V rings are idle once both streams are done
-      sStat[wg * 128 + row] = make_float2(m_used, l_run);
-      named_bar_sync(1, 256);
-      const float2 other = sStat[(1 - wg) * 128 + row];
-      const float m = fmaxf(m_used, other.x);
+      named_bar_sync(9, 512);
+      const float l_me = l_run + sStat[(sidx * 2 + 1 - half) * 128 + row].y;
+      const float2 o0 = sStat[((1 - sidx) * 2) * 128 + row];
+      const float2 o1 = sStat[((1 - sidx) * 2 + 1) * 128 + row];
+      const float m_ot = o0.x, l_ot = o0.y + o1.y;
+      const float m = fmaxf(m_used, m_ot);
       const float a_me = m_used > -INFINITY ? ex2(m_used - m) : 0.0f;
-      const float a_ot = other.x > -INFINITY ? ex2(other.x - m) : 0.0f;
-      const float l = l_run * a_me + other.y * a_ot;
+      const float a_ot = m_ot > -INFINITY ? ex2(m_ot - m) : 0.0f;
+      const float l = l_me * a_me + l_ot * a_ot;
       const float inv_l = l > 0.0f ? 1.0f / l : 0.0f;
-      // hand the partner its half of my accumulator, scaled to the common reference
-      float* give = mbuf + ((size_t)wg * 128 + row) * C::kMergeStride;
-#pragma unroll
-      for (int c = 0; c < HALF / 32; ++c) {
-        uint32_t o[32];
+      const int give_q = 2 * (1 - sidx) + half, keep_q = 2 * sidx + half;
+      float* give = mbuf + ((size_t)(sidx * 2 + half) * 128 + row) * C::kMergeStride;
+      {
+        uint32_t o[QW];
         if (cnt > 0) {
-          tmem_ld32(tO + (1 - wg) * HALF + c * 32, o);
+          if constexpr (QW == 32) tmem_ld32(tO + give_q * QW, o); else tmem_ld16(tO + give_q * QW, o);
           tmem_ld_wait();
         } else {
 #pragma unroll
-          for (int e = 0; e < 32; ++e) o[e] = 0u;
+          for (int e = 0; e < QW; ++e) o[e] = 0u;
         }
 #pragma unroll
-        for (int v = 0; v < 8; ++v)
-          *reinterpret_cast<float4*>(give + c * 32 + v * 4) =
+        for (int v = 0; v < QW / 4; ++v)
+          *reinterpret_cast<float4*>(give + v * 4) =
               make_float4(__uint_as_float(o[v * 4]) * a_me, __uint_as_float(o[v * 4 + 1]) * a_me,
                           __uint_as_float(o[v * 4 + 2]) * a_me, __uint_as_float(o[v * 4 + 3]) * a_me);
       }
-      named_bar_sync(1, 256);
+      named_bar_sync(9, 512);
       const int64_t tok = q0 + row;
-      const float* take = mbuf + ((size_t)(1 - wg) * 128 + row) * C::kMergeStride;
-      __nv_bfloat16* orow = p.O + (int64_t)batch * p.sB + (int64_t)head * p.sH + tok * p.sT + wg * HALF;
-#pragma unroll
-      for (int c = 0; c < HALF / 32; ++c) {
-        uint32_t o[32];
+      const float* take = mbuf + ((size_t)((1 - sidx) * 2 + half) * 128 + row) * C::kMergeStride;
+      __nv_bfloat16* orow = p.O + (int64_t)batch * p.sB + (int64_t)head * p.sH + tok * p.sT + keep_q * QW;
+      {
+        uint32_t o[QW];
         if (cnt > 0) {
-          tmem_ld32(tO + wg * HALF + c * 32, o);
+          if constexpr (QW == 32) tmem_ld32(tO + keep_q * QW, o); else tmem_ld16(tO + keep_q * QW, o);
           tmem_ld_wait();
         } else {
 #pragma unroll
-          for (int e = 0; e < 32; ++e) o[e] = 0u;
+          for (int e = 0; e < QW; ++e) o[e] = 0u;
         }
         if (tok < p.N) {
 #pragma unroll
-          for (int v = 0; v < 4; ++v) {
-            const float4 t0 = *reinterpret_cast<const float4*>(take + c * 32 + v * 8);
-            const float4 t1 = *reinterpret_cast<const float4*>(take + c * 32 + v * 8 + 4);
+          for (int v = 0; v < QW / 8; ++v) {
+            const float4 t0 = *reinterpret_cast<const float4*>(take + v * 8);
+            const float4 t1 = *reinterpret_cast<const float4*>(take + v * 8 + 4);
             const float tt[8] = {t0.x, t0.y, t0.z, t0.w, t1.x, t1.y, t1.z, t1.w};
             uint32_t w[4];
 #pragma unroll
@@ -484,18 +541,23 @@ __global__ void __launch_bounds__(kAttnThreads, 1)
               const __nv_bfloat162 h2 = __floats2bfloat162_rn(x0, x1);
               w[e] = *reinterpret_cast<const uint32_t*>(&h2);
             }
-            *reinterpret_cast<uint4*>(orow + c * 32 + v * 8) = make_uint4(w[0], w[1], w[2], w[3]);
+            *reinterpret_cast<uint4*>(orow + v * 8) = make_uint4(w[0], w[1], w[2], w[3]);
           }
         }
       }
-      if (p.lse && wg == 0 && tok < p.N)
+      if (p.lse && sidx == 0 && half == 0 && tok < p.N)
         p.lse[(int64_t)bh * p.N + tok] = l > 0.0f ? (m + log2f(l)) * 0.6931471805599453f : -INFINITY;
     }
   }
 
+  PROF_T(t_cta1);
   tc_fence_before();
   __syncthreads();
   if (warp == 1) tmem_dealloc(tmem_base, kTmemCols);
+  PROF_T(t_cta2);
+  PROF_ADD(13, t_cta0, t_cta1);  // CTA lifetime of the sampled lanes up to the final barrier
+  PROF_ADD(14, t_cta1, t_cta2);  // final barrier + dealloc
+  PROF_ADD(15, t_cta0, t_cta0 + 1);
 }
 
 // ------------------------------------------------------------------------------------------------
@@ -581,5 +643,17 @@ int launch_attn(const sparsp_shape& s, const Geometry& g, const void* Q, const v
   if (g.d == 128 && g.b == 64) return launch_attn_t<128, 64>(s, g, Q, K, V, p, st);
   return launch_attn_t<128, 128>(s, g, Q, K, V, p, st);
 }
+
+#ifdef SPARSP_ATTN_PROFILE
+extern "C" __attribute__((visibility("default"))) int sparsp_debug_attn_profile(unsigned long long* out16, int reset) {
+  cudaDeviceSynchronize();
+  cudaMemcpyFromSymbol(out16, g_attn_prof, sizeof(g_attn_prof));
+  if (reset) {
+    unsigned long long z[16] = {0};
+    cudaMemcpyToSymbol(g_attn_prof, z, sizeof z);
+  }
+  return 0;
+}
+#endif
 
 }  // namespace sparsp

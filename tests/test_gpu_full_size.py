@@ -1,0 +1,104 @@
+"""GPU parity at the full sizes of the five workloads, in the launch configuration bench.py times.
+
+Inputs are generated on the device with the shared seeded generator and copied to the host, so both
+sides see the same bits.  Masks, unions, counts, offsets and volumes are compared in full with the
+oracle; the packed buffer is compared in full, in device memory, against a library gather driven by
+the ORACLE's entry list; attention is compared on a seeded sample of (head, query block) units the
+oracle computes one by one (first block, last ragged block, one block per virtual rank, the
+video/text boundary, random ones)."""
+import numpy as np
+import pytest
+import torch
+
+import parity_util as pu
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def binding():
+    from paper_2609_32197_b200 import binding as b
+    b.lib()
+    assert torch.cuda.is_available()
+    return b
+
+
+def _placement(oracle, synth, wl, name):
+    if name == "contiguous":
+        return oracle.placement_contiguous(wl.n_blocks, wl.ranks)
+    if name == "periodic":
+        return oracle.placement_periodic(wl.n_blocks, wl.ranks, wl.block, wl.frame_tokens, wl.n_video)
+    return synth.shuffled_placement(wl.n_blocks, wl.ranks, seed=1).numpy()
+
+
+def _full_size(oracle, binding, name, n_attn_random):
+    from paper_2609_32197_b200 import synth
+    wl = synth.WORKLOADS[name]
+    H, d, b, P = wl.heads, wl.head_dim, wl.block, wl.ranks
+    Qd, Kd, Vd = synth.make_qkv(wl, "cuda")
+    Q, K, V = Qd.cpu(), Kd.cpu(), Vd.cpu()
+    N, NB = wl.n_tokens, wl.n_blocks
+    shape = binding.make_shape(H, d, wl.grid, wl.n_text, b)
+    ws = binding.make_workspace(shape, P)
+    pq, pk = oracle.pool(Q, b), oracle.pool(K, b)
+    sc = oracle.scores(pq, pk)
+    is_text = oracle.text_block_flags(wl.n_video, wl.n_text, b)
+    report = {}
+    for pct in (wl.topk_pct or (None,)):
+        k = wl.topk_abs if pct is None else oracle.resolve_topk(pct, wl.nb_video)
+        assert pct is None or k == binding.sparsp_resolve_topk(pct, binding.sparsp_geometry(shape).n_video_blocks)
+        # ---- step 1, in full
+        mask_ref, list_ref, count_ref = oracle.topk_mask(sc, is_text, k)
+        got = pu.gpu_block_mask(binding, shape, Qd, Kd, k, ws)
+        assert np.array_equal(got["pooled_q"][0].cpu().numpy().view(np.uint32), pq.view(np.uint32))
+        assert np.array_equal(got["pooled_k"][0].cpu().numpy().view(np.uint32), pk.view(np.uint32))
+        gm = pu.u32(got["mask"][0])
+        assert np.array_equal(gm, mask_ref), f"{name} k={k}: mask differs on {(gm != mask_ref).any(axis=2).sum()} rows"
+        assert np.array_equal(got["kv_list"][0].cpu().numpy(), list_ref)
+        assert np.array_equal(got["kv_count"][0].cpu().numpy(), count_ref)
+        for pname in wl.placements:
+            rank = _placement(oracle, synth, wl, pname)
+            # ---- step 2, in full
+            dg = pu.gpu_demand_pack(binding, shape, got["mask"], torch.as_tensor(rank).cuda(), P, 0, Kd, Vd, ws)
+            assert binding.sparsp_status(ws) == binding.SPARSP_OK
+            dref = pu.check_demand(oracle, binding, shape, mask_ref, rank, P, False, dg)
+            h_idx, j_idx = pu.oracle_entry_list(dref, rank, P, H, NB, False)
+            assert len(h_idx) == int(dref["total"].sum()) == dg["total_entries"]
+            pu.check_packed_full_on_device(Kd, Vd, b, dg["packed"], h_idx, j_idx)
+            report[(k, pname)] = int(dref["volume"].sum())
+            del dg
+        # ---- step 3, sampled
+        Od = torch.zeros_like(Qd)
+        binding.sparsp_sparse_attn_fwd(shape, Qd, Kd, Vd, got["mask"], 0.0, Od, None, ws)
+        torch.cuda.synchronize()
+        assert binding.sparsp_status(ws) == binding.SPARSP_OK, binding.sparsp_last_error()
+        extra = [wl.nb_video - 1, wl.nb_video] if wl.n_text else []
+        units = pu.sample_units(H, NB, _placement(oracle, synth, wl, wl.placements[0]), n_attn_random, 17, extra)
+        mx, mean = pu.check_attn_units(oracle, Q, K, V, mask_ref, b, Od, units)
+        # rows the sample does not cover: finite, and not left at the zero fill
+        assert bool(torch.isfinite(Od.float()).all())
+        assert bool((Od.float().abs().amax(dim=-1) > 0).all())
+        report[(k, "attn")] = (len(units), mx, mean)
+    print(name, report)
+    return report
+
+
+def test_mid_full_size(oracle_mod, binding):
+    _full_size(oracle_mod, binding, "mid", 24)
+
+
+def test_cog_like_full_size_text_blocks_and_shuffled_placement(oracle_mod, binding):
+    _full_size(oracle_mod, binding, "cog", 24)
+
+
+def test_wan_like_full_size_two_placements(oracle_mod, binding):
+    rep = _full_size(oracle_mod, binding, "wan", 8)
+    vols = {p: v for (k, p), v in rep.items() if p in ("contiguous", "periodic")}
+    assert set(vols) == {"contiguous", "periodic"}
+
+
+def test_hunyuan_like_full_size_topk_sweep(oracle_mod, binding):
+    rep = _full_size(oracle_mod, binding, "hunyuan", 4)
+    vols = sorted((k, v) for (k, p), v in rep.items() if p == "contiguous")
+    assert [k for k, _ in vols] == [47, 93, 233]
+    assert vols[0][1] < vols[1][1] < vols[2][1]  # more kept blocks, more demanded bytes
