@@ -43,6 +43,8 @@ constexpr int kAttnThreads = 608;
 constexpr int kIssuer1Warp = 18;  // warp 1 issues the MMAs of stream 0, warp 18 those of stream 1
 constexpr int kTmemCols = 512;
 constexpr float kGrowThreshold = 8.0f;
+constexpr long long kStaggerCycles = 6000;
+constexpr unsigned kSoftmaxSleepNs = 40;
 
 template <int D, int BLK>
 struct AttnCfg {
@@ -236,8 +238,11 @@ __global__ void __maxnreg__(96)
     // barrier and then arrives once on its "empty" barrier (count 2: one arrival per issuer) --
     // through tcgen05.commit after its MMAs if its stream uses the tile, directly otherwise.  The
     // two streams therefore never wait on each other's softmax, only on the shared K/V rings.
-    if (lane == 0 && n_tiles > 0) {
+    // The whole warp runs the loop (uniform control flow and uniform operands, so descriptors and
+    // addresses can live in uniform registers); one elected lane issues the tcgen05 instructions.
+    if (n_tiles > 0) {
       const int s = (warp == 1) ? 0 : 1;
+      const bool leader = elect_one();
       constexpr uint32_t kIdescQK = make_idesc_bf16(128, 128, 0, 0);
       constexpr uint32_t kIdescPV = make_idesc_bf16(128, D, 0, 1);
       const uint32_t tSs = tmem_base + s * 128;
@@ -266,20 +271,30 @@ __global__ void __maxnreg__(96)
         if (keep) {
           tc_fence_after();
           const uint64_t db0 = descV + (uint64_t)(((m % S) * C::kTileBytes) >> 4);
+          if (leader) {
 #pragma unroll
-          for (int kk = 0; kk < 8; ++kk)
-            mma_ts(tOs, tSs + kk * 8, db0 + (uint64_t)((kk * 2048) >> 4), kIdescPV, (kk > 0) ? 1u : started);
+            for (int kk = 0; kk < 8; ++kk)
+              mma_ts(tOs, tSs + kk * 8, db0 + (uint64_t)((kk * 2048) >> 4), kIdescPV, (kk > 0) ? 1u : started);
+            mma_commit(o_full + s);
+            mma_commit(v_empty + m % S);
+          }
           started = 1u;
-          mma_commit(o_full + s);
-          mma_commit(v_empty + m % S);
           PROF_T(t_v2);
           PROF_ADD(6, t_v1, t_v2);  // issuer issuing P V
-        } else {
+        } else if (leader) {
           mbar_arrive(v_empty + m % S);
         }
+        __syncwarp();
       };
 
       mbar_wait_bounded(bar_q, 0, s_abort, p.status, 11, p.wait_limit);
+      if (s == 1) {
+        // start stream 1 half a period late, so that its exponentials fall into stream 0's MMA
+        // phase instead of competing with stream 0's exponentials for the special-function unit
+        const long long t0 = clock64();
+        while (!mbar_test_wait(p_full + 0, 0) && clock64() - t0 < kStaggerCycles) {
+        }
+      }
       for (int n = 0; n < n_tiles; ++n) {
         const bool keep = (stream_mask(n) >> s) & 1;
         while (vdone < n - 1) handle_v(vdone++);  // a V stage is released at most two steps after its fill
@@ -289,21 +304,25 @@ __global__ void __maxnreg__(96)
         PROF_ADD(9, t_k0, t_k1);  // issuer waiting for K
         if (keep) {
           while (vdone <= last_kept) handle_v(vdone++);  // P V of the previous kept tile frees S_s
+          PROF_T(t_k3);
           tc_fence_after();
           const uint64_t db0 = descK + (uint64_t)(((n % S) * C::kTileBytes) >> 4);
+          if (leader) {
 #pragma unroll
-          for (int kk = 0; kk < D / 16; ++kk) {
-            const uint64_t off = (uint64_t)(((kk / 4) * 16384 + (kk % 4) * 32) >> 4);
-            mma_ss(tSs, descQ + off, db0 + off, kIdescQK, kk > 0 ? 1u : 0u);
+            for (int kk = 0; kk < D / 16; ++kk) {
+              const uint64_t off = (uint64_t)(((kk / 4) * 16384 + (kk % 4) * 32) >> 4);
+              mma_ss(tSs, descQ + off, db0 + off, kIdescQK, kk > 0 ? 1u : 0u);
+            }
+            mma_commit(s_full + s);
+            mma_commit(k_empty + n % S);
           }
-          mma_commit(s_full + s);
-          mma_commit(k_empty + n % S);
           last_kept = n;
           PROF_T(t_k2);
-          PROF_ADD(7, t_k1, t_k2);  // issuer issuing Q K^T
-        } else {
+          PROF_ADD(7, t_k3, t_k2);  // issuer issuing Q K^T
+        } else if (leader) {
           mbar_arrive(k_empty + n % S);
         }
+        __syncwarp();
       }
       while (vdone < n_tiles) handle_v(vdone++);
     }
@@ -339,7 +358,7 @@ __global__ void __maxnreg__(96)
       const int valid[2] = {min(nv, 32), max(nv - 32, 0)};
 
       PROF_T(t_a);
-      mbar_wait_bounded(s_full + sidx, cnt & 1, s_abort, p.status, 30 + sidx, p.wait_limit);
+      mbar_wait_bounded(s_full + sidx, cnt & 1, s_abort, p.status, 30 + sidx, p.wait_limit, kSoftmaxSleepNs);
       tc_fence_after();
       PROF_T(t_b);
 #ifdef SPARSP_ATTN_NOSOFTMAX  // tuning builds only: measure the MMA / TMA pipeline alone

@@ -13,6 +13,19 @@ __device__ __forceinline__ uint32_t smem_u32(const void* p) {
   return static_cast<uint32_t>(__cvta_generic_to_shared(p));
 }
 
+// One lane of a converged warp (a predicate the compiler can treat as warp-uniform control).
+__device__ __forceinline__ bool elect_one() {
+  uint32_t pred;
+  asm volatile(
+      "{\n\t"
+      ".reg .pred p;\n\t"
+      "elect.sync _|p, 0xffffffff;\n\t"
+      "selp.b32 %0, 1, 0, p;\n\t"
+      "}"
+      : "=r"(pred));
+  return pred != 0;
+}
+
 // ---- mbarrier ----------------------------------------------------------------------------------
 __device__ __forceinline__ void mbar_init(uint64_t* bar, uint32_t count) {
   asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(bar)), "r"(count) : "memory");
@@ -60,11 +73,15 @@ __device__ __forceinline__ bool mbar_test_wait(uint64_t* bar, uint32_t parity) {
 // abort flag (after which every later wait of the CTA returns at once, so control flow stays
 // uniform and the kernel drains quickly) and records `code`/`where` in the global status words.
 __device__ __forceinline__ void mbar_wait_bounded(uint64_t* bar, uint32_t parity, volatile int* abort_flag,
-                                                  int32_t* status, int where, long long limit_cycles) {
-  if (*abort_flag) return;
+                                                  int32_t* status, int where, long long limit_cycles,
+                                                  unsigned sleep_ns = 0) {
   if (mbar_try_wait(bar, parity)) return;
+  if (*abort_flag) return;
   const long long t0 = clock64();
   while (!mbar_try_wait(bar, parity)) {
+    // many-thread waiters back off, so that their polling does not take issue slots from the
+    // single-thread MMA issuer and TMA producer that share their scheduler
+    if (sleep_ns) __nanosleep(sleep_ns);
     if (*abort_flag) return;
     if (clock64() - t0 > limit_cycles) {
       *abort_flag = 1;
