@@ -153,6 +153,27 @@ SPARSP_API int sparsp_sparse_attn_fwd(const sparsp_shape* shape, const void* Q, 
                            const uint32_t* mask, float softmax_scale, void* O, float* lse,
                            void* workspace, void* stream);
 
+/* Planning without any allocation.  (No counterpart in the paper: an engineering variant of the
+ * planning half of sparsp_demand_pack.)
+ * For callers that are not allowed to allocate device memory -- for example a plug-in running inside a
+ * host application that has handed all GPU memory to its own pool, or a latency-critical loop that
+ * must never enter the driver's allocator -- and so cannot provide the workspace the other calls need.
+ * Computes exactly what sparsp_demand_pack computes with SPARSP_PLAN_ONLY (same definitions, layouts
+ * and argument meaning for union_mask, cnt, seg_offset, seg_total, volume_bytes; `flags` may only carry
+ * SPARSP_INCLUDE_LOCAL) but keeps its scratch (per-rank ownership bit words and table bases) in a
+ * 16.4 KB array that is part of the library image; every GPU that loads the library holds that array
+ * until the process exits.  The call itself allocates and frees nothing, on the host or on the device.
+ * Limits: n_ranks <= 64 and batch * n_ranks <= 1024, else SPARSP_ERR_CAPACITY (nothing is launched).
+ * The first call on each device looks up the array's device address (with that device current); make
+ * that first call before any stream capture begins.  All calls on a device share the one array: it
+ * keeps the previous call's contents, every word a call reads is rewritten by that call first (nothing
+ * needs to start at zero), and two calls whose kernels may overlap on the GPU (different streams
+ * without ordering) race on it -- serialise them. */
+SPARSP_API int sparsp_demand_plan_noalloc(const sparsp_shape* shape, const uint32_t* mask,
+                                          const int32_t* rank_of_block, int32_t n_ranks, int32_t flags,
+                                          uint32_t* union_mask, int32_t* cnt, int64_t* seg_offset,
+                                          int64_t* seg_total, int64_t* volume_bytes, void* stream);
+
 /* Synchronises `stream` and returns the workspace's status word in *code (SPARSP_OK if no kernel
  * reported a problem since the last reset), then resets it. */
 SPARSP_API int sparsp_status(void* workspace, void* stream, int32_t* code);

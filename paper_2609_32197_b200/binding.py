@@ -28,7 +28,7 @@ SPARSP_INCLUDE_LOCAL = 2
 EXPORTS = [
     "sparsp_geometry", "sparsp_resolve_topk", "sparsp_placement_contiguous", "sparsp_placement_periodic",
     "sparsp_workspace_bytes", "sparsp_block_mask", "sparsp_demand_pack", "sparsp_sparse_attn_fwd",
-    "sparsp_status", "sparsp_last_error", "sparsp_launch_count",
+    "sparsp_status", "sparsp_last_error", "sparsp_launch_count", "sparsp_demand_plan_noalloc",
 ]
 
 
@@ -155,6 +155,16 @@ def sparsp_demand_pack(shape, mask, rank_of_block, n_ranks, flags, K, V, union_m
                                     _ptr(union_mask), _ptr(cnt), _ptr(seg_offset), _ptr(seg_total),
                                     _ptr(volume_bytes), _ptr(packed), ctypes.c_int64(packed_capacity_bytes),
                                     _ptr(dst_base_bytes), _ptr(workspace), _stream()))
+
+
+def sparsp_demand_plan_noalloc(shape, mask, rank_of_block, n_ranks, flags, union_mask, cnt, seg_offset, seg_total,
+                               volume_bytes):
+    """Planning half of sparsp_demand_pack for callers that cannot allocate device memory: no workspace
+    argument, the scratch is a small array inside the library.  Outputs as for SPARSP_PLAN_ONLY."""
+    _check(lib().sparsp_demand_plan_noalloc(ctypes.byref(shape), _ptr(mask), _ptr(rank_of_block),
+                                            ctypes.c_int32(n_ranks), ctypes.c_int32(flags), _ptr(union_mask),
+                                            _ptr(cnt), _ptr(seg_offset), _ptr(seg_total), _ptr(volume_bytes),
+                                            _stream()))
 
 
 def sparsp_sparse_attn_fwd(shape, Q, K, V, mask, softmax_scale, O, lse, workspace):

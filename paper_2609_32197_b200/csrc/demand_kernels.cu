@@ -1,6 +1,8 @@
 // Step 2: per-rank per-head unions of required KV blocks, demand counts, exchange volume,
 // pack-order offsets, the entry table, and the gather of K/V tiles into per-consumer buffers.
 // Everything before the gather is small integer work on bit words; the gather is the HBM-bound part.
+#include <mutex>
+
 #include "common.cuh"
 
 namespace sparsp {
@@ -240,4 +242,89 @@ int launch_pack(const sparsp_shape& s, const Geometry& g, const void* K, const v
   return SPARSP_OK;
 }
 
+// ------------------------------------------------------------------------------------------------
+// Allocation-free planning call.  Its scratch (the per-rank ownership bit words and the per-consumer
+// table bases) lives in one file-scope device array instead of a caller-provided workspace, so a
+// caller that cannot allocate device memory at all can still obtain unions, counts, offsets and
+// volumes.  Every GPU that loads the library carries the array (kPlanScratchBytes) until exit.
+// ------------------------------------------------------------------------------------------------
+constexpr int kPlanMaxRanks = 64;         // n_ranks limit of the allocation-free call
+constexpr int kPlanMaxBatchRanks = 1024;  // batch * n_ranks limit
+constexpr int kPlanOwnWords = kPlanMaxRanks * (kMaxBlocks / 32);
+constexpr size_t kPlanScratchBytes = kPlanOwnWords * sizeof(uint32_t) + (kPlanMaxBatchRanks + 1) * sizeof(int64_t);
+
+static __device__ __align__(256) unsigned char g_plan_scratch[kPlanScratchBytes];
+
+constexpr int kMaxDevices = 64;
+static std::mutex g_plan_mutex;
+static void* g_plan_scratch_addr[kMaxDevices] = {nullptr};
+
+// Device address of g_plan_scratch on the current device.  In host code the array's name is only a
+// handle, so the address is resolved once per device with that device current.
+static int plan_scratch_address(void** out) {
+  int dev = 0;
+  SPARSP_CUDA_OK(cudaGetDevice(&dev));
+  if (dev < 0 || dev >= kMaxDevices) {
+    set_error("device ordinal %d outside 0..%d", dev, kMaxDevices - 1);
+    return SPARSP_ERR_UNSUPPORTED;
+  }
+  std::lock_guard<std::mutex> lock(g_plan_mutex);
+  if (!g_plan_scratch_addr[dev]) {
+    void* ptr = nullptr;
+    SPARSP_CUDA_OK(cudaGetSymbolAddress(&ptr, g_plan_scratch));
+    g_plan_scratch_addr[dev] = ptr;
+  }
+  *out = g_plan_scratch_addr[dev];
+  return SPARSP_OK;
+}
+
 }  // namespace sparsp
+
+using namespace sparsp;
+
+extern "C" SPARSP_API int sparsp_demand_plan_noalloc(const sparsp_shape* shape, const uint32_t* mask,
+                                                     const int32_t* rank_of_block, int32_t n_ranks,
+                                                     int32_t flags, uint32_t* union_mask, int32_t* cnt,
+                                                     int64_t* seg_offset, int64_t* seg_total,
+                                                     int64_t* volume_bytes, void* stream) {
+  Geometry g;
+  int rc = make_geometry(shape, &g);
+  if (rc != SPARSP_OK) return rc;
+  if (n_ranks < 1 || n_ranks > kPlanMaxRanks || (int64_t)g.B * n_ranks > kPlanMaxBatchRanks) {
+    set_error("sparsp_demand_plan_noalloc supports n_ranks <= %d and batch * n_ranks <= %d (got %d, %lld)",
+              kPlanMaxRanks, kPlanMaxBatchRanks, n_ranks, (long long)g.B * n_ranks);
+    return SPARSP_ERR_CAPACITY;
+  }
+  if (flags & ~SPARSP_INCLUDE_LOCAL) {
+    set_error("sparsp_demand_plan_noalloc accepts only SPARSP_INCLUDE_LOCAL (got 0x%x)", flags);
+    return SPARSP_ERR_INVALID_ARG;
+  }
+  if (!mask || !rank_of_block || !union_mask || !cnt || !seg_offset || !seg_total || !volume_bytes) {
+    set_error("sparsp_demand_plan_noalloc: NULL argument");
+    return SPARSP_ERR_INVALID_ARG;
+  }
+  if ((uintptr_t)seg_offset % 8 || (uintptr_t)seg_total % 8 || (uintptr_t)volume_bytes % 8 ||
+      (uintptr_t)mask % 4 || (uintptr_t)union_mask % 4 || (uintptr_t)cnt % 4 || (uintptr_t)rank_of_block % 4) {
+    set_error("sparsp_demand_plan_noalloc: misaligned argument");
+    return SPARSP_ERR_INVALID_ARG;
+  }
+  void* scratch = nullptr;
+  if ((rc = plan_scratch_address(&scratch)) != SPARSP_OK) return rc;
+  uint32_t* own = (uint32_t*)scratch;                                       // [P][Wd], fully rewritten
+  int64_t* ent_base = (int64_t*)((char*)scratch + kPlanOwnWords * sizeof(uint32_t));  // [B*P] + total
+  int64_t* n_entries = ent_base + kPlanMaxBatchRanks;
+  const int P = n_ranks;
+  const int include_local = (flags & SPARSP_INCLUDE_LOCAL) ? 1 : 0;
+  const int64_t entry_bytes = 2LL * g.b * g.d * 2;
+  cudaStream_t st = (cudaStream_t)stream;
+  own_kernel<<<(P * g.Wd + 127) / 128, 128, 0, st>>>(rank_of_block, g.NB, g.Wd, P, own);
+  const int64_t n_u = (int64_t)g.B * P * g.H * g.Wd;
+  union_kernel<<<(int)((n_u + 127) / 128), 128, 0, st>>>(mask, rank_of_block, g.B, g.H, g.NB, g.Wd, P, union_mask);
+  const int64_t n_c = (int64_t)g.B * P * P * g.H;
+  count_kernel<<<(int)((n_c + 127) / 128), 128, 0, st>>>(union_mask, own, g.B, g.H, g.Wd, P, cnt);
+  scan_kernel<<<1, 1024, 0, st>>>(cnt, g.B, g.H, P, include_local, entry_bytes, seg_offset, seg_total,
+                                  volume_bytes, ent_base, n_entries);
+  count_launch(4);
+  SPARSP_CUDA_OK(cudaGetLastError());
+  return SPARSP_OK;
+}
