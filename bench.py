@@ -32,7 +32,10 @@ FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustain
 NOMINAL = {"hbm_gbs": 8000.0, "bf16_tflops": 2250.0}
 # dram__bytes_read.sum + dram__bytes_write.sum per launch of the attention kernel, from the ncu
 # captures summarised under profiles/ (None = not captured for that workload).
-ATTN_DRAM_TRAFFIC = {}
+ATTN_DRAM_TRAFFIC = {
+    ("mid", 58): 588.8e6,            # profiles/attn_fwd_kernel_mid_and_hunyuan4.md, full workload
+    ("hunyuan", 93): 6 * 722.2e6,     # same file: 4-head capture scaled by heads (24 / 4)
+}
 
 
 def load_peaks():
@@ -133,7 +136,7 @@ def run_ours(args):
     import torch
     import torch.distributed as dist
 
-    from paper_2609_32197_b200 import binding, synth
+    from paper_2609_32197_b200 import binding, dist_util, synth
 
     rank = int(os.environ.get("RANK", 0))
     world = int(os.environ.get("WORLD_SIZE", 1))
@@ -145,9 +148,7 @@ def run_ours(args):
     binding.lib()
 
     wl, placement = resolve_workload(args)
-    if rank != 0:  # every rank its own replica of the workload
-        wl = synth.Workload(wl.name, wl.heads, wl.head_dim, wl.grid, wl.n_text, wl.block, wl.topk_abs,
-                            wl.topk_pct, wl.ranks, wl.placements, seed=wl.seed + rank)
+    wl = dist_util.replica_workload(wl, rank)  # every rank its own replica of the workload
     H, d, b, P = wl.heads, wl.head_dim, wl.block, wl.ranks
     shape = binding.make_shape(H, d, wl.grid, wl.n_text, b)
     g = binding.sparsp_geometry(shape)
@@ -281,15 +282,13 @@ def run_ours(args):
         e2e_ms = e0.elapsed_time(e1) / e2e_steps
 
     # max over ranks (device-timed), whole-job totals
-    if world > 1:
-        t = torch.tensor([total_ms, e2e_ms, attn_ms, pack_ms, mask_ms], dtype=torch.float64, device=dev)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        total_ms, e2e_ms, attn_ms, pack_ms, mask_ms = t.tolist()
-        f = torch.tensor([flops, float(launches)], dtype=torch.float64, device=dev)
-        dist.all_reduce(f, op=dist.ReduceOp.SUM)
-        flops_all, launches_all = f.tolist()
-    else:
-        flops_all, launches_all = flops, launches
+    tm, tot = dist_util.reduce_over_ranks(
+        {"total": total_ms, "e2e": e2e_ms if e2e_ms == e2e_ms else 0.0, "attn": attn_ms, "pack": pack_ms, "mask": mask_ms},
+        {"flops": flops, "launches": float(launches)}, dev)
+    total_ms, attn_ms, pack_ms, mask_ms = tm["total"], tm["attn"], tm["pack"], tm["mask"]
+    if e2e_ms == e2e_ms:
+        e2e_ms = tm["e2e"]
+    flops_all, launches_all = tot["flops"], tot["launches"]
     ms_per_step = total_ms / args.steps
 
     peaks = load_peaks()
