@@ -213,3 +213,65 @@ def test_invalid_arguments_are_rejected_on_the_host(binding):
                                    d["union_mask"], d["cnt"], d["seg_offset"], d["seg_total"], d["volume_bytes"],
                                    x, 16, None, ws)
     assert e.value.code == binding.SPARSP_ERR_INVALID_ARG
+
+
+def _stack_batches(xs, layout):
+    """list of [H][N][d] CPU tensors -> device tensor [B][H][N][d] or [B][N][H][d]"""
+    t = torch.stack(xs, 0).cuda()
+    return t.contiguous() if layout == "HND" else t.permute(0, 2, 1, 3).contiguous()
+
+
+@pytest.mark.parametrize("layout", ["HND", "NHD"])
+def test_batch_of_two(oracle_mod, binding, layout):
+    """Batch is an independent outer dimension: each batch item must match the oracle run on it alone."""
+    b, d, H, P, k = 64, 64, 2, 3, 4
+    wls = [_workload("b0", H, d, (3, 9, 13), 40, b, k, P, seed=31), _workload("b1", H, d, (3, 9, 13), 40, b, k, P, seed=32)]
+    data = [_gen(w) for w in wls]
+    N, NB = wls[0].n_tokens, wls[0].n_blocks
+    shape = binding.make_shape(H, d, wls[0].grid, 40, b, batch=2, layout=layout)
+    Qd, Kd, Vd = (_stack_batches([x[i] for x in data], layout) for i in range(3))
+    ws = binding.make_workspace(shape, P)
+    mo = binding.alloc_mask_outputs(shape, k, with_list=True, with_pooled=True)
+    binding.sparsp_block_mask(shape, Qd, Kd, k, mo["mask"], mo["kv_list"], mo["kv_count"], mo["pooled_q"],
+                              mo["pooled_k"], ws)
+    rank = np.array([(j * 2) % P for j in range(NB)], np.int32)
+    dg = pu.gpu_demand_pack(binding, shape, mo["mask"], torch.as_tensor(rank).cuda(), P, 0, Kd, Vd, ws)
+    Od = torch.zeros_like(Qd)
+    lse = torch.zeros(2, H, N, dtype=torch.float32, device="cuda")
+    binding.sparsp_sparse_attn_fwd(shape, Qd, Kd, Vd, mo["mask"], 0.0, Od, lse, ws)
+    torch.cuda.synchronize()
+    assert binding.sparsp_status(ws) == binding.SPARSP_OK
+    entry = 2 * b * d * 2
+    packed = dg["packed"].cpu().numpy()
+    cursor = 0
+    for bi, (Q, K, V) in enumerate(data):
+        ref = oracle_mod.block_mask(Q, K, b, k, 40)
+        assert np.array_equal(pu.u32(mo["mask"][bi]), ref["mask"])
+        assert np.array_equal(mo["kv_list"][bi].cpu().numpy(), ref["kv_list"])
+        assert np.array_equal(mo["pooled_k"][bi].cpu().numpy().view(np.uint32), ref["pk"].view(np.uint32))
+        dref = oracle_mod.demand(ref["mask"], rank, P, b, d)
+        assert np.array_equal(pu.u32(dg["union_mask"][bi]), dref["U"])
+        assert np.array_equal(dg["cnt"][bi].cpu().numpy(), dref["cnt"])
+        assert np.array_equal(dg["seg_offset"][bi].cpu().numpy(), dref["seg_off"])
+        assert np.array_equal(dg["volume_bytes"][bi].cpu().numpy(), dref["volume"])
+        pref = oracle_mod.pack(K, V, dref["U"], rank, b, P, dref["total"])
+        assert np.array_equal(packed[cursor:cursor + pref.size], pref), f"packed bytes of batch item {bi}"
+        cursor += pref.size
+        O_b = Od[bi] if layout == "HND" else Od[bi].permute(1, 0, 2)
+        units = [(h, i) for h in range(H) for i in range(NB)]
+        pu.check_attn_units(oracle_mod, Q, K, V, ref["mask"], b, O_b, units, lse_gpu=lse[bi])
+    assert (packed[cursor:] == 0xAB).all()
+
+
+def test_degenerate_shapes(oracle_mod, binding):
+    """One block only; k = 1; a virtual rank that owns nothing; odd block count with block = 128."""
+    # (a) a single ragged block: NB = 1, k = 1, P = 2 (rank 1 owns nothing)
+    wl = _workload("one", 2, 128, (1, 5, 9), 0, 128, 1, 2, seed=41)  # 45 tokens
+    _run_all(oracle_mod, binding, wl, np.zeros(1, np.int32))
+    # (b) k = 1 on several blocks, odd NB with block 128 (the last CTA holds a single query block)
+    wl = _workload("odd", 2, 64, (3, 10, 21), 0, 128, 1, 4, seed=42)  # 630 tokens -> 5 blocks
+    _run_all(oracle_mod, binding, wl, np.array([0, 0, 2, 2, 3], np.int32))  # rank 1 owns nothing
+    # (c) odd NB with block 64: the last stacked Q tile has an empty lower half
+    wl = _workload("odd64", 2, 128, (3, 10, 21), 0, 64, 2, 2, seed=43)  # 630 tokens -> 10 blocks ... use 9
+    wl = _workload("odd64", 2, 128, (3, 9, 21), 0, 64, 2, 2, seed=43)  # 567 tokens -> 9 blocks
+    _run_all(oracle_mod, binding, wl, oracle_mod.placement_contiguous(9, 2))
