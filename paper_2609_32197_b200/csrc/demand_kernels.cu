@@ -172,16 +172,64 @@ int launch_demand(const Geometry& g, const uint32_t* mask, const int32_t* rank_o
 }
 
 // ------------------------------------------------------------------------------------------------
-// Gather.  Work item = one K or V tile of one entry (block x d bf16 = 8..32 KiB).  Persistent CTAs
-// stride over the items; a CTA moves a tile with 16-byte loads and stores, kUnroll independent loads
-// in flight per thread, fully coalesced when a tile's rows are adjacent in memory.  Rows at or
-// beyond N are written as zeros.
+// Gather.  All K and V tiles of all entries form one flat sequence of 16-byte vectors (tile t of the
+// sequence = K or V tile of entry t/2).  Persistent CTAs take chunks of kPackThreads * kPackUnroll
+// consecutive vectors, so the bytes in flight per SM do not depend on the tile size (8..32 KiB); loads
+// and stores are fully coalesced when a tile's rows are adjacent in memory.  Rows at or beyond N are
+// written as zeros.
 // ------------------------------------------------------------------------------------------------
 constexpr int kPackThreads = 256;
 constexpr int kPackUnroll = 8;
 
 template <int D>
 __global__ void __launch_bounds__(kPackThreads) pack_kernel(
+    const __nv_bfloat16* __restrict__ K, const __nv_bfloat16* __restrict__ V,
+    const PackEntry* __restrict__ entries, const int64_t* __restrict__ n_entries_p, int H, int b,
+    int64_t N, int64_t sB, int64_t sH, int64_t sT, unsigned char* __restrict__ packed) {
+  constexpr int VPR = D / 8;                // 16-byte vectors per row
+  const int vpt = b * VPR;                  // vectors per tile (a power of two)
+  const int vpt_shift = 31 - __clz(vpt);
+  const int64_t n_vec = 2 * (*n_entries_p) * (int64_t)vpt;
+  constexpr int64_t kChunk = (int64_t)kPackThreads * kPackUnroll;
+  for (int64_t base = (int64_t)blockIdx.x * kChunk; base < n_vec; base += (int64_t)gridDim.x * kChunk) {
+    uint4 buf[kPackUnroll];
+    uint4* dst[kPackUnroll];
+#pragma unroll
+    for (int u = 0; u < kPackUnroll; ++u) {
+      const int64_t g = base + u * kPackThreads + threadIdx.x;
+      buf[u] = make_uint4(0u, 0u, 0u, 0u);
+      dst[u] = nullptr;
+      if (g < n_vec) {
+        const int64_t tile = g >> vpt_shift;
+        const int v = (int)(g & (vpt - 1));
+        const int4 raw = __ldg(reinterpret_cast<const int4*>(entries) + (tile >> 1));
+        PackEntry e;
+        e.dst_byte = (int64_t)(((uint64_t)(uint32_t)raw.y << 32) | (uint32_t)raw.x);
+        e.bh = raw.z;
+        e.j = raw.w;
+        if (e.j >= 0) {
+          const int which = (int)(tile & 1);
+          const int row = v / VPR, col = v % VPR;
+          const int64_t tok = (int64_t)e.j * b + row;
+          dst[u] = reinterpret_cast<uint4*>(packed + e.dst_byte + (int64_t)which * vpt * 16) + v;
+          if (tok < N) {
+            const int64_t batch = e.bh / H, head = e.bh % H;
+            const __nv_bfloat16* src = (which ? V : K) + batch * sB + head * sH + tok * sT;
+            buf[u] = __ldcs(reinterpret_cast<const uint4*>(src) + col);
+          }
+        }
+      }
+    }
+#pragma unroll
+    for (int u = 0; u < kPackUnroll; ++u)
+      if (dst[u]) __stcs(dst[u], buf[u]);
+  }
+}
+
+// Per-tile variant for large tiles (>= 16 KiB): one K or V tile per CTA step, the entry record is read
+// once per tile.  Measured faster than the flat variant when a tile alone fills a CTA's loads in flight.
+template <int D>
+__global__ void __launch_bounds__(kPackThreads) pack_tile_kernel(
     const __nv_bfloat16* __restrict__ K, const __nv_bfloat16* __restrict__ V,
     const PackEntry* __restrict__ entries, const int64_t* __restrict__ n_entries_p, int H, int b,
     int64_t N, int64_t sB, int64_t sH, int64_t sT, unsigned char* __restrict__ packed) {
@@ -229,14 +277,23 @@ int launch_pack(const sparsp_shape& s, const Geometry& g, const void* K, const v
   const int grid = sms * 8;
   auto k = (const __nv_bfloat16*)K;
   auto v = (const __nv_bfloat16*)V;
-  if (g.d == 64)
-    pack_kernel<64><<<grid, kPackThreads, 0, st>>>(k, v, entries, n_entries, g.H, g.b, g.N,
-                                                   s.stride_batch, s.stride_head, s.stride_token,
-                                                   (unsigned char*)packed);
-  else
-    pack_kernel<128><<<grid, kPackThreads, 0, st>>>(k, v, entries, n_entries, g.H, g.b, g.N,
-                                                    s.stride_batch, s.stride_head, s.stride_token,
-                                                    (unsigned char*)packed);
+  const bool small_tiles = g.b * g.d / 8 < 1024;  // 8 KiB tiles: several tiles per CTA step
+  unsigned char* out = (unsigned char*)packed;
+  if (small_tiles) {
+    if (g.d == 64)
+      pack_kernel<64><<<grid, kPackThreads, 0, st>>>(k, v, entries, n_entries, g.H, g.b, g.N, s.stride_batch,
+                                                     s.stride_head, s.stride_token, out);
+    else
+      pack_kernel<128><<<grid, kPackThreads, 0, st>>>(k, v, entries, n_entries, g.H, g.b, g.N, s.stride_batch,
+                                                      s.stride_head, s.stride_token, out);
+  } else {
+    if (g.d == 64)
+      pack_tile_kernel<64><<<grid, kPackThreads, 0, st>>>(k, v, entries, n_entries, g.H, g.b, g.N,
+                                                          s.stride_batch, s.stride_head, s.stride_token, out);
+    else
+      pack_tile_kernel<128><<<grid, kPackThreads, 0, st>>>(k, v, entries, n_entries, g.H, g.b, g.N,
+                                                           s.stride_batch, s.stride_head, s.stride_token, out);
+  }
   count_launch();
   SPARSP_CUDA_OK(cudaGetLastError());
   return SPARSP_OK;
