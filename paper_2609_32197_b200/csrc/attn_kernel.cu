@@ -43,8 +43,14 @@ constexpr int kAttnThreads = 608;
 constexpr int kIssuer1Warp = 18;  // warp 1 issues the MMAs of stream 0, warp 18 those of stream 1
 constexpr int kTmemCols = 512;
 constexpr float kGrowThreshold = 8.0f;
-constexpr long long kStaggerCycles = 6000;
-constexpr unsigned kSoftmaxSleepNs = 40;
+// Tuning switches (compile-time): packed fp32x2 arithmetic in the exponential loop, and how many of
+// the exponentials go to the FMA pipe instead of the special-function unit (every n-th pair; 0 = none).
+#ifndef SPARSP_TUNE_F32X2
+#define SPARSP_TUNE_F32X2 1
+#endif
+#ifndef SPARSP_TUNE_POLY
+#define SPARSP_TUNE_POLY 4
+#endif
 
 template <int D, int BLK>
 struct AttnCfg {
@@ -82,6 +88,45 @@ __device__ unsigned long long g_attn_prof[16];
 #define PROF_T(var)
 #define PROF_ADD(slot, a, b)
 #endif
+
+// Packed fp32 pairs (one instruction for two lanes' worth of fused multiply-add / add).
+__device__ __forceinline__ float2 ffma2(float2 a, float2 b, float2 c) {
+  unsigned long long ra, rb, rc, rd;
+  float2 d;
+  asm("mov.b64 %0, {%1, %2};" : "=l"(ra) : "f"(a.x), "f"(a.y));
+  asm("mov.b64 %0, {%1, %2};" : "=l"(rb) : "f"(b.x), "f"(b.y));
+  asm("mov.b64 %0, {%1, %2};" : "=l"(rc) : "f"(c.x), "f"(c.y));
+  asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(rd) : "l"(ra), "l"(rb), "l"(rc));
+  asm("mov.b64 {%0, %1}, %2;" : "=f"(d.x), "=f"(d.y) : "l"(rd));
+  return d;
+}
+__device__ __forceinline__ float2 fadd2(float2 a, float2 b) {
+  unsigned long long ra, rb, rd;
+  float2 d;
+  asm("mov.b64 %0, {%1, %2};" : "=l"(ra) : "f"(a.x), "f"(a.y));
+  asm("mov.b64 %0, {%1, %2};" : "=l"(rb) : "f"(b.x), "f"(b.y));
+  asm("add.rn.f32x2 %0, %1, %2;" : "=l"(rd) : "l"(ra), "l"(rb));
+  asm("mov.b64 {%0, %1}, %2;" : "=f"(d.x), "=f"(d.y) : "l"(rd));
+  return d;
+}
+
+// 2^x for a pair of fp32 values on the FMA/ALU pipes (no special-function unit): round-to-nearest
+// split x = i + f, f in [-0.5, 0.5], cubic minimax polynomial for 2^f (relative error 7.5e-5, far
+// below bf16 rounding), exponent added into the bit pattern.  x is clamped at -126 (result >= 2^-126).
+__device__ __forceinline__ float2 exp2_poly2(float2 x) {
+  const float kMagic = 12582912.0f;  // 1.5 * 2^23: adding it rounds to an integer in the low mantissa bits
+  x.x = fmaxf(x.x, -126.0f);
+  x.y = fmaxf(x.y, -126.0f);
+  const float2 t = fadd2(x, make_float2(kMagic, kMagic));
+  const float2 fi = fadd2(t, make_float2(-kMagic, -kMagic));
+  const float2 f = fadd2(x, make_float2(-fi.x, -fi.y));
+  float2 q = ffma2(f, make_float2(0.0551716685f, 0.0551716685f), make_float2(0.2426111251f, 0.2426111251f));
+  q = ffma2(q, f, make_float2(0.6932609677f, 0.6932609677f));
+  q = ffma2(q, f, make_float2(0.9999280572f, 0.9999280572f));
+  q.x = __int_as_float(__float_as_int(q.x) + (__float_as_int(t.x) << 23));
+  q.y = __int_as_float(__float_as_int(q.y) + (__float_as_int(t.y) << 23));
+  return q;
+}
 
 __device__ __forceinline__ void named_bar_sync(int id, int n) {
   asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(n) : "memory");
@@ -288,13 +333,6 @@ __global__ void __maxnreg__(96)
       };
 
       mbar_wait_bounded(bar_q, 0, s_abort, p.status, 11, p.wait_limit);
-      if (s == 1) {
-        // start stream 1 half a period late, so that its exponentials fall into stream 0's MMA
-        // phase instead of competing with stream 0's exponentials for the special-function unit
-        const long long t0 = clock64();
-        while (!mbar_test_wait(p_full + 0, 0) && clock64() - t0 < kStaggerCycles) {
-        }
-      }
       for (int n = 0; n < n_tiles; ++n) {
         const bool keep = (stream_mask(n) >> s) & 1;
         while (vdone < n - 1) handle_v(vdone++);  // a V stage is released at most two steps after its fill
@@ -358,7 +396,7 @@ __global__ void __maxnreg__(96)
       const int valid[2] = {min(nv, 32), max(nv - 32, 0)};
 
       PROF_T(t_a);
-      mbar_wait_bounded(s_full + sidx, cnt & 1, s_abort, p.status, 30 + sidx, p.wait_limit, kSoftmaxSleepNs);
+      mbar_wait_bounded(s_full + sidx, cnt & 1, s_abort, p.status, 30 + sidx, p.wait_limit);
       tc_fence_after();
       PROF_T(t_b);
 #ifdef SPARSP_ATTN_NOSOFTMAX  // tuning builds only: measure the MMA / TMA pipeline alone
@@ -413,12 +451,26 @@ __global__ void __maxnreg__(96)
       // exponentials; bf16 P overwrites S in place: my keys [64*half, 64*half+64) go to columns
       // [32*half, 32*half+32)
       float lsum = 0.0f;
+      float2 lsum2 = make_float2(0.0f, 0.0f);
       const float neg_m = -m_used;
 #pragma unroll
       for (int c = 0; c < 2; ++c) {
         uint32_t pk[16];
         const float* svc = sv + c * 32;
         if (valid[c] == 32) {
+#if SPARSP_TUNE_F32X2
+          const float2 sc2 = make_float2(p.scale_log2, p.scale_log2), nm2 = make_float2(neg_m, neg_m);
+#pragma unroll
+          for (int e = 0; e < 16; ++e) {
+            const float2 x = ffma2(make_float2(svc[2 * e], svc[2 * e + 1]), sc2, nm2);
+            const float2 pp = (SPARSP_TUNE_POLY > 0 && (e % (SPARSP_TUNE_POLY > 0 ? SPARSP_TUNE_POLY : 1)) == 1)
+                                  ? exp2_poly2(x)
+                                  : make_float2(ex2(x.x), ex2(x.y));
+            lsum2 = fadd2(lsum2, pp);
+            const __nv_bfloat162 h2 = __floats2bfloat162_rn(pp.x, pp.y);
+            pk[e] = *reinterpret_cast<const uint32_t*>(&h2);
+          }
+#else
 #pragma unroll
           for (int e = 0; e < 16; ++e) {
             const float p0 = ex2(fmaf(svc[2 * e], p.scale_log2, neg_m));
@@ -427,6 +479,7 @@ __global__ void __maxnreg__(96)
             const __nv_bfloat162 h2 = __floats2bfloat162_rn(p0, p1);
             pk[e] = *reinterpret_cast<const uint32_t*>(&h2);
           }
+#endif
         } else if (valid[c] > 0) {
 #pragma unroll
           for (int e = 0; e < 16; ++e) {
@@ -442,7 +495,7 @@ __global__ void __maxnreg__(96)
         }
         tmem_st16(tS + half * 32 + c * 16, pk);
       }
-      l_run += lsum;
+      l_run += lsum + (lsum2.x + lsum2.y);
       PROF_T(t_e);
       tmem_st_wait();
       tc_fence_before();
