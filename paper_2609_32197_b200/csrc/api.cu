@@ -90,6 +90,8 @@ WsLayout make_layout(const Geometry& g, int P) {
   off += align_up(pooled, 256);
   L.pooled_k = off;
   off += align_up(pooled, 256);
+  L.scores = off;  // pooled-Q x pooled-K^T, fp32 [B][H][NB][NB]
+  off += align_up((int64_t)g.B * g.H * g.NB * g.NB * 4, 256);
   L.own = off;
   off += align_up((int64_t)P * g.Wd * 4, 256);
   L.ent_base = off;
@@ -196,7 +198,7 @@ int sparsp_block_mask(const sparsp_shape* shape, const void* Q, const void* K, i
   float* pk = pooled_k ? pooled_k : (float*)(ws + L.pooled_k);
   cudaStream_t st = (cudaStream_t)stream;
   SPARSP_TRY(launch_pool(*shape, g, Q, K, pq, pk, st));
-  SPARSP_TRY(launch_score_topk(g, pq, pk, topk_video, mask, kv_list, kv_count, st));
+  SPARSP_TRY(launch_score_topk(g, pq, pk, (float*)(ws + L.scores), topk_video, mask, kv_list, kv_count, st));
   return SPARSP_OK;
 }
 

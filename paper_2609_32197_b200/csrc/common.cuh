@@ -34,7 +34,7 @@ struct PackEntry {
 };
 
 struct WsLayout {
-  int64_t status, pooled_q, pooled_k, own, ent_base, n_entries, entries, total;
+  int64_t status, pooled_q, pooled_k, scores, own, ent_base, n_entries, entries, total;
 };
 
 void set_error(const char* fmt, ...);
@@ -57,8 +57,8 @@ inline int64_t align_up(int64_t x, int64_t a) { return (x + a - 1) / a * a; }
 // launchers implemented in the kernel files -------------------------------------------------
 int launch_pool(const sparsp_shape& s, const Geometry& g, const void* Q, const void* K, float* pq,
                 float* pk, cudaStream_t st);
-int launch_score_topk(const Geometry& g, const float* pq, const float* pk, int topk, uint32_t* mask,
-                      int32_t* kv_list, int32_t* kv_count, cudaStream_t st);
+int launch_score_topk(const Geometry& g, const float* pq, const float* pk, float* scores, int topk,
+                      uint32_t* mask, int32_t* kv_list, int32_t* kv_count, cudaStream_t st);
 int launch_demand(const Geometry& g, const uint32_t* mask, const int32_t* rank_of_block, int P,
                   int flags, uint32_t* U, int32_t* cnt, int64_t* seg_off, int64_t* seg_total,
                   int64_t* volume, const int64_t* dst_base, int64_t capacity, char* ws,

@@ -1,4 +1,5 @@
-// Step 1: mean-pool Q and K per block, score pooled-Q x pooled-K^T per head, warp-level top-k.
+// Step 1: mean-pool Q and K per block, score pooled-Q x pooled-K^T per head (fp32 SIMT GEMM with a
+// fixed accumulation order), warp-level top-k per row.
 //
 // Arithmetic contract (the result decides which blocks are kept, so it is fixed to the operation):
 //   pool : fp32 sum of the block's valid tokens in ascending token order starting from 0, then one
@@ -96,14 +97,81 @@ int launch_pool(const sparsp_shape& s, const Geometry& g, const void* Q, const v
 }
 
 // ------------------------------------------------------------------------------------------------
-// score + top-k.  A CTA owns ROWS = WARPS*RPW query blocks of one (batch, head); pooled K streams
-// through shared memory in 32-block tiles; lane l of a warp computes the scores of column l of the
-// tile for the warp's RPW rows.  Scores stay in shared memory as order-preserving uint32 keys and
-// the warp then selects its rows' k largest by a 32-step radix search with ballots.
+// score: S[bh][i][j] = sum_c pQ[i][c] * pK[j][c] as one fused-multiply-add chain per output, c
+// ascending (a no-split-K SIMT GEMM).  A CTA computes a 64 x 64 tile; a thread owns 4 rows x 4
+// columns (columns tx, tx+16, tx+32, tx+48 so that its 16-byte shared-memory reads of pooled K never
+// conflict), i.e. 16 independent chains fed by 8 vector loads per 4 channels.  Scores go to a
+// workspace buffer: at most 83 MB, written and read once, ~25 us of HBM time on the largest workload.
 // ------------------------------------------------------------------------------------------------
-constexpr int kScoreWarps = 8;
-constexpr int kScoreRPW = 2;
-constexpr int kScoreRows = kScoreWarps * kScoreRPW;
+constexpr int kScoreTile = 64;
+constexpr int kScoreThreads = 256;
+
+template <int D>
+__global__ void __launch_bounds__(kScoreThreads) score_kernel(const float* __restrict__ pq,
+                                                              const float* __restrict__ pk, int NB,
+                                                              float* __restrict__ scores) {
+  constexpr int LD = D + 4;  // row pitch in floats: 16 bytes of skew per row
+  extern __shared__ __align__(16) unsigned char smem_raw[];
+  float* sQ = reinterpret_cast<float*>(smem_raw);  // [64][LD]
+  float* sK = sQ + kScoreTile * LD;                // [64][LD]
+  const int64_t bh = blockIdx.z;
+  const int row0 = blockIdx.y * kScoreTile, col0 = blockIdx.x * kScoreTile;
+  const int tx = threadIdx.x & 15, ty = threadIdx.x >> 4;
+
+  for (int idx = threadIdx.x; idx < kScoreTile * (D / 4); idx += kScoreThreads) {
+    const int r = idx / (D / 4), c4 = idx % (D / 4);
+    float4 q = make_float4(0.f, 0.f, 0.f, 0.f), k = q;
+    if (row0 + r < NB) q = __ldg(reinterpret_cast<const float4*>(pq + (bh * NB + row0 + r) * D) + c4);
+    if (col0 + r < NB) k = __ldg(reinterpret_cast<const float4*>(pk + (bh * NB + col0 + r) * D) + c4);
+    *reinterpret_cast<float4*>(sQ + r * LD + c4 * 4) = q;
+    *reinterpret_cast<float4*>(sK + r * LD + c4 * 4) = k;
+  }
+  __syncthreads();
+
+  float acc[4][4];
+#pragma unroll
+  for (int i = 0; i < 4; ++i)
+#pragma unroll
+    for (int j = 0; j < 4; ++j) acc[i][j] = 0.0f;
+
+#pragma unroll 4
+  for (int c = 0; c < D; c += 4) {
+    float4 q[4], k[4];
+#pragma unroll
+    for (int i = 0; i < 4; ++i) q[i] = *reinterpret_cast<const float4*>(sQ + (ty * 4 + i) * LD + c);
+#pragma unroll
+    for (int j = 0; j < 4; ++j) k[j] = *reinterpret_cast<const float4*>(sK + (tx + 16 * j) * LD + c);
+#pragma unroll
+    for (int i = 0; i < 4; ++i)
+#pragma unroll
+      for (int j = 0; j < 4; ++j) {
+        float a = acc[i][j];
+        a = __fmaf_rn(q[i].x, k[j].x, a);
+        a = __fmaf_rn(q[i].y, k[j].y, a);
+        a = __fmaf_rn(q[i].z, k[j].z, a);
+        a = __fmaf_rn(q[i].w, k[j].w, a);
+        acc[i][j] = a;
+      }
+  }
+#pragma unroll
+  for (int i = 0; i < 4; ++i) {
+    const int r = row0 + ty * 4 + i;
+    if (r >= NB) continue;
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+      const int cidx = col0 + tx + 16 * j;
+      if (cidx < NB) scores[(bh * NB + r) * NB + cidx] = acc[i][j];
+    }
+  }
+}
+
+// ------------------------------------------------------------------------------------------------
+// top-k: one warp per (batch, head, query block) row.  The row's scores become order-preserving
+// uint32 keys in shared memory; the warp finds the k-th largest key by a 32-step radix search with
+// ballots/popcounts, breaks ties towards the lower index, forces the text blocks on, and emits the
+// mask words and the ascending kept list by ballot-prefix compaction.
+// ------------------------------------------------------------------------------------------------
+constexpr int kTopkWarps = 8;
 
 __device__ __forceinline__ uint32_t score_key(float s) {
   if (s == 0.0f) s = 0.0f;  // -0 -> +0 so that they compare equal
@@ -111,107 +179,83 @@ __device__ __forceinline__ uint32_t score_key(float s) {
   return (u & 0x80000000u) ? ~u : (u | 0x80000000u);
 }
 
-template <int D>
-__global__ void __launch_bounds__(kScoreWarps * 32) score_topk_kernel(
-    const float* __restrict__ pq, const float* __restrict__ pk, int NB, int Wd, int nb_cand, int topk,
-    int kept_cap, uint32_t* __restrict__ mask, int32_t* __restrict__ kv_list,
-    int32_t* __restrict__ kv_count) {
+__global__ void __launch_bounds__(kTopkWarps * 32) topk_kernel(const float* __restrict__ scores, int64_t n_rows,
+                                                               int NB, int Wd, int nb_cand, int topk,
+                                                               int kept_cap, uint32_t* __restrict__ mask,
+                                                               int32_t* __restrict__ kv_list,
+                                                               int32_t* __restrict__ kv_count) {
   extern __shared__ __align__(16) unsigned char smem_raw[];
-  float* sQ = reinterpret_cast<float*>(smem_raw);                 // [ROWS][D]
-  float* sK = sQ + kScoreRows * D;                                // [32][D+1]
-  uint32_t* sS = reinterpret_cast<uint32_t*>(sK + 32 * (D + 1));  // [ROWS][NBpad]
   const int NBpad = Wd * 32;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const int64_t bh = blockIdx.y;
-  const int row0 = blockIdx.x * kScoreRows;
-
-  for (int idx = threadIdx.x; idx < kScoreRows * D; idx += blockDim.x) {
-    const int r = row0 + idx / D;
-    sQ[idx] = r < NB ? pq[(bh * NB + r) * D + idx % D] : 0.0f;
-  }
-
+  uint32_t* keys = reinterpret_cast<uint32_t*>(smem_raw) + warp * NBpad;
+  const int64_t row = (int64_t)blockIdx.x * kTopkWarps + warp;  // (batch*H + head) * NB + i
+  if (row >= n_rows) return;
+  const float* srow = scores + row * NB;
   for (int t = 0; t < Wd; ++t) {
-    __syncthreads();
-    for (int idx = threadIdx.x; idx < 32 * D; idx += blockDim.x) {
-      const int jj = idx / D, c = idx % D;
-      const int j = t * 32 + jj;
-      sK[jj * (D + 1) + c] = j < NB ? pk[(bh * NB + j) * D + c] : 0.0f;
-    }
-    __syncthreads();
-    float acc[kScoreRPW];
-#pragma unroll
-    for (int r = 0; r < kScoreRPW; ++r) acc[r] = 0.0f;
-    const float* kcol = sK + lane * (D + 1);
-#pragma unroll 8
-    for (int c = 0; c < D; ++c) {
-      const float kv = kcol[c];
-#pragma unroll
-      for (int r = 0; r < kScoreRPW; ++r)
-        acc[r] = __fmaf_rn(sQ[(warp * kScoreRPW + r) * D + c], kv, acc[r]);
-    }
-#pragma unroll
-    for (int r = 0; r < kScoreRPW; ++r)
-      sS[(warp * kScoreRPW + r) * NBpad + t * 32 + lane] = score_key(acc[r]);
+    const int j = t * 32 + lane;
+    keys[j] = j < NB ? score_key(__ldcs(srow + j)) : 0u;
   }
   __syncwarp();
 
   const uint32_t lt_mask = (1u << lane) - 1u;
-  for (int r = 0; r < kScoreRPW; ++r) {
-    const int i = row0 + warp * kScoreRPW + r;
-    if (i >= NB) break;  // warp-uniform
-    const uint32_t* keys = sS + (warp * kScoreRPW + r) * NBpad;
-    // largest T with |{ candidates : key >= T }| >= topk  ==> T is the topk-th largest key
-    uint32_t T = 0;
-    for (int bit = 31; bit >= 0; --bit) {
-      const uint32_t trial = T | (1u << bit);
-      int c = 0;
-      for (int t = 0; t < Wd; ++t) {
-        const int j = t * 32 + lane;
-        c += (j < nb_cand && keys[j] >= trial) ? 1 : 0;
-      }
-      c = __reduce_add_sync(0xffffffffu, c);
-      if (c >= topk) T = trial;
-    }
-    int gt = 0;
+  // largest T with |{ candidates : key >= T }| >= topk  ==> T is the topk-th largest key
+  uint32_t T = 0;
+  for (int bit = 31; bit >= 0; --bit) {
+    const uint32_t trial = T | (1u << bit);
+    int c = 0;
     for (int t = 0; t < Wd; ++t) {
       const int j = t * 32 + lane;
-      gt += (j < nb_cand && keys[j] > T) ? 1 : 0;
+      c += (j < nb_cand && keys[j] >= trial) ? 1 : 0;
     }
-    gt = __reduce_add_sync(0xffffffffu, gt);
-    const int need_eq = topk - gt;  // ties at T taken in ascending index order
-    int eq_seen = 0, out_pos = 0;
-    const int64_t row = bh * NB + i;
-    for (int t = 0; t < Wd; ++t) {
-      const int j = t * 32 + lane;
-      const bool cand = j < nb_cand;
-      const uint32_t key = keys[j];
-      const bool is_eq = cand && key == T;
-      const uint32_t eq_ballot = __ballot_sync(0xffffffffu, is_eq);
-      const bool take_eq = is_eq && (eq_seen + __popc(eq_ballot & lt_mask) < need_eq);
-      eq_seen += __popc(eq_ballot);
-      const bool keep = (cand && key > T) || take_eq || (j >= nb_cand && j < NB);
-      const uint32_t word = __ballot_sync(0xffffffffu, keep);
-      if (lane == 0) mask[row * Wd + t] = word;
-      if (kv_list && keep) {
-        const int pos = out_pos + __popc(word & lt_mask);
-        if (pos < kept_cap) kv_list[row * kept_cap + pos] = j;
-      }
-      out_pos += __popc(word);
-    }
-    if (kv_count && lane == 0) kv_count[row] = out_pos;
+    c = __reduce_add_sync(0xffffffffu, c);
+    if (c >= topk) T = trial;
   }
+  int gt = 0;
+  for (int t = 0; t < Wd; ++t) {
+    const int j = t * 32 + lane;
+    gt += (j < nb_cand && keys[j] > T) ? 1 : 0;
+  }
+  gt = __reduce_add_sync(0xffffffffu, gt);
+  const int need_eq = topk - gt;  // ties at T taken in ascending index order
+  int eq_seen = 0, out_pos = 0;
+  for (int t = 0; t < Wd; ++t) {
+    const int j = t * 32 + lane;
+    const bool cand = j < nb_cand;
+    const uint32_t key = keys[j];
+    const bool is_eq = cand && key == T;
+    const uint32_t eq_ballot = __ballot_sync(0xffffffffu, is_eq);
+    const bool take_eq = is_eq && (eq_seen + __popc(eq_ballot & lt_mask) < need_eq);
+    eq_seen += __popc(eq_ballot);
+    const bool keep = (cand && key > T) || take_eq || (j >= nb_cand && j < NB);
+    const uint32_t word = __ballot_sync(0xffffffffu, keep);
+    if (lane == 0) mask[row * Wd + t] = word;
+    if (kv_list && keep) {
+      const int pos = out_pos + __popc(word & lt_mask);
+      if (pos < kept_cap) kv_list[row * kept_cap + pos] = j;
+    }
+    out_pos += __popc(word);
+  }
+  if (kv_count && lane == 0) kv_count[row] = out_pos;
 }
 
-int launch_score_topk(const Geometry& g, const float* pq, const float* pk, int topk, uint32_t* mask,
-                      int32_t* kv_list, int32_t* kv_count, cudaStream_t st) {
+int launch_score_topk(const Geometry& g, const float* pq, const float* pk, float* scores, int topk,
+                      uint32_t* mask, int32_t* kv_list, int32_t* kv_count, cudaStream_t st) {
   const int kept_cap = topk + (g.NB - g.nb_cand);
-  const size_t smem = (size_t)(kScoreRows * g.d + 32 * (g.d + 1) + kScoreRows * g.Wd * 32) * 4;
-  dim3 grid((g.NB + kScoreRows - 1) / kScoreRows, g.B * g.H);
-  auto kern = g.d == 64 ? score_topk_kernel<64> : score_topk_kernel<128>;
-  SPARSP_CUDA_OK(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
-  kern<<<grid, kScoreWarps * 32, smem, st>>>(pq, pk, g.NB, g.Wd, g.nb_cand, topk, kept_cap, mask,
-                                            kv_list, kv_count);
-  count_launch();
+  {
+    const size_t smem = (size_t)2 * kScoreTile * (g.d + 4) * 4;
+    const int nt = (g.NB + kScoreTile - 1) / kScoreTile;
+    dim3 grid(nt, nt, g.B * g.H);
+    auto kern = g.d == 64 ? score_kernel<64> : score_kernel<128>;
+    SPARSP_CUDA_OK(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+    kern<<<grid, kScoreThreads, smem, st>>>(pq, pk, g.NB, scores);
+  }
+  {
+    const int64_t n_rows = (int64_t)g.B * g.H * g.NB;
+    const size_t smem = (size_t)kTopkWarps * g.Wd * 32 * 4;
+    topk_kernel<<<(unsigned)((n_rows + kTopkWarps - 1) / kTopkWarps), kTopkWarps * 32, smem, st>>>(
+        scores, n_rows, g.NB, g.Wd, g.nb_cand, topk, kept_cap, mask, kv_list, kv_count);
+  }
+  count_launch(2);
   SPARSP_CUDA_OK(cudaGetLastError());
   return SPARSP_OK;
 }
