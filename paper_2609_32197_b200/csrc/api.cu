@@ -1,5 +1,8 @@
 // extern "C" entry points of the SparSP library: argument checking, workspace carving, launch order.
 #include <cstring>
+#include <map>
+#include <mutex>
+#include <utility>
 
 #include "common.cuh"
 
@@ -18,6 +21,22 @@ void set_error(const char* fmt, ...) {
 int cuda_fail(cudaError_t e, const char* what) {
   set_error("CUDA error %d (%s) in %s", (int)e, cudaGetErrorString(e), what);
   return SPARSP_ERR_CUDA;
+}
+
+cudaError_t ensure_dynamic_smem(const void* func, int bytes) {
+  static std::mutex mu;
+  static std::map<std::pair<const void*, int>, int> limit;
+  int dev = 0;
+  cudaError_t e = cudaGetDevice(&dev);
+  if (e != cudaSuccess) return e;
+  std::lock_guard<std::mutex> lock(mu);
+  int& cur = limit[std::make_pair(func, dev)];
+  if (bytes > cur) {
+    e = cudaFuncSetAttribute(func, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes);
+    if (e != cudaSuccess) return e;
+    cur = bytes;
+  }
+  return cudaSuccess;
 }
 
 int make_geometry(const sparsp_shape* s, Geometry* g) {
@@ -92,6 +111,8 @@ WsLayout make_layout(const Geometry& g, int P) {
   off += align_up(pooled, 256);
   L.scores = off;  // pooled-Q x pooled-K^T, fp32 [B][H][NB][NB]
   off += align_up((int64_t)g.B * g.H * g.NB * g.NB * 4, 256);
+  L.pairs = off;  // query-block pairs of the attention CTAs, int32 [B][H][ceil(NB/2)][2]
+  off += align_up((int64_t)g.B * g.H * ((g.NB + 1) / 2) * 2 * 4, 256);
   L.own = off;
   off += align_up((int64_t)P * g.Wd * 4, 256);
   L.ent_base = off;

@@ -29,6 +29,7 @@ using namespace ptx;
 
 struct AttnParams {
   const uint32_t* mask;
+  const int32_t* pairs;  // [B*H][ceil(NB/2)][2] query blocks of each CTA (second may be -1)
   __nv_bfloat16* O;
   float* lse;
   int32_t* status;
@@ -165,8 +166,10 @@ __global__ void __maxnreg__(96)
   PROF_T(t_cta0);
   const int bh = blockIdx.y;
   const int batch = bh / p.H, head = bh % p.H;
-  const int i0 = blockIdx.x * 2;  // first of the CTA's two query blocks
-  const int64_t q0 = (int64_t)i0 * BLK;
+  // the CTA's two query blocks (any two blocks of the head: a pairing pass picks partners whose kept
+  // lists overlap); blk[1] < 0 means the CTA has a single block
+  const int32_t* pr = p.pairs + ((int64_t)bh * gridDim.x + blockIdx.x) * 2;
+  const int blk[2] = {pr[0], pr[1]};
 
   // ---- setup ------------------------------------------------------------------------------
   if (tid == 0) {
@@ -193,14 +196,15 @@ __global__ void __maxnreg__(96)
     tmem_relinquish();
   }
   if (warp == 0) {
-    // union of the two mask rows -> ascending entry list; flag bit q = kept by query block i0 + q
-    const uint32_t* mrow = p.mask + ((int64_t)bh * p.NB + i0) * p.Wd;
+    // union of the two mask rows -> ascending entry list; flag bit q = kept by query block blk[q]
+    const uint32_t* mrow0 = p.mask + ((int64_t)bh * p.NB + blk[0]) * p.Wd;
+    const uint32_t* mrow1 = p.mask + ((int64_t)bh * p.NB + max(blk[1], 0)) * p.Wd;
     int running = 0;
     for (int w0 = 0; w0 < p.Wd; w0 += 32) {
       const int w = w0 + lane;
       uint32_t rb[2];
-      rb[0] = (w < p.Wd) ? mrow[w] : 0u;
-      rb[1] = (w < p.Wd && i0 + 1 < p.NB) ? mrow[p.Wd + w] : 0u;
+      rb[0] = (w < p.Wd) ? mrow0[w] : 0u;
+      rb[1] = (w < p.Wd && blk[1] >= 0) ? mrow1[w] : 0u;
       uint32_t u = rb[0] | rb[1];
       const int mine = __popc(u);
       int incl = mine;
@@ -235,11 +239,15 @@ __global__ void __maxnreg__(96)
     // ================================ TMA producer ========================================
     if (lane == 0 && n_tiles > 0) {
       mbar_expect_tx(bar_q, C::kQTiles * C::kQBytes);
+      // a Q tile is 128 rows: one 128-token block, or two 64-token blocks stacked (an absent second
+      // block re-reads the first: finite data whose rows are never used)
 #pragma unroll
-      for (int t = 0; t < C::kQTiles; ++t)
+      for (int q = 0; q < 2; ++q) {
+        const int tok = (blk[q] >= 0 ? blk[q] : blk[0]) * BLK;
+        unsigned char* dst = C::kSplitKV ? sQ + q * (BLK * 128) : sQ + q * C::kQBytes;
 #pragma unroll
-        for (int c = 0; c < D / 64; ++c)
-          tma_load_4d(sQ + t * C::kQBytes + c * 16384, &tmQ, bar_q, c * 64, (int)q0 + t * 128, head, batch);
+        for (int c = 0; c < D / 64; ++c) tma_load_4d(dst + c * 16384, &tmQ, bar_q, c * 64, tok, head, batch);
+      }
       auto load_tile = [&](unsigned char* dst, const CUtensorMap* tm, uint64_t* bar, int n) {
 #ifdef SPARSP_ATTN_NOLOAD  // tuning builds only: reuse stale tiles to take TMA traffic out of the picture
         if (n >= S) {
@@ -524,7 +532,7 @@ __global__ void __maxnreg__(96)
       // the row's two threads add their partial sums; each writes its half of the columns
       named_bar_sync(pair_bar, 64);
       const float l = l_run + sStat[(sidx * 2 + 1 - half) * 128 + row].y;
-      const int64_t tok = q0 + sidx * 128 + row;
+      const int64_t tok = blk[sidx] >= 0 ? (int64_t)blk[sidx] * BLK + row : p.N;
       const float inv_l = l > 0.0f ? 1.0f / l : 0.0f;
       __nv_bfloat16* orow = p.O + (int64_t)batch * p.sB + (int64_t)head * p.sH + tok * p.sT + half * (D / 2);
 #pragma unroll
@@ -587,7 +595,7 @@ __global__ void __maxnreg__(96)
                           __uint_as_float(o[v * 4 + 2]) * a_me, __uint_as_float(o[v * 4 + 3]) * a_me);
       }
       named_bar_sync(9, 512);
-      const int64_t tok = q0 + row;
+      const int64_t tok = blk[rh] >= 0 ? (int64_t)blk[rh] * BLK + (row & 63) : p.N;
       const float* take = mbuf + ((size_t)((1 - sidx) * 2 + half) * 128 + row) * C::kMergeStride;
       __nv_bfloat16* orow = p.O + (int64_t)batch * p.sB + (int64_t)head * p.sH + tok * p.sT + keep_q * QW;
       {
@@ -630,6 +638,80 @@ __global__ void __maxnreg__(96)
   PROF_ADD(13, t_cta0, t_cta1);  // CTA lifetime of the sampled lanes up to the final barrier
   PROF_ADD(14, t_cta1, t_cta2);  // final barrier + dealloc
   PROF_ADD(15, t_cta0, t_cta0 + 1);
+}
+
+// ------------------------------------------------------------------------------------------------
+// Pairing pass: which two query blocks of a head share a CTA.  Blocks i and i+D are paired in
+// stripes (i mod 2D < D), leftovers pair up consecutively.  With `search` the offset D in 1..NB/2 that
+// maximises the summed overlap |M[i] & M[i+D]| of the kept lists is chosen per (batch, head) --
+// video attention is multi-diagonal, so the best partner of a block is typically the same position a
+// fixed number of blocks away; the more two stacked blocks share, the less of a 128-row tile's work
+// is masked away.  Without `search`, D = 1 (neighbours).  One CTA per (batch, head).
+// ------------------------------------------------------------------------------------------------
+constexpr int kPairThreads = 256;
+constexpr int kPairSample = 4;
+
+__global__ void __launch_bounds__(kPairThreads) pair_kernel(const uint32_t* __restrict__ mask, int NB, int Wd,
+                                                            int search, int32_t* __restrict__ pairs) {
+  extern __shared__ __align__(16) unsigned char smem_raw[];
+  uint32_t* m = reinterpret_cast<uint32_t*>(smem_raw);                  // [NB][Wd]
+  uint8_t* used = reinterpret_cast<uint8_t*>(m + (size_t)NB * Wd);      // [NB]
+  __shared__ int s_score[kPairThreads];
+  __shared__ int s_d[kPairThreads];
+  const int bh = blockIdx.x;
+  const uint32_t* src = mask + (int64_t)bh * NB * Wd;
+  for (int idx = threadIdx.x; idx < NB * Wd; idx += kPairThreads) m[idx] = src[idx];
+  for (int idx = threadIdx.x; idx < NB; idx += kPairThreads) used[idx] = 0;
+  __syncthreads();
+  int best = -1, best_d = 1;
+  if (search) {
+    for (int d = 1 + threadIdx.x; d <= NB / 2; d += kPairThreads) {
+      int score = 0;
+      for (int i = 0; i + d < NB; i += kPairSample)  // every kPairSample-th row is enough to rank offsets
+        for (int w = 0; w < Wd; ++w) score += __popc(m[i * Wd + w] & m[(i + d) * Wd + w]);
+      if (score > best) {
+        best = score;
+        best_d = d;
+      }
+    }
+  }
+  s_score[threadIdx.x] = best;
+  s_d[threadIdx.x] = best_d;
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    for (int t = 1; t < kPairThreads; ++t)
+      if (s_score[t] > best || (s_score[t] == best && s_score[t] >= 0 && s_d[t] < best_d)) {
+        best = s_score[t];
+        best_d = s_d[t];
+      }
+    int32_t* out = pairs + (int64_t)bh * ((NB + 1) / 2) * 2;
+    int c = 0;
+    for (int i = 0; i < NB; ++i) {
+      const int j = i + best_d;
+      if (!used[i] && j < NB && !used[j]) {
+        used[i] = used[j] = 1;
+        out[2 * c] = i;
+        out[2 * c + 1] = j;
+        ++c;
+      }
+    }
+    int prev = -1;
+    for (int i = 0; i < NB; ++i) {
+      if (used[i]) continue;
+      if (prev < 0) {
+        prev = i;
+      } else {
+        out[2 * c] = prev;
+        out[2 * c + 1] = i;
+        ++c;
+        prev = -1;
+      }
+    }
+    if (prev >= 0) {
+      out[2 * c] = prev;
+      out[2 * c + 1] = -1;
+    }
+  }
 }
 
 // ------------------------------------------------------------------------------------------------
@@ -679,12 +761,12 @@ static int launch_attn_t(const sparsp_shape& s, const Geometry& g, const void* Q
                          const AttnParams& p, cudaStream_t st) {
   CUtensorMap tq, tk, tv;
   int rc;
-  if ((rc = make_tmap(&tq, Q, s, g, 128)) != SPARSP_OK) return rc;
+  if ((rc = make_tmap(&tq, Q, s, g, BLK)) != SPARSP_OK) return rc;
   if ((rc = make_tmap(&tk, K, s, g, BLK)) != SPARSP_OK) return rc;
   if ((rc = make_tmap(&tv, V, s, g, BLK)) != SPARSP_OK) return rc;
   auto kern = attn_fwd_kernel<D, BLK>;
   const int smem = AttnCfg<D, BLK>::kDynamic;
-  SPARSP_CUDA_OK(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
+  SPARSP_CUDA_OK(ensure_dynamic_smem((const void*)kern, smem));
   dim3 grid((unsigned)((g.NB + 1) / 2), (unsigned)(g.B * g.H));
   kern<<<grid, kAttnThreads, smem, st>>>(tq, tk, tv, p);
   count_launch();
@@ -695,8 +777,16 @@ static int launch_attn_t(const sparsp_shape& s, const Geometry& g, const void* Q
 int launch_attn(const sparsp_shape& s, const Geometry& g, const void* Q, const void* K, const void* V,
                 const uint32_t* mask, float scale, void* O, float* lse, char* ws, const WsLayout& L,
                 cudaStream_t st) {
+  int32_t* pairs = (int32_t*)(ws + L.pairs);
+  {
+    const size_t smem = (size_t)g.NB * g.Wd * 4 + g.NB;
+    SPARSP_CUDA_OK(ensure_dynamic_smem((const void*)pair_kernel, (int)smem));
+    pair_kernel<<<g.B * g.H, kPairThreads, smem, st>>>(mask, g.NB, g.Wd, g.b == 64 ? 1 : 0, pairs);
+    count_launch();
+  }
   AttnParams p;
   p.mask = mask;
+  p.pairs = pairs;
   p.O = (__nv_bfloat16*)O;
   p.lse = lse;
   p.status = (int32_t*)(ws + L.status);

@@ -34,7 +34,7 @@ struct PackEntry {
 };
 
 struct WsLayout {
-  int64_t status, pooled_q, pooled_k, scores, own, ent_base, n_entries, entries, total;
+  int64_t status, pooled_q, pooled_k, scores, pairs, own, ent_base, n_entries, entries, total;
 };
 
 void set_error(const char* fmt, ...);
@@ -45,6 +45,10 @@ inline void count_launch(int n = 1) { g_launches.fetch_add(n, std::memory_order_
 int make_geometry(const sparsp_shape* s, Geometry* g);
 int check_strides(const sparsp_shape* s, const Geometry& g);
 WsLayout make_layout(const Geometry& g, int n_ranks);
+
+// Raises a kernel's dynamic shared-memory limit to at least `bytes` on the current device; remembers
+// what was set per (kernel, device) so that the driver call is made only when the limit must grow.
+cudaError_t ensure_dynamic_smem(const void* func, int bytes);
 
 inline int64_t align_up(int64_t x, int64_t a) { return (x + a - 1) / a * a; }
 

@@ -246,7 +246,7 @@ int launch_score_topk(const Geometry& g, const float* pq, const float* pk, float
     const int nt = (g.NB + kScoreTile - 1) / kScoreTile;
     dim3 grid(nt, nt, g.B * g.H);
     auto kern = g.d == 64 ? score_kernel<64> : score_kernel<128>;
-    SPARSP_CUDA_OK(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+    SPARSP_CUDA_OK(ensure_dynamic_smem((const void*)kern, (int)smem));
     kern<<<grid, kScoreThreads, smem, st>>>(pq, pk, g.NB, scores);
   }
   {
