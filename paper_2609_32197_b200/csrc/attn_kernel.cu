@@ -654,62 +654,45 @@ constexpr int kPairSample = 4;
 __global__ void __launch_bounds__(kPairThreads) pair_kernel(const uint32_t* __restrict__ mask, int NB, int Wd,
                                                             int search, int32_t* __restrict__ pairs) {
   extern __shared__ __align__(16) unsigned char smem_raw[];
-  uint32_t* m = reinterpret_cast<uint32_t*>(smem_raw);                  // [NB][Wd]
-  uint8_t* used = reinterpret_cast<uint8_t*>(m + (size_t)NB * Wd);      // [NB]
-  __shared__ int s_score[kPairThreads];
-  __shared__ int s_d[kPairThreads];
+  uint32_t* m = reinterpret_cast<uint32_t*>(smem_raw);  // [NB][Wd]
+  __shared__ unsigned int s_best;                        // (score << 10) | (1023 - D): max = best score, smallest D
   const int bh = blockIdx.x;
-  const uint32_t* src = mask + (int64_t)bh * NB * Wd;
-  for (int idx = threadIdx.x; idx < NB * Wd; idx += kPairThreads) m[idx] = src[idx];
-  for (int idx = threadIdx.x; idx < NB; idx += kPairThreads) used[idx] = 0;
-  __syncthreads();
-  int best = -1, best_d = 1;
+  if (threadIdx.x == 0) s_best = (0u << 10) | (1023u - 1u);  // default D = 1
   if (search) {
+    const uint32_t* src = mask + (int64_t)bh * NB * Wd;
+    for (int idx = threadIdx.x; idx < NB * Wd; idx += kPairThreads) m[idx] = src[idx];
+    __syncthreads();
     for (int d = 1 + threadIdx.x; d <= NB / 2; d += kPairThreads) {
-      int score = 0;
+      unsigned int score = 0;
       for (int i = 0; i + d < NB; i += kPairSample)  // every kPairSample-th row is enough to rank offsets
         for (int w = 0; w < Wd; ++w) score += __popc(m[i * Wd + w] & m[(i + d) * Wd + w]);
-      if (score > best) {
-        best = score;
-        best_d = d;
-      }
+      atomicMax(&s_best, (score << 10) | (unsigned int)(1023 - d));
     }
   }
-  s_score[threadIdx.x] = best;
-  s_d[threadIdx.x] = best_d;
   __syncthreads();
-  if (threadIdx.x == 0) {
-    for (int t = 1; t < kPairThreads; ++t)
-      if (s_score[t] > best || (s_score[t] == best && s_score[t] >= 0 && s_d[t] < best_d)) {
-        best = s_score[t];
-        best_d = s_d[t];
+  const int D = 1023 - (int)(s_best & 1023u);
+  // stripes: rows with (i mod 2D) < D pair with i + D; the rows of the last partial stripe that have
+  // no partner form one consecutive run and pair up as neighbours
+  const int full = NB / (2 * D), R = NB % (2 * D);
+  const int np_last = max(R - D, 0), lo_end = min(R, D);
+  int32_t* out = pairs + (int64_t)bh * ((NB + 1) / 2) * 2;
+  for (int i = threadIdx.x; i < NB; i += kPairThreads) {
+    const int st = i / (2 * D), pos = i % (2 * D);
+    if (st < full) {
+      if (pos < D) {
+        out[2 * (st * D + pos)] = i;
+        out[2 * (st * D + pos) + 1] = i + D;
       }
-    int32_t* out = pairs + (int64_t)bh * ((NB + 1) / 2) * 2;
-    int c = 0;
-    for (int i = 0; i < NB; ++i) {
-      const int j = i + best_d;
-      if (!used[i] && j < NB && !used[j]) {
-        used[i] = used[j] = 1;
+    } else if (pos < np_last) {
+      out[2 * (full * D + pos)] = i;
+      out[2 * (full * D + pos) + 1] = i + D;
+    } else if (pos < lo_end) {
+      const int k = pos - np_last, n_left = lo_end - np_last;
+      if ((k & 1) == 0) {
+        const int c = full * D + np_last + k / 2;
         out[2 * c] = i;
-        out[2 * c + 1] = j;
-        ++c;
+        out[2 * c + 1] = (k + 1 < n_left) ? i + 1 : -1;
       }
-    }
-    int prev = -1;
-    for (int i = 0; i < NB; ++i) {
-      if (used[i]) continue;
-      if (prev < 0) {
-        prev = i;
-      } else {
-        out[2 * c] = prev;
-        out[2 * c + 1] = i;
-        ++c;
-        prev = -1;
-      }
-    }
-    if (prev >= 0) {
-      out[2 * c] = prev;
-      out[2 * c + 1] = -1;
     }
   }
 }
@@ -779,7 +762,7 @@ int launch_attn(const sparsp_shape& s, const Geometry& g, const void* Q, const v
                 cudaStream_t st) {
   int32_t* pairs = (int32_t*)(ws + L.pairs);
   {
-    const size_t smem = (size_t)g.NB * g.Wd * 4 + g.NB;
+    const size_t smem = (size_t)g.NB * g.Wd * 4;
     SPARSP_CUDA_OK(ensure_dynamic_smem((const void*)pair_kernel, (int)smem));
     pair_kernel<<<g.B * g.H, kPairThreads, smem, st>>>(mask, g.NB, g.Wd, g.b == 64 ? 1 : 0, pairs);
     count_launch();
