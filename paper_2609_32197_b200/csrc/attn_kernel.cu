@@ -50,7 +50,7 @@ constexpr float kGrowThreshold = 8.0f;
 #define SPARSP_TUNE_F32X2 1
 #endif
 #ifndef SPARSP_TUNE_POLY
-#define SPARSP_TUNE_POLY 4
+#define SPARSP_TUNE_POLY 3
 #endif
 
 template <int D, int BLK>
