@@ -33,8 +33,8 @@ NOMINAL = {"hbm_gbs": 8000.0, "bf16_tflops": 2250.0}
 # dram__bytes_read.sum + dram__bytes_write.sum per launch of the attention kernel, from the ncu
 # captures summarised under profiles/ (None = not captured for that workload).
 ATTN_DRAM_TRAFFIC = {
-    ("mid", 58): 588.8e6,            # profiles/attn_fwd_kernel_mid_and_hunyuan4.md, full workload
-    ("hunyuan", 93): 6 * 722.2e6,     # same file: 4-head capture scaled by heads (24 / 4)
+    ("mid", 58): 590.7e6,            # profiles/attn_fwd_kernel_mid_and_hunyuan4.md, full workload
+    ("hunyuan", 93): 6 * 748.3e6,     # same file: 4-head capture scaled by heads (24 / 4)
 }
 
 
@@ -323,11 +323,11 @@ def run_ours(args):
         "pack_gbs": pack_gbs,
         "pack_pct_hbm": {"of_measured": pack_gbs / peaks["hbm_gbs"], "of_nominal": pack_gbs / NOMINAL["hbm_gbs"]},
         "volume_bytes_total": volume,
-        "roofline": {"bound": "tensor", "kernel": "attn_fwd_kernel", "achieved": attn_tflops,
+        "roofline": {"bound": "tensor", "kernel": "attn_fwd_kernel (+ pair_kernel, timed together)", "achieved": attn_tflops,
                      "peak": peaks["bf16_tflops"], "peak_source": peaks["source"] + " burst", "unit": "TFLOP/s",
                      "frac": attn_tflops / peaks["bf16_tflops"],
                      "traffic": ATTN_DRAM_TRAFFIC.get((wl.name, k))},
-        "roofline_pack": {"bound": "hbm", "kernel": "pack_kernel", "achieved": pack_gbs, "peak": peaks["hbm_gbs"],
+        "roofline_pack": {"bound": "hbm", "kernel": "pack_kernel" if b * d < 8192 else "pack_tile_kernel", "achieved": pack_gbs, "peak": peaks["hbm_gbs"],
                           "peak_source": peaks["source"], "unit": "GB/s", "frac": pack_gbs / peaks["hbm_gbs"],
                           "algorithmic_bytes": pack_bytes},
         "e2e": {"value": None if e2e_ms != e2e_ms else flops_all / (e2e_ms * 1e-3) / 1e12, "unit": "TFLOP/s",
