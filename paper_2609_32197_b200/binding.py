@@ -54,8 +54,14 @@ def lib() -> ctypes.CDLL:
     global _lib
     if _lib is None:
         if not os.path.exists(LIB_PATH):
-            raise RuntimeError(f"{LIB_PATH} is missing: build it with `python -m paper_2609_32197_b200.build` "
-                               "(there is no CPU fallback)")
+            # not built yet (e.g. a fresh checkout): compile it in-tree with nvcc; if that is impossible
+            # the call fails loudly -- there is no CPU fallback
+            try:
+                from . import build as _build
+                _build.build()
+            except Exception as exc:  # noqa: BLE001
+                raise RuntimeError(f"{LIB_PATH} is missing and could not be built with nvcc ({exc}); "
+                                   "there is no CPU fallback") from exc
         L = ctypes.CDLL(LIB_PATH)
         L.sparsp_last_error.restype = ctypes.c_char_p
         L.sparsp_launch_count.restype = ctypes.c_int64
