@@ -303,6 +303,17 @@ __global__ void __maxnreg__(96)
       const uint64_t descQ = make_smem_desc(smem_u32(sQ + (C::kSplitKV ? 0 : s) * C::kQBytes), 16, 1024);
       const uint64_t descK = make_smem_desc(smem_u32(sK), 16, 1024);
       const uint64_t descV = make_smem_desc(smem_u32(sV), 16384, 1024);
+      // low words of the descriptors per K step (stage 0); a stage adds kTileBytes/16 to the low word
+      const uint32_t hiQK = (uint32_t)(descK >> 32), hiV = (uint32_t)(descV >> 32);
+      uint32_t qlo[D / 16], klo[D / 16], vlo[8];
+#pragma unroll
+      for (int kk = 0; kk < D / 16; ++kk) {
+        const uint32_t off = (uint32_t)(((kk / 4) * 16384 + (kk % 4) * 32) >> 4);
+        qlo[kk] = (uint32_t)descQ + off;
+        klo[kk] = (uint32_t)descK + off;
+      }
+#pragma unroll
+      for (int kk = 0; kk < 8; ++kk) vlo[kk] = (uint32_t)descV + (uint32_t)((kk * 2048) >> 4);
       int vdone = 0;       // tiles whose V obligation (P V or plain release) has been handled
       int last_kept = -1;  // last tile whose Q K^T this stream has issued
       int pcnt = 0;        // P tiles consumed
@@ -323,11 +334,11 @@ __global__ void __maxnreg__(96)
         PROF_ADD(10, t_v0, t_v1);  // issuer waiting for V
         if (keep) {
           tc_fence_after();
-          const uint64_t db0 = descV + (uint64_t)(((m % S) * C::kTileBytes) >> 4);
+          const uint32_t stage_off = (uint32_t)(((m % S) * C::kTileBytes) >> 4);
           if (leader) {
 #pragma unroll
             for (int kk = 0; kk < 8; ++kk)
-              mma_ts(tOs, tSs + kk * 8, db0 + (uint64_t)((kk * 2048) >> 4), kIdescPV, (kk > 0) ? 1u : started);
+              mma_ts_lohi(tOs, tSs + kk * 8, vlo[kk] + stage_off, hiV, kIdescPV, (kk > 0) ? 1u : started);
             mma_commit(o_full + s);
             mma_commit(v_empty + m % S);
           }
@@ -352,13 +363,11 @@ __global__ void __maxnreg__(96)
           while (vdone <= last_kept) handle_v(vdone++);  // P V of the previous kept tile frees S_s
           PROF_T(t_k3);
           tc_fence_after();
-          const uint64_t db0 = descK + (uint64_t)(((n % S) * C::kTileBytes) >> 4);
+          const uint32_t stage_off = (uint32_t)(((n % S) * C::kTileBytes) >> 4);
           if (leader) {
 #pragma unroll
-            for (int kk = 0; kk < D / 16; ++kk) {
-              const uint64_t off = (uint64_t)(((kk / 4) * 16384 + (kk % 4) * 32) >> 4);
-              mma_ss(tSs, descQ + off, db0 + off, kIdescQK, kk > 0 ? 1u : 0u);
-            }
+            for (int kk = 0; kk < D / 16; ++kk)
+              mma_ss_lohi(tSs, qlo[kk], hiQK, klo[kk] + stage_off, hiQK, kIdescQK, kk > 0 ? 1u : 0u);
             mma_commit(s_full + s);
             mma_commit(k_empty + n % S);
           }
