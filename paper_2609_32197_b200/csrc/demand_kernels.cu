@@ -1,9 +1,11 @@
 // Step 2: per-rank per-head unions of required KV blocks, demand counts, exchange volume,
 // pack-order offsets, the entry table, and the gather of K/V tiles into per-consumer buffers.
 // Everything before the gather is small integer work on bit words; the gather is the HBM-bound part.
+#include <algorithm>
 #include <mutex>
 
 #include "common.cuh"
+#include "sm100_ptx.cuh"
 
 namespace sparsp {
 
@@ -265,6 +267,118 @@ __global__ void __launch_bounds__(kPackThreads) pack_tile_kernel(
   }
 }
 
+// ------------------------------------------------------------------------------------------------
+// Bulk-copy gather for layouts in which a tile's rows are adjacent in memory ([B][H][N][d]): one warp
+// per CTA streams whole tiles global -> shared -> global with the TMA bulk engine (cp.async.bulk), a
+// ring of n_stages tile buffers per warp (1, 2 or 4 warps per CTA for 32, 16, 8 KiB tiles, so that the
+// bytes in flight per SM do not depend on the tile size), loads running n_stages-1 tiles ahead of the
+// stores.
+// No thread touches the data, except to zero the missing rows of a ragged last block.
+// ------------------------------------------------------------------------------------------------
+constexpr int kBulkMaxStages = 8;
+#ifndef SPARSP_TUNE_PACK_BULK
+#define SPARSP_TUNE_PACK_BULK 1
+#endif
+constexpr bool kPackUseBulk = SPARSP_TUNE_PACK_BULK != 0;
+
+__device__ __forceinline__ void bulk_load(void* smem_dst, const void* gsrc, uint32_t bytes, uint64_t* bar) {
+  asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(
+                   ptx::smem_u32(smem_dst)),
+               "l"(gsrc), "r"(bytes), "r"(ptx::smem_u32(bar))
+               : "memory");
+}
+__device__ __forceinline__ void bulk_store(void* gdst, const void* smem_src, uint32_t bytes) {
+  asm volatile("cp.async.bulk.global.shared::cta.bulk_group [%0], [%1], %2;" ::"l"(gdst),
+               "r"(ptx::smem_u32(smem_src)), "r"(bytes)
+               : "memory");
+  asm volatile("cp.async.bulk.commit_group;" ::: "memory");
+}
+
+template <int D>
+__global__ void __launch_bounds__(128) pack_bulk_kernel(const __nv_bfloat16* __restrict__ K,
+                                                       const __nv_bfloat16* __restrict__ V,
+                                                       const PackEntry* __restrict__ entries,
+                                                       const int64_t* __restrict__ n_entries_p, int H, int b,
+                                                       int64_t N, int64_t sB, int64_t sH, int n_stages,
+                                                       unsigned char* __restrict__ packed,
+                                                       int32_t* __restrict__ status) {
+  extern __shared__ __align__(128) unsigned char smem_raw[];
+  __shared__ uint64_t full_all[4 * kBulkMaxStages];
+  __shared__ int s_abort;
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  const int n_warps = blockDim.x >> 5;
+  const uint32_t tile_bytes = (uint32_t)b * D * 2;
+  uint64_t* full = full_all + warp * kBulkMaxStages;
+  unsigned char* ring = smem_raw + (size_t)warp * n_stages * tile_bytes;  // this warp's buffers
+  const int64_t unit = (int64_t)blockIdx.x * n_warps + warp, n_units = (int64_t)gridDim.x * n_warps;
+  const int64_t n_items = 2 * (*n_entries_p);
+  const int64_t n_local = n_items > unit ? (n_items - unit + n_units - 1) / n_units : 0;
+  if (threadIdx.x == 0) s_abort = 0;
+  if (lane == 0) {
+    for (int st = 0; st < n_stages; ++st) ptx::mbar_init(full + st, 1);
+    ptx::mbar_init_fence();
+  }
+  __syncthreads();
+
+  // source address and valid byte count of local item q (0 valid bytes = entry skipped for capacity)
+  auto locate = [&](int64_t q, const unsigned char*& src, unsigned char*& dst, uint32_t& valid) {
+    const int64_t item = unit + q * n_units;
+    const int4 raw = __ldg(reinterpret_cast<const int4*>(entries) + (item >> 1));
+    const int64_t dst_byte = (int64_t)(((uint64_t)(uint32_t)raw.y << 32) | (uint32_t)raw.x);
+    const int bh = raw.z, j = raw.w;
+    const int which = (int)(item & 1);
+    if (j < 0) {
+      valid = 0;
+      src = nullptr;
+      dst = nullptr;
+      return;
+    }
+    const int64_t batch = bh / H, head = bh % H, tok0 = (int64_t)j * b;
+    const int64_t n_valid = min((int64_t)b, N - tok0);
+    valid = (uint32_t)(n_valid * D * 2);
+    src = reinterpret_cast<const unsigned char*>((which ? V : K) + batch * sB + head * sH + tok0 * D);
+    dst = packed + dst_byte + (int64_t)which * tile_bytes;
+  };
+  auto issue_load = [&](int64_t q) {
+    const unsigned char* src;
+    unsigned char* dst;
+    uint32_t valid;
+    locate(q, src, dst, valid);
+    uint64_t* bar = full + q % n_stages;
+    if (valid == 0) {
+      ptx::mbar_arrive(bar);  // nothing to move: complete the phase directly
+    } else {
+      ptx::mbar_expect_tx(bar, valid);
+      bulk_load(ring + (size_t)(q % n_stages) * tile_bytes, src, valid, bar);
+    }
+  };
+
+  if (lane == 0)
+    for (int64_t q = 0; q < n_stages - 1 && q < n_local; ++q) issue_load(q);
+  for (int64_t q = 0; q < n_local; ++q) {
+    const unsigned char* src;
+    unsigned char* dst;
+    uint32_t valid;
+    locate(q, src, dst, valid);  // same values in every lane
+    unsigned char* buf = ring + (size_t)(q % n_stages) * tile_bytes;
+    ptx::mbar_wait_bounded(full + q % n_stages, (uint32_t)((q / n_stages) & 1), &s_abort, status, 50, 200000000LL);
+    if (valid != 0 && valid < tile_bytes) {  // ragged last block: zero the missing rows
+      for (uint32_t o = valid + lane * 16; o < tile_bytes; o += 32 * 16)
+        *reinterpret_cast<uint4*>(buf + o) = make_uint4(0u, 0u, 0u, 0u);
+      ptx::fence_proxy_async_smem();
+    }
+    __syncwarp();
+    if (lane == 0) {
+      if (valid != 0) bulk_store(dst, buf, tile_bytes);
+      // the buffer of item q-1 may be refilled once its store has read it
+      asm volatile("cp.async.bulk.wait_group.read 1;" ::: "memory");
+      if (q + n_stages - 1 < n_local) issue_load(q + n_stages - 1);
+    }
+    __syncwarp();
+  }
+  if (lane == 0) asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");
+}
+
 int launch_pack(const sparsp_shape& s, const Geometry& g, const void* K, const void* V, void* packed,
                 int64_t capacity, int P, char* ws, const WsLayout& L, cudaStream_t st) {
   (void)capacity;
@@ -279,7 +393,24 @@ int launch_pack(const sparsp_shape& s, const Geometry& g, const void* K, const v
   auto v = (const __nv_bfloat16*)V;
   const bool small_tiles = g.b * g.d / 8 < 1024;  // 8 KiB tiles: several tiles per CTA step
   unsigned char* out = (unsigned char*)packed;
-  if (small_tiles) {
+  const bool rows_adjacent = s.stride_token == g.d;
+  if (rows_adjacent && kPackUseBulk) {
+    // TMA bulk path: a ring of whole-tile buffers per CTA, one CTA per SM
+    const int tile_bytes = g.b * g.d * 2;
+    const int n_warps = std::max(1, std::min(4, (32 * 1024) / tile_bytes));
+    const int n_stages = 5;  // per warp: 160 KiB of tile buffers per CTA whatever the tile size
+    const int smem = n_warps * n_stages * tile_bytes;
+    int32_t* status = (int32_t*)(ws + L.status);
+    if (g.d == 64) {
+      SPARSP_CUDA_OK(ensure_dynamic_smem((const void*)pack_bulk_kernel<64>, smem));
+      pack_bulk_kernel<64><<<sms, 32 * n_warps, smem, st>>>(k, v, entries, n_entries, g.H, g.b, g.N,
+                                                            s.stride_batch, s.stride_head, n_stages, out, status);
+    } else {
+      SPARSP_CUDA_OK(ensure_dynamic_smem((const void*)pack_bulk_kernel<128>, smem));
+      pack_bulk_kernel<128><<<sms, 32 * n_warps, smem, st>>>(k, v, entries, n_entries, g.H, g.b, g.N,
+                                                             s.stride_batch, s.stride_head, n_stages, out, status);
+    }
+  } else if (small_tiles) {
     if (g.d == 64)
       pack_kernel<64><<<grid, kPackThreads, 0, st>>>(k, v, entries, n_entries, g.H, g.b, g.N, s.stride_batch,
                                                      s.stride_head, s.stride_token, out);
