@@ -69,7 +69,13 @@ struct AttnCfg {
   static constexpr int kOffStat = kOffEntF + kMaxBlocks;         // float2 [2 streams][2 halves][128]
   static constexpr int kOffMax = kOffStat + 2 * 2 * 128 * 8;     // float [2 parities][2][2][128]
   static constexpr int kOffBars = kOffMax + 2 * 2 * 2 * 128 * 4;
-  static constexpr int kNumBars = 1 + 4 * kStages + 6;
+  static constexpr int kNumBars = 1 + 4 * kStages + 8;
+  // head_dim 64 leaves tensor-memory room for P next to S (S 2x128 + P 2x64 + O 2x64 = 512 columns):
+  // Q K^T of the next tile can then start as soon as the softmax warps have READ S, instead of
+  // waiting for P V to finish reading P out of the same columns.
+  static constexpr bool kDecoupledP = (D == 64);
+  static constexpr int kColP = 256;                       // first P column (decoupled layout)
+  static constexpr int kColO = kDecoupledP ? 384 : 256;   // first O column
   static constexpr int kOffMisc = kOffBars + 8 * kNumBars;
   static constexpr int kTotal = kOffMisc + 32;
   static constexpr int kDynamic = kTotal + 1024;  // slack for the 1024-byte alignment of the base
@@ -158,6 +164,7 @@ __global__ void __maxnreg__(96)
   uint64_t* s_full = v_empty + S;  // [2] S_s written by Q K^T
   uint64_t* p_full = s_full + 2;   // [2] P_s written by the stream's 8 softmax warps (one arrival each)
   uint64_t* o_full = p_full + 2;   // [2] a P V of stream s has completed
+  uint64_t* s_free = o_full + 2;   // [2] S_s has been read into registers (decoupled-P layout only)
   uint32_t* s_tmem = reinterpret_cast<uint32_t*>(smem + C::kOffMisc);
   int* s_nent = reinterpret_cast<int*>(smem + C::kOffMisc + 4);
   volatile int* s_abort = reinterpret_cast<volatile int*>(smem + C::kOffMisc + 8);
@@ -187,6 +194,7 @@ __global__ void __maxnreg__(96)
       mbar_init(s_full + s, 1);
       mbar_init(p_full + s, 8);
       mbar_init(o_full + s, 1);
+      mbar_init(s_free + s, 8);
     }
     mbar_init_fence();
     *s_abort = 0;
@@ -299,7 +307,10 @@ __global__ void __maxnreg__(96)
       constexpr uint32_t kIdescQK = make_idesc_bf16(128, 128, 0, 0);
       constexpr uint32_t kIdescPV = make_idesc_bf16(128, D, 0, 1);
       const uint32_t tSs = tmem_base + s * 128;
-      const uint32_t tOs = tmem_base + 256 + s * D;
+      const uint32_t tPs = C::kDecoupledP ? tmem_base + C::kColP + s * 64 : tSs;  // bf16 P (A operand of P V)
+      const uint32_t tOs = tmem_base + C::kColO + s * D;
+      int qcnt = 0;  // Q K^T tiles issued
+      constexpr int kVLag = (S >= 4) ? S - 2 : 1;
       const uint64_t descQ = make_smem_desc(smem_u32(sQ + (C::kSplitKV ? 0 : s) * C::kQBytes), 16, 1024);
       const uint64_t descK = make_smem_desc(smem_u32(sK), 16, 1024);
       const uint64_t descV = make_smem_desc(smem_u32(sV), 16384, 1024);
@@ -338,7 +349,7 @@ __global__ void __maxnreg__(96)
           if (leader) {
 #pragma unroll
             for (int kk = 0; kk < 8; ++kk)
-              mma_ts_lohi(tOs, tSs + kk * 8, vlo[kk] + stage_off, hiV, kIdescPV, (kk > 0) ? 1u : started);
+              mma_ts_lohi(tOs, tPs + kk * 8, vlo[kk] + stage_off, hiV, kIdescPV, (kk > 0) ? 1u : started);
             mma_commit(o_full + s);
             mma_commit(v_empty + m % S);
           }
@@ -354,13 +365,19 @@ __global__ void __maxnreg__(96)
       mbar_wait_bounded(bar_q, 0, s_abort, p.status, 11, p.wait_limit);
       for (int n = 0; n < n_tiles; ++n) {
         const bool keep = (stream_mask(n) >> s) & 1;
-        while (vdone < n - 1) handle_v(vdone++);  // a V stage is released at most two steps after its fill
+        // a V stage is released at most kVLag + 1 steps after its fill (always fewer than the ring has stages)
+        while (vdone < n - kVLag) handle_v(vdone++);
         PROF_T(t_k0);
         mbar_wait_bounded(k_full + n % S, (n / S) & 1, s_abort, p.status, 12, p.wait_limit);
         PROF_T(t_k1);
         PROF_ADD(9, t_k0, t_k1);  // issuer waiting for K
         if (keep) {
-          while (vdone <= last_kept) handle_v(vdone++);  // P V of the previous kept tile frees S_s
+          if (C::kDecoupledP) {
+            // S_s is free once the softmax warps have loaded the previous tile's scores
+            if (qcnt > 0) mbar_wait_bounded(s_free + s, (qcnt - 1) & 1, s_abort, p.status, 24 + s, p.wait_limit);
+          } else {
+            while (vdone <= last_kept) handle_v(vdone++);  // P V of the previous kept tile frees S_s
+          }
           PROF_T(t_k3);
           tc_fence_after();
           const uint32_t stage_off = (uint32_t)(((n % S) * C::kTileBytes) >> 4);
@@ -371,9 +388,12 @@ __global__ void __maxnreg__(96)
             mma_commit(s_full + s);
             mma_commit(k_empty + n % S);
           }
-          last_kept = n;
+          ++qcnt;
           PROF_T(t_k2);
           PROF_ADD(7, t_k3, t_k2);  // issuer issuing Q K^T
+          if (C::kDecoupledP)
+            while (vdone <= last_kept) handle_v(vdone++);  // P V of the previous kept tile, after this Q K^T
+          last_kept = n;
         } else if (leader) {
           mbar_arrive(k_empty + n % S);
         }
@@ -391,7 +411,8 @@ __global__ void __maxnreg__(96)
     const int pair_bar = 1 + sidx * 4 + rgrp;  // named barrier shared with the row's other thread
     const uint32_t lane_off = (uint32_t)(rgrp * 32) << 16;
     const uint32_t tS = tmem_base + sidx * 128 + lane_off;
-    const uint32_t tO = tmem_base + 256 + sidx * D + lane_off;
+    const uint32_t tP = (C::kDecoupledP ? tmem_base + C::kColP + sidx * 64 : tmem_base + sidx * 128) + lane_off;
+    const uint32_t tO = tmem_base + C::kColO + sidx * D + lane_off;
     float m_used = -INFINITY;  // reference maximum (log2 domain) of the row's exponentials
     float l_run = 0.0f;        // this thread's share of the row sum
     int cnt = 0;
@@ -427,6 +448,12 @@ __global__ void __maxnreg__(96)
       tmem_ld32(tS + half * 64, reinterpret_cast<uint32_t*>(sv));
       tmem_ld32(tS + half * 64 + 32, reinterpret_cast<uint32_t*>(sv) + 32);
       tmem_ld_wait();
+      if (C::kDecoupledP) {
+        // S is in registers: let the issuer start the next Q K^T
+        tc_fence_before();
+        __syncwarp();
+        if (lane == 0) mbar_arrive(s_free + sidx);
+      }
       float mx = -INFINITY;
 #pragma unroll
       for (int c = 0; c < 2; ++c) {
@@ -445,6 +472,11 @@ __global__ void __maxnreg__(96)
       named_bar_sync(pair_bar, 64);
       mx = fmaxf(mx, mslot[(1 - half) * 128 + row]) * p.scale_log2;
       PROF_T(t_c);
+      if (C::kDecoupledP && cnt > 0) {
+        // the previous P V must have finished reading P (and updating O) before either is touched
+        mbar_wait_bounded(o_full + sidx, (cnt - 1) & 1, s_abort, p.status, 34 + sidx, p.wait_limit);
+        tc_fence_after();
+      }
       const float m_new = fmaxf(m_used, mx);
       const bool grow = m_new > m_used + kGrowThreshold || (m_used == -INFINITY && m_new > -INFINITY);
       if (__any_sync(0xffffffffu, grow)) {
@@ -510,7 +542,7 @@ __global__ void __maxnreg__(96)
 #pragma unroll
           for (int e = 0; e < 16; ++e) pk[e] = 0u;
         }
-        tmem_st16(tS + half * 32 + c * 16, pk);
+        tmem_st16(tP + half * 32 + c * 16, pk);
       }
       l_run += lsum + (lsum2.x + lsum2.y);
       PROF_T(t_e);
