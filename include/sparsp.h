@@ -153,6 +153,27 @@ SPARSP_API int sparsp_sparse_attn_fwd(const sparsp_shape* shape, const void* Q, 
                            const uint32_t* mask, float softmax_scale, void* O, float* lse,
                            void* workspace, void* stream);
 
+/* Consumer side of the demand-routed exchange (Section 5.1: in round k a rank receives from the
+ * producer at ring distance k exactly the blocks it selected; Section 7: the attention over each
+ * arriving part is merged with the running result by online softmax).
+ *
+ * sparsp_hop_mask: the mask of ONE hop,
+ *   hop_mask[b,h,i,:] = (rank_of_block[i] == consumer) ? mask[b,h,i,:] AND own[producer,:] : 0,
+ * i.e. the consumer rank's query blocks restricted to the KV blocks the producer owns.  Feeding it to
+ * sparsp_sparse_attn_fwd (with lse) gives that hop's partial result; rows without any kept key come
+ * out as zeros with lse = -inf.
+ *   mask, hop_mask  uint32 [B][H][NB][Wd];  rank_of_block  DEVICE int32 [NB]
+ *
+ * sparsp_attn_merge: log-sum-exp merge of two partial results over disjoint key sets,
+ *   lse = log(exp(lse_a) + exp(lse_b)),  O = O_a * exp(lse_a - lse) + O_b * exp(lse_b - lse),
+ * computed in fp32, O rounded to bf16.  O may alias O_a or O_b (and lse alias lse_a or lse_b).
+ *   O_a, O_b, O  bf16, strided as in `shape`;  lse_a, lse_b, lse  fp32 [B][H][N] */
+SPARSP_API int sparsp_hop_mask(const sparsp_shape* shape, const uint32_t* mask, const int32_t* rank_of_block,
+                               int32_t n_ranks, int32_t consumer, int32_t producer, uint32_t* hop_mask,
+                               void* stream);
+SPARSP_API int sparsp_attn_merge(const sparsp_shape* shape, const void* O_a, const float* lse_a, const void* O_b,
+                                 const float* lse_b, void* O, float* lse, void* stream);
+
 /* Planning without any allocation.  (No counterpart in the paper: an engineering variant of the
  * planning half of sparsp_demand_pack.)
  * For callers that are not allowed to allocate device memory -- for example a plug-in running inside a

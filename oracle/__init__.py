@@ -255,3 +255,36 @@ def attn_dense_masked(Q, K, V, mask: np.ndarray, b: int, scale: float | None = N
     lib().oracle_attn_dense_masked(_p(Qs), _p(Ks), _p(Vs), _p(mask), _i64(H), _i64(N), _i64(d),
                                    _i64(b), ctypes.c_double(sc), _p(out), _p(rowsum))
     return out, rowsum
+
+
+# ---------------------------------------------------------------------------------------------
+# consumer-side pipeline ("next" rows): per-hop masks and log-sum-exp merging of partial results
+# ---------------------------------------------------------------------------------------------
+def hop_mask(mask: np.ndarray, rank_of_block: np.ndarray, consumer: int, producer: int) -> np.ndarray:
+    """Rows of the consumer rank's query blocks, restricted to the KV blocks the producer owns
+    (the blocks that travel in one hop of the demand-routed exchange, Section 5.1); all else zero."""
+    mask = np.ascontiguousarray(mask, dtype=np.uint32)
+    H, NB, Wd = mask.shape
+    own = np.zeros(Wd, dtype=np.uint32)
+    for j in range(NB):
+        if rank_of_block[j] == producer:
+            own[j >> 5] |= np.uint32(1 << (j & 31))
+    out = np.zeros_like(mask)
+    for i in range(NB):
+        if rank_of_block[i] == consumer:
+            out[:, i, :] = mask[:, i, :] & own
+    return out
+
+
+def attn_merge(oa: np.ndarray, la: np.ndarray, ob: np.ndarray, lb: np.ndarray):
+    """Log-sum-exp merge of two partial results over disjoint key sets. oa/ob [..., d] fp32, la/lb [...]."""
+    oa = np.ascontiguousarray(oa, dtype=np.float32)
+    ob = np.ascontiguousarray(ob, dtype=np.float32)
+    la = np.ascontiguousarray(la, dtype=np.float32)
+    lb = np.ascontiguousarray(lb, dtype=np.float32)
+    d = oa.shape[-1]
+    rows = oa.size // d
+    out = np.empty_like(oa)
+    lse = np.empty_like(la)
+    lib().oracle_attn_merge(_p(oa), _p(la), _p(ob), _p(lb), _i64(rows), _i64(d), _p(out), _p(lse))
+    return out, lse

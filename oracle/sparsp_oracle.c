@@ -287,6 +287,10 @@ void oracle_attn_rows(const uint16_t* Q, const uint16_t* K, const uint16_t* V, c
           for (int64_t c = 0; c < d; ++c) acc[c] += p * (double)bf16_to_f32(v[c]);
         }
       }
+      if (denom == 0.0) { /* no kept key (only possible for hop-restricted masks): zero row, lse = -inf */
+        if (lse) lse[u * b + r] = -INFINITY;
+        continue;
+      }
       for (int64_t c = 0; c < d; ++c) o[c] = (float)(acc[c] / denom);
       if (lse) lse[u * b + r] = (float)(m + log(denom));
     }
@@ -344,6 +348,32 @@ void oracle_attn_dense_masked(const uint16_t* Q, const uint16_t* K, const uint16
       free(s);
       free(pr);
     }
+  }
+}
+
+/* ------------------------------------------------------------------------------------------------
+ * Merging partial attention results (ring-attention style, Section 2.3 / Section 7: per-hop partial
+ * outputs are combined by online softmax).  For two partial results over DISJOINT key sets, each
+ * normalised by its own sum and carrying lse = log(sum of exp of its scaled logits):
+ *   lse = log(exp(lse_a) + exp(lse_b));  O = O_a * exp(lse_a - lse) + O_b * exp(lse_b - lse)
+ * An empty part has lse = -inf and weight 0.  fp64 throughout.  rows x d.
+ * ---------------------------------------------------------------------------------------------- */
+void oracle_attn_merge(const float* oa, const float* la, const float* ob, const float* lb, int64_t rows,
+                       int64_t d, float* out, float* lse) {
+#pragma omp parallel for schedule(static)
+  for (int64_t r = 0; r < rows; ++r) {
+    const double a = la[r], b = lb[r];
+    const double m = a > b ? a : b;
+    if (m == -INFINITY) {
+      for (int64_t c = 0; c < d; ++c) out[r * d + c] = 0.0f;
+      lse[r] = -INFINITY;
+      continue;
+    }
+    const double ea = exp(a - m), eb = exp(b - m);
+    const double tot = ea + eb;
+    for (int64_t c = 0; c < d; ++c)
+      out[r * d + c] = (float)(((double)oa[r * d + c] * ea + (double)ob[r * d + c] * eb) / tot);
+    lse[r] = (float)(m + log(tot));
   }
 }
 

@@ -29,6 +29,7 @@ EXPORTS = [
     "sparsp_geometry", "sparsp_resolve_topk", "sparsp_placement_contiguous", "sparsp_placement_periodic",
     "sparsp_workspace_bytes", "sparsp_block_mask", "sparsp_demand_pack", "sparsp_sparse_attn_fwd",
     "sparsp_status", "sparsp_last_error", "sparsp_launch_count", "sparsp_demand_plan_noalloc",
+    "sparsp_hop_mask", "sparsp_attn_merge",
 ]
 
 
@@ -177,6 +178,16 @@ def sparsp_sparse_attn_fwd(shape, Q, K, V, mask, softmax_scale, O, lse, workspac
     _check(lib().sparsp_sparse_attn_fwd(ctypes.byref(shape), _ptr(Q), _ptr(K), _ptr(V), _ptr(mask),
                                         ctypes.c_float(softmax_scale), _ptr(O), _ptr(lse), _ptr(workspace),
                                         _stream()))
+
+
+def sparsp_hop_mask(shape, mask, rank_of_block, n_ranks, consumer, producer, hop_mask):
+    _check(lib().sparsp_hop_mask(ctypes.byref(shape), _ptr(mask), _ptr(rank_of_block), ctypes.c_int32(n_ranks),
+                                 ctypes.c_int32(consumer), ctypes.c_int32(producer), _ptr(hop_mask), _stream()))
+
+
+def sparsp_attn_merge(shape, O_a, lse_a, O_b, lse_b, O, lse):
+    _check(lib().sparsp_attn_merge(ctypes.byref(shape), _ptr(O_a), _ptr(lse_a), _ptr(O_b), _ptr(lse_b), _ptr(O),
+                                   _ptr(lse), _stream()))
 
 
 def sparsp_status(workspace) -> int:

@@ -292,6 +292,36 @@ int sparsp_sparse_attn_fwd(const sparsp_shape* shape, const void* Q, const void*
                      (cudaStream_t)stream);
 }
 
+int sparsp_hop_mask(const sparsp_shape* shape, const uint32_t* mask, const int32_t* rank_of_block, int32_t n_ranks,
+                    int32_t consumer, int32_t producer, uint32_t* hop_mask, void* stream) {
+  Geometry g;
+  SPARSP_TRY(make_geometry(shape, &g));
+  if (n_ranks < 1 || n_ranks > kMaxRanks || consumer < 0 || consumer >= n_ranks || producer < 0 ||
+      producer >= n_ranks) {
+    set_error("consumer/producer %d/%d outside 0..%d", consumer, producer, n_ranks - 1);
+    return SPARSP_ERR_INVALID_ARG;
+  }
+  SPARSP_TRY(check_ptr(mask, "mask", 4));
+  SPARSP_TRY(check_ptr(rank_of_block, "rank_of_block", 4));
+  SPARSP_TRY(check_ptr(hop_mask, "hop_mask", 4));
+  return launch_hop_mask(g, mask, rank_of_block, consumer, producer, hop_mask, (cudaStream_t)stream);
+}
+
+int sparsp_attn_merge(const sparsp_shape* shape, const void* O_a, const float* lse_a, const void* O_b,
+                      const float* lse_b, void* O, float* lse, void* stream) {
+  Geometry g;
+  SPARSP_TRY(make_geometry(shape, &g));
+  SPARSP_TRY(check_supported(g));
+  SPARSP_TRY(check_strides(shape, g));
+  SPARSP_TRY(check_ptr(O_a, "O_a"));
+  SPARSP_TRY(check_ptr(O_b, "O_b"));
+  SPARSP_TRY(check_ptr(O, "O"));
+  SPARSP_TRY(check_ptr(lse_a, "lse_a", 4));
+  SPARSP_TRY(check_ptr(lse_b, "lse_b", 4));
+  SPARSP_TRY(check_ptr(lse, "lse", 4));
+  return launch_attn_merge(*shape, g, O_a, lse_a, O_b, lse_b, O, lse, (cudaStream_t)stream);
+}
+
 int sparsp_status(void* workspace, void* stream, int32_t* code) {
   SPARSP_TRY(check_ptr(workspace, "workspace", 256));
   if (!code) {

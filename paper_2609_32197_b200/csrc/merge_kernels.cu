@@ -1,0 +1,95 @@
+// Consumer-side helpers of the demand-routed exchange: the mask of one hop (consumer rank's query
+// blocks x producer rank's KV blocks) and the log-sum-exp merge of per-hop partial attention results.
+// Both are small element-wise kernels; the merge is HBM-bound (reads two outputs, writes one).
+#include "common.cuh"
+
+namespace sparsp {
+
+// hop[b][h][i][w] = rank[i] == consumer ? mask[b][h][i][w] & own_producer[w] : 0.  Thread per word.
+__global__ void hop_mask_kernel(const uint32_t* __restrict__ mask, const int32_t* __restrict__ rank, int NB,
+                                int Wd, int64_t n_words, int consumer, int producer,
+                                uint32_t* __restrict__ hop) {
+  const int64_t idx = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+  if (idx >= n_words) return;
+  const int w = (int)(idx % Wd);
+  const int i = (int)((idx / Wd) % NB);
+  uint32_t out = 0;
+  if (rank[i] == consumer) {
+    uint32_t own = 0;
+    for (int t = 0; t < 32; ++t) {
+      const int j = w * 32 + t;
+      if (j < NB && rank[j] == producer) own |= 1u << t;
+    }
+    out = mask[idx] & own;
+  }
+  hop[idx] = out;
+}
+
+// Thread per (row, 8 columns).  O_a, O_b, O: bf16 with the shape's strides; lse: fp32 [B][H][N].
+template <int D>
+__global__ void attn_merge_kernel(const __nv_bfloat16* __restrict__ Oa, const float* __restrict__ la,
+                                  const __nv_bfloat16* __restrict__ Ob, const float* __restrict__ lb,
+                                  __nv_bfloat16* __restrict__ O, float* __restrict__ lse, int H, int64_t N,
+                                  int64_t sB, int64_t sH, int64_t sT, int64_t n_rows) {
+  constexpr int VPR = D / 8;
+  const int64_t idx = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+  const int64_t row = idx / VPR;
+  const int col = (int)(idx % VPR);
+  if (row >= n_rows) return;
+  const int64_t tok = row % N, bh = row / N;
+  const int64_t off = (bh / H) * sB + (bh % H) * sH + tok * sT + col * 8;
+  const float a = la[row], b = lb[row];
+  const float m = fmaxf(a, b);
+  float wa = 0.0f, wb = 0.0f, out_lse = -INFINITY;
+  if (m > -INFINITY) {
+    const float ea = __expf(a - m), eb = __expf(b - m);
+    const float tot = ea + eb;
+    wa = ea / tot;
+    wb = eb / tot;
+    out_lse = m + __logf(tot);
+  }
+  const uint4 va = *reinterpret_cast<const uint4*>(Oa + off);
+  const uint4 vb = *reinterpret_cast<const uint4*>(Ob + off);
+  const uint32_t xa[4] = {va.x, va.y, va.z, va.w}, xb[4] = {vb.x, vb.y, vb.z, vb.w};
+  uint32_t r[4];
+#pragma unroll
+  for (int e = 0; e < 4; ++e) {
+    const float a0 = __uint_as_float(xa[e] << 16), a1 = __uint_as_float(xa[e] & 0xffff0000u);
+    const float b0 = __uint_as_float(xb[e] << 16), b1 = __uint_as_float(xb[e] & 0xffff0000u);
+    const __nv_bfloat162 h2 = __floats2bfloat162_rn(a0 * wa + b0 * wb, a1 * wa + b1 * wb);
+    r[e] = *reinterpret_cast<const uint32_t*>(&h2);
+  }
+  *reinterpret_cast<uint4*>(O + off) = make_uint4(r[0], r[1], r[2], r[3]);
+  if (col == 0) lse[row] = out_lse;
+}
+
+int launch_hop_mask(const Geometry& g, const uint32_t* mask, const int32_t* rank, int consumer, int producer,
+                    uint32_t* hop, cudaStream_t st) {
+  const int64_t n_words = (int64_t)g.B * g.H * g.NB * g.Wd;
+  hop_mask_kernel<<<(unsigned)((n_words + 255) / 256), 256, 0, st>>>(mask, rank, g.NB, g.Wd, n_words, consumer,
+                                                                     producer, hop);
+  count_launch();
+  SPARSP_CUDA_OK(cudaGetLastError());
+  return SPARSP_OK;
+}
+
+int launch_attn_merge(const sparsp_shape& s, const Geometry& g, const void* Oa, const float* la, const void* Ob,
+                      const float* lb, void* O, float* lse, cudaStream_t st) {
+  const int64_t n_rows = (int64_t)g.B * g.H * g.N;
+  const int64_t threads = n_rows * (g.d / 8);
+  const unsigned grid = (unsigned)((threads + 255) / 256);
+  auto a = (const __nv_bfloat16*)Oa;
+  auto b = (const __nv_bfloat16*)Ob;
+  auto o = (__nv_bfloat16*)O;
+  if (g.d == 64)
+    attn_merge_kernel<64><<<grid, 256, 0, st>>>(a, la, b, lb, o, lse, g.H, g.N, s.stride_batch, s.stride_head,
+                                                s.stride_token, n_rows);
+  else
+    attn_merge_kernel<128><<<grid, 256, 0, st>>>(a, la, b, lb, o, lse, g.H, g.N, s.stride_batch, s.stride_head,
+                                                 s.stride_token, n_rows);
+  count_launch();
+  SPARSP_CUDA_OK(cudaGetLastError());
+  return SPARSP_OK;
+}
+
+}  // namespace sparsp

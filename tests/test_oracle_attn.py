@@ -110,3 +110,46 @@ def test_explicit_scale_and_sampled_units(oracle_mod):
     part, _ = oracle_mod.attn_rows(Q, K, V, words, b, [(1, 2), (0, 0)], scale=0.3)
     assert np.array_equal(part[0], full[1, 2 * b:3 * b])
     assert np.array_equal(part[1], full[0, 0:b])
+
+
+def test_hop_partials_merge_to_full_attention(oracle_mod):
+    """Ring-style decomposition: attention of a consumer rank over each producer's blocks separately,
+    merged by log-sum-exp, equals attention over all kept blocks at once (and library SDPA)."""
+    rng = np.random.default_rng(6)
+    H, b, d, NB, P = 2, 64, 16, 6, 3
+    N = NB * b - 11
+    Q, K, V = _rand_qkv(rng, H, N, d)
+    M = rng.random((H, NB, NB)) < 0.5
+    for i in range(NB):
+        M[:, i, i] = True
+    words = _mask_words(M)
+    rank = np.array([0, 1, 2, 2, 0, 1], np.int32)
+    full, full_lse = oracle_mod.attn_all(Q, K, V, words, b)
+    for r in range(P):
+        acc = np.zeros_like(full)
+        acc_lse = np.full(full_lse.shape, -np.inf, np.float32)
+        for p in range(P):
+            hm = oracle_mod.hop_mask(words, rank, r, p)
+            # brute-force check of the hop mask definition
+            for h in range(H):
+                for i in range(NB):
+                    for j in range(NB):
+                        bit = (int(hm[h, i, j >> 5]) >> (j & 31)) & 1
+                        assert bit == int(M[h, i, j] and rank[i] == r and rank[j] == p)
+            part, part_lse = oracle_mod.attn_all(Q, K, V, hm, b)
+            acc, acc_lse = oracle_mod.attn_merge(acc, acc_lse, part, part_lse)
+        rows = np.repeat(rank == r, b)[:N]
+        assert np.abs(acc[:, rows] - full[:, rows]).max() < 1e-5
+        assert np.abs(acc_lse[:, rows] - full_lse[:, rows]).max() < 1e-5
+        assert np.all(acc_lse[:, ~rows] == -np.inf) and not acc[:, ~rows].any()
+
+
+def test_merge_special_cases(oracle_mod):
+    oa = np.array([[1.0, 2.0], [3.0, 4.0], [0.0, 0.0]], np.float32)
+    ob = np.array([[5.0, 6.0], [7.0, 8.0], [0.0, 0.0]], np.float32)
+    la = np.array([0.0, -np.inf, -np.inf], np.float32)
+    lb = np.array([0.0, 2.0, -np.inf], np.float32)
+    out, lse = oracle_mod.attn_merge(oa, la, ob, lb)
+    assert np.allclose(out[0], [3.0, 4.0]) and np.isclose(lse[0], np.log(2.0))   # equal weights: mean
+    assert np.allclose(out[1], [7.0, 8.0]) and lse[1] == 2.0                      # empty part a
+    assert not out[2].any() and lse[2] == -np.inf                                 # both empty
