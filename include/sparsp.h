@@ -168,6 +168,24 @@ SPARSP_API int sparsp_sparse_attn_fwd(const sparsp_shape* shape, const void* Q, 
  *   lse = log(exp(lse_a) + exp(lse_b)),  O = O_a * exp(lse_a - lse) + O_b * exp(lse_b - lse),
  * computed in fp32, O rounded to bf16.  O may alias O_a or O_b (and lse alias lse_a or lse_b).
  *   O_a, O_b, O  bf16, strided as in `shape`;  lse_a, lse_b, lse  fp32 [B][H][N] */
+/* sparsp_sparse_attn_fwd_packed: step 3 as the CONSUMER rank sees it after the exchange (Section 6: packed
+ * blocks arrive in the consumer's slot; here they are read in place, through the locally derived offsets of
+ * Section 5.2, instead of being scattered back first).  Computes the rows of the consumer's query blocks
+ * only; a kept KV block the consumer owns is read from K / V, every other kept block from the consumer's
+ * packed buffer as written by sparsp_demand_pack WITHOUT SPARSP_INCLUDE_LOCAL -- K and V of blocks owned by
+ * other ranks are never touched.  Rows of other ranks' query blocks are left unwritten.
+ *   mask, rank_of_block, union_mask, seg_offset, seg_total   as for / from sparsp_demand_pack
+ *   consumer         0 .. n_ranks-1
+ *   packed, packed_capacity_bytes, dst_base_bytes             the buffer sparsp_demand_pack filled, with the
+ *                    same bases (NULL = dense); bases must be multiples of the tile size block*d*2
+ *   O, lse           as for sparsp_sparse_attn_fwd */
+SPARSP_API int sparsp_sparse_attn_fwd_packed(const sparsp_shape* shape, const void* Q, const void* K, const void* V,
+                                             const uint32_t* mask, const int32_t* rank_of_block, int32_t n_ranks,
+                                             int32_t consumer, const uint32_t* union_mask,
+                                             const int64_t* seg_offset, const int64_t* seg_total, const void* packed,
+                                             int64_t packed_capacity_bytes, const int64_t* dst_base_bytes,
+                                             float softmax_scale, void* O, float* lse, void* workspace,
+                                             void* stream);
 SPARSP_API int sparsp_hop_mask(const sparsp_shape* shape, const uint32_t* mask, const int32_t* rank_of_block,
                                int32_t n_ranks, int32_t consumer, int32_t producer, uint32_t* hop_mask,
                                void* stream);

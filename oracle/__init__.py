@@ -288,3 +288,44 @@ def attn_merge(oa: np.ndarray, la: np.ndarray, ob: np.ndarray, lb: np.ndarray):
     lse = np.empty_like(la)
     lib().oracle_attn_merge(_p(oa), _p(la), _p(ob), _p(lb), _i64(rows), _i64(d), _p(out), _p(lse))
     return out, lse
+
+
+def consumer_view(K, V, packed: np.ndarray, dem: dict, rank_of_block: np.ndarray, b: int, consumer: int,
+                  dst_base: np.ndarray | None = None):
+    """What consumer rank r can see after the exchange: its own K/V blocks from the original tensors,
+    the blocks it demanded from other ranks out of ITS packed buffer (entry order: producer ascending,
+    head ascending, block ascending; entry = K tile then V tile), and NaN everywhere else -- so that an
+    attention over this view proves that nothing but local blocks and packed entries is needed.
+    -> (K_r, V_r) fp32 [H][NB*b][d]."""
+    Ks, Vs = _u16(K), _u16(V)
+    H, N, d = Ks.shape
+    NB = n_blocks(N, b)
+    P = dem["cnt"].shape[0]
+    entry = 2 * b * d * 2
+    if dst_base is None:
+        dst_base = np.concatenate([[0], np.cumsum(dem["total"])[:-1]]).astype(np.int64) * entry
+
+    def bf16_to_f32(u16):
+        return (u16.astype(np.uint32) << 16).view(np.float32)
+
+    Kr = np.full((H, NB * b, d), np.nan, dtype=np.float32)
+    Vr = np.full((H, NB * b, d), np.nan, dtype=np.float32)
+    for j in range(NB):
+        if rank_of_block[j] == consumer:
+            n_j = min(b, N - j * b)
+            Kr[:, j * b:j * b + n_j] = bf16_to_f32(Ks[:, j * b:j * b + n_j])
+            Vr[:, j * b:j * b + n_j] = bf16_to_f32(Vs[:, j * b:j * b + n_j])
+    for p in range(P):
+        if p == consumer:
+            continue
+        for h in range(H):
+            words = dem["U"][consumer, h]
+            pos = int(dem["seg_off"][consumer, p, h])
+            for j in range(NB):
+                if rank_of_block[j] == p and (int(words[j >> 5]) >> (j & 31)) & 1:
+                    off = int(dst_base[consumer]) + pos * entry
+                    tile = packed[off:off + entry].view(np.uint16).reshape(2, b, d)
+                    Kr[h, j * b:(j + 1) * b] = bf16_to_f32(tile[0])
+                    Vr[h, j * b:(j + 1) * b] = bf16_to_f32(tile[1])
+                    pos += 1
+    return Kr, Vr

@@ -29,7 +29,7 @@ EXPORTS = [
     "sparsp_geometry", "sparsp_resolve_topk", "sparsp_placement_contiguous", "sparsp_placement_periodic",
     "sparsp_workspace_bytes", "sparsp_block_mask", "sparsp_demand_pack", "sparsp_sparse_attn_fwd",
     "sparsp_status", "sparsp_last_error", "sparsp_launch_count", "sparsp_demand_plan_noalloc",
-    "sparsp_hop_mask", "sparsp_attn_merge",
+    "sparsp_hop_mask", "sparsp_attn_merge", "sparsp_sparse_attn_fwd_packed",
 ]
 
 
@@ -178,6 +178,17 @@ def sparsp_sparse_attn_fwd(shape, Q, K, V, mask, softmax_scale, O, lse, workspac
     _check(lib().sparsp_sparse_attn_fwd(ctypes.byref(shape), _ptr(Q), _ptr(K), _ptr(V), _ptr(mask),
                                         ctypes.c_float(softmax_scale), _ptr(O), _ptr(lse), _ptr(workspace),
                                         _stream()))
+
+
+def sparsp_sparse_attn_fwd_packed(shape, Q, K, V, mask, rank_of_block, n_ranks, consumer, union_mask, seg_offset,
+                                  seg_total, packed, packed_capacity_bytes, dst_base_bytes, softmax_scale, O, lse,
+                                  workspace):
+    _check(lib().sparsp_sparse_attn_fwd_packed(ctypes.byref(shape), _ptr(Q), _ptr(K), _ptr(V), _ptr(mask),
+                                               _ptr(rank_of_block), ctypes.c_int32(n_ranks), ctypes.c_int32(consumer),
+                                               _ptr(union_mask), _ptr(seg_offset), _ptr(seg_total), _ptr(packed),
+                                               ctypes.c_int64(packed_capacity_bytes), _ptr(dst_base_bytes),
+                                               ctypes.c_float(softmax_scale), _ptr(O), _ptr(lse), _ptr(workspace),
+                                               _stream()))
 
 
 def sparsp_hop_mask(shape, mask, rank_of_block, n_ranks, consumer, producer, hop_mask):

@@ -113,6 +113,10 @@ WsLayout make_layout(const Geometry& g, int P) {
   off += align_up((int64_t)g.B * g.H * g.NB * g.NB * 4, 256);
   L.pairs = off;  // query-block pairs of the attention CTAs, int32 [B][H][ceil(NB/2)][2]
   off += align_up((int64_t)g.B * g.H * ((g.NB + 1) / 2) * 2 * 4, 256);
+  L.slot = off;  // packed-buffer slot of every KV block for one consumer, int32 [B][H][NB]
+  off += align_up((int64_t)g.B * g.H * g.NB * 4, 256);
+  L.tile_base = off;  // first packed tile of that consumer per batch item, int64 [B]
+  off += align_up((int64_t)g.B * 8, 256);
   L.own = off;
   off += align_up((int64_t)P * g.Wd * 4, 256);
   L.ent_base = off;
@@ -290,6 +294,47 @@ int sparsp_sparse_attn_fwd(const sparsp_shape* shape, const void* Q, const void*
   const WsLayout L = make_layout(g, 1);
   return launch_attn(*shape, g, Q, K, V, mask, softmax_scale, O, lse, (char*)workspace, L,
                      (cudaStream_t)stream);
+}
+
+int sparsp_sparse_attn_fwd_packed(const sparsp_shape* shape, const void* Q, const void* K, const void* V,
+                                  const uint32_t* mask, const int32_t* rank_of_block, int32_t n_ranks,
+                                  int32_t consumer, const uint32_t* union_mask, const int64_t* seg_offset,
+                                  const int64_t* seg_total, const void* packed, int64_t packed_capacity_bytes,
+                                  const int64_t* dst_base_bytes, float softmax_scale, void* O, float* lse,
+                                  void* workspace, void* stream) {
+  Geometry g;
+  SPARSP_TRY(make_geometry(shape, &g));
+  SPARSP_TRY(check_supported(g));
+  SPARSP_TRY(check_strides(shape, g));
+  if (n_ranks < 1 || n_ranks > kMaxRanks || consumer < 0 || consumer >= n_ranks) {
+    set_error("consumer %d outside 0..%d", consumer, n_ranks - 1);
+    return SPARSP_ERR_INVALID_ARG;
+  }
+  SPARSP_TRY(check_ptr(Q, "Q"));
+  SPARSP_TRY(check_ptr(K, "K"));
+  SPARSP_TRY(check_ptr(V, "V"));
+  SPARSP_TRY(check_ptr(O, "O"));
+  SPARSP_TRY(check_ptr(mask, "mask", 4));
+  SPARSP_TRY(check_ptr(rank_of_block, "rank_of_block", 4));
+  SPARSP_TRY(check_ptr(union_mask, "union_mask", 4));
+  SPARSP_TRY(check_ptr(seg_offset, "seg_offset", 8));
+  SPARSP_TRY(check_ptr(seg_total, "seg_total", 8));
+  SPARSP_TRY(check_ptr(packed, "packed", 16));
+  SPARSP_TRY(check_ptr(workspace, "workspace", 256));
+  if (lse && (uintptr_t)lse % 4) return check_ptr((void*)1, "lse", 4);
+  if (dst_base_bytes && (uintptr_t)dst_base_bytes % 8) return check_ptr((void*)1, "dst_base_bytes", 8);
+  if (!(softmax_scale >= 0.0f)) {
+    set_error("softmax_scale must be >= 0");
+    return SPARSP_ERR_INVALID_ARG;
+  }
+  if (packed_capacity_bytes < (int64_t)g.b * g.d * 2) {
+    set_error("packed_capacity_bytes is smaller than one tile");
+    return SPARSP_ERR_INVALID_ARG;
+  }
+  const WsLayout L = make_layout(g, 1);
+  return launch_attn_packed(*shape, g, Q, K, V, mask, rank_of_block, n_ranks, consumer, union_mask, seg_offset,
+                            seg_total, packed, packed_capacity_bytes, dst_base_bytes, softmax_scale, O, lse,
+                            (char*)workspace, L, (cudaStream_t)stream);
 }
 
 int sparsp_hop_mask(const sparsp_shape* shape, const uint32_t* mask, const int32_t* rank_of_block, int32_t n_ranks,

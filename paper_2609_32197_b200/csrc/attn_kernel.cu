@@ -20,6 +20,8 @@
 // more than 2^8 since the reference last moved.
 // Every mbarrier wait is bounded; a wait that runs out sets SPARSP_ERR_TIMEOUT in the status word
 // and raises a CTA-wide flag that makes all later waits fall through, so the CTA still drains.
+#include <algorithm>
+
 #include "common.cuh"
 #include "sm100_ptx.cuh"
 
@@ -30,6 +32,11 @@ using namespace ptx;
 struct AttnParams {
   const uint32_t* mask;
   const int32_t* pairs;  // [B*H][ceil(NB/2)][2] query blocks of each CTA (second may be -1)
+  // packed-source mode (NULL = every tile comes from K / V): slot[bh][j] = entry index of KV block j in
+  // the consumer's packed buffer, or -1 if the consumer owns the block; tile_base = index of the
+  // consumer's first tile in the packed tensor map (a device scalar)
+  const int32_t* slot;
+  const int64_t* tile_base;
   __nv_bfloat16* O;
   float* lse;
   int32_t* status;
@@ -68,7 +75,8 @@ struct AttnCfg {
   static constexpr int kOffEntF = kOffEntJ + 2 * kMaxBlocks;     // uint8 [1024] bit q: kept by query block q
   static constexpr int kOffStat = kOffEntF + kMaxBlocks;         // float2 [2 streams][2 halves][128]
   static constexpr int kOffMax = kOffStat + 2 * 2 * 128 * 8;     // float [2 parities][2][2][128]
-  static constexpr int kOffBars = kOffMax + 2 * 2 * 2 * 128 * 4;
+  static constexpr int kOffSlot = kOffMax + 2 * 2 * 2 * 128 * 4;  // int32 [1024] packed-buffer slot per list entry
+  static constexpr int kOffBars = kOffSlot + 4 * kMaxBlocks;
   static constexpr int kNumBars = 1 + 4 * kStages + 8;
   // head_dim 64 leaves tensor-memory room for P next to S (S 2x128 + P 2x64 + O 2x64 = 512 columns):
   // Q K^T of the next tile can then start as soon as the softmax warps have READ S, instead of
@@ -142,7 +150,8 @@ __device__ __forceinline__ void named_bar_sync(int id, int n) {
 template <int D, int BLK>
 __global__ void __maxnreg__(96)
     attn_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmK,
-                    const __grid_constant__ CUtensorMap tmV, const AttnParams p) {
+                    const __grid_constant__ CUtensorMap tmV, const __grid_constant__ CUtensorMap tmP,
+                    const AttnParams p) {
   using C = AttnCfg<D, BLK>;
   constexpr int S = C::kStages;
   extern __shared__ unsigned char smem_dyn[];
@@ -155,6 +164,7 @@ __global__ void __maxnreg__(96)
   uint8_t* sEntF = smem + C::kOffEntF;
   float2* sStat = reinterpret_cast<float2*>(smem + C::kOffStat);
   float* sMax = reinterpret_cast<float*>(smem + C::kOffMax);
+  int32_t* sSlot = reinterpret_cast<int32_t*>(smem + C::kOffSlot);
   uint64_t* bars = reinterpret_cast<uint64_t*>(smem + C::kOffBars);
   uint64_t* bar_q = bars;
   uint64_t* k_full = bars + 1;
@@ -205,13 +215,13 @@ __global__ void __maxnreg__(96)
   }
   if (warp == 0) {
     // union of the two mask rows -> ascending entry list; flag bit q = kept by query block blk[q]
-    const uint32_t* mrow0 = p.mask + ((int64_t)bh * p.NB + blk[0]) * p.Wd;
+    const uint32_t* mrow0 = p.mask + ((int64_t)bh * p.NB + max(blk[0], 0)) * p.Wd;
     const uint32_t* mrow1 = p.mask + ((int64_t)bh * p.NB + max(blk[1], 0)) * p.Wd;
     int running = 0;
     for (int w0 = 0; w0 < p.Wd; w0 += 32) {
       const int w = w0 + lane;
       uint32_t rb[2];
-      rb[0] = (w < p.Wd) ? mrow0[w] : 0u;
+      rb[0] = (w < p.Wd && blk[0] >= 0) ? mrow0[w] : 0u;
       rb[1] = (w < p.Wd && blk[1] >= 0) ? mrow1[w] : 0u;
       uint32_t u = rb[0] | rb[1];
       const int mine = __popc(u);
@@ -227,6 +237,7 @@ __global__ void __maxnreg__(96)
         u &= u - 1;
         sEntJ[pos] = (uint16_t)(w * 32 + t);
         sEntF[pos] = (uint8_t)(((rb[0] >> t) & 1u) | (((rb[1] >> t) & 1u) << 1));
+        if (p.slot) sSlot[pos] = p.slot[(int64_t)bh * p.NB + w * 32 + t];
         ++pos;
       }
       running += __shfl_sync(0xffffffffu, incl, 31);
@@ -251,11 +262,12 @@ __global__ void __maxnreg__(96)
       // block re-reads the first: finite data whose rows are never used)
 #pragma unroll
       for (int q = 0; q < 2; ++q) {
-        const int tok = (blk[q] >= 0 ? blk[q] : blk[0]) * BLK;
+        const int tok = max(blk[q] >= 0 ? blk[q] : blk[0], 0) * BLK;
         unsigned char* dst = C::kSplitKV ? sQ + q * (BLK * 128) : sQ + q * C::kQBytes;
 #pragma unroll
         for (int c = 0; c < D / 64; ++c) tma_load_4d(dst + c * 16384, &tmQ, bar_q, c * 64, tok, head, batch);
       }
+      const int tile_base = p.slot ? (int)p.tile_base[batch] : 0;
       auto load_tile = [&](unsigned char* dst, const CUtensorMap* tm, uint64_t* bar, int n) {
 #ifdef SPARSP_ATTN_NOLOAD  // tuning builds only: reuse stale tiles to take TMA traffic out of the picture
         if (n >= S) {
@@ -268,9 +280,18 @@ __global__ void __maxnreg__(96)
         for (int e = 0; e < C::kEPT; ++e) {
           const int ent = min(n * C::kEPT + e, n_ent - 1);  // an absent second half re-reads the last entry
           const int j = sEntJ[ent];
+          const int slot = p.slot ? sSlot[ent] : -1;
+          if (slot < 0) {
 #pragma unroll
-          for (int c = 0; c < D / 64; ++c)
-            tma_load_4d(dst + c * 16384 + e * (BLK * 128), tm, bar, c * 64, j * BLK, head, batch);
+            for (int c = 0; c < D / 64; ++c)
+              tma_load_4d(dst + c * 16384 + e * (BLK * 128), tm, bar, c * 64, j * BLK, head, batch);
+          } else {
+            // remote block: its K tile and V tile are consecutive tiles of the consumer's packed buffer
+            const int tile = tile_base + 2 * slot + (tm == &tmV ? 1 : 0);
+#pragma unroll
+            for (int c = 0; c < D / 64; ++c)
+              tma_load_4d(dst + c * 16384 + e * (BLK * 128), &tmP, bar, c * 64, 0, tile, 0);
+          }
         }
       };
       int kn = 0, vn = 0;
@@ -780,22 +801,76 @@ static int make_tmap(CUtensorMap* out, const void* base, const sparsp_shape& s, 
   return SPARSP_OK;
 }
 
+// Packed buffer viewed as a sequence of (block x d) bf16 tiles: dims (d, block, n_tiles, 1).
+static int make_packed_tmap(CUtensorMap* out, const void* packed, int64_t capacity_bytes, const Geometry& g) {
+  EncodeTiledFn enc = get_encode_fn();
+  if (!enc) {
+    set_error("cuTensorMapEncodeTiled is not available from the driver");
+    return SPARSP_ERR_CUDA;
+  }
+  const int64_t tile_bytes = (int64_t)g.b * g.d * 2;
+  const int64_t n_tiles = capacity_bytes / tile_bytes;
+  if (n_tiles < 1 || n_tiles > 0x7fffffff) {
+    set_error("packed buffer holds %lld tiles: outside 1..2^31-1", (long long)n_tiles);
+    return SPARSP_ERR_INVALID_ARG;
+  }
+  cuuint64_t dims[4] = {(cuuint64_t)g.d, (cuuint64_t)g.b, (cuuint64_t)n_tiles, 1};
+  cuuint64_t strides[3] = {(cuuint64_t)g.d * 2, (cuuint64_t)tile_bytes, (cuuint64_t)(tile_bytes * n_tiles)};
+  cuuint32_t box[4] = {64, (cuuint32_t)g.b, 1, 1};
+  cuuint32_t estr[4] = {1, 1, 1, 1};
+  CUresult r = enc(out, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void*>(packed), dims, strides, box, estr,
+                   CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                   CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  if (r != CUDA_SUCCESS) {
+    set_error("cuTensorMapEncodeTiled (packed) failed with %d", (int)r);
+    return SPARSP_ERR_CUDA;
+  }
+  return SPARSP_OK;
+}
+
 template <int D, int BLK>
 static int launch_attn_t(const sparsp_shape& s, const Geometry& g, const void* Q, const void* K, const void* V,
-                         const AttnParams& p, cudaStream_t st) {
-  CUtensorMap tq, tk, tv;
+                         const void* packed, int64_t packed_capacity, const AttnParams& p, cudaStream_t st) {
+  CUtensorMap tq, tk, tv, tp;
   int rc;
   if ((rc = make_tmap(&tq, Q, s, g, BLK)) != SPARSP_OK) return rc;
   if ((rc = make_tmap(&tk, K, s, g, BLK)) != SPARSP_OK) return rc;
   if ((rc = make_tmap(&tv, V, s, g, BLK)) != SPARSP_OK) return rc;
+  if (packed) {
+    if ((rc = make_packed_tmap(&tp, packed, packed_capacity, g)) != SPARSP_OK) return rc;
+  } else {
+    tp = tk;  // never used without a slot table
+  }
   auto kern = attn_fwd_kernel<D, BLK>;
   const int smem = AttnCfg<D, BLK>::kDynamic;
   SPARSP_CUDA_OK(ensure_dynamic_smem((const void*)kern, smem));
   dim3 grid((unsigned)((g.NB + 1) / 2), (unsigned)(g.B * g.H));
-  kern<<<grid, kAttnThreads, smem, st>>>(tq, tk, tv, p);
+  kern<<<grid, kAttnThreads, smem, st>>>(tq, tk, tv, tp, p);
   count_launch();
   SPARSP_CUDA_OK(cudaGetLastError());
   return SPARSP_OK;
+}
+
+static int launch_attn_common(const sparsp_shape& s, const Geometry& g, const void* Q, const void* K, const void* V,
+                              const void* packed, int64_t packed_capacity, AttnParams p, float scale, void* O,
+                              float* lse, char* ws, const WsLayout& L, cudaStream_t st) {
+  p.O = (__nv_bfloat16*)O;
+  p.lse = lse;
+  p.status = (int32_t*)(ws + L.status);
+  p.N = g.N;
+  p.sB = s.stride_batch;
+  p.sH = s.stride_head;
+  p.sT = s.stride_token;
+  p.H = g.H;
+  p.NB = g.NB;
+  p.Wd = g.Wd;
+  const float sc = scale > 0.0f ? scale : 1.0f / sqrtf((float)g.d);
+  p.scale_log2 = sc * 1.4426950408889634f;
+  p.wait_limit = 200000000LL;  // about 0.1 s of SM clocks
+  if (g.d == 64 && g.b == 64) return launch_attn_t<64, 64>(s, g, Q, K, V, packed, packed_capacity, p, st);
+  if (g.d == 64 && g.b == 128) return launch_attn_t<64, 128>(s, g, Q, K, V, packed, packed_capacity, p, st);
+  if (g.d == 128 && g.b == 64) return launch_attn_t<128, 64>(s, g, Q, K, V, packed, packed_capacity, p, st);
+  return launch_attn_t<128, 128>(s, g, Q, K, V, packed, packed_capacity, p, st);
 }
 
 int launch_attn(const sparsp_shape& s, const Geometry& g, const void* Q, const void* K, const void* V,
@@ -811,23 +886,109 @@ int launch_attn(const sparsp_shape& s, const Geometry& g, const void* Q, const v
   AttnParams p;
   p.mask = mask;
   p.pairs = pairs;
-  p.O = (__nv_bfloat16*)O;
-  p.lse = lse;
-  p.status = (int32_t*)(ws + L.status);
-  p.N = g.N;
-  p.sB = s.stride_batch;
-  p.sH = s.stride_head;
-  p.sT = s.stride_token;
-  p.H = g.H;
-  p.NB = g.NB;
-  p.Wd = g.Wd;
-  const float sc = scale > 0.0f ? scale : 1.0f / sqrtf((float)g.d);
-  p.scale_log2 = sc * 1.4426950408889634f;
-  p.wait_limit = 200000000LL;  // about 0.1 s of SM clocks
-  if (g.d == 64 && g.b == 64) return launch_attn_t<64, 64>(s, g, Q, K, V, p, st);
-  if (g.d == 64 && g.b == 128) return launch_attn_t<64, 128>(s, g, Q, K, V, p, st);
-  if (g.d == 128 && g.b == 64) return launch_attn_t<128, 64>(s, g, Q, K, V, p, st);
-  return launch_attn_t<128, 128>(s, g, Q, K, V, p, st);
+  p.slot = nullptr;
+  p.tile_base = nullptr;
+  return launch_attn_common(s, g, Q, K, V, nullptr, 0, p, scale, O, lse, ws, L, st);
+}
+
+// ------------------------------------------------------------------------------------------------
+// Packed-source attention for one consumer rank: pairs are formed among the consumer's own query
+// blocks, and every kept KV block the consumer does not own is read from the consumer's packed buffer.
+// ------------------------------------------------------------------------------------------------
+// pairs of the consumer's blocks (ascending, neighbours in that order); the rest of the table is (-1, -1)
+__global__ void pair_rank_kernel(const int32_t* __restrict__ rank, int NB, int consumer, int32_t* __restrict__ pairs) {
+  const int n_pairs = (NB + 1) / 2;
+  int32_t* out = pairs + (int64_t)blockIdx.x * n_pairs * 2;
+  for (int i = threadIdx.x; i < 2 * n_pairs; i += blockDim.x) out[i] = -1;
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    int k = 0;
+    for (int i = 0; i < NB; ++i)
+      if (rank[i] == consumer) out[k++] = i;  // pair c = entries 2c and 2c+1
+  }
+}
+
+// slot[bh][j] = entry index of block j inside the consumer's packed buffer (pack order: producer ascending,
+// head ascending, block ascending), for every block of the consumer's union that another rank owns.  One warp
+// per (batch, producer, head).  The table must have been filled with -1.  Also writes tile_base[b].
+__global__ void slot_kernel(const uint32_t* __restrict__ U, const int32_t* __restrict__ rank,
+                            const int64_t* __restrict__ seg_off, const int64_t* __restrict__ seg_total,
+                            const int64_t* __restrict__ dst_base, int B, int H, int NB, int Wd, int P, int consumer,
+                            int64_t tile_bytes, int32_t* __restrict__ slot, int64_t* __restrict__ tile_base) {
+  const int64_t wid = ((int64_t)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
+  const int lane = threadIdx.x & 31;
+  if (wid < B && lane == 0) {  // first tile of the consumer's buffer for batch item wid
+    const int64_t br = wid * P + consumer;
+    int64_t base;
+    if (dst_base) {
+      base = dst_base[br];
+    } else {
+      base = 0;
+      for (int64_t t = 0; t < br; ++t) base += seg_total[t] * 2 * tile_bytes;
+    }
+    tile_base[wid] = base / tile_bytes;
+  }
+  const int64_t n_seg = (int64_t)B * P * H;
+  if (wid >= n_seg) return;
+  const int h = (int)(wid % H);
+  const int prod = (int)((wid / H) % P);
+  const int bb = (int)(wid / ((int64_t)H * P));
+  if (prod == consumer) return;
+  const uint32_t* u = U + ((int64_t)(bb * P + consumer) * H + h) * Wd;
+  const int64_t first = seg_off[((int64_t)(bb * P + consumer) * P + prod) * H + h];
+  int32_t* out = slot + (int64_t)(bb * H + h) * NB;
+  int running = 0;
+  for (int w0 = 0; w0 < Wd; w0 += 32) {
+    const int w = w0 + lane;
+    uint32_t bits = 0;
+    if (w < Wd) {
+      uint32_t own = 0;
+      for (int t = 0; t < 32; ++t) {
+        const int j = w * 32 + t;
+        if (j < NB && rank[j] == prod) own |= 1u << t;
+      }
+      bits = u[w] & own;
+    }
+    const int mine = __popc(bits);
+    int incl = mine;
+#pragma unroll
+    for (int sft = 1; sft < 32; sft <<= 1) {
+      const int v = __shfl_up_sync(0xffffffffu, incl, sft);
+      if (lane >= sft) incl += v;
+    }
+    int pos = running + incl - mine;
+    while (bits) {
+      const int t = __ffs(bits) - 1;
+      bits &= bits - 1;
+      out[w * 32 + t] = (int32_t)(first + pos);
+      ++pos;
+    }
+    running += __shfl_sync(0xffffffffu, incl, 31);
+  }
+}
+
+int launch_attn_packed(const sparsp_shape& s, const Geometry& g, const void* Q, const void* K, const void* V,
+                       const uint32_t* mask, const int32_t* rank, int P, int consumer, const uint32_t* U,
+                       const int64_t* seg_off, const int64_t* seg_total, const void* packed, int64_t capacity,
+                       const int64_t* dst_base, float scale, void* O, float* lse, char* ws, const WsLayout& L,
+                       cudaStream_t st) {
+  int32_t* pairs = (int32_t*)(ws + L.pairs);
+  int32_t* slot = (int32_t*)(ws + L.slot);
+  int64_t* tile_base = (int64_t*)(ws + L.tile_base);
+  const int64_t tile_bytes = (int64_t)g.b * g.d * 2;
+  SPARSP_CUDA_OK(cudaMemsetAsync(slot, 0xFF, (size_t)g.B * g.H * g.NB * 4, st));
+  pair_rank_kernel<<<g.B * g.H, 128, 0, st>>>(rank, g.NB, consumer, pairs);
+  const int64_t n_warps = std::max<int64_t>((int64_t)g.B * P * g.H, g.B);
+  slot_kernel<<<(unsigned)((n_warps * 32 + 255) / 256), 256, 0, st>>>(U, rank, seg_off, seg_total, dst_base, g.B, g.H,
+                                                                    g.NB, g.Wd, P, consumer, tile_bytes, slot,
+                                                                    tile_base);
+  count_launch(2);
+  AttnParams p;
+  p.mask = mask;
+  p.pairs = pairs;
+  p.slot = slot;
+  p.tile_base = tile_base;
+  return launch_attn_common(s, g, Q, K, V, packed, capacity, p, scale, O, lse, ws, L, st);
 }
 
 #ifdef SPARSP_ATTN_PROFILE

@@ -34,7 +34,7 @@ struct PackEntry {
 };
 
 struct WsLayout {
-  int64_t status, pooled_q, pooled_k, scores, pairs, own, ent_base, n_entries, entries, total;
+  int64_t status, pooled_q, pooled_k, scores, pairs, slot, tile_base, own, ent_base, n_entries, entries, total;
 };
 
 void set_error(const char* fmt, ...);
@@ -73,6 +73,11 @@ int launch_attn(const sparsp_shape& s, const Geometry& g, const void* Q, const v
                 const uint32_t* mask, float scale, void* O, float* lse, char* ws, const WsLayout& L,
                 cudaStream_t st);
 
+int launch_attn_packed(const sparsp_shape& s, const Geometry& g, const void* Q, const void* K, const void* V,
+                       const uint32_t* mask, const int32_t* rank, int P, int consumer, const uint32_t* U,
+                       const int64_t* seg_off, const int64_t* seg_total, const void* packed, int64_t capacity,
+                       const int64_t* dst_base, float scale, void* O, float* lse, char* ws, const WsLayout& L,
+                       cudaStream_t st);
 int launch_hop_mask(const Geometry& g, const uint32_t* mask, const int32_t* rank, int consumer, int producer,
                     uint32_t* hop, cudaStream_t st);
 int launch_attn_merge(const sparsp_shape& s, const Geometry& g, const void* Oa, const float* la, const void* Ob,

@@ -89,3 +89,103 @@ def test_merge_kernel_matches_oracle_elementwise(oracle_mod, binding):
     fin = np.isfinite(rl)
     assert np.abs(lse.cpu().numpy()[fin] - rl[fin]).max() < 1e-4
     assert np.array_equal(np.isneginf(lse.cpu().numpy()), np.isneginf(rl))
+
+
+@pytest.mark.parametrize("d,b,layout", [(128, 128, "HND"), (64, 64, "HND"), (128, 64, "NHD"), (64, 128, "HND")])
+def test_attention_reading_remote_blocks_from_the_packed_buffer(oracle_mod, binding, d, b, layout):
+    """The consumer-side attention must produce the consumer's rows from its own K/V blocks plus its
+    packed buffer alone: the K/V handed to it have every block the consumer does NOT own overwritten
+    with NaN, and the oracle computes the expected rows from the same restricted view."""
+    from paper_2609_32197_b200 import synth
+    H, P = 3, 3
+    # a few more kept blocks than the minimum: with very few, |O| grows past 4 where half a bf16 ulp (0.0156) of
+    # output rounding alone nearly uses up the bound
+    wl = synth.Workload("packed", H, d, (5, 11, 13), 70, b, 5 if b == 128 else 9, None, P, seed=61)
+    Q, K, V = synth.make_qkv(wl, "cpu")
+    N, NB = wl.n_tokens, wl.n_blocks
+    shape = binding.make_shape(H, d, wl.grid, wl.n_text, b, layout=layout)
+    Qd, Kd, Vd = (pu.to_layout(x.cuda(), layout) for x in (Q, K, V))
+    ws = binding.make_workspace(shape, P)
+    ref = oracle_mod.block_mask(Q, K, b, wl.topk_abs, wl.n_text)
+    mo = pu.gpu_block_mask(binding, shape, Qd, Kd, wl.topk_abs, ws)
+    rank = np.array([(j * 2 + j // 3) % P for j in range(NB)], np.int32)
+    rank_d = torch.as_tensor(rank).cuda()
+    dg = pu.gpu_demand_pack(binding, shape, mo["mask"], rank_d, P, 0, Kd, Vd, ws)
+    dref = oracle_mod.demand(ref["mask"], rank, P, b, d)
+    packed_ref = oracle_mod.pack(K, V, dref["U"], rank, b, P, dref["total"])
+    assert np.array_equal(dg["packed"].cpu().numpy()[:packed_ref.size], packed_ref)
+    blk_of_tok = np.arange(N) // b
+    for r in range(P):
+        # poison everything the consumer does not own
+        foreign = torch.as_tensor(rank[blk_of_tok] != r)
+        Kp, Vp = K.clone(), V.clone()
+        Kp[:, foreign] = float("nan")
+        Vp[:, foreign] = float("nan")
+        Kpd, Vpd = pu.to_layout(Kp.cuda(), layout), pu.to_layout(Vp.cuda(), layout)
+        O = torch.full_like(Qd, 7.0)
+        lse = torch.full((1, H, N), 7.0, dtype=torch.float32, device="cuda")
+        binding.sparsp_sparse_attn_fwd_packed(shape, Qd, Kpd, Vpd, mo["mask"], rank_d, P, r, dg["union_mask"],
+                                              dg["seg_offset"], dg["seg_total"], dg["packed"],
+                                              dg["packed"].numel() - 64, None, 0.0, O, lse, ws)
+        torch.cuda.synchronize()
+        assert binding.sparsp_status(ws) == binding.SPARSP_OK, binding.sparsp_last_error()
+        # oracle: attention over the consumer's restricted view (NaN outside local + packed blocks)
+        Kr, Vr = oracle_mod.consumer_view(K, V, packed_ref, dref, rank, b, r)
+        units = [(h, i) for h in range(H) for i in range(NB) if rank[i] == r]
+        Kv = torch.tensor(Kr[:, :N]).to(torch.bfloat16)
+        Vv = torch.tensor(Vr[:, :N]).to(torch.bfloat16)
+        got = pu.from_layout(O, layout)
+        mx, mean = pu.check_attn_units(oracle_mod, Q, Kv, Vv, ref["mask"], b, got, units, lse_gpu=lse[0])
+        # rows of other ranks are left as they were
+        other = torch.as_tensor(np.repeat(rank != r, b)[:N])
+        assert bool((got[:, other].float() == 7.0).all()) and bool((lse[0][:, other] == 7.0).all())
+
+
+def test_packed_attention_with_explicit_slot_bases(oracle_mod, binding):
+    """Consumer slots placed out of order with a gap between them: the attention finds its tiles
+    through the same bases the pack call was given."""
+    from paper_2609_32197_b200 import synth
+    H, P, d, b = 2, 2, 64, 64
+    wl = synth.Workload("packed_base", H, d, (4, 9, 11), 40, b, 6, None, P, seed=62)
+    Q, K, V = synth.make_qkv(wl, "cpu")
+    N, NB = wl.n_tokens, wl.n_blocks
+    shape = binding.make_shape(H, d, wl.grid, wl.n_text, b)
+    Qd, Kd, Vd = (x.cuda() for x in (Q, K, V))
+    ws = binding.make_workspace(shape, P)
+    mo = pu.gpu_block_mask(binding, shape, Qd, Kd, wl.topk_abs, ws)
+    rank = (np.arange(NB) % P).astype(np.int32)
+    rank_d = torch.as_tensor(rank).cuda()
+    plan = pu.gpu_demand_pack(binding, shape, mo["mask"], rank_d, P, binding.SPARSP_PLAN_ONLY, None, None, ws)
+    tot = plan["seg_total"][0].cpu().numpy()
+    entry = 2 * b * d * 2
+    base = np.array([[(int(tot[1]) + 3) * entry, 0]], np.int64)      # rank 1 first, 3 entries of gap, then rank 0
+    base_d = torch.as_tensor(base).cuda()
+    cap = int(tot.sum()) + 3
+    dg = pu.gpu_demand_pack(binding, shape, mo["mask"], rank_d, P, 0, Kd, Vd, ws, capacity_entries=cap, dst_base=base_d)
+    assert binding.sparsp_status(ws) == binding.SPARSP_OK
+    mask_np = pu.u32(mo["mask"][0])
+    blk_of_tok = np.arange(N) // b
+    for r in range(P):
+        foreign = torch.as_tensor(rank[blk_of_tok] != r)
+        Kp, Vp = K.clone(), V.clone()
+        Kp[:, foreign] = float("nan")
+        Vp[:, foreign] = float("nan")
+        O = torch.zeros_like(Qd)
+        lse = torch.zeros((1, H, N), dtype=torch.float32, device="cuda")
+        binding.sparsp_sparse_attn_fwd_packed(shape, Qd, Kp.cuda(), Vp.cuda(), mo["mask"], rank_d, P, r,
+                                              dg["union_mask"], dg["seg_offset"], dg["seg_total"], dg["packed"],
+                                              cap * entry, base_d, 0.0, O, lse, ws)
+        torch.cuda.synchronize()
+        assert binding.sparsp_status(ws) == binding.SPARSP_OK, binding.sparsp_last_error()
+        units = [(h, i) for h in range(H) for i in range(NB) if rank[i] == r]
+        pu.check_attn_units(oracle_mod, Q, K, V, mask_np, b, O, units, lse_gpu=lse[0])
+
+
+def test_packed_attention_rejects_bad_arguments(binding):
+    shape = binding.make_shape(2, 64, (2, 4, 8), 0, 64)
+    ws = binding.make_workspace(shape, 2)
+    z = torch.zeros(64, dtype=torch.uint8, device="cuda")
+    for consumer, cap in [(2, 1 << 20), (-1, 1 << 20), (0, -5)]:
+        with pytest.raises(RuntimeError):
+            binding.sparsp_sparse_attn_fwd_packed(shape, z, z, z, z, z, 2, consumer, z, z, z, z, cap, None, 0.0, z,
+                                                  None, ws)

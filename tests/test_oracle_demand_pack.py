@@ -209,3 +209,31 @@ def test_placements(oracle_mod):
     # text tail: round robin
     r = oracle_mod.placement_periodic(8, 2, 64, 3 * 64, 6 * 64)
     assert list(r[6:]) == [0, 1]
+
+
+def test_consumer_view_rebuilds_exactly_the_demanded_blocks(oracle_mod):
+    """Local blocks + the consumer's packed entries reproduce K/V on every block its rows keep, and
+    nothing else is available (NaN) -- the packed layout and the locally derived offsets suffice."""
+    rng = np.random.default_rng(11)
+    H, b, d, P = 2, 64, 8, 3
+    N = 5 * b + 30
+    NB = 6
+    K = torch.tensor(rng.standard_normal((H, N, d)), dtype=torch.float32).to(torch.bfloat16)
+    V = torch.tensor(rng.standard_normal((H, N, d)), dtype=torch.float32).to(torch.bfloat16)
+    M = rng.random((H, NB, NB)) < 0.4
+    rank = np.array([0, 1, 2, 2, 0, 1], np.int32)
+    dem = oracle_mod.demand(_mask_from_bool(M), rank, P, b, d)
+    packed = oracle_mod.pack(K, V, dem["U"], rank, b, P, dem["total"])
+    Kf = np.zeros((H, NB * b, d), np.float32)
+    Kf[:, :N] = K.float().numpy()
+    for r in range(P):
+        Kr, Vr = oracle_mod.consumer_view(K, V, packed, dem, rank, b, r)
+        for h in range(H):
+            for j in range(NB):
+                needed = rank[j] == r or any(M[h, i, j] for i in range(NB) if rank[i] == r)
+                blk = Kr[h, j * b:(j + 1) * b]
+                n_j = min(b, N - j * b)
+                if needed:
+                    assert np.array_equal(blk[:n_j], Kf[h, j * b:j * b + n_j])
+                else:
+                    assert np.isnan(blk).all()
