@@ -327,7 +327,7 @@ def run_ours(args):
                      "peak": peaks["bf16_tflops"], "peak_source": peaks["source"] + " burst", "unit": "TFLOP/s",
                      "frac": attn_tflops / peaks["bf16_tflops"],
                      "traffic": ATTN_DRAM_TRAFFIC.get((wl.name, k))},
-        "roofline_pack": {"bound": "hbm", "kernel": "pack_kernel" if b * d < 8192 else "pack_tile_kernel", "achieved": pack_gbs, "peak": peaks["hbm_gbs"],
+        "roofline_pack": {"bound": "hbm", "kernel": "pack_bulk_kernel", "achieved": pack_gbs, "peak": peaks["hbm_gbs"],
                           "peak_source": peaks["source"], "unit": "GB/s", "frac": pack_gbs / peaks["hbm_gbs"],
                           "algorithmic_bytes": pack_bytes},
         "e2e": {"value": None if e2e_ms != e2e_ms else flops_all / (e2e_ms * 1e-3) / 1e12, "unit": "TFLOP/s",
