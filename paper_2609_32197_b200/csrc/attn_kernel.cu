@@ -1,23 +1,26 @@
 // Step 3: block-sparse FlashAttention forward on tcgen05 tensor cores (sm_100a).
 //
-// A CTA owns two adjacent query blocks of one (batch, head) and runs two independent softmax
-// "streams" so that one stream's exponentials overlap the other stream's MMAs:
-//   block = 128: the two query blocks are two 128-row Q tiles; stream s = Q tile s.  The CTA walks
-//                the UNION of the two rows' kept KV blocks; a stream skips the blocks its own row
-//                does not keep, K/V tiles that both keep are loaded once.
-//   block = 64 : the two query blocks are stacked into ONE 128-row Q tile (full-rate M = 128 MMAs);
-//                a KV tile is two entries of the union list (128 keys, full-rate N = 128); each
-//                64x64 quadrant the mask does not keep is zeroed in P.  Stream s takes the KV tiles
-//                of parity s into its own accumulator; the two partial results are merged at the end.
-// Warp roles (608 threads): warp 0 = TMA producer (K ring and V ring, polled independently),
-// warps 1 and 18 = MMA issuers of stream 0 / 1 (one thread each, so the streams never serialise on
-// one instruction stream), warps 2-9 / 10-17 = softmax warps of stream 0 / 1.  A query row
-// is shared by TWO threads of different warps, each owning 64 of the tile's 128 key columns: a row
-// of S is read from tensor memory once, in 64 registers, and the pair exchanges its two partial row
-// maxima through shared memory behind a 64-thread named barrier.  Tensor memory: S_s (128 fp32 columns, overwritten in place by bf16 P_s, which
-// the P.V MMA reads straight from tensor memory) and O_s (d fp32 columns) per stream.
-// Online softmax is base-2 in fp32; O is rescaled lazily, only when a row's maximum has grown by
-// more than 2^8 since the reference last moved.
+// A CTA owns ONE 128-row Q tile of one (batch, head) and one fp32 accumulator O in tensor memory:
+//   block = 128: the Q tile is one query block; the CTA walks that block's kept KV blocks.
+//   block = 64 : two query blocks (chosen by a pairing pass so that their kept lists overlap) are stacked
+//                into the Q tile (full-rate M = 128 MMAs); a KV tile is two entries of the UNION of their
+//                kept lists (128 keys, full-rate N = 128); each 64x64 quadrant the mask does not keep is
+//                zeroed in P.
+// The scores S = Q K^T and the probabilities P are double-buffered in tensor memory (S: 2 x 128 fp32
+// columns, P: 2 x 64 columns of packed bf16, O: d columns), so that the tensor pipe always has the next
+// tiles' MMAs queued while the softmax of the current tile runs: Q K^T of tile n+2 starts as soon as the
+// scores of tile n have been READ, and P V of tile n is issued as soon as P_n is written.
+// Warp roles (384 threads = 3 warpgroups; the first hands most of its registers to the other two):
+//   warp 0      TMA producer (K ring and V ring, polled independently)
+//   warp 1      issues every Q K^T          warp 2      issues every P V
+//   warps 4-7   softmax of the even tiles   warps 8-11  softmax of the odd tiles
+// A softmax thread owns one query row of its tile: the whole 128-column row of S sits in registers.  The
+// two threads that own the same row (one per warpgroup) share the row's reference maximum through shared
+// memory and take their decisions strictly in tile order (a pair of 64-thread named barriers per row
+// group hands the turn back and forth); each keeps its own partial row sum.
+// Online softmax is base-2 in fp32; O is rescaled lazily, only when a row's maximum has grown by more
+// than 2^8 since the reference last moved -- the thread that decides so first waits for every P V
+// issued so far, then rescales the row of O.
 // Every mbarrier wait is bounded; a wait that runs out sets SPARSP_ERR_TIMEOUT in the status word
 // and raises a CTA-wide flag that makes all later waits fall through, so the CTA still drains.
 #include <algorithm>
@@ -31,7 +34,9 @@ using namespace ptx;
 
 struct AttnParams {
   const uint32_t* mask;
-  const int32_t* pairs;  // [B*H][ceil(NB/2)][2] query blocks of each CTA (second may be -1)
+  // block 64: [B*H][ceil(NB/2)][2] query blocks of each CTA (second may be -1); block 128: NULL (CTA x
+  // handles block x) or [B*H][2*ceil(NB/2)] query block of each CTA (-1 = none)
+  const int32_t* pairs;
   // packed-source mode (NULL = every tile comes from K / V): slot[bh][j] = entry index of KV block j in
   // the consumer's packed buffer, or -1 if the consumer owns the block; tile_base = index of the
   // consumer's first tile in the packed tensor map (a device scalar)
@@ -47,48 +52,42 @@ struct AttnParams {
   long long wait_limit;
 };
 
-constexpr int kAttnThreads = 608;
-constexpr int kIssuer1Warp = 18;  // warp 1 issues the MMAs of stream 0, warp 18 those of stream 1
+constexpr int kAttnThreads = 384;  // three warpgroups: utility warps, softmax of the even tiles, softmax of the odd tiles
+// register budget per thread after the warpgroups re-balance (128*72 + 256*216 = 384*168)
+#define SPARSP_REGS_UTILITY 72
+#define SPARSP_REGS_SOFTMAX 216
 constexpr int kTmemCols = 512;
 constexpr float kGrowThreshold = 8.0f;
-// Tuning switches (compile-time): packed fp32x2 arithmetic in the exponential loop, and how many of
-// the exponentials go to the FMA pipe instead of the special-function unit (every n-th pair; 0 = none).
-#ifndef SPARSP_TUNE_F32X2
-#define SPARSP_TUNE_F32X2 1
-#endif
+// Tuning switch (compile-time): how many of the exponentials go to the FMA pipe instead of the
+// special-function unit (every n-th pair; 0 = none).
 #ifndef SPARSP_TUNE_POLY
 #define SPARSP_TUNE_POLY 3
 #endif
 
 template <int D, int BLK>
 struct AttnCfg {
-  static constexpr bool kSplitKV = (BLK == 64);   // one Q tile, streams split the KV tiles
-  static constexpr int kQTiles = kSplitKV ? 1 : 2;
-  static constexpr int kEPT = 128 / BLK;          // union-list entries per 128-key KV tile
-  static constexpr int kStages = (D == 64) ? 4 : 2;
+  static constexpr bool kStacked = (BLK == 64);  // Q tile = two 64-token query blocks
+  static constexpr int kEPT = 128 / BLK;         // kept-list entries per 128-key KV tile
+  static constexpr int kStagesK = (D == 64) ? 4 : 3;
+  static constexpr int kStagesV = (D == 64) ? 4 : 2;
   static constexpr int kQBytes = 128 * D * 2;
   static constexpr int kTileBytes = 128 * D * 2;  // one K or V tile
   static constexpr int kOffQ = 0;
-  static constexpr int kOffK = kOffQ + kQTiles * kQBytes;
-  static constexpr int kOffV = kOffK + kStages * kTileBytes;
-  static constexpr int kOffEntJ = kOffV + kStages * kTileBytes;  // uint16 [1024] union list
-  static constexpr int kOffEntF = kOffEntJ + 2 * kMaxBlocks;     // uint8 [1024] bit q: kept by query block q
-  static constexpr int kOffStat = kOffEntF + kMaxBlocks;         // float2 [2 streams][2 halves][128]
-  static constexpr int kOffMax = kOffStat + 2 * 2 * 128 * 8;     // float [2 parities][2][2][128]
-  static constexpr int kOffSlot = kOffMax + 2 * 2 * 2 * 128 * 4;  // int32 [1024] packed-buffer slot per list entry
+  static constexpr int kOffK = kOffQ + kQBytes;
+  static constexpr int kOffV = kOffK + kStagesK * kTileBytes;
+  static constexpr int kOffEntJ = kOffV + kStagesV * kTileBytes;  // uint16 [1024] kept / union list
+  static constexpr int kOffEntF = kOffEntJ + 2 * kMaxBlocks;      // uint8 [1024] bit q: kept by query block q
+  static constexpr int kOffStat = kOffEntF + kMaxBlocks;          // float2 [2 warpgroups][128]
+  static constexpr int kOffRef = kOffStat + 2 * 128 * 8;          // float [128] reference maximum per row
+  static constexpr int kOffSlot = kOffRef + 128 * 4;              // int32 [1024] packed-buffer slot per list entry
   static constexpr int kOffBars = kOffSlot + 4 * kMaxBlocks;
-  static constexpr int kNumBars = 1 + 4 * kStages + 8;
-  // head_dim 64 leaves tensor-memory room for P next to S (S 2x128 + P 2x64 + O 2x64 = 512 columns):
-  // Q K^T of the next tile can then start as soon as the softmax warps have READ S, instead of
-  // waiting for P V to finish reading P out of the same columns.
-  static constexpr bool kDecoupledP = (D == 64);
-  static constexpr int kColP = 256;                       // first P column (decoupled layout)
-  static constexpr int kColO = kDecoupledP ? 384 : 256;   // first O column
+  static constexpr int kNumBars = 1 + 2 * (kStagesK + kStagesV) + 10;
+  static constexpr int kColS = 0;    // S buffers: columns [0, 256)
+  static constexpr int kColP = 256;  // P buffers: columns [256, 384)
+  static constexpr int kColO = 384;  // accumulator: columns [384, 384 + d)
   static constexpr int kOffMisc = kOffBars + 8 * kNumBars;
   static constexpr int kTotal = kOffMisc + 32;
   static constexpr int kDynamic = kTotal + 1024;  // slack for the 1024-byte alignment of the base
-  static constexpr int kMergeStride = D / 4 + 4;  // floats per row of the merge buffer
-  static_assert(4 * 128 * kMergeStride * 4 <= 2 * kStages * kTileBytes, "merge buffer must fit the K/V rings");
   static_assert(kDynamic <= 232448, "shared memory budget");
 };
 
@@ -98,7 +97,7 @@ struct AttnCfg {
 __device__ unsigned long long g_attn_prof[16];
 #define PROF_T(var) const long long var = clock64()
 #define PROF_ADD(slot, a, b) \
-  if (lane == 0 && (warp == 2 || warp == 1)) atomicAdd(&g_attn_prof[slot], (unsigned long long)((b) - (a)))
+  if (lane == 0 && (warp == 4 || warp == 1)) atomicAdd(&g_attn_prof[slot], (unsigned long long)((b) - (a)))
 #else
 #define PROF_T(var)
 #define PROF_ADD(slot, a, b)
@@ -148,12 +147,12 @@ __device__ __forceinline__ void named_bar_sync(int id, int n) {
 }
 
 template <int D, int BLK>
-__global__ void __maxnreg__(96)
+__global__ void __launch_bounds__(kAttnThreads, 1)
     attn_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmK,
                     const __grid_constant__ CUtensorMap tmV, const __grid_constant__ CUtensorMap tmP,
                     const AttnParams p) {
   using C = AttnCfg<D, BLK>;
-  constexpr int S = C::kStages;
+  constexpr int SK = C::kStagesK, SV = C::kStagesV;
   extern __shared__ unsigned char smem_dyn[];
   unsigned char* smem =
       reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_dyn) + 1023) & ~uintptr_t(1023));
@@ -163,18 +162,21 @@ __global__ void __maxnreg__(96)
   uint16_t* sEntJ = reinterpret_cast<uint16_t*>(smem + C::kOffEntJ);
   uint8_t* sEntF = smem + C::kOffEntF;
   float2* sStat = reinterpret_cast<float2*>(smem + C::kOffStat);
-  float* sMax = reinterpret_cast<float*>(smem + C::kOffMax);
+  volatile float* sRef = reinterpret_cast<volatile float*>(smem + C::kOffRef);
   int32_t* sSlot = reinterpret_cast<int32_t*>(smem + C::kOffSlot);
   uint64_t* bars = reinterpret_cast<uint64_t*>(smem + C::kOffBars);
   uint64_t* bar_q = bars;
   uint64_t* k_full = bars + 1;
-  uint64_t* k_empty = k_full + S;
-  uint64_t* v_full = k_empty + S;
-  uint64_t* v_empty = v_full + S;
-  uint64_t* s_full = v_empty + S;  // [2] S_s written by Q K^T
-  uint64_t* p_full = s_full + 2;   // [2] P_s written by the stream's 8 softmax warps (one arrival each)
-  uint64_t* o_full = p_full + 2;   // [2] a P V of stream s has completed
-  uint64_t* s_free = o_full + 2;   // [2] S_s has been read into registers (decoupled-P layout only)
+  uint64_t* k_empty = k_full + SK;
+  uint64_t* v_full = k_empty + SK;
+  uint64_t* v_empty = v_full + SV;
+  uint64_t* s_full = v_empty + SV;  // [2] S buffer written by a Q K^T
+  uint64_t* s_free = s_full + 2;    // [2] S buffer read into registers by its 4 softmax warps
+  uint64_t* p_full = s_free + 2;    // [2] P buffer written by its 4 softmax warps
+  // [4] the P V of tile n arrives on o_full[n % 4].  Four barriers, because a parity wait can only tell the
+  // phase a barrier is in from the one before: a softmax thread that wants P V n-1 or n-2 has itself seen
+  // P V n-4 complete, and P V n+2 cannot complete before that thread has stored P_n.
+  uint64_t* o_full = p_full + 2;
   uint32_t* s_tmem = reinterpret_cast<uint32_t*>(smem + C::kOffMisc);
   int* s_nent = reinterpret_cast<int*>(smem + C::kOffMisc + 4);
   volatile int* s_abort = reinterpret_cast<volatile int*>(smem + C::kOffMisc + 8);
@@ -183,10 +185,16 @@ __global__ void __maxnreg__(96)
   PROF_T(t_cta0);
   const int bh = blockIdx.y;
   const int batch = bh / p.H, head = bh % p.H;
-  // the CTA's two query blocks (any two blocks of the head: a pairing pass picks partners whose kept
-  // lists overlap); blk[1] < 0 means the CTA has a single block
-  const int32_t* pr = p.pairs + ((int64_t)bh * gridDim.x + blockIdx.x) * 2;
-  const int blk[2] = {pr[0], pr[1]};
+  // the CTA's query block(s); a negative entry means "absent"
+  int blk[2];
+  if (C::kStacked) {
+    const int32_t* pr = p.pairs + ((int64_t)bh * gridDim.x + blockIdx.x) * 2;
+    blk[0] = pr[0];
+    blk[1] = pr[1];
+  } else {
+    blk[0] = p.pairs ? p.pairs[(int64_t)bh * (2 * ((p.NB + 1) / 2)) + blockIdx.x] : (int)blockIdx.x;
+    blk[1] = -1;
+  }
 
   // ---- setup ------------------------------------------------------------------------------
   if (tid == 0) {
@@ -194,27 +202,30 @@ __global__ void __maxnreg__(96)
     prefetch_tmap(&tmK);
     prefetch_tmap(&tmV);
     mbar_init(bar_q, 1);
-    for (int s = 0; s < S; ++s) {
+    for (int s = 0; s < SK; ++s) {
       mbar_init(k_full + s, 1);
-      mbar_init(k_empty + s, 2);
+      mbar_init(k_empty + s, 1);
+    }
+    for (int s = 0; s < SV; ++s) {
       mbar_init(v_full + s, 1);
-      mbar_init(v_empty + s, 2);
+      mbar_init(v_empty + s, 1);
     }
     for (int s = 0; s < 2; ++s) {
       mbar_init(s_full + s, 1);
-      mbar_init(p_full + s, 8);
-      mbar_init(o_full + s, 1);
-      mbar_init(s_free + s, 8);
+      mbar_init(s_free + s, 4);
+      mbar_init(p_full + s, 4);
     }
+    for (int s = 0; s < 4; ++s) mbar_init(o_full + s, 1);
     mbar_init_fence();
     *s_abort = 0;
   }
+  if (tid >= 128 && tid < 256) sRef[tid - 128] = -INFINITY;
   if (warp == 1) {
     tmem_alloc(s_tmem, kTmemCols);
     tmem_relinquish();
   }
   if (warp == 0) {
-    // union of the two mask rows -> ascending entry list; flag bit q = kept by query block blk[q]
+    // union of the (up to) two mask rows -> ascending entry list; flag bit q = kept by query block blk[q]
     const uint32_t* mrow0 = p.mask + ((int64_t)bh * p.NB + max(blk[0], 0)) * p.Wd;
     const uint32_t* mrow1 = p.mask + ((int64_t)bh * p.NB + max(blk[1], 0)) * p.Wd;
     int running = 0;
@@ -251,357 +262,340 @@ __global__ void __maxnreg__(96)
   const int n_ent = *s_nent;
   const int n_tiles = (n_ent + C::kEPT - 1) / C::kEPT;
 
-  // which streams work on KV tile n
-  auto stream_mask = [&](int n) -> int { return C::kSplitKV ? (1 << (n & 1)) : (int)sEntF[n]; };
-
-  if (warp == 0) {
-    // ================================ TMA producer ========================================
-    if (lane == 0 && n_tiles > 0) {
-      mbar_expect_tx(bar_q, C::kQTiles * C::kQBytes);
-      // a Q tile is 128 rows: one 128-token block, or two 64-token blocks stacked (an absent second
-      // block re-reads the first: finite data whose rows are never used)
+  // the utility warpgroup hands most of its registers to the two softmax warpgroups (the re-balancing
+  // instruction sits inside each role's branch so that the register allocator sees which code runs
+  // under which limit)
+  if (warp < 4) {
+    asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(SPARSP_REGS_UTILITY));
+    if (warp == 0) {
+      // ================================ TMA producer ========================================
+      if (lane == 0 && n_tiles > 0) {
+        mbar_expect_tx(bar_q, C::kQBytes);
+        // a Q tile is 128 rows: one 128-token block, or two 64-token blocks stacked (an absent second
+        // block re-reads the first: finite data whose rows are never used)
 #pragma unroll
-      for (int q = 0; q < 2; ++q) {
-        const int tok = max(blk[q] >= 0 ? blk[q] : blk[0], 0) * BLK;
-        unsigned char* dst = C::kSplitKV ? sQ + q * (BLK * 128) : sQ + q * C::kQBytes;
+        for (int q = 0; q < C::kEPT; ++q) {
+          const int tok = max(blk[q] >= 0 ? blk[q] : blk[0], 0) * BLK;
 #pragma unroll
-        for (int c = 0; c < D / 64; ++c) tma_load_4d(dst + c * 16384, &tmQ, bar_q, c * 64, tok, head, batch);
-      }
-      const int tile_base = p.slot ? (int)p.tile_base[batch] : 0;
-      auto load_tile = [&](unsigned char* dst, const CUtensorMap* tm, uint64_t* bar, int n) {
+          for (int c = 0; c < D / 64; ++c)
+            tma_load_4d(sQ + c * 16384 + q * (BLK * 128), &tmQ, bar_q, c * 64, tok, head, batch);
+        }
+        const int tile_base = p.slot ? (int)p.tile_base[batch] : 0;
+        auto load_tile = [&](unsigned char* dst, const CUtensorMap* tm, uint64_t* bar, int n, int n_stages) {
 #ifdef SPARSP_ATTN_NOLOAD  // tuning builds only: reuse stale tiles to take TMA traffic out of the picture
-        if (n >= S) {
-          mbar_arrive(bar);
-          return;
-        }
+          if (n >= n_stages) {
+            mbar_arrive(bar);
+            return;
+          }
 #endif
-        mbar_expect_tx(bar, C::kTileBytes);
+          mbar_expect_tx(bar, C::kTileBytes);
 #pragma unroll
-        for (int e = 0; e < C::kEPT; ++e) {
-          const int ent = min(n * C::kEPT + e, n_ent - 1);  // an absent second half re-reads the last entry
-          const int j = sEntJ[ent];
-          const int slot = p.slot ? sSlot[ent] : -1;
-          if (slot < 0) {
+          for (int e = 0; e < C::kEPT; ++e) {
+            const int ent = min(n * C::kEPT + e, n_ent - 1);  // an absent second half re-reads the last entry
+            const int j = sEntJ[ent];
+            const int slot = p.slot ? sSlot[ent] : -1;
+            if (slot < 0) {
 #pragma unroll
-            for (int c = 0; c < D / 64; ++c)
-              tma_load_4d(dst + c * 16384 + e * (BLK * 128), tm, bar, c * 64, j * BLK, head, batch);
-          } else {
-            // remote block: its K tile and V tile are consecutive tiles of the consumer's packed buffer
-            const int tile = tile_base + 2 * slot + (tm == &tmV ? 1 : 0);
+              for (int c = 0; c < D / 64; ++c)
+                tma_load_4d(dst + c * 16384 + e * (BLK * 128), tm, bar, c * 64, j * BLK, head, batch);
+            } else {
+              // remote block: its K tile and V tile are consecutive tiles of the consumer's packed buffer
+              const int tile = tile_base + 2 * slot + (tm == &tmV ? 1 : 0);
 #pragma unroll
-            for (int c = 0; c < D / 64; ++c)
-              tma_load_4d(dst + c * 16384 + e * (BLK * 128), &tmP, bar, c * 64, 0, tile, 0);
+              for (int c = 0; c < D / 64; ++c)
+                tma_load_4d(dst + c * 16384 + e * (BLK * 128), &tmP, bar, c * 64, 0, tile, 0);
+            }
           }
-        }
-      };
-      int kn = 0, vn = 0;
-      const long long t0 = clock64();
-      while ((kn < n_tiles || vn < n_tiles) && !*s_abort) {
-        bool progressed = false;
-        if (kn < n_tiles && mbar_test_wait(k_empty + kn % S, ((kn / S) & 1) ^ 1)) {
-          load_tile(sK + (kn % S) * C::kTileBytes, &tmK, k_full + kn % S, kn);
-          ++kn;
-          progressed = true;
-        }
-        if (vn < n_tiles && mbar_test_wait(v_empty + vn % S, ((vn / S) & 1) ^ 1)) {
-          load_tile(sV + (vn % S) * C::kTileBytes, &tmV, v_full + vn % S, vn);
-          ++vn;
-          progressed = true;
-        }
-        if (!progressed && clock64() - t0 > p.wait_limit * 8) {
-          *s_abort = 1;
-          if (atomicCAS(p.status, 0, SPARSP_ERR_TIMEOUT) == 0) p.status[1] = 10;
+        };
+        int kn = 0, vn = 0;
+        const long long t0 = clock64();
+        while ((kn < n_tiles || vn < n_tiles) && !*s_abort) {
+          bool progressed = false;
+          if (kn < n_tiles && mbar_test_wait(k_empty + kn % SK, ((kn / SK) & 1) ^ 1)) {
+            load_tile(sK + (kn % SK) * C::kTileBytes, &tmK, k_full + kn % SK, kn, SK);
+            ++kn;
+            progressed = true;
+          }
+          if (vn < n_tiles && mbar_test_wait(v_empty + vn % SV, ((vn / SV) & 1) ^ 1)) {
+            load_tile(sV + (vn % SV) * C::kTileBytes, &tmV, v_full + vn % SV, vn, SV);
+            ++vn;
+            progressed = true;
+          }
+          if (!progressed && clock64() - t0 > p.wait_limit * 8) {
+            *s_abort = 1;
+            if (atomicCAS(p.status, 0, SPARSP_ERR_TIMEOUT) == 0) p.status[1] = 10;
+          }
         }
       }
-    }
-  } else if (warp == 1 || warp == kIssuer1Warp) {
-    // ================================ MMA issuers (one thread per stream) =================
-    // Each issuer walks ALL KV tiles in order and, for every tile, first observes the tile's "full"
-    // barrier and then arrives once on its "empty" barrier (count 2: one arrival per issuer) --
-    // through tcgen05.commit after its MMAs if its stream uses the tile, directly otherwise.  The
-    // two streams therefore never wait on each other's softmax, only on the shared K/V rings.
-    // The whole warp runs the loop (uniform control flow and uniform operands, so descriptors and
-    // addresses can live in uniform registers); one elected lane issues the tcgen05 instructions.
-    if (n_tiles > 0) {
-      const int s = (warp == 1) ? 0 : 1;
-      const bool leader = elect_one();
-      constexpr uint32_t kIdescQK = make_idesc_bf16(128, 128, 0, 0);
-      constexpr uint32_t kIdescPV = make_idesc_bf16(128, D, 0, 1);
-      const uint32_t tSs = tmem_base + s * 128;
-      const uint32_t tPs = C::kDecoupledP ? tmem_base + C::kColP + s * 64 : tSs;  // bf16 P (A operand of P V)
-      const uint32_t tOs = tmem_base + C::kColO + s * D;
-      int qcnt = 0;  // Q K^T tiles issued
-      constexpr int kVLag = (S >= 4) ? S - 2 : 1;
-      const uint64_t descQ = make_smem_desc(smem_u32(sQ + (C::kSplitKV ? 0 : s) * C::kQBytes), 16, 1024);
-      const uint64_t descK = make_smem_desc(smem_u32(sK), 16, 1024);
-      const uint64_t descV = make_smem_desc(smem_u32(sV), 16384, 1024);
-      // low words of the descriptors per K step (stage 0); a stage adds kTileBytes/16 to the low word
-      const uint32_t hiQK = (uint32_t)(descK >> 32), hiV = (uint32_t)(descV >> 32);
-      uint32_t qlo[D / 16], klo[D / 16], vlo[8];
+    } else if (warp == 1) {
+      // ================================ Q K^T issuer ========================================
+      // The whole warp runs the loop (uniform control flow and operands); one elected lane issues.
+      if (n_tiles > 0) {
+        const bool leader = elect_one();
+        constexpr uint32_t kIdescQK = make_idesc_bf16(128, 128, 0, 0);
+        const uint64_t descQ = make_smem_desc(smem_u32(sQ), 16, 1024);
+        const uint64_t descK = make_smem_desc(smem_u32(sK), 16, 1024);
+        const uint32_t hiQK = (uint32_t)(descK >> 32);
+        uint32_t qlo[D / 16], klo[D / 16];
 #pragma unroll
-      for (int kk = 0; kk < D / 16; ++kk) {
-        const uint32_t off = (uint32_t)(((kk / 4) * 16384 + (kk % 4) * 32) >> 4);
-        qlo[kk] = (uint32_t)descQ + off;
-        klo[kk] = (uint32_t)descK + off;
-      }
-#pragma unroll
-      for (int kk = 0; kk < 8; ++kk) vlo[kk] = (uint32_t)descV + (uint32_t)((kk * 2048) >> 4);
-      int vdone = 0;       // tiles whose V obligation (P V or plain release) has been handled
-      int last_kept = -1;  // last tile whose Q K^T this stream has issued
-      int pcnt = 0;        // P tiles consumed
-      uint32_t started = 0;
-
-      auto handle_v = [&](int m) {
-        const bool keep = (stream_mask(m) >> s) & 1;
-        if (keep) {
-          PROF_T(t_p0);
-          mbar_wait_bounded(p_full + s, pcnt & 1, s_abort, p.status, 20 + s, p.wait_limit);
-          ++pcnt;
-          PROF_T(t_p1);
-          PROF_ADD(8, t_p0, t_p1);  // issuer waiting for P
+        for (int kk = 0; kk < D / 16; ++kk) {
+          const uint32_t off = (uint32_t)(((kk / 4) * 16384 + (kk % 4) * 32) >> 4);
+          qlo[kk] = (uint32_t)descQ + off;
+          klo[kk] = (uint32_t)descK + off;
         }
-        PROF_T(t_v0);
-        mbar_wait_bounded(v_full + m % S, (m / S) & 1, s_abort, p.status, 22, p.wait_limit);
-        PROF_T(t_v1);
-        PROF_ADD(10, t_v0, t_v1);  // issuer waiting for V
-        if (keep) {
-          tc_fence_after();
-          const uint32_t stage_off = (uint32_t)(((m % S) * C::kTileBytes) >> 4);
-          if (leader) {
-#pragma unroll
-            for (int kk = 0; kk < 8; ++kk)
-              mma_ts_lohi(tOs, tPs + kk * 8, vlo[kk] + stage_off, hiV, kIdescPV, (kk > 0) ? 1u : started);
-            mma_commit(o_full + s);
-            mma_commit(v_empty + m % S);
-          }
-          started = 1u;
-          PROF_T(t_v2);
-          PROF_ADD(6, t_v1, t_v2);  // issuer issuing P V
-        } else if (leader) {
-          mbar_arrive(v_empty + m % S);
-        }
-        __syncwarp();
-      };
-
-      mbar_wait_bounded(bar_q, 0, s_abort, p.status, 11, p.wait_limit);
-      for (int n = 0; n < n_tiles; ++n) {
-        const bool keep = (stream_mask(n) >> s) & 1;
-        // a V stage is released at most kVLag + 1 steps after its fill (always fewer than the ring has stages)
-        while (vdone < n - kVLag) handle_v(vdone++);
-        PROF_T(t_k0);
-        mbar_wait_bounded(k_full + n % S, (n / S) & 1, s_abort, p.status, 12, p.wait_limit);
-        PROF_T(t_k1);
-        PROF_ADD(9, t_k0, t_k1);  // issuer waiting for K
-        if (keep) {
-          if (C::kDecoupledP) {
-            // S_s is free once the softmax warps have loaded the previous tile's scores
-            if (qcnt > 0) mbar_wait_bounded(s_free + s, (qcnt - 1) & 1, s_abort, p.status, 24 + s, p.wait_limit);
-          } else {
-            while (vdone <= last_kept) handle_v(vdone++);  // P V of the previous kept tile frees S_s
-          }
+        mbar_wait_bounded(bar_q, 0, s_abort, p.status, 11, p.wait_limit);
+        for (int n = 0; n < n_tiles; ++n) {
+          PROF_T(t_k0);
+          mbar_wait_bounded(k_full + n % SK, (n / SK) & 1, s_abort, p.status, 12, p.wait_limit);
+          PROF_T(t_k1);
+          PROF_ADD(9, t_k0, t_k1);  // issuer waiting for K
+          // S buffer n%2 is free once the softmax warps have loaded the scores of tile n-2
+          if (n >= 2) mbar_wait_bounded(s_free + (n & 1), ((n - 2) >> 1) & 1, s_abort, p.status, 24, p.wait_limit);
           PROF_T(t_k3);
+          PROF_ADD(8, t_k1, t_k3);  // issuer waiting for a free S buffer
           tc_fence_after();
-          const uint32_t stage_off = (uint32_t)(((n % S) * C::kTileBytes) >> 4);
+          const uint32_t stage_off = (uint32_t)(((n % SK) * C::kTileBytes) >> 4);
+          const uint32_t tS = tmem_base + C::kColS + (n & 1) * 128;
           if (leader) {
 #pragma unroll
             for (int kk = 0; kk < D / 16; ++kk)
-              mma_ss_lohi(tSs, qlo[kk], hiQK, klo[kk] + stage_off, hiQK, kIdescQK, kk > 0 ? 1u : 0u);
-            mma_commit(s_full + s);
-            mma_commit(k_empty + n % S);
+              mma_ss_lohi(tS, qlo[kk], hiQK, klo[kk] + stage_off, hiQK, kIdescQK, kk > 0 ? 1u : 0u);
+            mma_commit(s_full + (n & 1));
+            mma_commit(k_empty + n % SK);
           }
-          ++qcnt;
+          __syncwarp();
           PROF_T(t_k2);
           PROF_ADD(7, t_k3, t_k2);  // issuer issuing Q K^T
-          if (C::kDecoupledP)
-            while (vdone <= last_kept) handle_v(vdone++);  // P V of the previous kept tile, after this Q K^T
-          last_kept = n;
-        } else if (leader) {
-          mbar_arrive(k_empty + n % S);
         }
-        __syncwarp();
       }
-      while (vdone < n_tiles) handle_v(vdone++);
+    } else if (warp == 2) {
+      // ================================ P V issuer ==========================================
+      if (n_tiles > 0) {
+        const bool leader = elect_one();
+        constexpr uint32_t kIdescPV = make_idesc_bf16(128, D, 0, 1);
+        const uint64_t descV = make_smem_desc(smem_u32(sV), 16384, 1024);
+        const uint32_t hiV = (uint32_t)(descV >> 32);
+        uint32_t vlo[8];
+#pragma unroll
+        for (int kk = 0; kk < 8; ++kk) vlo[kk] = (uint32_t)descV + (uint32_t)((kk * 2048) >> 4);
+        const uint32_t tO = tmem_base + C::kColO;
+        for (int n = 0; n < n_tiles; ++n) {
+          mbar_wait_bounded(p_full + (n & 1), (n >> 1) & 1, s_abort, p.status, 20, p.wait_limit);
+          mbar_wait_bounded(v_full + n % SV, (n / SV) & 1, s_abort, p.status, 22, p.wait_limit);
+          tc_fence_after();
+          const uint32_t stage_off = (uint32_t)(((n % SV) * C::kTileBytes) >> 4);
+          const uint32_t tP = tmem_base + C::kColP + (n & 1) * 64;
+          if (leader) {
+#pragma unroll
+            for (int kk = 0; kk < 8; ++kk)
+              mma_ts_lohi(tO, tP + kk * 8, vlo[kk] + stage_off, hiV, kIdescPV, (kk > 0 || n > 0) ? 1u : 0u);
+            mma_commit(o_full + (n & 3));
+            mma_commit(v_empty + n % SV);
+          }
+          __syncwarp();
+        }
+      }
     }
-  } else if (warp >= 2 && warp < 18) {
-    // ================================ softmax warps =======================================
-    const int sidx = (warp - 2) >> 3;       // stream
-    const int half = ((warp - 2) >> 2) & 1;  // which 64 key columns of a tile this thread owns
-    const int rgrp = warp & 3;               // tensor-memory lane group this warp may access
+  } else {
+    asm volatile("setmaxnreg.inc.sync.aligned.u32 %0;" ::"n"(SPARSP_REGS_SOFTMAX));
+    // ================================ softmax warpgroups ==================================
+    const int wg = (warp >> 2) - 1;  // 0: even tiles, 1: odd tiles; also the S / P buffer this warpgroup uses
+    const int rgrp = warp & 3;       // tensor-memory lane group this warp may access
     const int row = rgrp * 32 + lane;
-    const int rh = row >> 6;                 // which query block of a stacked Q tile the row belongs to
-    const int pair_bar = 1 + sidx * 4 + rgrp;  // named barrier shared with the row's other thread
+    const int rh = row >> 6;         // which query block of a stacked Q tile the row belongs to
     const uint32_t lane_off = (uint32_t)(rgrp * 32) << 16;
-    const uint32_t tS = tmem_base + sidx * 128 + lane_off;
-    const uint32_t tP = (C::kDecoupledP ? tmem_base + C::kColP + sidx * 64 : tmem_base + sidx * 128) + lane_off;
-    const uint32_t tO = tmem_base + C::kColO + sidx * D + lane_off;
-    float m_used = -INFINITY;  // reference maximum (log2 domain) of the row's exponentials
-    float l_run = 0.0f;        // this thread's share of the row sum
-    int cnt = 0;
+    const uint32_t tS = tmem_base + C::kColS + wg * 128 + lane_off;
+    const uint32_t tP = tmem_base + C::kColP + wg * 64 + lane_off;
+    const uint32_t tO = tmem_base + C::kColO + lane_off;
+    const int bar_mine = 1 + wg * 4 + rgrp;         // I arrive here after my decision
+    const int bar_other = 1 + (1 - wg) * 4 + rgrp;  // the row group's other warp arrives here after its decision
+    float m_ref = -INFINITY;  // the row's reference maximum (log2 domain) as this thread last saw it
+    float l_run = 0.0f;       // this thread's partial row sum, relative to m_ref
+    int cnt = 0;              // tiles this warpgroup has processed
 
     PROF_T(t_loop0);
     PROF_ADD(11, t_cta0, t_loop0);  // prologue up to the softmax loop
-    for (int n = 0; n < n_tiles; ++n) {
-      if (!((stream_mask(n) >> sidx) & 1)) continue;
-      // kept / valid columns of my 64-column half (warp-uniform)
-      int nv;
-      if (C::kSplitKV) {
-        const int ent = n * 2 + half;
-        nv = 0;
-        if (ent < n_ent && ((sEntF[ent] >> rh) & 1)) nv = (int)min((int64_t)64, p.N - (int64_t)sEntJ[ent] * 64);
+    for (int n = wg; n < n_tiles; n += 2, ++cnt) {
+      // kept / valid key columns of each 64-column half of the tile (warp-uniform)
+      int vh[2];
+      if (C::kStacked) {
+#pragma unroll
+        for (int h = 0; h < 2; ++h) {
+          const int ent = n * 2 + h;
+          vh[h] = 0;
+          if (ent < n_ent && ((sEntF[ent] >> rh) & 1)) vh[h] = (int)min((int64_t)64, p.N - (int64_t)sEntJ[ent] * 64);
+        }
       } else {
-        nv = (int)min((int64_t)128, p.N - (int64_t)sEntJ[n] * 128) - 64 * half;
-        nv = max(0, min(64, nv));
+        const int nv = (int)min((int64_t)128, p.N - (int64_t)sEntJ[n] * 128);
+        vh[0] = min(nv, 64);
+        vh[1] = max(nv - 64, 0);
       }
-      const int valid[2] = {min(nv, 32), max(nv - 32, 0)};
 
       PROF_T(t_a);
-      mbar_wait_bounded(s_full + sidx, cnt & 1, s_abort, p.status, 30 + sidx, p.wait_limit);
+      mbar_wait_bounded(s_full + wg, cnt & 1, s_abort, p.status, 30 + wg, p.wait_limit);
       tc_fence_after();
       PROF_T(t_b);
-#ifdef SPARSP_ATTN_NOSOFTMAX  // tuning builds only: measure the MMA / TMA pipeline alone
+      float sv[128];
+#pragma unroll
+      for (int c = 0; c < 4; ++c) tmem_ld32(tS + c * 32, reinterpret_cast<uint32_t*>(sv) + c * 32);
+      tmem_ld_wait();
+      // S is in registers: the Q K^T of tile n+2 may overwrite the buffer
       tc_fence_before();
       __syncwarp();
-      if (lane == 0) mbar_arrive(p_full + sidx);
-      ++cnt;
+      if (lane == 0) mbar_arrive(s_free + wg);
+      PROF_T(t_b2);
+#ifdef SPARSP_ATTN_NOSOFTMAX  // tuning builds only: measure the MMA / TMA pipeline alone
+      if (n >= 2) mbar_wait_bounded(o_full + ((n - 2) & 3), ((n - 2) >> 2) & 1, s_abort, p.status, 34 + wg, p.wait_limit);
+      __syncwarp();
+      if (lane == 0) mbar_arrive(p_full + wg);
       continue;
 #endif
-      float sv[64];
-      tmem_ld32(tS + half * 64, reinterpret_cast<uint32_t*>(sv));
-      tmem_ld32(tS + half * 64 + 32, reinterpret_cast<uint32_t*>(sv) + 32);
-      tmem_ld_wait();
-      if (C::kDecoupledP) {
-        // S is in registers: let the issuer start the next Q K^T
-        tc_fence_before();
-        __syncwarp();
-        if (lane == 0) mbar_arrive(s_free + sidx);
-      }
+      // one flat instruction stream per 64-key half; a ragged half (the sequence ends inside it) first has
+      // its invalid columns set to -inf, an absent half (not kept by this row's query block) is skipped
       float mx = -INFINITY;
 #pragma unroll
-      for (int c = 0; c < 2; ++c) {
-        if (valid[c] == 32) {
+      for (int h = 0; h < 2; ++h) {
+        float* svh = sv + h * 64;
+        if (vh[h] > 0) {
+          if (vh[h] < 64) {
 #pragma unroll
-          for (int e = 0; e < 32; e += 2) mx = fmaxf(mx, fmaxf(sv[c * 32 + e], sv[c * 32 + e + 1]));
-        } else if (valid[c] > 0) {
+            for (int e = 0; e < 64; ++e) svh[e] = e < vh[h] ? svh[e] : -INFINITY;
+          }
+          float m0 = svh[0], m1 = svh[1], m2 = svh[2], m3 = svh[3];
 #pragma unroll
-          for (int e = 0; e < 32; ++e) mx = fmaxf(mx, e < valid[c] ? sv[c * 32 + e] : -INFINITY);
+          for (int e = 4; e < 64; e += 4) {
+            m0 = fmaxf(m0, svh[e]);
+            m1 = fmaxf(m1, svh[e + 1]);
+            m2 = fmaxf(m2, svh[e + 2]);
+            m3 = fmaxf(m3, svh[e + 3]);
+          }
+          mx = fmaxf(mx, fmaxf(fmaxf(m0, m1), fmaxf(m2, m3)));
         }
       }
-      // exchange the two halves' maxima (double-buffered by tile parity); the barrier also orders
-      // my partner's reads of S before my writes of P into the columns it read
-      float* mslot = sMax + (((cnt & 1) * 2 + sidx) * 2) * 128;
-      mslot[half * 128 + row] = mx;
-      named_bar_sync(pair_bar, 64);
-      mx = fmaxf(mx, mslot[(1 - half) * 128 + row]) * p.scale_log2;
+      mx *= p.scale_log2;
       PROF_T(t_c);
-      if (C::kDecoupledP && cnt > 0) {
-        // the previous P V must have finished reading P (and updating O) before either is touched
-        mbar_wait_bounded(o_full + sidx, (cnt - 1) & 1, s_abort, p.status, 34 + sidx, p.wait_limit);
-        tc_fence_after();
+
+      // ---- my turn to look at / move the row's reference maximum (strictly in tile order) ----
+      if (n > 0) named_bar_sync(bar_other, 64);
+      PROF_T(t_c2);
+      PROF_ADD(6, t_c, t_c2);  // waiting for my turn
+      {
+        const float m_cur = sRef[row];
+        if (m_cur != m_ref) {  // the other thread moved it since my last tile
+          l_run *= ex2(m_ref - m_cur);  // m_ref = -inf: l_run is 0 and stays 0
+          m_ref = m_cur;
+        }
       }
-      const float m_new = fmaxf(m_used, mx);
-      const bool grow = m_new > m_used + kGrowThreshold || (m_used == -INFINITY && m_new > -INFINITY);
+      const float m_new = fmaxf(m_ref, mx);
+      const bool grow = m_new > m_ref + kGrowThreshold || (m_ref == -INFINITY && m_new > -INFINITY);
       if (__any_sync(0xffffffffu, grow)) {
-        const float alpha = grow ? ex2(m_used - m_new) : 1.0f;  // m_used = -inf -> 0
-        if (cnt > 0) {  // S_s of this tile is complete, hence so is every earlier P V of the stream
+        const float alpha = grow ? ex2(m_ref - m_new) : 1.0f;  // m_ref = -inf -> 0
+        if (n > 0) {
+          // every P V issued so far must have landed in O before the row is rescaled; they complete in
+          // order, so the one of tile n-1 suffices
+          mbar_wait_bounded(o_full + ((n - 1) & 3), ((n - 1) >> 2) & 1, s_abort, p.status, 38, p.wait_limit);
+          tc_fence_after();
 #pragma unroll
-          for (int c = 0; c < D / 32; ++c) {  // my half of the accumulator's columns, 16 at a time
+          for (int c = 0; c < D / 16; ++c) {  // the row's accumulator, 16 columns at a time
             uint32_t o[16];
-            tmem_ld16(tO + half * (D / 2) + c * 16, o);
+            tmem_ld16(tO + c * 16, o);
             tmem_ld_wait();
 #pragma unroll
             for (int e = 0; e < 16; ++e) o[e] = __float_as_uint(__uint_as_float(o[e]) * alpha);
-            tmem_st16(tO + half * (D / 2) + c * 16, o);
+            tmem_st16(tO + c * 16, o);
           }
+          tmem_st_wait();
+          tc_fence_before();
         }
         l_run *= alpha;
-        if (grow) m_used = m_new;
+        if (grow) {
+          m_ref = m_new;
+          sRef[row] = m_new;
+        }
+      }
+      if (n + 1 < n_tiles) {
+        asm volatile("bar.arrive %0, %1;" ::"r"(bar_mine), "r"(64) : "memory");
       }
       PROF_T(t_d);
 
-      // exponentials; bf16 P overwrites S in place: my keys [64*half, 64*half+64) go to columns
-      // [32*half, 32*half+32)
-      float lsum = 0.0f;
+      // exponentials of keys [32c, 32c+32) -> packed bf16 columns [16c, 16c+16) of the P buffer
       float2 lsum2 = make_float2(0.0f, 0.0f);
-      const float neg_m = -m_used;
+      const float neg_m = -m_ref;
+      uint32_t pk[64];
+      const float2 sc2 = make_float2(p.scale_log2, p.scale_log2), nm2 = make_float2(neg_m, neg_m);
 #pragma unroll
-      for (int c = 0; c < 2; ++c) {
-        uint32_t pk[16];
-        const float* svc = sv + c * 32;
-        if (valid[c] == 32) {
-#if SPARSP_TUNE_F32X2
-          const float2 sc2 = make_float2(p.scale_log2, p.scale_log2), nm2 = make_float2(neg_m, neg_m);
+      for (int h = 0; h < 2; ++h) {
+        const float* svh = sv + h * 64;
+        uint32_t* pkh = pk + h * 32;
+        if (vh[h] > 0) {  // then the row has a finite reference maximum
 #pragma unroll
-          for (int e = 0; e < 16; ++e) {
-            const float2 x = ffma2(make_float2(svc[2 * e], svc[2 * e + 1]), sc2, nm2);
+          for (int e = 0; e < 32; ++e) {
+            const float2 x = ffma2(make_float2(svh[2 * e], svh[2 * e + 1]), sc2, nm2);
             const float2 pp = (SPARSP_TUNE_POLY > 0 && (e % (SPARSP_TUNE_POLY > 0 ? SPARSP_TUNE_POLY : 1)) == 1)
                                   ? exp2_poly2(x)
                                   : make_float2(ex2(x.x), ex2(x.y));
             lsum2 = fadd2(lsum2, pp);
             const __nv_bfloat162 h2 = __floats2bfloat162_rn(pp.x, pp.y);
-            pk[e] = *reinterpret_cast<const uint32_t*>(&h2);
+            pkh[e] = *reinterpret_cast<const uint32_t*>(&h2);
           }
-#else
+          if (vh[h] < 64) {
+            // columns past the end of the sequence: exactly zero in P (the polynomial path returns
+            // 2^-126 for them, which the row sum may keep)
 #pragma unroll
-          for (int e = 0; e < 16; ++e) {
-            const float p0 = ex2(fmaf(svc[2 * e], p.scale_log2, neg_m));
-            const float p1 = ex2(fmaf(svc[2 * e + 1], p.scale_log2, neg_m));
-            lsum += p0 + p1;
-            const __nv_bfloat162 h2 = __floats2bfloat162_rn(p0, p1);
-            pk[e] = *reinterpret_cast<const uint32_t*>(&h2);
-          }
-#endif
-        } else if (valid[c] > 0) {
-#pragma unroll
-          for (int e = 0; e < 16; ++e) {
-            const float p0 = 2 * e < valid[c] ? ex2(fmaf(svc[2 * e], p.scale_log2, neg_m)) : 0.0f;
-            const float p1 = 2 * e + 1 < valid[c] ? ex2(fmaf(svc[2 * e + 1], p.scale_log2, neg_m)) : 0.0f;
-            lsum += p0 + p1;
-            const __nv_bfloat162 h2 = __floats2bfloat162_rn(p0, p1);
-            pk[e] = *reinterpret_cast<const uint32_t*>(&h2);
+            for (int e = 0; e < 32; ++e) pkh[e] = 2 * e + 1 < vh[h] ? pkh[e] : (2 * e < vh[h] ? (pkh[e] & 0xffffu) : 0u);
           }
         } else {
 #pragma unroll
-          for (int e = 0; e < 16; ++e) pk[e] = 0u;
+          for (int e = 0; e < 32; ++e) pkh[e] = 0u;
         }
-        tmem_st16(tP + half * 32 + c * 16, pk);
       }
-      l_run += lsum + (lsum2.x + lsum2.y);
+      l_run += lsum2.x + lsum2.y;
       PROF_T(t_e);
+      // my P buffer was last read by the P V of tile n-2
+      if (n >= 2) {
+        mbar_wait_bounded(o_full + ((n - 2) & 3), ((n - 2) >> 2) & 1, s_abort, p.status, 34 + wg, p.wait_limit);
+        tc_fence_after();
+      }
+#pragma unroll
+      for (int c = 0; c < 4; ++c) tmem_st16(tP + c * 16, pk + c * 16);
       tmem_st_wait();
       tc_fence_before();
       __syncwarp();
-      if (lane == 0) mbar_arrive(p_full + sidx);
-      ++cnt;
+      if (lane == 0) mbar_arrive(p_full + wg);
       PROF_T(t_f);
-      PROF_ADD(0, t_a, t_b);  // wait for S
-      PROF_ADD(1, t_b, t_c);  // load + max + exchange
-      PROF_ADD(2, t_c, t_d);  // rescale decision
-      PROF_ADD(3, t_d, t_e);  // exponentials + P store
-      PROF_ADD(4, t_e, t_f);  // store wait + arrive
+      PROF_ADD(0, t_a, t_b);      // wait for S
+      PROF_ADD(1, t_b, t_b2);     // load of S
+      PROF_ADD(14, t_b2, t_c);    // row maximum
+      PROF_ADD(2, t_c, t_d);      // turn-taking + rescale decision
+      PROF_ADD(3, t_d, t_e);      // exponentials
+      PROF_ADD(4, t_e, t_f);      // wait for the P buffer + store + arrive
       PROF_ADD(5, t_a, t_a + 1);  // tile count
     }
 
-    // ---- epilogue -------------------------------------------------------------------------
+    // ---- epilogue: warpgroup x writes the column half x of every row ------------------------------
     PROF_T(t_ep0);
-    if (cnt > 0) {
-      mbar_wait_bounded(o_full + sidx, (cnt - 1) & 1, s_abort, p.status, 40 + sidx, p.wait_limit);
+    sStat[wg * 128 + row] = make_float2(m_ref, l_run);
+    named_bar_sync(9, 256);  // all tiles' decisions and P stores are done
+    if (n_tiles > 0) {
+      const int last = n_tiles - 1;
+      mbar_wait_bounded(o_full + (last & 3), (last >> 2) & 1, s_abort, p.status, 40, p.wait_limit);
       tc_fence_after();
     }
     PROF_T(t_ep1);
-    PROF_ADD(12, t_ep0, t_ep1);  // wait for the last P V
-    sStat[(sidx * 2 + half) * 128 + row] = make_float2(m_used, l_run);
-    if (!C::kSplitKV) {
-      // the row's two threads add their partial sums; each writes its half of the columns
-      named_bar_sync(pair_bar, 64);
-      const float l = l_run + sStat[(sidx * 2 + 1 - half) * 128 + row].y;
-      const int64_t tok = blk[sidx] >= 0 ? (int64_t)blk[sidx] * BLK + row : p.N;
+    {
+      constexpr int HW = D / 2;
+      const float m_fin = sRef[row];
+      const float2 st0 = sStat[row], st1 = sStat[128 + row];
+      const float l = (st0.y > 0.0f ? st0.y * ex2(st0.x - m_fin) : 0.0f) + (st1.y > 0.0f ? st1.y * ex2(st1.x - m_fin) : 0.0f);
       const float inv_l = l > 0.0f ? 1.0f / l : 0.0f;
-      __nv_bfloat16* orow = p.O + (int64_t)batch * p.sB + (int64_t)head * p.sH + tok * p.sT + half * (D / 2);
+      const int qb = C::kStacked ? blk[rh] : blk[0];
+      const int64_t tok = qb >= 0 ? (int64_t)qb * BLK + (C::kStacked ? (row & 63) : row) : p.N;
+      __nv_bfloat16* orow = p.O + (int64_t)batch * p.sB + (int64_t)head * p.sH + tok * p.sT + wg * HW;
 #pragma unroll
-      for (int c = 0; c < D / 64; ++c) {
+      for (int c = 0; c < HW / 32; ++c) {
         uint32_t o[32];
-        if (cnt > 0) {  // warp-uniform: tensor-memory loads are warp-collective
-          tmem_ld32(tO + half * (D / 2) + c * 32, o);
+        if (n_tiles > 0) {  // CTA-uniform: tensor-memory loads are warp-collective
+          tmem_ld32(tO + wg * HW + c * 32, o);
           tmem_ld_wait();
         } else {
 #pragma unroll
@@ -621,74 +615,8 @@ __global__ void __maxnreg__(96)
           }
         }
       }
-      if (p.lse && half == 0 && tok < p.N)
-        p.lse[(int64_t)bh * p.N + tok] = l > 0.0f ? (m_used + log2f(l)) * 0.6931471805599453f : -INFINITY;
-    } else {
-      // merge the two streams' partial results.  Thread (stream s, half h) finalises the column
-      // quarter 2s+h; it hands the other stream's thread of the same half the quarter that one
-      // finalises, scaled to the common reference maximum.
-      constexpr int QW = D / 4;
-      float* mbuf = reinterpret_cast<float*>(sK);  // K/V rings are idle once both streams are done
-      named_bar_sync(9, 512);
-      const float l_me = l_run + sStat[(sidx * 2 + 1 - half) * 128 + row].y;
-      const float2 o0 = sStat[((1 - sidx) * 2) * 128 + row];
-      const float2 o1 = sStat[((1 - sidx) * 2 + 1) * 128 + row];
-      const float m_ot = o0.x, l_ot = o0.y + o1.y;
-      const float m = fmaxf(m_used, m_ot);
-      const float a_me = m_used > -INFINITY ? ex2(m_used - m) : 0.0f;
-      const float a_ot = m_ot > -INFINITY ? ex2(m_ot - m) : 0.0f;
-      const float l = l_me * a_me + l_ot * a_ot;
-      const float inv_l = l > 0.0f ? 1.0f / l : 0.0f;
-      const int give_q = 2 * (1 - sidx) + half, keep_q = 2 * sidx + half;
-      float* give = mbuf + ((size_t)(sidx * 2 + half) * 128 + row) * C::kMergeStride;
-      {
-        uint32_t o[QW];
-        if (cnt > 0) {
-          if constexpr (QW == 32) tmem_ld32(tO + give_q * QW, o); else tmem_ld16(tO + give_q * QW, o);
-          tmem_ld_wait();
-        } else {
-#pragma unroll
-          for (int e = 0; e < QW; ++e) o[e] = 0u;
-        }
-#pragma unroll
-        for (int v = 0; v < QW / 4; ++v)
-          *reinterpret_cast<float4*>(give + v * 4) =
-              make_float4(__uint_as_float(o[v * 4]) * a_me, __uint_as_float(o[v * 4 + 1]) * a_me,
-                          __uint_as_float(o[v * 4 + 2]) * a_me, __uint_as_float(o[v * 4 + 3]) * a_me);
-      }
-      named_bar_sync(9, 512);
-      const int64_t tok = blk[rh] >= 0 ? (int64_t)blk[rh] * BLK + (row & 63) : p.N;
-      const float* take = mbuf + ((size_t)((1 - sidx) * 2 + half) * 128 + row) * C::kMergeStride;
-      __nv_bfloat16* orow = p.O + (int64_t)batch * p.sB + (int64_t)head * p.sH + tok * p.sT + keep_q * QW;
-      {
-        uint32_t o[QW];
-        if (cnt > 0) {
-          if constexpr (QW == 32) tmem_ld32(tO + keep_q * QW, o); else tmem_ld16(tO + keep_q * QW, o);
-          tmem_ld_wait();
-        } else {
-#pragma unroll
-          for (int e = 0; e < QW; ++e) o[e] = 0u;
-        }
-        if (tok < p.N) {
-#pragma unroll
-          for (int v = 0; v < QW / 8; ++v) {
-            const float4 t0 = *reinterpret_cast<const float4*>(take + v * 8);
-            const float4 t1 = *reinterpret_cast<const float4*>(take + v * 8 + 4);
-            const float tt[8] = {t0.x, t0.y, t0.z, t0.w, t1.x, t1.y, t1.z, t1.w};
-            uint32_t w[4];
-#pragma unroll
-            for (int e = 0; e < 4; ++e) {
-              const float x0 = (__uint_as_float(o[v * 8 + 2 * e]) * a_me + tt[2 * e]) * inv_l;
-              const float x1 = (__uint_as_float(o[v * 8 + 2 * e + 1]) * a_me + tt[2 * e + 1]) * inv_l;
-              const __nv_bfloat162 h2 = __floats2bfloat162_rn(x0, x1);
-              w[e] = *reinterpret_cast<const uint32_t*>(&h2);
-            }
-            *reinterpret_cast<uint4*>(orow + v * 8) = make_uint4(w[0], w[1], w[2], w[3]);
-          }
-        }
-      }
-      if (p.lse && sidx == 0 && half == 0 && tok < p.N)
-        p.lse[(int64_t)bh * p.N + tok] = l > 0.0f ? (m + log2f(l)) * 0.6931471805599453f : -INFINITY;
+      if (p.lse && wg == 0 && tok < p.N)
+        p.lse[(int64_t)bh * p.N + tok] = l > 0.0f ? (m_fin + log2f(l)) * 0.6931471805599453f : -INFINITY;
     }
   }
 
@@ -698,7 +626,6 @@ __global__ void __maxnreg__(96)
   if (warp == 1) tmem_dealloc(tmem_base, kTmemCols);
   PROF_T(t_cta2);
   PROF_ADD(13, t_cta0, t_cta1);  // CTA lifetime of the sampled lanes up to the final barrier
-  PROF_ADD(14, t_cta1, t_cta2);  // final barrier + dealloc
   PROF_ADD(15, t_cta0, t_cta0 + 1);
 }
 
@@ -844,7 +771,8 @@ static int launch_attn_t(const sparsp_shape& s, const Geometry& g, const void* Q
   auto kern = attn_fwd_kernel<D, BLK>;
   const int smem = AttnCfg<D, BLK>::kDynamic;
   SPARSP_CUDA_OK(ensure_dynamic_smem((const void*)kern, smem));
-  dim3 grid((unsigned)((g.NB + 1) / 2), (unsigned)(g.B * g.H));
+  // one CTA per 128-row Q tile: a 128-token block, or a pair of 64-token blocks
+  dim3 grid((unsigned)(BLK == 128 ? g.NB : (g.NB + 1) / 2), (unsigned)(g.B * g.H));
   kern<<<grid, kAttnThreads, smem, st>>>(tq, tk, tv, tp, p);
   count_launch();
   SPARSP_CUDA_OK(cudaGetLastError());
@@ -876,11 +804,12 @@ static int launch_attn_common(const sparsp_shape& s, const Geometry& g, const vo
 int launch_attn(const sparsp_shape& s, const Geometry& g, const void* Q, const void* K, const void* V,
                 const uint32_t* mask, float scale, void* O, float* lse, char* ws, const WsLayout& L,
                 cudaStream_t st) {
-  int32_t* pairs = (int32_t*)(ws + L.pairs);
-  {
+  int32_t* pairs = nullptr;  // block 128: CTA x handles query block x
+  if (g.b == 64) {
+    pairs = (int32_t*)(ws + L.pairs);
     const size_t smem = (size_t)g.NB * g.Wd * 4;
     SPARSP_CUDA_OK(ensure_dynamic_smem((const void*)pair_kernel, (int)smem));
-    pair_kernel<<<g.B * g.H, kPairThreads, smem, st>>>(mask, g.NB, g.Wd, g.b == 64 ? 1 : 0, pairs);
+    pair_kernel<<<g.B * g.H, kPairThreads, smem, st>>>(mask, g.NB, g.Wd, 1, pairs);
     count_launch();
   }
   AttnParams p;
