@@ -321,9 +321,14 @@ __global__ void __launch_bounds__(kAttnThreads, 1)
             ++vn;
             progressed = true;
           }
-          if (!progressed && clock64() - t0 > p.wait_limit * 8) {
-            *s_abort = 1;
-            if (atomicCAS(p.status, 0, SPARSP_ERR_TIMEOUT) == 0) p.status[1] = 10;
+          if (!progressed) {
+            // both rings are full: the loads run several tiles ahead of the MMAs, so polling slowly costs
+            // nothing and leaves this scheduler's issue slots to the softmax warps that share it
+            __nanosleep(200);
+            if (clock64() - t0 > p.wait_limit * 8) {
+              *s_abort = 1;
+              if (atomicCAS(p.status, 0, SPARSP_ERR_TIMEOUT) == 0) p.status[1] = 10;
+            }
           }
         }
       }
@@ -476,7 +481,9 @@ __global__ void __launch_bounds__(kAttnThreads, 1)
       PROF_T(t_c);
 
       // ---- my turn to look at / move the row's reference maximum (strictly in tile order) ----
+#ifndef SPARSP_ATTN_NOTURN  // (tuning builds only: without the hand-over the result is wrong)
       if (n > 0) named_bar_sync(bar_other, 64);
+#endif
       PROF_T(t_c2);
       PROF_ADD(6, t_c, t_c2);  // waiting for my turn
       {
@@ -513,9 +520,11 @@ __global__ void __launch_bounds__(kAttnThreads, 1)
           sRef[row] = m_new;
         }
       }
+#ifndef SPARSP_ATTN_NOTURN
       if (n + 1 < n_tiles) {
         asm volatile("bar.arrive %0, %1;" ::"r"(bar_mine), "r"(64) : "memory");
       }
+#endif
       PROF_T(t_d);
 
       // exponentials of keys [32c, 32c+32) -> packed bf16 columns [16c, 16c+16) of the P buffer
