@@ -1,18 +1,22 @@
 // Step 3: block-sparse FlashAttention forward on tcgen05 tensor cores (sm_100a).
 //
-// A CTA owns ONE 128-row Q tile of one (batch, head) and one fp32 accumulator O in tensor memory:
-//   block = 128: the Q tile is one query block; the CTA walks that block's kept KV blocks.
+// Work item = ONE 128-row Q tile of one (batch, head) with one fp32 accumulator O in tensor memory:
+//   block = 128: the Q tile is one query block; the item walks that block's kept KV blocks.
 //   block = 64 : two query blocks (chosen by a pairing pass so that their kept lists overlap) are stacked
 //                into the Q tile (full-rate M = 128 MMAs); a KV tile is two entries of the UNION of their
 //                kept lists (128 keys, full-rate N = 128); each 64x64 quadrant the mask does not keep is
 //                zeroed in P.
+// The kernel is persistent: one CTA per SM walks items c, c + grid, c + 2 grid, ...; the next item's kept
+// list, Q tile, first K/V tiles and first Q K^T overlap the current item's last tiles and its epilogue.
 // The scores S = Q K^T and the probabilities P are double-buffered in tensor memory (S: 2 x 128 fp32
 // columns, P: 2 x 64 columns of packed bf16, O: d columns), so that the tensor pipe always has the next
-// tiles' MMAs queued while the softmax of the current tile runs: Q K^T of tile n+2 starts as soon as the
-// scores of tile n have been READ, and P V of tile n is issued as soon as P_n is written.
+// tiles' MMAs queued while the softmax of the current tile runs: Q K^T of tile g+2 starts as soon as the
+// scores of tile g have been READ, and P V of tile g is issued as soon as P_g is written.  Tiles are
+// numbered g = 0, 1, 2, ... across the CTA's items; every ring, buffer and barrier phase follows g.
 // Warp roles (384 threads = 3 warpgroups; the first hands most of its registers to the other two):
-//   warp 0      TMA producer (K ring and V ring, polled independently)
+//   warp 0      TMA producer (Q per item; K ring and V ring, polled independently)
 //   warp 1      issues every Q K^T          warp 2      issues every P V
+//   warp 3      builds the kept / union list of the NEXT items (two list buffers)
 //   warps 4-7   softmax of the even tiles   warps 8-11  softmax of the odd tiles
 // A softmax thread owns one query row of its tile: the whole 128-column row of S sits in registers.  The
 // two threads that own the same row (one per warpgroup) share the row's reference maximum through shared
@@ -24,6 +28,8 @@
 // Every mbarrier wait is bounded; a wait that runs out sets SPARSP_ERR_TIMEOUT in the status word
 // and raises a CTA-wide flag that makes all later waits fall through, so the CTA still drains.
 #include <algorithm>
+#include <cstdlib>
+#include <type_traits>
 
 #include "common.cuh"
 #include "sm100_ptx.cuh"
@@ -34,8 +40,8 @@ using namespace ptx;
 
 struct AttnParams {
   const uint32_t* mask;
-  // block 64: [B*H][ceil(NB/2)][2] query blocks of each CTA (second may be -1); block 128: NULL (CTA x
-  // handles block x) or [B*H][2*ceil(NB/2)] query block of each CTA (-1 = none)
+  // block 64: [B*H][ceil(NB/2)][2] query blocks of each item (second may be -1); block 128: NULL (item x
+  // handles block x) or [B*H][2*ceil(NB/2)] query block of each item (-1 = none)
   const int32_t* pairs;
   // packed-source mode (NULL = every tile comes from K / V): slot[bh][j] = entry index of KV block j in
   // the consumer's packed buffer, or -1 if the consumer owns the block; tile_base = index of the
@@ -48,6 +54,8 @@ struct AttnParams {
   int64_t N;
   int64_t sB, sH, sT;
   int H, NB, Wd;
+  int per_bh;   // work items per (batch, head): NB (block 128) or ceil(NB/2) (block 64)
+  int n_items;  // B * H * per_bh
   float scale_log2;  // softmax scale * log2(e)
   long long wait_limit;
 };
@@ -75,33 +83,21 @@ struct AttnCfg {
   static constexpr int kOffQ = 0;
   static constexpr int kOffK = kOffQ + kQBytes;
   static constexpr int kOffV = kOffK + kStagesK * kTileBytes;
-  static constexpr int kOffEntJ = kOffV + kStagesV * kTileBytes;  // uint16 [1024] kept / union list
-  static constexpr int kOffEntF = kOffEntJ + 2 * kMaxBlocks;      // uint8 [1024] bit q: kept by query block q
-  static constexpr int kOffStat = kOffEntF + kMaxBlocks;          // float2 [2 warpgroups][128]
-  static constexpr int kOffRef = kOffStat + 2 * 128 * 8;          // float [128] reference maximum per row
-  static constexpr int kOffSlot = kOffRef + 128 * 4;              // int32 [1024] packed-buffer slot per list entry
-  static constexpr int kOffBars = kOffSlot + 4 * kMaxBlocks;
-  static constexpr int kNumBars = 1 + 2 * (kStagesK + kStagesV) + 10;
+  static constexpr int kOffEntJ = kOffV + kStagesV * kTileBytes;  // uint16 [2][1024] kept / union list
+  static constexpr int kOffEntF = kOffEntJ + 2 * 2 * kMaxBlocks;  // uint8 [2][1024] bit q: kept by query block q
+  static constexpr int kOffSlot = kOffEntF + 2 * kMaxBlocks;      // int32 [2][1024] packed-buffer slot per entry
+  static constexpr int kOffStat = kOffSlot + 2 * 4 * kMaxBlocks;  // float2 [2 items][2 warpgroups][128]
+  static constexpr int kOffRef = kOffStat + 2 * 2 * 128 * 8;      // float [3 items][128] reference maximum per row
+  static constexpr int kOffBars = kOffRef + 3 * 128 * 4;
+  static constexpr int kNumBars = 2 + 2 * (kStagesK + kStagesV) + 10 + 1 + 4;
   static constexpr int kColS = 0;    // S buffers: columns [0, 256)
   static constexpr int kColP = 256;  // P buffers: columns [256, 384)
   static constexpr int kColO = 384;  // accumulator: columns [384, 384 + d)
   static constexpr int kOffMisc = kOffBars + 8 * kNumBars;
-  static constexpr int kTotal = kOffMisc + 32;
+  static constexpr int kTotal = kOffMisc + 64;
   static constexpr int kDynamic = kTotal + 1024;  // slack for the 1024-byte alignment of the base
   static_assert(kDynamic <= 232448, "shared memory budget");
 };
-
-#ifdef SPARSP_ATTN_PROFILE
-// Optional cycle accounting for tuning builds: per-phase SM-clock totals of one softmax lane and of
-// the MMA thread of every CTA.  Off in normal builds.
-__device__ unsigned long long g_attn_prof[16];
-#define PROF_T(var) const long long var = clock64()
-#define PROF_ADD(slot, a, b) \
-  if (lane == 0 && (warp == 4 || warp == 1)) atomicAdd(&g_attn_prof[slot], (unsigned long long)((b) - (a)))
-#else
-#define PROF_T(var)
-#define PROF_ADD(slot, a, b)
-#endif
 
 // Packed fp32 pairs (one instruction for two lanes' worth of fused multiply-add / add).
 __device__ __forceinline__ float2 ffma2(float2 a, float2 b, float2 c) {
@@ -159,49 +155,44 @@ __global__ void __launch_bounds__(kAttnThreads, 1)
   unsigned char* sQ = smem + C::kOffQ;
   unsigned char* sK = smem + C::kOffK;
   unsigned char* sV = smem + C::kOffV;
-  uint16_t* sEntJ = reinterpret_cast<uint16_t*>(smem + C::kOffEntJ);
-  uint8_t* sEntF = smem + C::kOffEntF;
-  float2* sStat = reinterpret_cast<float2*>(smem + C::kOffStat);
-  volatile float* sRef = reinterpret_cast<volatile float*>(smem + C::kOffRef);
-  int32_t* sSlot = reinterpret_cast<int32_t*>(smem + C::kOffSlot);
+  uint16_t* sEntJ = reinterpret_cast<uint16_t*>(smem + C::kOffEntJ);  // [2][kMaxBlocks]
+  uint8_t* sEntF = smem + C::kOffEntF;                                // [2][kMaxBlocks]
+  int32_t* sSlot = reinterpret_cast<int32_t*>(smem + C::kOffSlot);    // [2][kMaxBlocks]
+  float2* sStat = reinterpret_cast<float2*>(smem + C::kOffStat);      // [2][2][128]
+  volatile float* sRef = reinterpret_cast<volatile float*>(smem + C::kOffRef);  // [3][128]
   uint64_t* bars = reinterpret_cast<uint64_t*>(smem + C::kOffBars);
-  uint64_t* bar_q = bars;
-  uint64_t* k_full = bars + 1;
+  uint64_t* q_full = bars;          // the item's Q tile has landed
+  uint64_t* q_free = bars + 1;      // every Q K^T of the item has completed: Q may be overwritten
+  uint64_t* k_full = bars + 2;
   uint64_t* k_empty = k_full + SK;
   uint64_t* v_full = k_empty + SK;
   uint64_t* v_empty = v_full + SV;
   uint64_t* s_full = v_empty + SV;  // [2] S buffer written by a Q K^T
   uint64_t* s_free = s_full + 2;    // [2] S buffer read into registers by its 4 softmax warps
   uint64_t* p_full = s_free + 2;    // [2] P buffer written by its 4 softmax warps
-  // [4] the P V of tile n arrives on o_full[n % 4].  Four barriers, because a parity wait can only tell the
-  // phase a barrier is in from the one before: a softmax thread that wants P V n-1 or n-2 has itself seen
-  // P V n-4 complete, and P V n+2 cannot complete before that thread has stored P_n.
+  // [4] the P V of tile g arrives on o_full[g % 4].  Four barriers, because a parity wait can only tell the
+  // phase a barrier is in from the one before: a softmax thread that wants P V g-1 or g-2 has itself seen
+  // P V g-4 complete, and P V g+2 cannot complete before that thread has stored P_g.
   uint64_t* o_full = p_full + 2;
+  uint64_t* o_drained = o_full + 4;      // the item's accumulator has been read out by all 8 softmax warps
+  uint64_t* list_ready = o_drained + 1;  // [2] list buffer filled
+  uint64_t* list_free = list_ready + 2;  // [2] list buffer no longer needed by its 11 readers
   uint32_t* s_tmem = reinterpret_cast<uint32_t*>(smem + C::kOffMisc);
-  int* s_nent = reinterpret_cast<int*>(smem + C::kOffMisc + 4);
-  volatile int* s_abort = reinterpret_cast<volatile int*>(smem + C::kOffMisc + 8);
+  volatile int* s_abort = reinterpret_cast<volatile int*>(smem + C::kOffMisc + 4);
+  int* s_nent = reinterpret_cast<int*>(smem + C::kOffMisc + 8);   // [2]
+  int* s_blk = reinterpret_cast<int*>(smem + C::kOffMisc + 16);   // [2][2] the item's query block(s); < 0 = absent
+  constexpr int kListReaders = 11;  // producer, two issuers, eight softmax warps
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-  PROF_T(t_cta0);
-  const int bh = blockIdx.y;
-  const int batch = bh / p.H, head = bh % p.H;
-  // the CTA's query block(s); a negative entry means "absent"
-  int blk[2];
-  if (C::kStacked) {
-    const int32_t* pr = p.pairs + ((int64_t)bh * gridDim.x + blockIdx.x) * 2;
-    blk[0] = pr[0];
-    blk[1] = pr[1];
-  } else {
-    blk[0] = p.pairs ? p.pairs[(int64_t)bh * (2 * ((p.NB + 1) / 2)) + blockIdx.x] : (int)blockIdx.x;
-    blk[1] = -1;
-  }
+  const int G = (int)gridDim.x;
 
   // ---- setup ------------------------------------------------------------------------------
   if (tid == 0) {
     prefetch_tmap(&tmQ);
     prefetch_tmap(&tmK);
     prefetch_tmap(&tmV);
-    mbar_init(bar_q, 1);
+    mbar_init(q_full, 1);
+    mbar_init(q_free, 1);
     for (int s = 0; s < SK; ++s) {
       mbar_init(k_full + s, 1);
       mbar_init(k_empty + s, 1);
@@ -214,197 +205,250 @@ __global__ void __launch_bounds__(kAttnThreads, 1)
       mbar_init(s_full + s, 1);
       mbar_init(s_free + s, 4);
       mbar_init(p_full + s, 4);
+      mbar_init(list_ready + s, 1);
+      mbar_init(list_free + s, kListReaders);
     }
     for (int s = 0; s < 4; ++s) mbar_init(o_full + s, 1);
+    mbar_init(o_drained, 8);
     mbar_init_fence();
     *s_abort = 0;
   }
-  if (tid >= 128 && tid < 256) sRef[tid - 128] = -INFINITY;
+  sRef[tid] = -INFINITY;  // 3 x 128 entries, 384 threads
   if (warp == 1) {
     tmem_alloc(s_tmem, kTmemCols);
     tmem_relinquish();
-  }
-  if (warp == 0) {
-    // union of the (up to) two mask rows -> ascending entry list; flag bit q = kept by query block blk[q]
-    const uint32_t* mrow0 = p.mask + ((int64_t)bh * p.NB + max(blk[0], 0)) * p.Wd;
-    const uint32_t* mrow1 = p.mask + ((int64_t)bh * p.NB + max(blk[1], 0)) * p.Wd;
-    int running = 0;
-    for (int w0 = 0; w0 < p.Wd; w0 += 32) {
-      const int w = w0 + lane;
-      uint32_t rb[2];
-      rb[0] = (w < p.Wd && blk[0] >= 0) ? mrow0[w] : 0u;
-      rb[1] = (w < p.Wd && blk[1] >= 0) ? mrow1[w] : 0u;
-      uint32_t u = rb[0] | rb[1];
-      const int mine = __popc(u);
-      int incl = mine;
-#pragma unroll
-      for (int s = 1; s < 32; s <<= 1) {
-        const int v = __shfl_up_sync(0xffffffffu, incl, s);
-        if (lane >= s) incl += v;
-      }
-      int pos = running + incl - mine;
-      while (u) {
-        const int t = __ffs(u) - 1;
-        u &= u - 1;
-        sEntJ[pos] = (uint16_t)(w * 32 + t);
-        sEntF[pos] = (uint8_t)(((rb[0] >> t) & 1u) | (((rb[1] >> t) & 1u) << 1));
-        if (p.slot) sSlot[pos] = p.slot[(int64_t)bh * p.NB + w * 32 + t];
-        ++pos;
-      }
-      running += __shfl_sync(0xffffffffu, incl, 31);
-    }
-    if (lane == 0) *s_nent = running;
   }
   tc_fence_before();
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem_base = *s_tmem;
-  const int n_ent = *s_nent;
-  const int n_tiles = (n_ent + C::kEPT - 1) / C::kEPT;
 
   // the utility warpgroup hands most of its registers to the two softmax warpgroups (the re-balancing
   // instruction sits inside each role's branch so that the register allocator sees which code runs
   // under which limit)
   if (warp < 4) {
     asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(SPARSP_REGS_UTILITY));
-    if (warp == 0) {
-      // ================================ TMA producer ========================================
-      if (lane == 0 && n_tiles > 0) {
-        mbar_expect_tx(bar_q, C::kQBytes);
-        // a Q tile is 128 rows: one 128-token block, or two 64-token blocks stacked (an absent second
-        // block re-reads the first: finite data whose rows are never used)
-#pragma unroll
-        for (int q = 0; q < C::kEPT; ++q) {
-          const int tok = max(blk[q] >= 0 ? blk[q] : blk[0], 0) * BLK;
-#pragma unroll
-          for (int c = 0; c < D / 64; ++c)
-            tma_load_4d(sQ + c * 16384 + q * (BLK * 128), &tmQ, bar_q, c * 64, tok, head, batch);
+    if (warp == 3) {
+      // ================================ list builder ========================================
+      // union of the item's (up to) two mask rows -> ascending entry list; flag bit q = kept by query
+      // block blk[q].  Runs up to two items ahead of the consumers.
+      int i = 0;
+      for (int it = blockIdx.x; it < p.n_items; it += G, ++i) {
+        const int buf = i & 1;
+        if (i >= 2) mbar_wait_bounded(list_free + buf, ((i - 2) >> 1) & 1, s_abort, p.status, 50, p.wait_limit);
+        const int bh = it / p.per_bh, x = it - bh * p.per_bh;
+        int blk[2];
+        if (C::kStacked) {
+          const int32_t* pr = p.pairs + ((int64_t)bh * p.per_bh + x) * 2;
+          blk[0] = pr[0];
+          blk[1] = pr[1];
+        } else {
+          blk[0] = p.pairs ? p.pairs[(int64_t)bh * (2 * ((p.NB + 1) / 2)) + x] : x;
+          blk[1] = -1;
         }
-        const int tile_base = p.slot ? (int)p.tile_base[batch] : 0;
-        auto load_tile = [&](unsigned char* dst, const CUtensorMap* tm, uint64_t* bar, int n, int n_stages) {
-#ifdef SPARSP_ATTN_NOLOAD  // tuning builds only: reuse stale tiles to take TMA traffic out of the picture
-          if (n >= n_stages) {
-            mbar_arrive(bar);
-            return;
-          }
-#endif
-          mbar_expect_tx(bar, C::kTileBytes);
+        uint16_t* entJ = sEntJ + buf * kMaxBlocks;
+        uint8_t* entF = sEntF + buf * kMaxBlocks;
+        int32_t* entS = sSlot + buf * kMaxBlocks;
+        const uint32_t* mrow0 = p.mask + ((int64_t)bh * p.NB + max(blk[0], 0)) * p.Wd;
+        const uint32_t* mrow1 = p.mask + ((int64_t)bh * p.NB + max(blk[1], 0)) * p.Wd;
+        int running = 0;
+        for (int w0 = 0; w0 < p.Wd; w0 += 32) {
+          const int w = w0 + lane;
+          uint32_t rb[2];
+          rb[0] = (w < p.Wd && blk[0] >= 0) ? mrow0[w] : 0u;
+          rb[1] = (w < p.Wd && blk[1] >= 0) ? mrow1[w] : 0u;
+          uint32_t u = rb[0] | rb[1];
+          const int mine = __popc(u);
+          int incl = mine;
 #pragma unroll
-          for (int e = 0; e < C::kEPT; ++e) {
-            const int ent = min(n * C::kEPT + e, n_ent - 1);  // an absent second half re-reads the last entry
-            const int j = sEntJ[ent];
-            const int slot = p.slot ? sSlot[ent] : -1;
-            if (slot < 0) {
+          for (int s = 1; s < 32; s <<= 1) {
+            const int v = __shfl_up_sync(0xffffffffu, incl, s);
+            if (lane >= s) incl += v;
+          }
+          int pos = running + incl - mine;
+          while (u) {
+            const int t = __ffs(u) - 1;
+            u &= u - 1;
+            entJ[pos] = (uint16_t)(w * 32 + t);
+            entF[pos] = (uint8_t)(((rb[0] >> t) & 1u) | (((rb[1] >> t) & 1u) << 1));
+            if (p.slot) entS[pos] = p.slot[(int64_t)bh * p.NB + w * 32 + t];
+            ++pos;
+          }
+          running += __shfl_sync(0xffffffffu, incl, 31);
+        }
+        if (lane == 0) {
+          s_nent[buf] = running;
+          s_blk[buf * 2] = blk[0];
+          s_blk[buf * 2 + 1] = blk[1];
+        }
+        __syncwarp();
+        if (lane == 0) mbar_arrive(list_ready + buf);
+      }
+    } else if (warp == 0) {
+      // ================================ TMA producer ========================================
+      if (lane == 0) {
+        int i = 0, kn = 0, vn = 0, qc = 0;  // items seen; K / V tiles loaded so far; items that had tiles
+        for (int it = blockIdx.x; it < p.n_items; it += G, ++i) {
+          const int buf = i & 1;
+          mbar_wait_bounded(list_ready + buf, (i >> 1) & 1, s_abort, p.status, 51, p.wait_limit);
+          const int n_ent = s_nent[buf];
+          const int n_tiles = (n_ent + C::kEPT - 1) / C::kEPT;
+          const int bh = it / p.per_bh;
+          const int batch = bh / p.H, head = bh % p.H;
+          const uint16_t* entJ = sEntJ + buf * kMaxBlocks;
+          const int32_t* entS = sSlot + buf * kMaxBlocks;
+          if (n_tiles > 0) {
+            // the Q tile may be overwritten once every Q K^T of the previous item has completed
+            if (qc > 0) mbar_wait_bounded(q_free, (qc - 1) & 1, s_abort, p.status, 52, p.wait_limit);
+            ++qc;
+            mbar_expect_tx(q_full, C::kQBytes);
+            // a Q tile is 128 rows: one 128-token block, or two 64-token blocks stacked (an absent second
+            // block re-reads the first: finite data whose rows are never used)
+#pragma unroll
+            for (int q = 0; q < C::kEPT; ++q) {
+              const int bq = s_blk[buf * 2 + q] >= 0 ? s_blk[buf * 2 + q] : s_blk[buf * 2];
+              const int tok = max(bq, 0) * BLK;
 #pragma unroll
               for (int c = 0; c < D / 64; ++c)
-                tma_load_4d(dst + c * 16384 + e * (BLK * 128), tm, bar, c * 64, j * BLK, head, batch);
-            } else {
-              // remote block: its K tile and V tile are consecutive tiles of the consumer's packed buffer
-              const int tile = tile_base + 2 * slot + (tm == &tmV ? 1 : 0);
+                tma_load_4d(sQ + c * 16384 + q * (BLK * 128), &tmQ, q_full, c * 64, tok, head, batch);
+            }
+            const int tile_base = p.slot ? (int)p.tile_base[batch] : 0;
+            auto load_tile = [&](unsigned char* dst, const CUtensorMap* tm, uint64_t* bar, int n) {
+              mbar_expect_tx(bar, C::kTileBytes);
 #pragma unroll
-              for (int c = 0; c < D / 64; ++c)
-                tma_load_4d(dst + c * 16384 + e * (BLK * 128), &tmP, bar, c * 64, 0, tile, 0);
+              for (int e = 0; e < C::kEPT; ++e) {
+                const int ent = min(n * C::kEPT + e, n_ent - 1);  // an absent second half re-reads the last entry
+                const int j = entJ[ent];
+                const int slot = p.slot ? entS[ent] : -1;
+                if (slot < 0) {
+#pragma unroll
+                  for (int c = 0; c < D / 64; ++c)
+                    tma_load_4d(dst + c * 16384 + e * (BLK * 128), tm, bar, c * 64, j * BLK, head, batch);
+                } else {
+                  // remote block: its K tile and V tile are consecutive tiles of the consumer's packed buffer
+                  const int tile = tile_base + 2 * slot + (tm == &tmV ? 1 : 0);
+#pragma unroll
+                  for (int c = 0; c < D / 64; ++c)
+                    tma_load_4d(dst + c * 16384 + e * (BLK * 128), &tmP, bar, c * 64, 0, tile, 0);
+                }
+              }
+            };
+            const int k0 = kn, v0 = vn, k_end = kn + n_tiles, v_end = vn + n_tiles;
+            const long long t0 = clock64();
+            while ((kn < k_end || vn < v_end) && !*s_abort) {
+              bool progressed = false;
+              if (kn < k_end && mbar_test_wait(k_empty + kn % SK, ((kn / SK) & 1) ^ 1)) {
+                load_tile(sK + (kn % SK) * C::kTileBytes, &tmK, k_full + kn % SK, kn - k0);
+                ++kn;
+                progressed = true;
+              }
+              if (vn < v_end && mbar_test_wait(v_empty + vn % SV, ((vn / SV) & 1) ^ 1)) {
+                load_tile(sV + (vn % SV) * C::kTileBytes, &tmV, v_full + vn % SV, vn - v0);
+                ++vn;
+                progressed = true;
+              }
+              if (!progressed) {
+                // both rings are full: the loads run several tiles ahead of the MMAs, so polling slowly
+                // costs nothing and leaves this scheduler's issue slots to the softmax warps that share it
+                __nanosleep(200);
+                if (clock64() - t0 > p.wait_limit * 8) {
+                  *s_abort = 1;
+                  if (atomicCAS(p.status, 0, SPARSP_ERR_TIMEOUT) == 0) p.status[1] = 10;
+                }
+              }
+            }
+            if (*s_abort) {  // keep the tile counters in step with the other roles
+              kn = k_end;
+              vn = v_end;
             }
           }
-        };
-        int kn = 0, vn = 0;
-        const long long t0 = clock64();
-        while ((kn < n_tiles || vn < n_tiles) && !*s_abort) {
-          bool progressed = false;
-          if (kn < n_tiles && mbar_test_wait(k_empty + kn % SK, ((kn / SK) & 1) ^ 1)) {
-            load_tile(sK + (kn % SK) * C::kTileBytes, &tmK, k_full + kn % SK, kn, SK);
-            ++kn;
-            progressed = true;
-          }
-          if (vn < n_tiles && mbar_test_wait(v_empty + vn % SV, ((vn / SV) & 1) ^ 1)) {
-            load_tile(sV + (vn % SV) * C::kTileBytes, &tmV, v_full + vn % SV, vn, SV);
-            ++vn;
-            progressed = true;
-          }
-          if (!progressed) {
-            // both rings are full: the loads run several tiles ahead of the MMAs, so polling slowly costs
-            // nothing and leaves this scheduler's issue slots to the softmax warps that share it
-            __nanosleep(200);
-            if (clock64() - t0 > p.wait_limit * 8) {
-              *s_abort = 1;
-              if (atomicCAS(p.status, 0, SPARSP_ERR_TIMEOUT) == 0) p.status[1] = 10;
-            }
-          }
+          mbar_arrive(list_free + buf);
         }
       }
     } else if (warp == 1) {
       // ================================ Q K^T issuer ========================================
       // The whole warp runs the loop (uniform control flow and operands); one elected lane issues.
-      if (n_tiles > 0) {
-        const bool leader = elect_one();
-        constexpr uint32_t kIdescQK = make_idesc_bf16(128, 128, 0, 0);
-        const uint64_t descQ = make_smem_desc(smem_u32(sQ), 16, 1024);
-        const uint64_t descK = make_smem_desc(smem_u32(sK), 16, 1024);
-        const uint32_t hiQK = (uint32_t)(descK >> 32);
-        uint32_t qlo[D / 16], klo[D / 16];
+      const bool leader = elect_one();
+      constexpr uint32_t kIdescQK = make_idesc_bf16(128, 128, 0, 0);
+      const uint64_t descQ = make_smem_desc(smem_u32(sQ), 16, 1024);
+      const uint64_t descK = make_smem_desc(smem_u32(sK), 16, 1024);
+      const uint32_t hiQK = (uint32_t)(descK >> 32);
+      uint32_t qlo[D / 16], klo[D / 16];
 #pragma unroll
-        for (int kk = 0; kk < D / 16; ++kk) {
-          const uint32_t off = (uint32_t)(((kk / 4) * 16384 + (kk % 4) * 32) >> 4);
-          qlo[kk] = (uint32_t)descQ + off;
-          klo[kk] = (uint32_t)descK + off;
-        }
-        mbar_wait_bounded(bar_q, 0, s_abort, p.status, 11, p.wait_limit);
-        for (int n = 0; n < n_tiles; ++n) {
-          PROF_T(t_k0);
-          mbar_wait_bounded(k_full + n % SK, (n / SK) & 1, s_abort, p.status, 12, p.wait_limit);
-          PROF_T(t_k1);
-          PROF_ADD(9, t_k0, t_k1);  // issuer waiting for K
-          // S buffer n%2 is free once the softmax warps have loaded the scores of tile n-2
-          if (n >= 2) mbar_wait_bounded(s_free + (n & 1), ((n - 2) >> 1) & 1, s_abort, p.status, 24, p.wait_limit);
-          PROF_T(t_k3);
-          PROF_ADD(8, t_k1, t_k3);  // issuer waiting for a free S buffer
-          tc_fence_after();
-          const uint32_t stage_off = (uint32_t)(((n % SK) * C::kTileBytes) >> 4);
-          const uint32_t tS = tmem_base + C::kColS + (n & 1) * 128;
-          if (leader) {
-#pragma unroll
-            for (int kk = 0; kk < D / 16; ++kk)
-              mma_ss_lohi(tS, qlo[kk], hiQK, klo[kk] + stage_off, hiQK, kIdescQK, kk > 0 ? 1u : 0u);
-            mma_commit(s_full + (n & 1));
-            mma_commit(k_empty + n % SK);
-          }
-          __syncwarp();
-          PROF_T(t_k2);
-          PROF_ADD(7, t_k3, t_k2);  // issuer issuing Q K^T
-        }
+      for (int kk = 0; kk < D / 16; ++kk) {
+        const uint32_t off = (uint32_t)(((kk / 4) * 16384 + (kk % 4) * 32) >> 4);
+        qlo[kk] = (uint32_t)descQ + off;
+        klo[kk] = (uint32_t)descK + off;
       }
-    } else if (warp == 2) {
-      // ================================ P V issuer ==========================================
-      if (n_tiles > 0) {
-        const bool leader = elect_one();
-        constexpr uint32_t kIdescPV = make_idesc_bf16(128, D, 0, 1);
-        const uint64_t descV = make_smem_desc(smem_u32(sV), 16384, 1024);
-        const uint32_t hiV = (uint32_t)(descV >> 32);
-        uint32_t vlo[8];
+      int i = 0, g = 0, qc = 0;
+      for (int it = blockIdx.x; it < p.n_items; it += G, ++i) {
+        const int buf = i & 1;
+        mbar_wait_bounded(list_ready + buf, (i >> 1) & 1, s_abort, p.status, 53, p.wait_limit);
+        const int n_tiles = (s_nent[buf] + C::kEPT - 1) / C::kEPT;
+        if (n_tiles > 0) {
+          mbar_wait_bounded(q_full, qc & 1, s_abort, p.status, 11, p.wait_limit);
+          ++qc;
+          for (int n = 0; n < n_tiles; ++n, ++g) {
+            mbar_wait_bounded(k_full + g % SK, (g / SK) & 1, s_abort, p.status, 12, p.wait_limit);
+            // S buffer g%2 is free once the softmax warps have loaded the scores of tile g-2
+            if (g >= 2) mbar_wait_bounded(s_free + (g & 1), ((g - 2) >> 1) & 1, s_abort, p.status, 24, p.wait_limit);
+            tc_fence_after();
+            const uint32_t stage_off = (uint32_t)(((g % SK) * C::kTileBytes) >> 4);
+            const uint32_t tS = tmem_base + C::kColS + (g & 1) * 128;
+            if (leader) {
 #pragma unroll
-        for (int kk = 0; kk < 8; ++kk) vlo[kk] = (uint32_t)descV + (uint32_t)((kk * 2048) >> 4);
-        const uint32_t tO = tmem_base + C::kColO;
-        for (int n = 0; n < n_tiles; ++n) {
-          mbar_wait_bounded(p_full + (n & 1), (n >> 1) & 1, s_abort, p.status, 20, p.wait_limit);
-          mbar_wait_bounded(v_full + n % SV, (n / SV) & 1, s_abort, p.status, 22, p.wait_limit);
+              for (int kk = 0; kk < D / 16; ++kk)
+                mma_ss_lohi(tS, qlo[kk], hiQK, klo[kk] + stage_off, hiQK, kIdescQK, kk > 0 ? 1u : 0u);
+              mma_commit(s_full + (g & 1));
+              mma_commit(k_empty + g % SK);
+              if (n == n_tiles - 1) mma_commit(q_free);
+            }
+            __syncwarp();
+          }
+        }
+        if (lane == 0) mbar_arrive(list_free + buf);
+        __syncwarp();
+      }
+    } else {
+      // ================================ P V issuer ==========================================
+      const bool leader = elect_one();
+      constexpr uint32_t kIdescPV = make_idesc_bf16(128, D, 0, 1);
+      const uint64_t descV = make_smem_desc(smem_u32(sV), 16384, 1024);
+      const uint32_t hiV = (uint32_t)(descV >> 32);
+      uint32_t vlo[8];
+#pragma unroll
+      for (int kk = 0; kk < 8; ++kk) vlo[kk] = (uint32_t)descV + (uint32_t)((kk * 2048) >> 4);
+      const uint32_t tO = tmem_base + C::kColO;
+      int i = 0, g = 0;
+      for (int it = blockIdx.x; it < p.n_items; it += G, ++i) {
+        const int buf = i & 1;
+        mbar_wait_bounded(list_ready + buf, (i >> 1) & 1, s_abort, p.status, 54, p.wait_limit);
+        const int n_tiles = (s_nent[buf] + C::kEPT - 1) / C::kEPT;
+        // the previous item's accumulator must have been read out before this item's first P V overwrites it
+        if (i > 0) mbar_wait_bounded(o_drained, (i - 1) & 1, s_abort, p.status, 55, p.wait_limit);
+        for (int n = 0; n < n_tiles; ++n, ++g) {
+          mbar_wait_bounded(p_full + (g & 1), (g >> 1) & 1, s_abort, p.status, 20, p.wait_limit);
+          mbar_wait_bounded(v_full + g % SV, (g / SV) & 1, s_abort, p.status, 22, p.wait_limit);
           tc_fence_after();
-          const uint32_t stage_off = (uint32_t)(((n % SV) * C::kTileBytes) >> 4);
-          const uint32_t tP = tmem_base + C::kColP + (n & 1) * 64;
+          const uint32_t stage_off = (uint32_t)(((g % SV) * C::kTileBytes) >> 4);
+          const uint32_t tP = tmem_base + C::kColP + (g & 1) * 64;
           if (leader) {
 #pragma unroll
             for (int kk = 0; kk < 8; ++kk)
               mma_ts_lohi(tO, tP + kk * 8, vlo[kk] + stage_off, hiV, kIdescPV, (kk > 0 || n > 0) ? 1u : 0u);
-            mma_commit(o_full + (n & 3));
-            mma_commit(v_empty + n % SV);
+            mma_commit(o_full + (g & 3));
+            mma_commit(v_empty + g % SV);
           }
           __syncwarp();
         }
+        if (lane == 0) mbar_arrive(list_free + buf);
+        __syncwarp();
       }
     }
   } else {
     asm volatile("setmaxnreg.inc.sync.aligned.u32 %0;" ::"n"(SPARSP_REGS_SOFTMAX));
     // ================================ softmax warpgroups ==================================
-    const int wg = (warp >> 2) - 1;  // 0: even tiles, 1: odd tiles; also the S / P buffer this warpgroup uses
+    const int wg = (warp >> 2) - 1;  // 0: even tiles g, 1: odd tiles; also the S / P buffer this warpgroup uses
     const int rgrp = warp & 3;       // tensor-memory lane group this warp may access
     const int row = rgrp * 32 + lane;
     const int rh = row >> 6;         // which query block of a stacked Q tile the row belongs to
@@ -414,205 +458,209 @@ __global__ void __launch_bounds__(kAttnThreads, 1)
     const uint32_t tO = tmem_base + C::kColO + lane_off;
     const int bar_mine = 1 + wg * 4 + rgrp;         // I arrive here after my decision
     const int bar_other = 1 + (1 - wg) * 4 + rgrp;  // the row group's other warp arrives here after its decision
-    float m_ref = -INFINITY;  // the row's reference maximum (log2 domain) as this thread last saw it
-    float l_run = 0.0f;       // this thread's partial row sum, relative to m_ref
-    int cnt = 0;              // tiles this warpgroup has processed
 
-    PROF_T(t_loop0);
-    PROF_ADD(11, t_cta0, t_loop0);  // prologue up to the softmax loop
-    for (int n = wg; n < n_tiles; n += 2, ++cnt) {
-      // kept / valid key columns of each 64-column half of the tile (warp-uniform)
-      int vh[2];
-      if (C::kStacked) {
-#pragma unroll
-        for (int h = 0; h < 2; ++h) {
-          const int ent = n * 2 + h;
-          vh[h] = 0;
-          if (ent < n_ent && ((sEntF[ent] >> rh) & 1)) vh[h] = (int)min((int64_t)64, p.N - (int64_t)sEntJ[ent] * 64);
-        }
-      } else {
-        const int nv = (int)min((int64_t)128, p.N - (int64_t)sEntJ[n] * 128);
-        vh[0] = min(nv, 64);
-        vh[1] = max(nv - 64, 0);
-      }
+    int i = 0, g0 = 0;  // items seen; number of the item's first tile
+    for (int it = blockIdx.x; it < p.n_items; it += G, ++i) {
+      const int buf = i & 1;
+      volatile float* ref = sRef + (i % 3) * 128;
+      mbar_wait_bounded_inline(list_ready + buf, (i >> 1) & 1, s_abort, 56, p.wait_limit);
+      const int n_ent = s_nent[buf];
+      const int n_tiles = (n_ent + C::kEPT - 1) / C::kEPT;
+      const uint16_t* entJ = sEntJ + buf * kMaxBlocks;
+      const uint8_t* entF = sEntF + buf * kMaxBlocks;
+      const int bh = it / p.per_bh;
+      const int batch = bh / p.H, head = bh % p.H;
+      float m_ref = -INFINITY;  // the row's reference maximum (log2 domain) as this thread last saw it
+      float l_run = 0.0f;       // this thread's partial row sum, relative to m_ref
 
-      PROF_T(t_a);
-      mbar_wait_bounded(s_full + wg, cnt & 1, s_abort, p.status, 30 + wg, p.wait_limit);
-      tc_fence_after();
-      PROF_T(t_b);
-      float sv[128];
+      // One tile of this warpgroup.  kRagged = the sequence ends inside the tile (possible only for the item's
+      // last tile): that variant carries the column masking, the common one stays small.
+      auto do_tile = [&](auto ragged_tag, const int n) {
+        constexpr bool kRagged = decltype(ragged_tag)::value;
+        const int g = g0 + n;
+        // kept / valid key columns of each 64-column half of the tile (warp-uniform)
+        int vh[2];
+        if (C::kStacked) {
 #pragma unroll
-      for (int c = 0; c < 4; ++c) tmem_ld32(tS + c * 32, reinterpret_cast<uint32_t*>(sv) + c * 32);
-      tmem_ld_wait();
-      // S is in registers: the Q K^T of tile n+2 may overwrite the buffer
-      tc_fence_before();
-      __syncwarp();
-      if (lane == 0) mbar_arrive(s_free + wg);
-      PROF_T(t_b2);
-#ifdef SPARSP_ATTN_NOSOFTMAX  // tuning builds only: measure the MMA / TMA pipeline alone
-      if (n >= 2) mbar_wait_bounded(o_full + ((n - 2) & 3), ((n - 2) >> 2) & 1, s_abort, p.status, 34 + wg, p.wait_limit);
-      __syncwarp();
-      if (lane == 0) mbar_arrive(p_full + wg);
-      continue;
-#endif
-      // one flat instruction stream per 64-key half; a ragged half (the sequence ends inside it) first has
-      // its invalid columns set to -inf, an absent half (not kept by this row's query block) is skipped
-      float mx = -INFINITY;
-#pragma unroll
-      for (int h = 0; h < 2; ++h) {
-        float* svh = sv + h * 64;
-        if (vh[h] > 0) {
-          if (vh[h] < 64) {
-#pragma unroll
-            for (int e = 0; e < 64; ++e) svh[e] = e < vh[h] ? svh[e] : -INFINITY;
-          }
-          float m0 = svh[0], m1 = svh[1], m2 = svh[2], m3 = svh[3];
-#pragma unroll
-          for (int e = 4; e < 64; e += 4) {
-            m0 = fmaxf(m0, svh[e]);
-            m1 = fmaxf(m1, svh[e + 1]);
-            m2 = fmaxf(m2, svh[e + 2]);
-            m3 = fmaxf(m3, svh[e + 3]);
-          }
-          mx = fmaxf(mx, fmaxf(fmaxf(m0, m1), fmaxf(m2, m3)));
-        }
-      }
-      mx *= p.scale_log2;
-      PROF_T(t_c);
-
-      // ---- my turn to look at / move the row's reference maximum (strictly in tile order) ----
-#ifndef SPARSP_ATTN_NOTURN  // (tuning builds only: without the hand-over the result is wrong)
-      if (n > 0) named_bar_sync(bar_other, 64);
-#endif
-      PROF_T(t_c2);
-      PROF_ADD(6, t_c, t_c2);  // waiting for my turn
-      {
-        const float m_cur = sRef[row];
-        if (m_cur != m_ref) {  // the other thread moved it since my last tile
-          l_run *= ex2(m_ref - m_cur);  // m_ref = -inf: l_run is 0 and stays 0
-          m_ref = m_cur;
-        }
-      }
-      const float m_new = fmaxf(m_ref, mx);
-      const bool grow = m_new > m_ref + kGrowThreshold || (m_ref == -INFINITY && m_new > -INFINITY);
-      if (__any_sync(0xffffffffu, grow)) {
-        const float alpha = grow ? ex2(m_ref - m_new) : 1.0f;  // m_ref = -inf -> 0
-        if (n > 0) {
-          // every P V issued so far must have landed in O before the row is rescaled; they complete in
-          // order, so the one of tile n-1 suffices
-          mbar_wait_bounded(o_full + ((n - 1) & 3), ((n - 1) >> 2) & 1, s_abort, p.status, 38, p.wait_limit);
-          tc_fence_after();
-#pragma unroll
-          for (int c = 0; c < D / 16; ++c) {  // the row's accumulator, 16 columns at a time
-            uint32_t o[16];
-            tmem_ld16(tO + c * 16, o);
-            tmem_ld_wait();
-#pragma unroll
-            for (int e = 0; e < 16; ++e) o[e] = __float_as_uint(__uint_as_float(o[e]) * alpha);
-            tmem_st16(tO + c * 16, o);
-          }
-          tmem_st_wait();
-          tc_fence_before();
-        }
-        l_run *= alpha;
-        if (grow) {
-          m_ref = m_new;
-          sRef[row] = m_new;
-        }
-      }
-#ifndef SPARSP_ATTN_NOTURN
-      if (n + 1 < n_tiles) {
-        asm volatile("bar.arrive %0, %1;" ::"r"(bar_mine), "r"(64) : "memory");
-      }
-#endif
-      PROF_T(t_d);
-
-      // exponentials of keys [32c, 32c+32) -> packed bf16 columns [16c, 16c+16) of the P buffer
-      float2 lsum2 = make_float2(0.0f, 0.0f);
-      const float neg_m = -m_ref;
-      uint32_t pk[64];
-      const float2 sc2 = make_float2(p.scale_log2, p.scale_log2), nm2 = make_float2(neg_m, neg_m);
-#pragma unroll
-      for (int h = 0; h < 2; ++h) {
-        const float* svh = sv + h * 64;
-        uint32_t* pkh = pk + h * 32;
-        if (vh[h] > 0) {  // then the row has a finite reference maximum
-#pragma unroll
-          for (int e = 0; e < 32; ++e) {
-            const float2 x = ffma2(make_float2(svh[2 * e], svh[2 * e + 1]), sc2, nm2);
-            const float2 pp = (SPARSP_TUNE_POLY > 0 && (e % (SPARSP_TUNE_POLY > 0 ? SPARSP_TUNE_POLY : 1)) == 1)
-                                  ? exp2_poly2(x)
-                                  : make_float2(ex2(x.x), ex2(x.y));
-            lsum2 = fadd2(lsum2, pp);
-            const __nv_bfloat162 h2 = __floats2bfloat162_rn(pp.x, pp.y);
-            pkh[e] = *reinterpret_cast<const uint32_t*>(&h2);
-          }
-          if (vh[h] < 64) {
-            // columns past the end of the sequence: exactly zero in P (the polynomial path returns
-            // 2^-126 for them, which the row sum may keep)
-#pragma unroll
-            for (int e = 0; e < 32; ++e) pkh[e] = 2 * e + 1 < vh[h] ? pkh[e] : (2 * e < vh[h] ? (pkh[e] & 0xffffu) : 0u);
+          for (int h = 0; h < 2; ++h) {
+            const int ent = n * 2 + h;
+            vh[h] = 0;
+            if (ent < n_ent && ((entF[ent] >> rh) & 1)) vh[h] = (int)min((int64_t)64, p.N - (int64_t)entJ[ent] * 64);
           }
         } else {
+          const int nv = (int)min((int64_t)128, p.N - (int64_t)entJ[n] * 128);
+          vh[0] = min(nv, 64);
+          vh[1] = max(nv - 64, 0);
+        }
+
+        mbar_wait_bounded_inline(s_full + wg, (g >> 1) & 1, s_abort, 30 + wg, p.wait_limit);
+        tc_fence_after();
+        float sv[128];
 #pragma unroll
-          for (int e = 0; e < 32; ++e) pkh[e] = 0u;
+        for (int c = 0; c < 4; ++c) tmem_ld32(tS + c * 32, reinterpret_cast<uint32_t*>(sv) + c * 32);
+        tmem_ld_wait();
+        // S is in registers: the Q K^T of tile g+2 may overwrite the buffer
+        tc_fence_before();
+        __syncwarp();
+        if (lane == 0) mbar_arrive(s_free + wg);
+
+        // one flat instruction stream per 64-key half; a ragged half (the sequence ends inside it) first has
+        // its invalid columns set to -inf, an absent half (not kept by this row's query block) is skipped
+        float mx = -INFINITY;
+#pragma unroll
+        for (int h = 0; h < 2; ++h) {
+          float* svh = sv + h * 64;
+          if (vh[h] > 0) {
+            if (kRagged && vh[h] < 64) {
+#pragma unroll
+              for (int e = 0; e < 64; ++e) svh[e] = e < vh[h] ? svh[e] : -INFINITY;
+            }
+            float m0 = svh[0], m1 = svh[1], m2 = svh[2], m3 = svh[3];
+#pragma unroll
+            for (int e = 4; e < 64; e += 4) {
+              m0 = fmaxf(m0, svh[e]);
+              m1 = fmaxf(m1, svh[e + 1]);
+              m2 = fmaxf(m2, svh[e + 2]);
+              m3 = fmaxf(m3, svh[e + 3]);
+            }
+            mx = fmaxf(mx, fmaxf(fmaxf(m0, m1), fmaxf(m2, m3)));
+          }
+        }
+        mx *= p.scale_log2;
+
+        // ---- my turn to look at / move the row's reference maximum (strictly in tile order) ----
+        if (n > 0) named_bar_sync(bar_other, 64);
+        {
+          const float m_cur = ref[row];
+          if (m_cur != m_ref) {  // the other thread moved it since my last tile
+            l_run *= ex2(m_ref - m_cur);  // m_ref = -inf: l_run is 0 and stays 0
+            m_ref = m_cur;
+          }
+        }
+        const float m_new = fmaxf(m_ref, mx);
+        const bool grow = m_new > m_ref + kGrowThreshold || (m_ref == -INFINITY && m_new > -INFINITY);
+        if (__any_sync(0xffffffffu, grow)) {
+          const float alpha = grow ? ex2(m_ref - m_new) : 1.0f;  // m_ref = -inf -> 0
+          if (n > 0) {
+            // every P V of the item issued so far must have landed in O before the row is rescaled; they
+            // complete in order, so the one of tile g-1 suffices
+            mbar_wait_bounded_inline(o_full + ((g - 1) & 3), ((g - 1) >> 2) & 1, s_abort, 38, p.wait_limit);
+            tc_fence_after();
+#pragma unroll 1
+            for (int c = 0; c < D / 16; ++c) {  // the row's accumulator, 16 columns at a time (rare: kept small)
+              uint32_t o[16];
+              tmem_ld16(tO + c * 16, o);
+              tmem_ld_wait();
+#pragma unroll
+              for (int e = 0; e < 16; ++e) o[e] = __float_as_uint(__uint_as_float(o[e]) * alpha);
+              tmem_st16(tO + c * 16, o);
+            }
+            tmem_st_wait();
+            tc_fence_before();
+          }
+          l_run *= alpha;
+          if (grow) {
+            m_ref = m_new;
+            ref[row] = m_new;
+          }
+        }
+        if (n + 1 < n_tiles) {
+          asm volatile("bar.arrive %0, %1;" ::"r"(bar_mine), "r"(64) : "memory");
+        }
+
+        // exponentials of keys [64h, 64h+64) -> packed bf16 columns [32h, 32h+32) of the P buffer
+        float2 lsum2 = make_float2(0.0f, 0.0f);
+        const float neg_m = -m_ref;
+        uint32_t pk[64];
+        const float2 sc2 = make_float2(p.scale_log2, p.scale_log2), nm2 = make_float2(neg_m, neg_m);
+#pragma unroll
+        for (int h = 0; h < 2; ++h) {
+          const float* svh = sv + h * 64;
+          uint32_t* pkh = pk + h * 32;
+          if (vh[h] > 0) {  // then the row has a finite reference maximum
+#pragma unroll
+            for (int e = 0; e < 32; ++e) {
+              const float2 x = ffma2(make_float2(svh[2 * e], svh[2 * e + 1]), sc2, nm2);
+              const float2 pp = (SPARSP_TUNE_POLY > 0 && (e % (SPARSP_TUNE_POLY > 0 ? SPARSP_TUNE_POLY : 1)) == 1)
+                                    ? exp2_poly2(x)
+                                    : make_float2(ex2(x.x), ex2(x.y));
+              lsum2 = fadd2(lsum2, pp);
+              const __nv_bfloat162 h2 = __floats2bfloat162_rn(pp.x, pp.y);
+              pkh[e] = *reinterpret_cast<const uint32_t*>(&h2);
+            }
+            if (kRagged && vh[h] < 64) {
+              // columns past the end of the sequence: exactly zero in P (the polynomial path returns
+              // 2^-126 for them, which the row sum may keep)
+#pragma unroll
+              for (int e = 0; e < 32; ++e) pkh[e] = 2 * e + 1 < vh[h] ? pkh[e] : (2 * e < vh[h] ? (pkh[e] & 0xffffu) : 0u);
+            }
+          } else {
+#pragma unroll
+            for (int e = 0; e < 32; ++e) pkh[e] = 0u;
+          }
+        }
+        l_run += lsum2.x + lsum2.y;
+        // my P buffer was last read by the P V of tile g-2
+        if (g >= 2) {
+          mbar_wait_bounded_inline(o_full + ((g - 2) & 3), ((g - 2) >> 2) & 1, s_abort, 34 + wg, p.wait_limit);
+          tc_fence_after();
+        }
+#pragma unroll
+        for (int c = 0; c < 4; ++c) tmem_st16(tP + c * 16, pk + c * 16);
+        tmem_st_wait();
+        tc_fence_before();
+        __syncwarp();
+        if (lane == 0) mbar_arrive(p_full + wg);
+      };
+      for (int n = (wg - g0) & 1; n < n_tiles; n += 2) {
+        // entries ascend, so only the last tile can reach past the end of the sequence
+        const bool ragged = n == n_tiles - 1 && (int64_t)(entJ[n_ent - 1] + 1) * BLK > p.N;
+        if (ragged) {
+          do_tile(std::true_type{}, n);
+        } else {
+          do_tile(std::false_type{}, n);
         }
       }
-      l_run += lsum2.x + lsum2.y;
-      PROF_T(t_e);
-      // my P buffer was last read by the P V of tile n-2
-      if (n >= 2) {
-        mbar_wait_bounded(o_full + ((n - 2) & 3), ((n - 2) >> 2) & 1, s_abort, p.status, 34 + wg, p.wait_limit);
+
+      // ---- item epilogue: warpgroup x writes the column half x of every row -------------------------
+      sStat[(buf * 2 + wg) * 128 + row] = make_float2(m_ref, l_run);
+      named_bar_sync(9, 256);  // all of the item's decisions and P stores are done
+      if (n_tiles > 0) {
+        const int last = g0 + n_tiles - 1;
+        mbar_wait_bounded_inline(o_full + (last & 3), (last >> 2) & 1, s_abort, 40, p.wait_limit);
         tc_fence_after();
       }
-#pragma unroll
-      for (int c = 0; c < 4; ++c) tmem_st16(tP + c * 16, pk + c * 16);
-      tmem_st_wait();
-      tc_fence_before();
-      __syncwarp();
-      if (lane == 0) mbar_arrive(p_full + wg);
-      PROF_T(t_f);
-      PROF_ADD(0, t_a, t_b);      // wait for S
-      PROF_ADD(1, t_b, t_b2);     // load of S
-      PROF_ADD(14, t_b2, t_c);    // row maximum
-      PROF_ADD(2, t_c, t_d);      // turn-taking + rescale decision
-      PROF_ADD(3, t_d, t_e);      // exponentials
-      PROF_ADD(4, t_e, t_f);      // wait for the P buffer + store + arrive
-      PROF_ADD(5, t_a, t_a + 1);  // tile count
-    }
-
-    // ---- epilogue: warpgroup x writes the column half x of every row ------------------------------
-    PROF_T(t_ep0);
-    sStat[wg * 128 + row] = make_float2(m_ref, l_run);
-    named_bar_sync(9, 256);  // all tiles' decisions and P stores are done
-    if (n_tiles > 0) {
-      const int last = n_tiles - 1;
-      mbar_wait_bounded(o_full + (last & 3), (last >> 2) & 1, s_abort, p.status, 40, p.wait_limit);
-      tc_fence_after();
-    }
-    PROF_T(t_ep1);
-    {
-      constexpr int HW = D / 2;
-      const float m_fin = sRef[row];
-      const float2 st0 = sStat[row], st1 = sStat[128 + row];
-      const float l = (st0.y > 0.0f ? st0.y * ex2(st0.x - m_fin) : 0.0f) + (st1.y > 0.0f ? st1.y * ex2(st1.x - m_fin) : 0.0f);
-      const float inv_l = l > 0.0f ? 1.0f / l : 0.0f;
-      const int qb = C::kStacked ? blk[rh] : blk[0];
-      const int64_t tok = qb >= 0 ? (int64_t)qb * BLK + (C::kStacked ? (row & 63) : row) : p.N;
-      __nv_bfloat16* orow = p.O + (int64_t)batch * p.sB + (int64_t)head * p.sH + tok * p.sT + wg * HW;
-#pragma unroll
-      for (int c = 0; c < HW / 32; ++c) {
-        uint32_t o[32];
+      {
+        constexpr int HW = D / 2;
+        const float m_fin = ref[row];
+        const float2 st0 = sStat[(buf * 2) * 128 + row], st1 = sStat[(buf * 2 + 1) * 128 + row];
+        // this reference buffer serves the item after next: no warp can be there before every warp has passed
+        // the barrier above, and the item before this one (its last user) is finished for all of them
+        sRef[((i + 2) % 3) * 128 + row] = -INFINITY;
+        const float l = (st0.y > 0.0f ? st0.y * ex2(st0.x - m_fin) : 0.0f) + (st1.y > 0.0f ? st1.y * ex2(st1.x - m_fin) : 0.0f);
+        const float inv_l = l > 0.0f ? 1.0f / l : 0.0f;
+        const int qb = C::kStacked ? s_blk[buf * 2 + rh] : s_blk[buf * 2];
+        const int64_t tok = qb >= 0 ? (int64_t)qb * BLK + (C::kStacked ? (row & 63) : row) : p.N;
+        __nv_bfloat16* orow = p.O + (int64_t)batch * p.sB + (int64_t)head * p.sH + tok * p.sT + wg * HW;
+        uint32_t o[HW];
         if (n_tiles > 0) {  // CTA-uniform: tensor-memory loads are warp-collective
-          tmem_ld32(tO + wg * HW + c * 32, o);
+#pragma unroll
+          for (int c = 0; c < HW / 32; ++c) tmem_ld32(tO + wg * HW + c * 32, o + c * 32);
           tmem_ld_wait();
         } else {
 #pragma unroll
-          for (int e = 0; e < 32; ++e) o[e] = 0u;
+          for (int e = 0; e < HW; ++e) o[e] = 0u;
+        }
+        // the accumulator is in registers: the next item's first P V may overwrite it
+        tc_fence_before();
+        __syncwarp();
+        if (lane == 0) {
+          mbar_arrive(o_drained);
+          mbar_arrive(list_free + buf);
         }
         if (tok < p.N) {
 #pragma unroll
-          for (int v = 0; v < 4; ++v) {
+          for (int v = 0; v < HW / 8; ++v) {
             uint32_t w[4];
 #pragma unroll
             for (int e = 0; e < 4; ++e) {
@@ -620,22 +668,20 @@ __global__ void __launch_bounds__(kAttnThreads, 1)
                                                               __uint_as_float(o[v * 8 + 2 * e + 1]) * inv_l);
               w[e] = *reinterpret_cast<const uint32_t*>(&h2);
             }
-            *reinterpret_cast<uint4*>(orow + c * 32 + v * 8) = make_uint4(w[0], w[1], w[2], w[3]);
+            *reinterpret_cast<uint4*>(orow + v * 8) = make_uint4(w[0], w[1], w[2], w[3]);
           }
         }
+        if (p.lse && wg == 0 && tok < p.N)
+          p.lse[(int64_t)bh * p.N + tok] = l > 0.0f ? (m_fin + log2f(l)) * 0.6931471805599453f : -INFINITY;
       }
-      if (p.lse && wg == 0 && tok < p.N)
-        p.lse[(int64_t)bh * p.N + tok] = l > 0.0f ? (m_fin + log2f(l)) * 0.6931471805599453f : -INFINITY;
+      g0 += n_tiles;
     }
   }
 
-  PROF_T(t_cta1);
   tc_fence_before();
   __syncthreads();
   if (warp == 1) tmem_dealloc(tmem_base, kTmemCols);
-  PROF_T(t_cta2);
-  PROF_ADD(13, t_cta0, t_cta1);  // CTA lifetime of the sampled lanes up to the final barrier
-  PROF_ADD(15, t_cta0, t_cta0 + 1);
+  if (tid == 0) report_abort(s_abort, p.status);
 }
 
 // ------------------------------------------------------------------------------------------------
@@ -780,9 +826,16 @@ static int launch_attn_t(const sparsp_shape& s, const Geometry& g, const void* Q
   auto kern = attn_fwd_kernel<D, BLK>;
   const int smem = AttnCfg<D, BLK>::kDynamic;
   SPARSP_CUDA_OK(ensure_dynamic_smem((const void*)kern, smem));
-  // one CTA per 128-row Q tile: a 128-token block, or a pair of 64-token blocks
-  dim3 grid((unsigned)(BLK == 128 ? g.NB : (g.NB + 1) / 2), (unsigned)(g.B * g.H));
-  kern<<<grid, kAttnThreads, smem, st>>>(tq, tk, tv, tp, p);
+  // work item = one 128-row Q tile (a 128-token block, or a pair of 64-token blocks); one persistent CTA per SM
+  AttnParams pp = p;
+  pp.per_bh = BLK == 128 ? g.NB : (g.NB + 1) / 2;
+  pp.n_items = g.B * g.H * pp.per_bh;
+  int dev = 0, sms = 0;
+  SPARSP_CUDA_OK(cudaGetDevice(&dev));
+  SPARSP_CUDA_OK(cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev));
+  static const int ctas_per_sm_x100 = getenv("SPARSP_TUNE_GRID") ? atoi(getenv("SPARSP_TUNE_GRID")) : 100;
+  dim3 grid((unsigned)std::min<long long>(pp.n_items, (long long)sms * ctas_per_sm_x100 / 100));
+  kern<<<grid, kAttnThreads, smem, st>>>(tq, tk, tv, tp, pp);
   count_launch();
   SPARSP_CUDA_OK(cudaGetLastError());
   return SPARSP_OK;
@@ -928,17 +981,5 @@ int launch_attn_packed(const sparsp_shape& s, const Geometry& g, const void* Q, 
   p.tile_base = tile_base;
   return launch_attn_common(s, g, Q, K, V, packed, capacity, p, scale, O, lse, ws, L, st);
 }
-
-#ifdef SPARSP_ATTN_PROFILE
-extern "C" __attribute__((visibility("default"))) int sparsp_debug_attn_profile(unsigned long long* out16, int reset) {
-  cudaDeviceSynchronize();
-  cudaMemcpyFromSymbol(out16, g_attn_prof, sizeof(g_attn_prof));
-  if (reset) {
-    unsigned long long z[16] = {0};
-    cudaMemcpyToSymbol(g_attn_prof, z, sizeof z);
-  }
-  return 0;
-}
-#endif
 
 }  // namespace sparsp

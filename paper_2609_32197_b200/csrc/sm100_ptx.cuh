@@ -72,16 +72,13 @@ __device__ __forceinline__ bool mbar_test_wait(uint64_t* bar, uint32_t parity) {
 // Bounded wait: gives up after `limit_cycles` SM clock cycles.  On give-up it raises the CTA-wide
 // abort flag (after which every later wait of the CTA returns at once, so control flow stays
 // uniform and the kernel drains quickly) and records `code`/`where` in the global status words.
-__device__ __forceinline__ void mbar_wait_bounded(uint64_t* bar, uint32_t parity, volatile int* abort_flag,
-                                                  int32_t* status, int where, long long limit_cycles,
-                                                  unsigned sleep_ns = 0) {
-  if (mbar_try_wait(bar, parity)) return;
+// The polling loop lives in one out-of-line function: the kernels that use it have dozens of waits and
+// their hot loops must stay small enough for the instruction caches.
+static __device__ __noinline__ void mbar_wait_slow(uint64_t* bar, uint32_t parity, volatile int* abort_flag,
+                                            int32_t* status, int where, long long limit_cycles) {
   if (*abort_flag) return;
   const long long t0 = clock64();
   while (!mbar_try_wait(bar, parity)) {
-    // many-thread waiters back off, so that their polling does not take issue slots from the
-    // single-thread MMA issuer and TMA producer that share their scheduler
-    if (sleep_ns) __nanosleep(sleep_ns);
     if (*abort_flag) return;
     if (clock64() - t0 > limit_cycles) {
       *abort_flag = 1;
@@ -92,6 +89,36 @@ __device__ __forceinline__ void mbar_wait_bounded(uint64_t* bar, uint32_t parity
       }
       return;
     }
+  }
+}
+__device__ __forceinline__ void mbar_wait_bounded(uint64_t* bar, uint32_t parity, volatile int* abort_flag,
+                                                  int32_t* status, int where, long long limit_cycles) {
+  if (mbar_try_wait(bar, parity)) return;
+  mbar_wait_slow(bar, parity, abort_flag, status, where, limit_cycles);
+}
+// Same, fully inline and as small as possible: for waits inside hot loops whose threads hold most of their
+// registers live (a call there would have to save them).  On give-up only the CTA-wide flag is set, to
+// `where` + 1; the kernel reports it to the status words once, at its end (report_abort below).
+__device__ __forceinline__ void mbar_wait_bounded_inline(uint64_t* bar, uint32_t parity, volatile int* abort_flag,
+                                                         int where, long long limit_cycles) {
+  if (mbar_try_wait(bar, parity)) return;
+  const long long t0 = clock64();
+  while (!mbar_try_wait(bar, parity)) {
+    if (*abort_flag) return;
+    if (clock64() - t0 > limit_cycles) {
+      *abort_flag = where + 1;
+      return;
+    }
+  }
+}
+// One thread, after the CTA's last barrier: turns a raised abort flag into the global status words
+// (unless an earlier report is already there).
+__device__ __forceinline__ void report_abort(volatile int* abort_flag, int32_t* status) {
+  const int a = *abort_flag;
+  if (a != 0 && atomicCAS(status, 0, -5 /* SPARSP_ERR_TIMEOUT */) == 0) {
+    status[1] = a - 1;
+    status[2] = (int)blockIdx.x;
+    status[3] = (int)blockIdx.y;
   }
 }
 
