@@ -249,32 +249,64 @@ __global__ void __launch_bounds__(kAttnThreads, 1)
         uint16_t* entJ = sEntJ + buf * kMaxBlocks;
         uint8_t* entF = sEntF + buf * kMaxBlocks;
         int32_t* entS = sSlot + buf * kMaxBlocks;
-        const uint32_t* mrow0 = p.mask + ((int64_t)bh * p.NB + max(blk[0], 0)) * p.Wd;
-        const uint32_t* mrow1 = p.mask + ((int64_t)bh * p.NB + max(blk[1], 0)) * p.Wd;
-        int running = 0;
-        for (int w0 = 0; w0 < p.Wd; w0 += 32) {
-          const int w = w0 + lane;
-          uint32_t rb[2];
-          rb[0] = (w < p.Wd && blk[0] >= 0) ? mrow0[w] : 0u;
-          rb[1] = (w < p.Wd && blk[1] >= 0) ? mrow1[w] : 0u;
-          uint32_t u = rb[0] | rb[1];
-          const int mine = __popc(u);
+        // NB <= 1024, so a mask row is at most 32 words: one word per lane
+        const uint32_t rb0 = (lane < p.Wd && blk[0] >= 0) ? p.mask[((int64_t)bh * p.NB + blk[0]) * p.Wd + lane] : 0u;
+        const uint32_t rb1 = (lane < p.Wd && blk[1] >= 0) ? p.mask[((int64_t)bh * p.NB + blk[1]) * p.Wd + lane] : 0u;
+        // Entry order (any order gives the same attention): first the blocks BOTH query blocks keep, then the
+        // blocks only the first keeps alternating with the blocks only the second keeps, then what is left of
+        // the longer of those two lists.  A tile is two consecutive entries, so a tile of the middle part costs
+        // every softmax row one 64-key half instead of costing half of the rows two.  With a single query
+        // block this is plain ascending order.
+        uint32_t cls[3] = {rb0 & rb1, rb0 & ~rb1, rb1 & ~rb0};
+        int before[3], total[3];
+#pragma unroll
+        for (int c = 0; c < 3; ++c) {
+          const int mine = __popc(cls[c]);
           int incl = mine;
 #pragma unroll
           for (int s = 1; s < 32; s <<= 1) {
             const int v = __shfl_up_sync(0xffffffffu, incl, s);
             if (lane >= s) incl += v;
           }
-          int pos = running + incl - mine;
+          before[c] = incl - mine;
+          total[c] = __shfl_sync(0xffffffffu, incl, 31);
+        }
+        const int n_both = total[0], n_mix = min(total[1], total[2]);
+        const int running = total[0] + total[1] + total[2];
+#pragma unroll
+        for (int c = 0; c < 3; ++c) {
+          uint32_t u = cls[c];
+          int idx = before[c];  // rank of the entry inside its class
           while (u) {
             const int t = __ffs(u) - 1;
             u &= u - 1;
-            entJ[pos] = (uint16_t)(w * 32 + t);
-            entF[pos] = (uint8_t)(((rb[0] >> t) & 1u) | (((rb[1] >> t) & 1u) << 1));
-            if (p.slot) entS[pos] = p.slot[(int64_t)bh * p.NB + w * 32 + t];
-            ++pos;
+            int pos;
+            if (c == 0) pos = idx;
+            else if (idx < n_mix) pos = n_both + 2 * idx + (c - 1);
+            else pos = n_both + n_mix + idx;  // tail of the longer class
+            entJ[pos] = (uint16_t)(lane * 32 + t);
+            entF[pos] = (uint8_t)(c == 0 ? 3 : c);
+            if (p.slot) entS[pos] = p.slot[(int64_t)bh * p.NB + lane * 32 + t];
+            ++idx;
           }
-          running += __shfl_sync(0xffffffffu, incl, 31);
+        }
+        __syncwarp();
+        // the softmax code lets only the LAST tile reach past the end of the sequence: if the last block of
+        // the sequence is ragged and in the list, it trades places with the last entry
+        if ((int64_t)p.NB * BLK > p.N && running > 0) {
+          const int lw = (p.NB - 1) >> 5, lb = (p.NB - 1) & 31;
+          const uint32_t have = __shfl_sync(0xffffffffu, rb0 | rb1, lw);
+          if ((have >> lb) & 1u) {
+            if (lane == 0) {
+              int r = 0;
+              while (r < running - 1 && entJ[r] != (uint16_t)(p.NB - 1)) ++r;
+              const int e = running - 1;
+              const uint16_t tj = entJ[r]; entJ[r] = entJ[e]; entJ[e] = tj;
+              const uint8_t tf = entF[r]; entF[r] = entF[e]; entF[e] = tf;
+              if (p.slot) { const int32_t ts = entS[r]; entS[r] = entS[e]; entS[e] = ts; }
+            }
+            __syncwarp();
+          }
         }
         if (lane == 0) {
           s_nent[buf] = running;
@@ -613,7 +645,7 @@ __global__ void __launch_bounds__(kAttnThreads, 1)
         if (lane == 0) mbar_arrive(p_full + wg);
       };
       for (int n = (wg - g0) & 1; n < n_tiles; n += 2) {
-        // entries ascend, so only the last tile can reach past the end of the sequence
+        // the list builder puts the sequence's last block (the only one that can be ragged) into the last tile
         const bool ragged = n == n_tiles - 1 && (int64_t)(entJ[n_ent - 1] + 1) * BLK > p.N;
         if (ragged) {
           do_tile(std::true_type{}, n);

@@ -98,10 +98,11 @@ def test_attention_reading_remote_blocks_from_the_packed_buffer(oracle_mod, bind
     with NaN, and the oracle computes the expected rows from the same restricted view."""
     from paper_2609_32197_b200 import synth
     H, P = 3, 3
-    # a few more kept blocks than the minimum: with very few, |O| grows past 4 where half a bf16 ulp (0.0156) of
-    # output rounding alone nearly uses up the bound
     wl = synth.Workload("packed", H, d, (5, 11, 13), 70, b, 5 if b == 128 else 9, None, P, seed=61)
     Q, K, V = synth.make_qkv(wl, "cpu")
+    # with this few kept blocks some outputs of the stock recipe pass 4, where half a bf16 ulp (0.0156) of
+    # output rounding alone nearly uses up the 2e-2 bound; halving V (exact in bf16) keeps |O| below 2.5
+    V = (V.float() * 0.5).to(torch.bfloat16)
     N, NB = wl.n_tokens, wl.n_blocks
     shape = binding.make_shape(H, d, wl.grid, wl.n_text, b, layout=layout)
     Qd, Kd, Vd = (pu.to_layout(x.cuda(), layout) for x in (Q, K, V))
