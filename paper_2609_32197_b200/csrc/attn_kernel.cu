@@ -13,11 +13,14 @@
 // tiles' MMAs queued while the softmax of the current tile runs: Q K^T of tile g+2 starts as soon as the
 // scores of tile g have been READ, and P V of tile g is issued as soon as P_g is written.  Tiles are
 // numbered g = 0, 1, 2, ... across the CTA's items; every ring, buffer and barrier phase follows g.
-// Warp roles (384 threads = 3 warpgroups; the first hands most of its registers to the other two):
-//   warp 0      TMA producer (Q per item; K ring and V ring, polled independently)
+// Warp roles (512 threads = 4 warpgroups; the first two hand most of their registers to the other two):
+//   warp 0      TMA producer of Q (per item) and of the K ring
 //   warp 1      issues every Q K^T          warp 2      issues every P V
-//   warp 3      builds the kept / union list of the NEXT items (two list buffers)
-//   warps 4-7   softmax of the even tiles   warps 8-11  softmax of the odd tiles
+//   warp 3      TMA producer of the V ring
+//   warp 4      builds the kept / union list of the NEXT items (two list buffers; warps 5-7 idle)
+//   warps 8-11  softmax of the even tiles   warps 12-15 softmax of the odd tiles
+// (A producer is one thread running a chain of dependent instructions next to busy softmax warps: it gets
+// an instruction issued every ~8 cycles, so K and V loads have a warp each and keep per-tile work minimal.)
 // A softmax thread owns one query row of its tile: the whole 128-column row of S sits in registers.  The
 // two threads that own the same row (one per warpgroup) share the row's reference maximum through shared
 // memory and take their decisions strictly in tile order (a pair of 64-thread named barriers per row
@@ -60,9 +63,10 @@ struct AttnParams {
   long long wait_limit;
 };
 
-constexpr int kAttnThreads = 384;  // three warpgroups: utility warps, softmax of the even tiles, softmax of the odd tiles
-// register budget per thread after the warpgroups re-balance (128*72 + 256*216 = 384*168)
-#define SPARSP_REGS_UTILITY 72
+constexpr int kAttnThreads = 512;  // four warpgroups: two of utility warps, softmax of the even tiles, softmax of the odd tiles
+// register budget per thread after the warpgroups re-balance (128*48 + 128*32 + 256*216 = 512*128)
+#define SPARSP_REGS_UTILITY 48
+#define SPARSP_REGS_UTILITY2 32
 #define SPARSP_REGS_SOFTMAX 216
 constexpr int kTmemCols = 512;
 constexpr float kGrowThreshold = 8.0f;
@@ -181,7 +185,7 @@ __global__ void __launch_bounds__(kAttnThreads, 1)
   volatile int* s_abort = reinterpret_cast<volatile int*>(smem + C::kOffMisc + 4);
   int* s_nent = reinterpret_cast<int*>(smem + C::kOffMisc + 8);   // [2]
   int* s_blk = reinterpret_cast<int*>(smem + C::kOffMisc + 16);   // [2][2] the item's query block(s); < 0 = absent
-  constexpr int kListReaders = 11;  // producer, two issuers, eight softmax warps
+  constexpr int kListReaders = 12;  // two producers, two issuers, eight softmax warps
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int G = (int)gridDim.x;
@@ -213,7 +217,7 @@ __global__ void __launch_bounds__(kAttnThreads, 1)
     mbar_init_fence();
     *s_abort = 0;
   }
-  sRef[tid] = -INFINITY;  // 3 x 128 entries, 384 threads
+  if (tid < 384) sRef[tid] = -INFINITY;  // 3 x 128 entries
   if (warp == 1) {
     tmem_alloc(s_tmem, kTmemCols);
     tmem_relinquish();
@@ -229,13 +233,193 @@ __global__ void __launch_bounds__(kAttnThreads, 1)
   if (warp < 4) {
     asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(SPARSP_REGS_UTILITY));
     if (warp == 3) {
-      // ================================ list builder ========================================
+      // ================================ TMA producer: V =====================================
+      if (lane == 0) {
+        int i = 0, vn = 0;  // items seen; V tiles loaded so far
+        for (int it = blockIdx.x; it < p.n_items; it += G, ++i) {
+          const int buf = i & 1;
+          mbar_wait_bounded_inline(list_ready + buf, (i >> 1) & 1, s_abort, 58, p.wait_limit);
+          const int n_ent = s_nent[buf];
+          const int n_tiles = (n_ent + C::kEPT - 1) / C::kEPT;
+          if (n_tiles > 0) {
+            const int bh = it / p.per_bh;
+            const int batch = bh / p.H, head = bh % p.H;
+            const uint16_t* entJ = sEntJ + buf * kMaxBlocks;
+            const int32_t* entS = sSlot + buf * kMaxBlocks;
+            const int tile_base = p.slot ? (int)p.tile_base[batch] : 0;
+            for (int n = 0; n < n_tiles; ++n, ++vn) {
+              const int st = vn % SV;
+              mbar_wait_bounded_inline(v_empty + st, ((vn / SV) & 1) ^ 1, s_abort, 59, p.wait_limit);
+              unsigned char* dst = sV + st * C::kTileBytes;
+              mbar_expect_tx(v_full + st, C::kTileBytes);
+  #pragma unroll
+              for (int e = 0; e < C::kEPT; ++e) {
+                const int ent = min(n * C::kEPT + e, n_ent - 1);
+                const int slot = p.slot ? entS[ent] : -1;
+                if (slot < 0) {
+                  const int tok = (int)entJ[ent] * BLK;
+  #pragma unroll
+                  for (int c = 0; c < D / 64; ++c)
+                    tma_load_4d(dst + c * 16384 + e * (BLK * 128), &tmV, v_full + st, c * 64, tok, head, batch);
+                } else {
+  #pragma unroll
+                  for (int c = 0; c < D / 64; ++c)
+                    tma_load_4d(dst + c * 16384 + e * (BLK * 128), &tmP, v_full + st, c * 64, 0, tile_base + 2 * slot + 1, 0);
+                }
+              }
+            }
+          }
+          mbar_arrive(list_free + buf);
+        }
+      }
+    } else if (warp == 0) {
+      // ================================ TMA producer: Q and K ===============================
+      if (lane == 0) {
+        int i = 0, kn = 0, qc = 0;  // items seen; K tiles loaded so far; items that had tiles
+        for (int it = blockIdx.x; it < p.n_items; it += G, ++i) {
+          const int buf = i & 1;
+          mbar_wait_bounded_inline(list_ready + buf, (i >> 1) & 1, s_abort, 51, p.wait_limit);
+          const int n_ent = s_nent[buf];
+          const int n_tiles = (n_ent + C::kEPT - 1) / C::kEPT;
+          if (n_tiles > 0) {
+            const int bh = it / p.per_bh;
+            const int batch = bh / p.H, head = bh % p.H;
+            const uint16_t* entJ = sEntJ + buf * kMaxBlocks;
+            const int32_t* entS = sSlot + buf * kMaxBlocks;
+            const int tile_base = p.slot ? (int)p.tile_base[batch] : 0;
+            for (int n = 0; n < n_tiles; ++n, ++kn) {
+              const int st = kn % SK;
+              mbar_wait_bounded_inline(k_empty + st, ((kn / SK) & 1) ^ 1, s_abort, 57, p.wait_limit);
+              unsigned char* dst = sK + st * C::kTileBytes;
+              mbar_expect_tx(k_full + st, C::kTileBytes);
+#pragma unroll
+              for (int e = 0; e < C::kEPT; ++e) {
+                const int ent = min(n * C::kEPT + e, n_ent - 1);  // an absent second half re-reads the last entry
+                const int slot = p.slot ? entS[ent] : -1;
+                if (slot < 0) {
+                  const int tok = (int)entJ[ent] * BLK;
+#pragma unroll
+                  for (int c = 0; c < D / 64; ++c)
+                    tma_load_4d(dst + c * 16384 + e * (BLK * 128), &tmK, k_full + st, c * 64, tok, head, batch);
+                } else {
+                  // remote block: its K tile and V tile are consecutive tiles of the consumer's packed buffer
+#pragma unroll
+                  for (int c = 0; c < D / 64; ++c)
+                    tma_load_4d(dst + c * 16384 + e * (BLK * 128), &tmP, k_full + st, c * 64, 0, tile_base + 2 * slot, 0);
+                }
+              }
+              if (n == 0) {
+                // the item's first K tile is on its way; now the Q tile, which may be overwritten once every
+                // Q K^T of the previous item has completed
+                if (qc > 0) mbar_wait_bounded_inline(q_free, (qc - 1) & 1, s_abort, 52, p.wait_limit);
+                ++qc;
+                mbar_expect_tx(q_full, C::kQBytes);
+                // a Q tile is 128 rows: one 128-token block, or two 64-token blocks stacked (an absent second
+                // block re-reads the first: finite data whose rows are never used)
+#pragma unroll
+                for (int q = 0; q < C::kEPT; ++q) {
+                  const int bq = s_blk[buf * 2 + q] >= 0 ? s_blk[buf * 2 + q] : s_blk[buf * 2];
+                  const int tok = max(bq, 0) * BLK;
+#pragma unroll
+                  for (int c = 0; c < D / 64; ++c)
+                    tma_load_4d(sQ + c * 16384 + q * (BLK * 128), &tmQ, q_full, c * 64, tok, head, batch);
+                }
+              }
+            }
+          }
+          mbar_arrive(list_free + buf);
+        }
+      }
+    } else if (warp == 1) {
+      // ================================ Q K^T issuer ========================================
+      // The whole warp runs the loop (uniform control flow and operands); one elected lane issues.
+      const bool leader = elect_one();
+      constexpr uint32_t kIdescQK = make_idesc_bf16(128, 128, 0, 0);
+      const uint64_t descQ = make_smem_desc(smem_u32(sQ), 16, 1024);
+      const uint64_t descK = make_smem_desc(smem_u32(sK), 16, 1024);
+      const uint32_t hiQK = (uint32_t)(descK >> 32);
+      uint32_t qlo[D / 16], klo[D / 16];
+#pragma unroll
+      for (int kk = 0; kk < D / 16; ++kk) {
+        const uint32_t off = (uint32_t)(((kk / 4) * 16384 + (kk % 4) * 32) >> 4);
+        qlo[kk] = (uint32_t)descQ + off;
+        klo[kk] = (uint32_t)descK + off;
+      }
+      int i = 0, g = 0, qc = 0;
+      for (int it = blockIdx.x; it < p.n_items; it += G, ++i) {
+        const int buf = i & 1;
+        mbar_wait_bounded_inline(list_ready + buf, (i >> 1) & 1, s_abort, 53, p.wait_limit);
+        const int n_tiles = (s_nent[buf] + C::kEPT - 1) / C::kEPT;
+        if (n_tiles > 0) {
+          mbar_wait_bounded_inline(q_full, qc & 1, s_abort, 11, p.wait_limit);
+          ++qc;
+          for (int n = 0; n < n_tiles; ++n, ++g) {
+            mbar_wait_bounded_inline(k_full + g % SK, (g / SK) & 1, s_abort, 12, p.wait_limit);
+            // S buffer g%2 is free once the softmax warps have loaded the scores of tile g-2
+            if (g >= 2) mbar_wait_bounded_inline(s_free + (g & 1), ((g - 2) >> 1) & 1, s_abort, 24, p.wait_limit);
+            tc_fence_after();
+            const uint32_t stage_off = (uint32_t)(((g % SK) * C::kTileBytes) >> 4);
+            const uint32_t tS = tmem_base + C::kColS + (g & 1) * 128;
+            if (leader) {
+#pragma unroll
+              for (int kk = 0; kk < D / 16; ++kk)
+                mma_ss_lohi(tS, qlo[kk], hiQK, klo[kk] + stage_off, hiQK, kIdescQK, kk > 0 ? 1u : 0u);
+              mma_commit(s_full + (g & 1));
+              mma_commit(k_empty + g % SK);
+              if (n == n_tiles - 1) mma_commit(q_free);
+            }
+            __syncwarp();
+          }
+        }
+        if (lane == 0) mbar_arrive(list_free + buf);
+        __syncwarp();
+      }
+    } else {
+      // ================================ P V issuer ==========================================
+      const bool leader = elect_one();
+      constexpr uint32_t kIdescPV = make_idesc_bf16(128, D, 0, 1);
+      const uint64_t descV = make_smem_desc(smem_u32(sV), 16384, 1024);
+      const uint32_t hiV = (uint32_t)(descV >> 32);
+      uint32_t vlo[8];
+#pragma unroll
+      for (int kk = 0; kk < 8; ++kk) vlo[kk] = (uint32_t)descV + (uint32_t)((kk * 2048) >> 4);
+      const uint32_t tO = tmem_base + C::kColO;
+      int i = 0, g = 0;
+      for (int it = blockIdx.x; it < p.n_items; it += G, ++i) {
+        const int buf = i & 1;
+        mbar_wait_bounded_inline(list_ready + buf, (i >> 1) & 1, s_abort, 54, p.wait_limit);
+        const int n_tiles = (s_nent[buf] + C::kEPT - 1) / C::kEPT;
+        // the previous item's accumulator must have been read out before this item's first P V overwrites it
+        if (i > 0) mbar_wait_bounded_inline(o_drained, (i - 1) & 1, s_abort, 55, p.wait_limit);
+        for (int n = 0; n < n_tiles; ++n, ++g) {
+          mbar_wait_bounded_inline(p_full + (g & 1), (g >> 1) & 1, s_abort, 20, p.wait_limit);
+          mbar_wait_bounded_inline(v_full + g % SV, (g / SV) & 1, s_abort, 22, p.wait_limit);
+          tc_fence_after();
+          const uint32_t stage_off = (uint32_t)(((g % SV) * C::kTileBytes) >> 4);
+          const uint32_t tP = tmem_base + C::kColP + (g & 1) * 64;
+          if (leader) {
+#pragma unroll
+            for (int kk = 0; kk < 8; ++kk)
+              mma_ts_lohi(tO, tP + kk * 8, vlo[kk] + stage_off, hiV, kIdescPV, (kk > 0 || n > 0) ? 1u : 0u);
+            mma_commit(o_full + (g & 3));
+            mma_commit(v_empty + g % SV);
+          }
+          __syncwarp();
+        }
+        if (lane == 0) mbar_arrive(list_free + buf);
+        __syncwarp();
+      }
+    }
+  } else if (warp < 8) {
+    asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(SPARSP_REGS_UTILITY2));
+    // ================================ list builder ========================================
+    if (warp == 4) {
       // union of the item's (up to) two mask rows -> ascending entry list; flag bit q = kept by query
       // block blk[q].  Runs up to two items ahead of the consumers.
       int i = 0;
       for (int it = blockIdx.x; it < p.n_items; it += G, ++i) {
         const int buf = i & 1;
-        if (i >= 2) mbar_wait_bounded(list_free + buf, ((i - 2) >> 1) & 1, s_abort, p.status, 50, p.wait_limit);
+        if (i >= 2) mbar_wait_bounded_inline(list_free + buf, ((i - 2) >> 1) & 1, s_abort, 50, p.wait_limit);
         const int bh = it / p.per_bh, x = it - bh * p.per_bh;
         int blk[2];
         if (C::kStacked) {
@@ -316,171 +500,11 @@ __global__ void __launch_bounds__(kAttnThreads, 1)
         __syncwarp();
         if (lane == 0) mbar_arrive(list_ready + buf);
       }
-    } else if (warp == 0) {
-      // ================================ TMA producer ========================================
-      if (lane == 0) {
-        int i = 0, kn = 0, vn = 0, qc = 0;  // items seen; K / V tiles loaded so far; items that had tiles
-        for (int it = blockIdx.x; it < p.n_items; it += G, ++i) {
-          const int buf = i & 1;
-          mbar_wait_bounded(list_ready + buf, (i >> 1) & 1, s_abort, p.status, 51, p.wait_limit);
-          const int n_ent = s_nent[buf];
-          const int n_tiles = (n_ent + C::kEPT - 1) / C::kEPT;
-          const int bh = it / p.per_bh;
-          const int batch = bh / p.H, head = bh % p.H;
-          const uint16_t* entJ = sEntJ + buf * kMaxBlocks;
-          const int32_t* entS = sSlot + buf * kMaxBlocks;
-          if (n_tiles > 0) {
-            // the Q tile may be overwritten once every Q K^T of the previous item has completed
-            if (qc > 0) mbar_wait_bounded(q_free, (qc - 1) & 1, s_abort, p.status, 52, p.wait_limit);
-            ++qc;
-            mbar_expect_tx(q_full, C::kQBytes);
-            // a Q tile is 128 rows: one 128-token block, or two 64-token blocks stacked (an absent second
-            // block re-reads the first: finite data whose rows are never used)
-#pragma unroll
-            for (int q = 0; q < C::kEPT; ++q) {
-              const int bq = s_blk[buf * 2 + q] >= 0 ? s_blk[buf * 2 + q] : s_blk[buf * 2];
-              const int tok = max(bq, 0) * BLK;
-#pragma unroll
-              for (int c = 0; c < D / 64; ++c)
-                tma_load_4d(sQ + c * 16384 + q * (BLK * 128), &tmQ, q_full, c * 64, tok, head, batch);
-            }
-            const int tile_base = p.slot ? (int)p.tile_base[batch] : 0;
-            auto load_tile = [&](unsigned char* dst, const CUtensorMap* tm, uint64_t* bar, int n) {
-              mbar_expect_tx(bar, C::kTileBytes);
-#pragma unroll
-              for (int e = 0; e < C::kEPT; ++e) {
-                const int ent = min(n * C::kEPT + e, n_ent - 1);  // an absent second half re-reads the last entry
-                const int j = entJ[ent];
-                const int slot = p.slot ? entS[ent] : -1;
-                if (slot < 0) {
-#pragma unroll
-                  for (int c = 0; c < D / 64; ++c)
-                    tma_load_4d(dst + c * 16384 + e * (BLK * 128), tm, bar, c * 64, j * BLK, head, batch);
-                } else {
-                  // remote block: its K tile and V tile are consecutive tiles of the consumer's packed buffer
-                  const int tile = tile_base + 2 * slot + (tm == &tmV ? 1 : 0);
-#pragma unroll
-                  for (int c = 0; c < D / 64; ++c)
-                    tma_load_4d(dst + c * 16384 + e * (BLK * 128), &tmP, bar, c * 64, 0, tile, 0);
-                }
-              }
-            };
-            const int k0 = kn, v0 = vn, k_end = kn + n_tiles, v_end = vn + n_tiles;
-            const long long t0 = clock64();
-            while ((kn < k_end || vn < v_end) && !*s_abort) {
-              bool progressed = false;
-              if (kn < k_end && mbar_test_wait(k_empty + kn % SK, ((kn / SK) & 1) ^ 1)) {
-                load_tile(sK + (kn % SK) * C::kTileBytes, &tmK, k_full + kn % SK, kn - k0);
-                ++kn;
-                progressed = true;
-              }
-              if (vn < v_end && mbar_test_wait(v_empty + vn % SV, ((vn / SV) & 1) ^ 1)) {
-                load_tile(sV + (vn % SV) * C::kTileBytes, &tmV, v_full + vn % SV, vn - v0);
-                ++vn;
-                progressed = true;
-              }
-              if (!progressed) {
-                // both rings are full: the loads run several tiles ahead of the MMAs, so polling slowly
-                // costs nothing and leaves this scheduler's issue slots to the softmax warps that share it
-                __nanosleep(200);
-                if (clock64() - t0 > p.wait_limit * 8) {
-                  *s_abort = 1;
-                  if (atomicCAS(p.status, 0, SPARSP_ERR_TIMEOUT) == 0) p.status[1] = 10;
-                }
-              }
-            }
-            if (*s_abort) {  // keep the tile counters in step with the other roles
-              kn = k_end;
-              vn = v_end;
-            }
-          }
-          mbar_arrive(list_free + buf);
-        }
-      }
-    } else if (warp == 1) {
-      // ================================ Q K^T issuer ========================================
-      // The whole warp runs the loop (uniform control flow and operands); one elected lane issues.
-      const bool leader = elect_one();
-      constexpr uint32_t kIdescQK = make_idesc_bf16(128, 128, 0, 0);
-      const uint64_t descQ = make_smem_desc(smem_u32(sQ), 16, 1024);
-      const uint64_t descK = make_smem_desc(smem_u32(sK), 16, 1024);
-      const uint32_t hiQK = (uint32_t)(descK >> 32);
-      uint32_t qlo[D / 16], klo[D / 16];
-#pragma unroll
-      for (int kk = 0; kk < D / 16; ++kk) {
-        const uint32_t off = (uint32_t)(((kk / 4) * 16384 + (kk % 4) * 32) >> 4);
-        qlo[kk] = (uint32_t)descQ + off;
-        klo[kk] = (uint32_t)descK + off;
-      }
-      int i = 0, g = 0, qc = 0;
-      for (int it = blockIdx.x; it < p.n_items; it += G, ++i) {
-        const int buf = i & 1;
-        mbar_wait_bounded(list_ready + buf, (i >> 1) & 1, s_abort, p.status, 53, p.wait_limit);
-        const int n_tiles = (s_nent[buf] + C::kEPT - 1) / C::kEPT;
-        if (n_tiles > 0) {
-          mbar_wait_bounded(q_full, qc & 1, s_abort, p.status, 11, p.wait_limit);
-          ++qc;
-          for (int n = 0; n < n_tiles; ++n, ++g) {
-            mbar_wait_bounded(k_full + g % SK, (g / SK) & 1, s_abort, p.status, 12, p.wait_limit);
-            // S buffer g%2 is free once the softmax warps have loaded the scores of tile g-2
-            if (g >= 2) mbar_wait_bounded(s_free + (g & 1), ((g - 2) >> 1) & 1, s_abort, p.status, 24, p.wait_limit);
-            tc_fence_after();
-            const uint32_t stage_off = (uint32_t)(((g % SK) * C::kTileBytes) >> 4);
-            const uint32_t tS = tmem_base + C::kColS + (g & 1) * 128;
-            if (leader) {
-#pragma unroll
-              for (int kk = 0; kk < D / 16; ++kk)
-                mma_ss_lohi(tS, qlo[kk], hiQK, klo[kk] + stage_off, hiQK, kIdescQK, kk > 0 ? 1u : 0u);
-              mma_commit(s_full + (g & 1));
-              mma_commit(k_empty + g % SK);
-              if (n == n_tiles - 1) mma_commit(q_free);
-            }
-            __syncwarp();
-          }
-        }
-        if (lane == 0) mbar_arrive(list_free + buf);
-        __syncwarp();
-      }
-    } else {
-      // ================================ P V issuer ==========================================
-      const bool leader = elect_one();
-      constexpr uint32_t kIdescPV = make_idesc_bf16(128, D, 0, 1);
-      const uint64_t descV = make_smem_desc(smem_u32(sV), 16384, 1024);
-      const uint32_t hiV = (uint32_t)(descV >> 32);
-      uint32_t vlo[8];
-#pragma unroll
-      for (int kk = 0; kk < 8; ++kk) vlo[kk] = (uint32_t)descV + (uint32_t)((kk * 2048) >> 4);
-      const uint32_t tO = tmem_base + C::kColO;
-      int i = 0, g = 0;
-      for (int it = blockIdx.x; it < p.n_items; it += G, ++i) {
-        const int buf = i & 1;
-        mbar_wait_bounded(list_ready + buf, (i >> 1) & 1, s_abort, p.status, 54, p.wait_limit);
-        const int n_tiles = (s_nent[buf] + C::kEPT - 1) / C::kEPT;
-        // the previous item's accumulator must have been read out before this item's first P V overwrites it
-        if (i > 0) mbar_wait_bounded(o_drained, (i - 1) & 1, s_abort, p.status, 55, p.wait_limit);
-        for (int n = 0; n < n_tiles; ++n, ++g) {
-          mbar_wait_bounded(p_full + (g & 1), (g >> 1) & 1, s_abort, p.status, 20, p.wait_limit);
-          mbar_wait_bounded(v_full + g % SV, (g / SV) & 1, s_abort, p.status, 22, p.wait_limit);
-          tc_fence_after();
-          const uint32_t stage_off = (uint32_t)(((g % SV) * C::kTileBytes) >> 4);
-          const uint32_t tP = tmem_base + C::kColP + (g & 1) * 64;
-          if (leader) {
-#pragma unroll
-            for (int kk = 0; kk < 8; ++kk)
-              mma_ts_lohi(tO, tP + kk * 8, vlo[kk] + stage_off, hiV, kIdescPV, (kk > 0 || n > 0) ? 1u : 0u);
-            mma_commit(o_full + (g & 3));
-            mma_commit(v_empty + g % SV);
-          }
-          __syncwarp();
-        }
-        if (lane == 0) mbar_arrive(list_free + buf);
-        __syncwarp();
-      }
     }
   } else {
     asm volatile("setmaxnreg.inc.sync.aligned.u32 %0;" ::"n"(SPARSP_REGS_SOFTMAX));
     // ================================ softmax warpgroups ==================================
-    const int wg = (warp >> 2) - 1;  // 0: even tiles g, 1: odd tiles; also the S / P buffer this warpgroup uses
+    const int wg = (warp >> 2) - 2;  // 0: even tiles g, 1: odd tiles; also the S / P buffer this warpgroup uses
     const int rgrp = warp & 3;       // tensor-memory lane group this warp may access
     const int row = rgrp * 32 + lane;
     const int rh = row >> 6;         // which query block of a stacked Q tile the row belongs to
