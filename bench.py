@@ -323,7 +323,7 @@ def run_ours(args):
         "pack_gbs": pack_gbs,
         "pack_pct_hbm": {"of_measured": pack_gbs / peaks["hbm_gbs"], "of_nominal": pack_gbs / NOMINAL["hbm_gbs"]},
         "volume_bytes_total": volume,
-        "roofline": {"bound": "tensor", "kernel": "attn_fwd_kernel (+ pair_kernel, timed together)", "achieved": attn_tflops,
+        "roofline": {"bound": "tensor", "kernel": "attn_fwd_kernel (+ attn_prep_kernel, timed together)", "achieved": attn_tflops,
                      "peak": peaks["bf16_tflops"], "peak_source": peaks["source"] + " burst", "unit": "TFLOP/s",
                      "frac": attn_tflops / peaks["bf16_tflops"],
                      "traffic": ATTN_DRAM_TRAFFIC.get((wl.name, k))},

@@ -117,6 +117,8 @@ WsLayout make_layout(const Geometry& g, int P) {
   off += align_up((int64_t)g.B * g.H * g.NB * 4, 256);
   L.tile_base = off;  // first packed tile of that consumer per batch item, int64 [B]
   off += align_up((int64_t)g.B * 8, 256);
+  L.knorm = off;  // largest key norm of every KV block, fp32 [B][H][NB] (attention: bound on the scores of a tile)
+  off += align_up((int64_t)g.B * g.H * g.NB * 4, 256);
   L.own = off;
   off += align_up((int64_t)P * g.Wd * 4, 256);
   L.ent_base = off;

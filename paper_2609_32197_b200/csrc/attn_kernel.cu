@@ -51,6 +51,9 @@ struct AttnParams {
   // consumer's first tile in the packed tensor map (a device scalar)
   const int32_t* slot;
   const int64_t* tile_base;
+  // largest key norm (L2) of every KV block, [B*H][NB], or NULL: lets a softmax row skip the row-maximum pass
+  // of a tile whose scores provably stay within 2^kSkipMargin of the row's reference maximum
+  const float* knorm;
   __nv_bfloat16* O;
   float* lse;
   int32_t* status;
@@ -70,10 +73,11 @@ constexpr int kAttnThreads = 512;  // four warpgroups: two of utility warps, sof
 #define SPARSP_REGS_SOFTMAX 216
 constexpr int kTmemCols = 512;
 constexpr float kGrowThreshold = 8.0f;
+constexpr float kSkipMargin = 64.0f;  // 2^64 * (keys of a sequence) * |V| stays far inside fp32
 // Tuning switch (compile-time): how many of the exponentials go to the FMA pipe instead of the
 // special-function unit (every n-th pair; 0 = none).
 #ifndef SPARSP_TUNE_POLY
-#define SPARSP_TUNE_POLY 3
+#define SPARSP_TUNE_POLY 4
 #endif
 
 template <int D, int BLK>
@@ -90,7 +94,8 @@ struct AttnCfg {
   static constexpr int kOffEntJ = kOffV + kStagesV * kTileBytes;  // uint16 [2][1024] kept / union list
   static constexpr int kOffEntF = kOffEntJ + 2 * 2 * kMaxBlocks;  // uint8 [2][1024] bit q: kept by query block q
   static constexpr int kOffSlot = kOffEntF + 2 * kMaxBlocks;      // int32 [2][1024] packed-buffer slot per entry
-  static constexpr int kOffStat = kOffSlot + 2 * 4 * kMaxBlocks;  // float2 [2 items][2 warpgroups][128]
+  static constexpr int kOffEntN = kOffSlot + 2 * 4 * kMaxBlocks;  // float [2][1024] largest key norm of the entry's block
+  static constexpr int kOffStat = kOffEntN + 2 * 4 * kMaxBlocks;  // float2 [2 items][2 warpgroups][128]
   static constexpr int kOffRef = kOffStat + 2 * 2 * 128 * 8;      // float [3 items][128] reference maximum per row
   static constexpr int kOffBars = kOffRef + 3 * 128 * 4;
   static constexpr int kNumBars = 2 + 2 * (kStagesK + kStagesV) + 10 + 1 + 4;
@@ -162,6 +167,7 @@ __global__ void __launch_bounds__(kAttnThreads, 1)
   uint16_t* sEntJ = reinterpret_cast<uint16_t*>(smem + C::kOffEntJ);  // [2][kMaxBlocks]
   uint8_t* sEntF = smem + C::kOffEntF;                                // [2][kMaxBlocks]
   int32_t* sSlot = reinterpret_cast<int32_t*>(smem + C::kOffSlot);    // [2][kMaxBlocks]
+  float* sEntN = reinterpret_cast<float*>(smem + C::kOffEntN);        // [2][kMaxBlocks]
   float2* sStat = reinterpret_cast<float2*>(smem + C::kOffStat);      // [2][2][128]
   volatile float* sRef = reinterpret_cast<volatile float*>(smem + C::kOffRef);  // [3][128]
   uint64_t* bars = reinterpret_cast<uint64_t*>(smem + C::kOffBars);
@@ -433,6 +439,7 @@ __global__ void __launch_bounds__(kAttnThreads, 1)
         uint16_t* entJ = sEntJ + buf * kMaxBlocks;
         uint8_t* entF = sEntF + buf * kMaxBlocks;
         int32_t* entS = sSlot + buf * kMaxBlocks;
+        float* entN = sEntN + buf * kMaxBlocks;
         // NB <= 1024, so a mask row is at most 32 words: one word per lane
         const uint32_t rb0 = (lane < p.Wd && blk[0] >= 0) ? p.mask[((int64_t)bh * p.NB + blk[0]) * p.Wd + lane] : 0u;
         const uint32_t rb1 = (lane < p.Wd && blk[1] >= 0) ? p.mask[((int64_t)bh * p.NB + blk[1]) * p.Wd + lane] : 0u;
@@ -471,6 +478,7 @@ __global__ void __launch_bounds__(kAttnThreads, 1)
             entJ[pos] = (uint16_t)(lane * 32 + t);
             entF[pos] = (uint8_t)(c == 0 ? 3 : c);
             if (p.slot) entS[pos] = p.slot[(int64_t)bh * p.NB + lane * 32 + t];
+            if (p.knorm) entN[pos] = p.knorm[(int64_t)bh * p.NB + lane * 32 + t];
             ++idx;
           }
         }
@@ -488,6 +496,7 @@ __global__ void __launch_bounds__(kAttnThreads, 1)
               const uint16_t tj = entJ[r]; entJ[r] = entJ[e]; entJ[e] = tj;
               const uint8_t tf = entF[r]; entF[r] = entF[e]; entF[e] = tf;
               if (p.slot) { const int32_t ts = entS[r]; entS[r] = entS[e]; entS[e] = ts; }
+              if (p.knorm) { const float tn = entN[r]; entN[r] = entN[e]; entN[e] = tn; }
             }
             __syncwarp();
           }
@@ -524,8 +533,10 @@ __global__ void __launch_bounds__(kAttnThreads, 1)
       const int n_tiles = (n_ent + C::kEPT - 1) / C::kEPT;
       const uint16_t* entJ = sEntJ + buf * kMaxBlocks;
       const uint8_t* entF = sEntF + buf * kMaxBlocks;
+      const float* entN = sEntN + buf * kMaxBlocks;
       const int bh = it / p.per_bh;
       const int batch = bh / p.H, head = bh % p.H;
+      float q_bound = INFINITY;  // |q_row| * softmax scale * log2(e) (+0.1 %), once known
       float m_ref = -INFINITY;  // the row's reference maximum (log2 domain) as this thread last saw it
       float l_run = 0.0f;       // this thread's partial row sum, relative to m_ref
 
@@ -555,14 +566,48 @@ __global__ void __launch_bounds__(kAttnThreads, 1)
 #pragma unroll
         for (int c = 0; c < 4; ++c) tmem_ld32(tS + c * 32, reinterpret_cast<uint32_t*>(sv) + c * 32);
         tmem_ld_wait();
+        if (p.knorm != nullptr && n < 2 && n_tiles >= n + 3) {
+          // My first tile of the item: the norm of my query row, read from the Q tile in shared memory (any
+          // order of its 16-byte units will do, so the swizzle does not matter).  Q is still there: its last
+          // Q K^T cannot have been issued before this warp releases the S buffer below.
+          float ss = 0.0f;
+#pragma unroll
+          for (int c = 0; c < D / 64; ++c) {
+#pragma unroll
+            for (int k = 0; k < 8; ++k) {
+              const uint4 v = *reinterpret_cast<const uint4*>(sQ + c * 16384 + row * 128 + (((k + lane) & 7) << 4));
+              const uint32_t w[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+              for (int e = 0; e < 4; ++e) {
+                const float lo = __uint_as_float(w[e] << 16), hi = __uint_as_float(w[e] & 0xffff0000u);
+                ss = fmaf(lo, lo, ss);
+                ss = fmaf(hi, hi, ss);
+              }
+            }
+          }
+          q_bound = sqrtf(ss) * p.scale_log2 * 1.001f;
+        }
         // S is in registers: the Q K^T of tile g+2 may overwrite the buffer
         tc_fence_before();
         __syncwarp();
         if (lane == 0) mbar_arrive(s_free + wg);
 
+        // Cauchy-Schwarz: no score of this tile exceeds |q| * max |k| * scale.  If that bound stays within
+        // 2^kSkipMargin of the row's reference maximum (which only grows, so the value this thread saw last
+        // will do) for all 32 rows of the warp, the reference need not move and the row-maximum pass is
+        // skipped: the exponentials stay below 2^kSkipMargin, harmless in fp32 / bf16, and the result does
+        // not depend on the reference.
+        bool skip = false;
+        if (!kRagged && p.knorm != nullptr) {
+          float kn = entN[n * C::kEPT];
+          if (C::kStacked) kn = fmaxf(kn, entN[min(n * 2 + 1, n_ent - 1)]);
+          skip = __all_sync(0xffffffffu, q_bound * kn <= m_ref + kSkipMargin);
+        }
+
         // one flat instruction stream per 64-key half; a ragged half (the sequence ends inside it) first has
         // its invalid columns set to -inf, an absent half (not kept by this row's query block) is skipped
         float mx = -INFINITY;
+        if (!skip)
 #pragma unroll
         for (int h = 0; h < 2; ++h) {
           float* svh = sv + h * 64;
@@ -595,7 +640,7 @@ __global__ void __launch_bounds__(kAttnThreads, 1)
         }
         const float m_new = fmaxf(m_ref, mx);
         const bool grow = m_new > m_ref + kGrowThreshold || (m_ref == -INFINITY && m_new > -INFINITY);
-        if (__any_sync(0xffffffffu, grow)) {
+        if (!skip && __any_sync(0xffffffffu, grow)) {
           const float alpha = grow ? ex2(m_ref - m_new) : 1.0f;  // m_ref = -inf -> 0
           if (n > 0) {
             // every P V of the item issued so far must have landed in O before the row is rescaled; they
@@ -751,12 +796,10 @@ __global__ void __launch_bounds__(kAttnThreads, 1)
 constexpr int kPairThreads = 256;
 constexpr int kPairSample = 4;
 
-__global__ void __launch_bounds__(kPairThreads) pair_kernel(const uint32_t* __restrict__ mask, int NB, int Wd,
-                                                            int search, int32_t* __restrict__ pairs) {
-  extern __shared__ __align__(16) unsigned char smem_raw[];
+__device__ __forceinline__ void pair_body(const uint32_t* __restrict__ mask, int NB, int Wd, int search,
+                                          int32_t* __restrict__ pairs, int bh, unsigned char* smem_raw) {
   uint32_t* m = reinterpret_cast<uint32_t*>(smem_raw);  // [NB][Wd]
   __shared__ unsigned int s_best;                        // (score << 10) | (1023 - D): max = best score, smallest D
-  const int bh = blockIdx.x;
   if (threadIdx.x == 0) s_best = (0u << 10) | (1023u - 1u);  // default D = 1
   if (search) {
     const uint32_t* src = mask + (int64_t)bh * NB * Wd;
@@ -919,15 +962,84 @@ static int launch_attn_common(const sparsp_shape& s, const Geometry& g, const vo
   return launch_attn_t<128, 128>(s, g, Q, K, V, packed, packed_capacity, p, st);
 }
 
+// Largest L2 norm of the keys of every KV block (times 1.001), fp32 [B*H][NB]: with the norm of a query row it
+// bounds the scores of a tile.  One warp per (batch, head, block); d/8 lanes read one token (16 bytes each).
+template <int D>
+__device__ __forceinline__ void knorm_body(const __nv_bfloat16* __restrict__ K, int64_t sB, int64_t sH, int64_t sT,
+                                           int H, int NB, int b, int64_t N, int64_t n_units, float* __restrict__ out,
+                                           int64_t unit) {
+  constexpr int LPT = D / 8;       // lanes per token
+  constexpr int TPW = 32 / LPT;    // tokens per warp pass
+  if (unit >= n_units) return;
+  const int lane = threadIdx.x & 31;
+  const int j = (int)(unit % NB);
+  const int64_t bh = unit / NB;
+  const int64_t batch = bh / H, head = bh % H;
+  const __nv_bfloat16* base = K + batch * sB + head * sH;
+  float best = 0.0f;
+#pragma unroll 8
+  for (int t0 = 0; t0 < b; t0 += TPW) {
+    const int64_t tok = (int64_t)j * b + t0 + lane / LPT;
+    float ss = 0.0f;
+    if (tok < N && t0 + lane / LPT < b) {
+      const uint4 v = *reinterpret_cast<const uint4*>(base + tok * sT + (lane % LPT) * 8);
+      const uint32_t w[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+      for (int e = 0; e < 4; ++e) {
+        const float lo = __uint_as_float(w[e] << 16), hi = __uint_as_float(w[e] & 0xffff0000u);
+        ss = fmaf(lo, lo, ss);
+        ss = fmaf(hi, hi, ss);
+      }
+    }
+#pragma unroll
+    for (int sft = 1; sft < LPT; sft <<= 1) ss += __shfl_xor_sync(0xffffffffu, ss, sft);
+    best = fmaxf(best, ss);
+  }
+#pragma unroll
+  for (int sft = LPT; sft < 32; sft <<= 1) best = fmaxf(best, __shfl_xor_sync(0xffffffffu, best, sft));
+  if (lane == 0) out[unit] = sqrtf(best) * 1.001f;
+}
+
+// One launch for the two passes that precede the attention kernel and do not depend on each other: blocks
+// [0, n_pair) choose the query-block pairs of one (batch, head) each (block 64 only), the rest take the largest
+// key norm of every KV block (times 1.001), fp32 [B*H][NB], one warp per block and d/8 lanes per token: with the
+// norm of a query row it bounds the scores of a tile.
+template <int D>
+__global__ void __launch_bounds__(kPairThreads) attn_prep_kernel(const uint32_t* __restrict__ mask, int NB, int Wd,
+                                                                 int32_t* __restrict__ pairs, int n_pair,
+                                                                 const __nv_bfloat16* __restrict__ K, int64_t sB,
+                                                                 int64_t sH, int64_t sT, int H, int b, int64_t N,
+                                                                 int64_t n_units, float* __restrict__ knorm) {
+  extern __shared__ __align__(16) unsigned char smem_raw[];
+  if ((int)blockIdx.x < n_pair) {
+    pair_body(mask, NB, Wd, 1, pairs, (int)blockIdx.x, smem_raw);
+  } else {
+    const int64_t unit = ((int64_t)(blockIdx.x - n_pair) * kPairThreads + threadIdx.x) >> 5;
+    knorm_body<D>(K, sB, sH, sT, H, NB, b, N, n_units, knorm, unit);
+  }
+}
+
 int launch_attn(const sparsp_shape& s, const Geometry& g, const void* Q, const void* K, const void* V,
                 const uint32_t* mask, float scale, void* O, float* lse, char* ws, const WsLayout& L,
                 cudaStream_t st) {
-  int32_t* pairs = nullptr;  // block 128: CTA x handles query block x
-  if (g.b == 64) {
-    pairs = (int32_t*)(ws + L.pairs);
-    const size_t smem = (size_t)g.NB * g.Wd * 4;
-    SPARSP_CUDA_OK(ensure_dynamic_smem((const void*)pair_kernel, (int)smem));
-    pair_kernel<<<g.B * g.H, kPairThreads, smem, st>>>(mask, g.NB, g.Wd, 1, pairs);
+  int32_t* pairs = nullptr;  // block 128: item x handles query block x
+  float* knorm = (float*)(ws + L.knorm);
+  {
+    const int n_pair = g.b == 64 ? g.B * g.H : 0;
+    if (n_pair) pairs = (int32_t*)(ws + L.pairs);
+    const size_t smem = n_pair ? (size_t)g.NB * g.Wd * 4 : 0;
+    const int64_t n_units = (int64_t)g.B * g.H * g.NB;
+    const unsigned blocks = (unsigned)(n_pair + (n_units * 32 + kPairThreads - 1) / kPairThreads);
+    const int64_t sB = s.stride_batch > 0 ? s.stride_batch : 0;
+    if (g.d == 64) {
+      SPARSP_CUDA_OK(ensure_dynamic_smem((const void*)attn_prep_kernel<64>, (int)smem));
+      attn_prep_kernel<64><<<blocks, kPairThreads, smem, st>>>(mask, g.NB, g.Wd, pairs, n_pair, (const __nv_bfloat16*)K, sB,
+                                                             s.stride_head, s.stride_token, g.H, g.b, g.N, n_units, knorm);
+    } else {
+      SPARSP_CUDA_OK(ensure_dynamic_smem((const void*)attn_prep_kernel<128>, (int)smem));
+      attn_prep_kernel<128><<<blocks, kPairThreads, smem, st>>>(mask, g.NB, g.Wd, pairs, n_pair, (const __nv_bfloat16*)K, sB,
+                                                              s.stride_head, s.stride_token, g.H, g.b, g.N, n_units, knorm);
+    }
     count_launch();
   }
   AttnParams p;
@@ -935,6 +1047,7 @@ int launch_attn(const sparsp_shape& s, const Geometry& g, const void* Q, const v
   p.pairs = pairs;
   p.slot = nullptr;
   p.tile_base = nullptr;
+  p.knorm = knorm;
   return launch_attn_common(s, g, Q, K, V, nullptr, 0, p, scale, O, lse, ws, L, st);
 }
 
@@ -1035,6 +1148,7 @@ int launch_attn_packed(const sparsp_shape& s, const Geometry& g, const void* Q, 
   p.pairs = pairs;
   p.slot = slot;
   p.tile_base = tile_base;
+  p.knorm = nullptr;  // remote keys live in the packed buffer: every tile takes its row maximum
   return launch_attn_common(s, g, Q, K, V, packed, capacity, p, scale, O, lse, ws, L, st);
 }
 

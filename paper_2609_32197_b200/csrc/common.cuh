@@ -34,7 +34,7 @@ struct PackEntry {
 };
 
 struct WsLayout {
-  int64_t status, pooled_q, pooled_k, scores, pairs, slot, tile_base, own, ent_base, n_entries, entries, total;
+  int64_t status, pooled_q, pooled_k, scores, pairs, slot, tile_base, knorm, own, ent_base, n_entries, entries, total;
 };
 
 void set_error(const char* fmt, ...);
