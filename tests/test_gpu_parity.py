@@ -275,3 +275,51 @@ def test_degenerate_shapes(oracle_mod, binding):
     wl = _workload("odd64", 2, 128, (3, 10, 21), 0, 64, 2, 2, seed=43)  # 630 tokens -> 10 blocks ... use 9
     wl = _workload("odd64", 2, 128, (3, 9, 21), 0, 64, 2, 2, seed=43)  # 567 tokens -> 9 blocks
     _run_all(oracle_mod, binding, wl, oracle_mod.placement_contiguous(9, 2))
+
+
+@pytest.mark.parametrize("d,b", [(128, 128), (64, 64), (128, 64)])
+@pytest.mark.parametrize("jump", [30.0, 100.0])
+def test_scores_far_above_the_first_tile(oracle_mod, binding, d, b, jump):
+    """The kernel skips a tile's row-maximum pass when a norm bound shows the scores stay within 2^64 of the
+    row's reference.  Here the first kept block scores 0 and a later one `jump` (log2 units) higher: 30 stays
+    inside the bound (exponentials up to 2^30 against the old reference), 100 does not (reference must move).
+    Both must give the oracle's result: the mean of V over the high-scoring block, to 2^-jump."""
+    H = 2
+    NB = 6
+    N = NB * b - 5                                   # ragged last block
+    rng = np.random.default_rng(17)
+    scale_log2 = 1.4426950408889634 / np.sqrt(d)
+    a = 4.0
+    bb = jump / (a * scale_log2)                     # a * bb * scale * log2(e) = jump; both exact enough in bf16
+    Q = torch.zeros(H, N, d, dtype=torch.bfloat16)
+    K = torch.zeros(H, N, d, dtype=torch.bfloat16)
+    Q[:, :, 0] = a
+    Q[:, :, 1:] = torch.tensor(rng.standard_normal((H, N, d - 1)) * 0.05).to(torch.bfloat16)
+    K[:, :, 1:] = torch.tensor(rng.standard_normal((H, N, d - 1)) * 0.05).to(torch.bfloat16)
+    K[:, 3 * b:4 * b, 0] = bb                        # block 3 scores `jump` above the others
+    V = torch.tensor(rng.standard_normal((H, N, d))).to(torch.bfloat16)
+    M = np.zeros((H, NB, NB), bool)
+    M[:, :, 0] = True
+    M[:, :, 1] = True
+    M[:, :, 3] = True
+    M[:, ::2, 5] = True                              # every other query block also keeps the ragged block
+    words = np.zeros((H, NB, 1), np.uint32)
+    for h in range(H):
+        for i in range(NB):
+            for j in range(NB):
+                if M[h, i, j]:
+                    words[h, i, 0] |= np.uint32(1 << j)
+    shape = binding.make_shape(H, d, (1, 1, N), 0, b)
+    ws = binding.make_workspace(shape, 2)
+    Qd, Kd, Vd = Q.cuda(), K.cuda(), V.cuda()
+    mask_d = torch.as_tensor(words.view(np.int32)).cuda()
+    O = torch.zeros_like(Qd)
+    lse = torch.zeros(1, H, N, dtype=torch.float32, device="cuda")
+    binding.sparsp_sparse_attn_fwd(shape, Qd, Kd, Vd, mask_d, 0.0, O, lse, ws)
+    torch.cuda.synchronize()
+    assert binding.sparsp_status(ws) == binding.SPARSP_OK
+    units = [(h, i) for h in range(H) for i in range(NB)]
+    pu.check_attn_units(oracle_mod, Q, K, V, words, b, O, units, lse_gpu=lse[0])
+    # closed form: the high block dominates by 2^jump, so every row is the mean of V over block 3
+    want = V[:, 3 * b:4 * b].float().mean(1)
+    assert (O.float().cpu() - want[:, None, :]).abs().max() < 2e-2
