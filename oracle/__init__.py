@@ -165,6 +165,37 @@ def topk_mask(sc: np.ndarray, is_text: np.ndarray, k: int):
     return mask, kv_list, kv_count
 
 
+def exp2c(x: np.ndarray) -> np.ndarray:
+    """The fixed-arithmetic 2^x of the CDF-threshold mode (fp32)."""
+    x = np.ascontiguousarray(x, dtype=np.float32)
+    y = np.empty_like(x)
+    lib().oracle_exp2c_array(_p(x), _i64(x.size), _p(y))
+    return y
+
+
+def cdf_mask(sc: np.ndarray, is_text: np.ndarray, tau: float, scale: float):
+    """CDF-threshold selection -> (mask [H][NB][Wd] uint32, kv_count [H][NB])."""
+    sc = np.ascontiguousarray(sc, dtype=np.float32)
+    is_text = np.ascontiguousarray(is_text, dtype=np.uint8)
+    H, NB, _ = sc.shape
+    mask = np.empty((H, NB, n_words(NB)), dtype=np.uint32)
+    kv_count = np.empty((H, NB), dtype=np.int32)
+    lib().oracle_cdf_mask(_p(sc), _p(is_text), _i64(H), _i64(NB), ctypes.c_float(tau), ctypes.c_float(scale),
+                          _p(mask), _p(kv_count))
+    return mask, kv_count
+
+
+def block_mask_cdf(Q, K, b: int, tau: float, n_text: int = 0, scale: float = 0.0):
+    """Whole step 1 in CDF-threshold mode (scale 0 means 1/sqrt(d))."""
+    H, N, d = Q.shape
+    pq, pk = pool(Q, b), pool(K, b)
+    sc = scores(pq, pk)
+    is_text = text_block_flags(N - n_text, n_text, b)
+    sc_scale = np.float32(scale) if scale > 0 else np.float32(1.0) / np.sqrt(np.float32(d))
+    mask, kv_count = cdf_mask(sc, is_text, tau, float(sc_scale))
+    return dict(mask=mask, kv_count=kv_count, pq=pq, pk=pk, scores=sc, is_text=is_text, scale=float(sc_scale))
+
+
 def block_mask(Q, K, b: int, k: int, n_text: int = 0):
     """Whole step 1: pool -> scores -> top-k.  Returns dict with mask, kv_list, kv_count, pq, pk."""
     H, N, d = Q.shape

@@ -159,6 +159,112 @@ void oracle_topk_mask(const float* scores, const uint8_t* is_text, int64_t H, in
 }
 
 /* ------------------------------------------------------------------------------------------------
+ * Step 1c, CDF-threshold mode (Section 8.1: keep the key blocks with the highest scores until their
+ * cumulative attention mass reaches the threshold tau).  Per (h, i), over the candidate KV blocks
+ * (is_text[j] == 0):   p_j = exp(scale * (S_j - max S)),  Z = sum p_j,  keep the smallest set
+ * { j : S_j >= v } (v one of the row's scores) whose mass reaches tau * Z; blocks with equal scores
+ * are kept or dropped together; every text block is kept.  The arithmetic is fixed so that the kept
+ * set is a well-defined integer result (all fp32):
+ *   x_j  = (S_j - max S) * (scale * log2 e)        one subtraction, one multiplication
+ *   p_j  = exp2c(x_j)                              below
+ *   sums = 32 partial sums (partial l adds the terms with j = l mod 32, j ascending, from 0),
+ *          combined by a butterfly: for s = 16, 8, 4, 2, 1: partial[l] += partial[l xor s]
+ *   theta = tau * Z;  mass(v) = the same sum over { j : S_j >= v }
+ * exp2c(x): x clamped below at -125; i = nearest integer (ties to even); f = x - i; degree-5 Horner
+ * polynomial in f with fused multiply-adds; i added into the exponent field.
+ * ---------------------------------------------------------------------------------------------- */
+static float oracle_exp2c(float x) {
+  if (x < -125.0f) x = -125.0f;
+  const float fi = rintf(x);
+  const float f = x - fi;
+  float p = 0.0013400432653725147f;
+  p = fmaf(p, f, 0.009676037356257439f);
+  p = fmaf(p, f, 0.05550327152013779f);
+  p = fmaf(p, f, 0.2402210682630539f);
+  p = fmaf(p, f, 0.6931471824645996f);
+  p = fmaf(p, f, 1.0000001192092896f);
+  int32_t bits;
+  memcpy(&bits, &p, 4);
+  bits += (int32_t)fi * (1 << 23);
+  memcpy(&p, &bits, 4);
+  return p;
+}
+
+void oracle_exp2c_array(const float* x, int64_t n, float* y) {
+  for (int64_t t = 0; t < n; ++t) y[t] = oracle_exp2c(x[t]);
+}
+
+/* sum of e[j] over the candidates j with take[j] != 0, in the fixed order described above */
+static float tree_sum32(const float* e, const uint8_t* take, int64_t n) {
+  float part[32];
+  for (int l = 0; l < 32; ++l) {
+    float acc = 0.0f;
+    for (int64_t j = l; j < n; j += 32)
+      if (take[j]) acc = acc + e[j];
+    part[l] = acc;
+  }
+  for (int s = 16; s >= 1; s >>= 1) {
+    float nxt[32];
+    for (int l = 0; l < 32; ++l) nxt[l] = part[l] + part[l ^ s];
+    memcpy(part, nxt, sizeof part);
+  }
+  return part[0];
+}
+
+void oracle_cdf_mask(const float* scores, const uint8_t* is_text, int64_t H, int64_t NB, float tau,
+                     float scale, uint32_t* mask, int32_t* kv_count) {
+  const int64_t Wd = ceil_div64(NB, 32);
+  const float c = scale * 1.4426950408889634f;
+#pragma omp parallel for collapse(2) schedule(static)
+  for (int64_t h = 0; h < H; ++h) {
+    for (int64_t i = 0; i < NB; ++i) {
+      const float* srow = scores + (h * NB + i) * NB;
+      float* e = (float*)malloc((size_t)NB * sizeof(float));
+      uint8_t* take = (uint8_t*)malloc((size_t)NB);
+      cand_t* cand = (cand_t*)malloc((size_t)NB * sizeof(cand_t));
+      int64_t nc = 0;
+      float mx = -INFINITY;
+      for (int64_t j = 0; j < NB; ++j)
+        if (!is_text[j] && srow[j] > mx) mx = srow[j];
+      for (int64_t j = 0; j < NB; ++j) {
+        e[j] = 0.0f;
+        take[j] = 0;
+        if (!is_text[j]) {
+          e[j] = oracle_exp2c((srow[j] - mx) * c);
+          take[j] = 1;
+          cand[nc].s = srow[j];
+          cand[nc].j = (int32_t)j;
+          ++nc;
+        }
+      }
+      const float theta = tau * tree_sum32(e, take, NB);
+      qsort(cand, (size_t)nc, sizeof(cand_t), cand_cmp);
+      /* grow the set one group of equal scores at a time, highest first */
+      for (int64_t j = 0; j < NB; ++j) take[j] = 0;
+      int64_t t = 0;
+      while (t < nc) {
+        const float v = cand[t].s;
+        while (t < nc && cand[t].s == v) take[cand[t++].j] = 1;
+        if (tree_sum32(e, take, NB) >= theta) break;
+      }
+      uint32_t* row = mask + (h * NB + i) * Wd;
+      for (int64_t w = 0; w < Wd; ++w) row[w] = 0u;
+      int64_t cnt = 0;
+      for (int64_t j = 0; j < NB; ++j) {
+        if (take[j] || is_text[j]) {
+          row[j >> 5] |= 1u << (j & 31);
+          ++cnt;
+        }
+      }
+      if (kv_count) kv_count[h * NB + i] = (int32_t)cnt;
+      free(e);
+      free(take);
+      free(cand);
+    }
+  }
+}
+
+/* ------------------------------------------------------------------------------------------------
  * Step 2a/2b.  With Q_r = { i : rank_of_block[i] = r } and P(j) = rank_of_block[j]:
  *   U[r][h]       = OR over i in Q_r of M[h][i]                       (bit words)
  *   D[r][h][p]    = U[r][h] AND own[p]          own[p] = { j : P(j) = p }
