@@ -172,7 +172,10 @@ def run_ours(args):
     entry = 2 * b * d * 2
 
     def step_mask():
-        binding.sparsp_block_mask(shape, Q, K, k, mo["mask"], mo["kv_list"], mo["kv_count"], None, None, ws)
+        if args.tau > 0:  # CDF-threshold selection instead of top-k (rows keep different numbers of blocks)
+            binding.sparsp_block_mask_cdf(shape, Q, K, args.tau, 0.0, mo["mask"], mo["kv_count"], None, None, ws)
+        else:
+            binding.sparsp_block_mask(shape, Q, K, k, mo["mask"], mo["kv_list"], mo["kv_count"], None, None, ws)
 
     def step_plan():
         binding.sparsp_demand_pack(shape, mo["mask"], rank_d, P, binding.SPARSP_PLAN_ONLY, None, None,
@@ -310,7 +313,8 @@ def run_ours(args):
         "data": "synthetic",
         "config": {
             "workload": wl.name, "heads": H, "head_dim": d, "grid": list(wl.grid), "n_text": wl.n_text,
-            "tokens": N, "block": b, "n_blocks": NB, "topk_blocks": k, "kept_pairs": kept_pairs,
+            "tokens": N, "block": b, "n_blocks": NB, "topk_blocks": (k if args.tau <= 0 else None),
+            "selection": ("top-k" if args.tau <= 0 else "cdf tau=%g" % args.tau), "kept_pairs": kept_pairs,
             "virtual_ranks": P, "placement": placement, "layout": "[H][N][d]",
             "l2_policy": "inputs larger than L2 (Q+K+V = %.0f MB)" % (3 * Q.numel() * 2 / 1e6),
         },
@@ -326,7 +330,7 @@ def run_ours(args):
         "roofline": {"bound": "tensor", "kernel": "attn_fwd_kernel (+ attn_prep_kernel, timed together)", "achieved": attn_tflops,
                      "peak": peaks["bf16_tflops"], "peak_source": peaks["source"] + " burst", "unit": "TFLOP/s",
                      "frac": attn_tflops / peaks["bf16_tflops"],
-                     "traffic": ATTN_DRAM_TRAFFIC.get((wl.name, k))},
+                     "traffic": ATTN_DRAM_TRAFFIC.get((wl.name, k)) if args.tau <= 0 else None},
         "roofline_pack": {"bound": "hbm", "kernel": "pack_bulk_kernel", "achieved": pack_gbs, "peak": peaks["hbm_gbs"],
                           "peak_source": peaks["source"], "unit": "GB/s", "frac": pack_gbs / peaks["hbm_gbs"],
                           "algorithmic_bytes": pack_bytes},
@@ -456,6 +460,7 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="mid", choices=["tiny", "mid", "cog", "wan", "hunyuan"])
     ap.add_argument("--pct", type=int, default=0, help="top-k as a percentage of the video blocks")
+    ap.add_argument("--tau", type=float, default=0.0, help="CDF-threshold selection with this mass instead of top-k (ours only)")
     ap.add_argument("--placement", default=None, choices=[None, "contiguous", "periodic", "shuffle"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true", help="skip the host-buffer end-to-end leg")

@@ -104,6 +104,29 @@ SPARSP_API int sparsp_block_mask(const sparsp_shape* shape, const void* Q, const
                       uint32_t* mask, int32_t* kv_list, int32_t* kv_count, float* pooled_q,
                       float* pooled_k, void* workspace, void* stream);
 
+/* Step 1, CDF-threshold selection (Section 8.1: for each query, keep the key blocks with the highest
+ * scores until their cumulative attention mass reaches the threshold).  Same pooling and scores as
+ * sparsp_block_mask; per row, over the text-free blocks:
+ *   p_j = exp(score_scale * (S_j - max S)),  Z = sum_j p_j,
+ *   keep the smallest set { j : S_j >= v } (v one of the row's scores) whose mass reaches tau * Z --
+ *   blocks with equal scores (-0 == +0) are kept or dropped together -- then every text block.
+ * The arithmetic is fixed (all fp32): x_j = (S_j - max S) * (score_scale * log2 e), one subtraction and
+ * one multiplication; p_j = 2^x_j by clamping x at -125, splitting off the nearest integer (ties to
+ * even) and a degree-5 Horner polynomial of the remainder with fused multiply-adds (coefficients
+ * 0.0013400432653725147, 0.009676037356257439, 0.05550327152013779, 0.2402210682630539,
+ * 0.6931471824645996, 1.0000001192092896), the integer part added into the exponent field; every sum
+ * is 32 partial sums (partial l adds the terms with j = l mod 32 in ascending order, from 0) combined
+ * by a butterfly (s = 16, 8, 4, 2, 1: partial[l] += partial[l xor s]); theta = tau * Z.
+ *   tau          in   (0, 1]
+ *   score_scale  in   0 means 1/sqrt(d)
+ *   mask         out  uint32 [B][H][NB][Wd]   (rows keep different numbers of blocks)
+ *   kv_count     out  int32 [B][H][NB]; may be NULL
+ *   pooled_q/k   out  fp32 [B][H][NB][d]; may be NULL
+ */
+SPARSP_API int sparsp_block_mask_cdf(const sparsp_shape* shape, const void* Q, const void* K, float tau,
+                          float score_scale, uint32_t* mask, int32_t* kv_count, float* pooled_q,
+                          float* pooled_k, void* workspace, void* stream);
+
 /* Step 2 -- demand and packing for n_ranks virtual ranks (Section 4.2, Eq. "receiver-demand" and
  * Eq. "sparse-exchange-volume"; Section 5.2: head-preserving demand, row-major packing with
  * locally derived offsets; Section 6: one slot per (producer, consumer) pair).

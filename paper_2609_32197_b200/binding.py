@@ -29,7 +29,7 @@ EXPORTS = [
     "sparsp_geometry", "sparsp_resolve_topk", "sparsp_placement_contiguous", "sparsp_placement_periodic",
     "sparsp_workspace_bytes", "sparsp_block_mask", "sparsp_demand_pack", "sparsp_sparse_attn_fwd",
     "sparsp_status", "sparsp_last_error", "sparsp_launch_count", "sparsp_demand_plan_noalloc",
-    "sparsp_hop_mask", "sparsp_attn_merge", "sparsp_sparse_attn_fwd_packed",
+    "sparsp_hop_mask", "sparsp_attn_merge", "sparsp_sparse_attn_fwd_packed", "sparsp_block_mask_cdf",
 ]
 
 
@@ -153,6 +153,12 @@ def sparsp_block_mask(shape, Q, K, topk_video, mask, kv_list, kv_count, pooled_q
     _check(lib().sparsp_block_mask(ctypes.byref(shape), _ptr(Q), _ptr(K), ctypes.c_int32(topk_video),
                                    _ptr(mask), _ptr(kv_list), _ptr(kv_count), _ptr(pooled_q),
                                    _ptr(pooled_k), _ptr(workspace), _stream()))
+
+
+def sparsp_block_mask_cdf(shape, Q, K, tau, score_scale, mask, kv_count, pooled_q, pooled_k, workspace):
+    _check(lib().sparsp_block_mask_cdf(ctypes.byref(shape), _ptr(Q), _ptr(K), ctypes.c_float(tau),
+                                       ctypes.c_float(score_scale), _ptr(mask), _ptr(kv_count), _ptr(pooled_q),
+                                       _ptr(pooled_k), _ptr(workspace), _stream()))
 
 
 def sparsp_demand_pack(shape, mask, rank_of_block, n_ranks, flags, K, V, union_mask, cnt, seg_offset,

@@ -1,4 +1,5 @@
 // extern "C" entry points of the SparSP library: argument checking, workspace carving, launch order.
+#include <cmath>
 #include <cstring>
 #include <map>
 #include <mutex>
@@ -226,6 +227,42 @@ int sparsp_block_mask(const sparsp_shape* shape, const void* Q, const void* K, i
   cudaStream_t st = (cudaStream_t)stream;
   SPARSP_TRY(launch_pool(*shape, g, Q, K, pq, pk, st));
   SPARSP_TRY(launch_score_topk(g, pq, pk, (float*)(ws + L.scores), topk_video, mask, kv_list, kv_count, st));
+  return SPARSP_OK;
+}
+
+int sparsp_block_mask_cdf(const sparsp_shape* shape, const void* Q, const void* K, float tau, float score_scale,
+                          uint32_t* mask, int32_t* kv_count, float* pooled_q, float* pooled_k, void* workspace,
+                          void* stream) {
+  Geometry g;
+  SPARSP_TRY(make_geometry(shape, &g));
+  SPARSP_TRY(check_supported(g));
+  SPARSP_TRY(check_strides(shape, g));
+  SPARSP_TRY(check_ptr(Q, "Q"));
+  SPARSP_TRY(check_ptr(K, "K"));
+  SPARSP_TRY(check_ptr(mask, "mask", 4));
+  SPARSP_TRY(check_ptr(workspace, "workspace", 256));
+  if (!(tau > 0.0f && tau <= 1.0f)) {
+    set_error("tau %g outside (0, 1]", (double)tau);
+    return SPARSP_ERR_INVALID_ARG;
+  }
+  if (!(score_scale >= 0.0f) || score_scale > 1e6f) {
+    set_error("score_scale %g must be 0 (meaning 1/sqrt(d)) or a positive finite number", (double)score_scale);
+    return SPARSP_ERR_INVALID_ARG;
+  }
+  if (g.nb_cand < 1) {
+    set_error("the sequence has no video block to choose from");
+    return SPARSP_ERR_INVALID_ARG;
+  }
+  if (pooled_q && (uintptr_t)pooled_q % 16) return check_ptr((void*)1, "pooled_q");
+  if (pooled_k && (uintptr_t)pooled_k % 16) return check_ptr((void*)1, "pooled_k");
+  char* ws = (char*)workspace;
+  const WsLayout L = make_layout(g, 1);
+  float* pq = pooled_q ? pooled_q : (float*)(ws + L.pooled_q);
+  float* pk = pooled_k ? pooled_k : (float*)(ws + L.pooled_k);
+  cudaStream_t st = (cudaStream_t)stream;
+  const float scale = score_scale > 0.0f ? score_scale : 1.0f / sqrtf((float)g.d);
+  SPARSP_TRY(launch_pool(*shape, g, Q, K, pq, pk, st));
+  SPARSP_TRY(launch_score_cdf(g, pq, pk, (float*)(ws + L.scores), tau, scale, mask, kv_count, st));
   return SPARSP_OK;
 }
 

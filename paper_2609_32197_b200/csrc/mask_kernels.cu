@@ -238,6 +238,113 @@ __global__ void __launch_bounds__(kTopkWarps * 32) topk_kernel(const float* __re
   if (kv_count && lane == 0) kv_count[row] = out_pos;
 }
 
+// ------------------------------------------------------------------------------------------------
+// CDF-threshold selection (Section 8.1): per row, softmax over the candidate scores, keep the smallest
+// top set by score (whole groups of equal scores) whose mass reaches tau.  Fixed fp32 arithmetic so that
+// the kept set is a well-defined integer result:
+//   x_j = (S_j - max S) * (scale * log2 e);  p_j = exp2c(x_j)  (clamp at -125, nearest-integer split,
+//   degree-5 Horner polynomial with fused multiply-adds, integer part added into the exponent field);
+//   every sum = 32 partial sums (lane l adds its terms j = l mod 32 in ascending order, from 0) combined
+//   by a butterfly (s = 16, 8, 4, 2, 1: partial[l] += partial[l xor s]);  theta = tau * Z.
+// One warp per row; the threshold is found by a 32-step search over the order-preserving key space,
+// which is valid because the mass of { key >= t } (nonnegative terms, fixed order) never grows with t.
+// ------------------------------------------------------------------------------------------------
+__device__ __forceinline__ float exp2c(float x) {
+  x = fmaxf(x, -125.0f);
+  const float fi = rintf(x);
+  const float f = x - fi;
+  float p = 0.0013400432653725147f;
+  p = fmaf(p, f, 0.009676037356257439f);
+  p = fmaf(p, f, 0.05550327152013779f);
+  p = fmaf(p, f, 0.2402210682630539f);
+  p = fmaf(p, f, 0.6931471824645996f);
+  p = fmaf(p, f, 1.0000001192092896f);
+  return __int_as_float(__float_as_int(p) + (int)fi * (1 << 23));
+}
+
+__device__ __forceinline__ float butterfly_sum(float v) {
+#pragma unroll
+  for (int s = 16; s >= 1; s >>= 1) v = __fadd_rn(v, __shfl_xor_sync(0xffffffffu, v, s));
+  return v;
+}
+
+__global__ void __launch_bounds__(kTopkWarps * 32) cdf_kernel(const float* __restrict__ scores, int64_t n_rows, int NB,
+                                                              int Wd, int nb_cand, float tau, float c,
+                                                              uint32_t* __restrict__ mask,
+                                                              int32_t* __restrict__ kv_count) {
+  extern __shared__ __align__(16) unsigned char smem_raw[];
+  const int NBpad = Wd * 32;
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  uint32_t* keys = reinterpret_cast<uint32_t*>(smem_raw) + (size_t)warp * 2 * NBpad;
+  float* e = reinterpret_cast<float*>(keys + NBpad);
+  const int64_t row = (int64_t)blockIdx.x * kTopkWarps + warp;  // (batch*H + head) * NB + i
+  if (row >= n_rows) return;
+  const float* srow = scores + row * NB;
+  float mx = -INFINITY;
+  for (int t = 0; t < Wd; ++t) {
+    const int j = t * 32 + lane;
+    const float s = j < nb_cand ? __ldcs(srow + j) : -INFINITY;
+    e[j] = s;
+    keys[j] = j < nb_cand ? score_key(s) : 0u;
+    mx = fmaxf(mx, s);
+  }
+#pragma unroll
+  for (int s = 16; s >= 1; s >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, s));
+  float acc = 0.0f;
+  for (int t = 0; t < Wd; ++t) {
+    const int j = t * 32 + lane;
+    float pj = 0.0f;
+    if (j < nb_cand) {
+      pj = exp2c(__fmul_rn(__fsub_rn(e[j], mx), c));
+      acc = __fadd_rn(acc, pj);
+    }
+    e[j] = pj;
+  }
+  const float theta = __fmul_rn(tau, butterfly_sum(acc));
+  // largest T with mass{ key >= T } >= theta
+  uint32_t T = 0;
+  for (int bit = 31; bit >= 0; --bit) {
+    const uint32_t trial = T | (1u << bit);
+    float m = 0.0f;
+    for (int t = 0; t < Wd; ++t) {
+      const int j = t * 32 + lane;
+      if (j < nb_cand && keys[j] >= trial) m = __fadd_rn(m, e[j]);
+    }
+    if (butterfly_sum(m) >= theta) T = trial;
+  }
+  int cnt = 0;
+  for (int t = 0; t < Wd; ++t) {
+    const int j = t * 32 + lane;
+    const bool keep = (j < nb_cand && keys[j] >= T) || (j >= nb_cand && j < NB);
+    const uint32_t word = __ballot_sync(0xffffffffu, keep);
+    if (lane == 0) mask[row * Wd + t] = word;
+    cnt += __popc(word);
+  }
+  if (kv_count && lane == 0) kv_count[row] = cnt;
+}
+
+int launch_score_cdf(const Geometry& g, const float* pq, const float* pk, float* scores, float tau, float scale,
+                     uint32_t* mask, int32_t* kv_count, cudaStream_t st) {
+  {
+    const size_t smem = (size_t)2 * kScoreTile * (g.d + 4) * 4;
+    const int nt = (g.NB + kScoreTile - 1) / kScoreTile;
+    dim3 grid(nt, nt, g.B * g.H);
+    auto kern = g.d == 64 ? score_kernel<64> : score_kernel<128>;
+    SPARSP_CUDA_OK(ensure_dynamic_smem((const void*)kern, (int)smem));
+    kern<<<grid, kScoreThreads, smem, st>>>(pq, pk, g.NB, scores);
+  }
+  {
+    const int64_t n_rows = (int64_t)g.B * g.H * g.NB;
+    const size_t smem = (size_t)kTopkWarps * 2 * g.Wd * 32 * 4;
+    const float c = scale * 1.4426950408889634f;  // fp32 product, as in the definition above
+    cdf_kernel<<<(unsigned)((n_rows + kTopkWarps - 1) / kTopkWarps), kTopkWarps * 32, smem, st>>>(
+        scores, n_rows, g.NB, g.Wd, g.nb_cand, tau, c, mask, kv_count);
+  }
+  count_launch(2);
+  SPARSP_CUDA_OK(cudaGetLastError());
+  return SPARSP_OK;
+}
+
 int launch_score_topk(const Geometry& g, const float* pq, const float* pk, float* scores, int topk,
                       uint32_t* mask, int32_t* kv_list, int32_t* kv_count, cudaStream_t st) {
   const int kept_cap = topk + (g.NB - g.nb_cand);
