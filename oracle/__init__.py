@@ -120,6 +120,56 @@ def placement_periodic(NB: int, P: int, b: int, frame_tokens: int, n_video: int)
     return out
 
 
+def placement_permutation(rank_of_block: np.ndarray, P: int, N: int, b: int):
+    """Section 4.3: the placement as a deterministic permutation from logical block coordinates to
+    (rank, offset) pairs, at the granularity of whole KV blocks.  Slots are ordered by rank, and inside a rank
+    by logical block index.  Returns (block_of_slot [NB], token_offset_of_slot [NB+1], first_slot_of_rank
+    [P+1]): slot s holds logical block block_of_slot[s], whose tokens start at token_offset_of_slot[s] in the
+    permuted sequence (the sequence's last block may be shorter than b)."""
+    NB = len(rank_of_block)
+    block_of_slot, first = [], [0]
+    for r in range(P):
+        block_of_slot += [j for j in range(NB) if rank_of_block[j] == r]
+        first.append(len(block_of_slot))
+    off = [0]
+    for j in block_of_slot:
+        off.append(off[-1] + min(b, N - j * b))
+    return (np.array(block_of_slot, np.int32), np.array(off, np.int64), np.array(first, np.int32))
+
+
+def permute_tokens(X, block_of_slot, token_offset_of_slot, b: int, inverse: bool = False):
+    """X [H][N][d] -> the same tokens in permuted order (or back, with inverse=True)."""
+    H, N, d = X.shape
+    Y = X.clone()
+    for s, j in enumerate(block_of_slot):
+        n_j = min(b, N - int(j) * b)
+        lo_new, lo_old = int(token_offset_of_slot[s]), int(j) * b
+        if inverse:
+            Y[:, lo_old:lo_old + n_j] = X[:, lo_new:lo_new + n_j]
+        else:
+            Y[:, lo_new:lo_new + n_j] = X[:, lo_old:lo_old + n_j]
+    return Y
+
+
+def sharing_histogram(mask: np.ndarray, rank_of_block: np.ndarray, P: int) -> np.ndarray:
+    """Section 3.1: for each remote K block a rank receives (per head), the fraction of that rank's local Q
+    blocks that access it.  hist[r][q], q = 0..100, counts the (head, remote block) pairs of consumer r whose
+    fraction, in whole percent rounded down, is q (a received block is accessed by at least one local Q block,
+    so a fraction below 1 % lands in bin 0)."""
+    H, NB, _ = mask.shape
+    hist = np.zeros((P, 101), np.int64)
+    for r in range(P):
+        local = [i for i in range(NB) if rank_of_block[i] == r]
+        for h in range(H):
+            for j in range(NB):
+                if rank_of_block[j] == r:
+                    continue
+                c = sum((int(mask[h, i, j >> 5]) >> (j & 31)) & 1 for i in local)
+                if c > 0:
+                    hist[r, (100 * c) // len(local)] += 1
+    return hist
+
+
 # ---------------------------------------------------------------------------------------------
 # step 1
 # ---------------------------------------------------------------------------------------------
