@@ -84,6 +84,32 @@ SPARSP_API int sparsp_placement_contiguous(const sparsp_shape* shape, int32_t n_
  * starting in the text tail get j mod G.  rank_of_block: HOST array of NB int32. */
 SPARSP_API int sparsp_placement_periodic(const sparsp_shape* shape, int32_t n_ranks, int32_t* rank_of_block);
 
+/* The placement as a permutation of whole KV blocks (Section 4.3: a deterministic permutation from logical
+ * block coordinates to (rank, offset) pairs, computed once per geometry and rank count, undone by its
+ * inverse).  Slots are ordered by rank and, inside a rank, by logical block index.
+ *   rank_of_block           in   HOST int32 [NB], values 0 .. n_ranks-1
+ *   block_of_slot           out  HOST int32 [NB]: the logical block held by slot s
+ *   token_offset_of_slot    out  HOST int64 [NB+1]: first token of slot s in the permuted sequence (the
+ *                                sequence's last block may be shorter than `block`); entry NB = N
+ *   first_slot_of_rank      out  HOST int32 [n_ranks+1]; may be NULL */
+SPARSP_API int sparsp_placement_permutation(const sparsp_shape* shape, int32_t n_ranks, const int32_t* rank_of_block,
+                                 int32_t* block_of_slot, int64_t* token_offset_of_slot,
+                                 int32_t* first_slot_of_rank);
+
+/* Applies that permutation (inverse = 0: logical order -> permuted order) or undoes it (inverse != 0) on a
+ * bf16 tensor strided as in `shape`; block membership is unchanged, tokens inside a block keep their order.
+ *   X in, Y out: DEVICE, different buffers;  block_of_slot, token_offset_of_slot: DEVICE copies of the above */
+SPARSP_API int sparsp_permute_tokens(const sparsp_shape* shape, const void* X, void* Y, const int32_t* block_of_slot,
+                          const int64_t* token_offset_of_slot, int32_t inverse, void* stream);
+
+/* How widely received K blocks are shared (Section 3.1): for every remote KV block j that consumer r
+ * receives for head h (some query block of r keeps it), the fraction of r's query blocks that keep it.
+ *   hist  out  DEVICE int64 [B][n_ranks][101]: hist[b][r][q] = number of such (h, j) pairs whose fraction,
+ *              in whole percent rounded down, is q
+ *   mask  uint32 [B][H][NB][Wd];  rank_of_block  DEVICE int32 [NB] */
+SPARSP_API int sparsp_sharing_histogram(const sparsp_shape* shape, const uint32_t* mask, const int32_t* rank_of_block,
+                             int32_t n_ranks, int64_t* hist, void* stream);
+
 /* Bytes of device workspace the three calls need for this shape and rank count. */
 SPARSP_API int sparsp_workspace_bytes(const sparsp_shape* shape, int32_t n_ranks, int64_t* bytes);
 

@@ -30,6 +30,7 @@ EXPORTS = [
     "sparsp_workspace_bytes", "sparsp_block_mask", "sparsp_demand_pack", "sparsp_sparse_attn_fwd",
     "sparsp_status", "sparsp_last_error", "sparsp_launch_count", "sparsp_demand_plan_noalloc",
     "sparsp_hop_mask", "sparsp_attn_merge", "sparsp_sparse_attn_fwd_packed", "sparsp_block_mask_cdf",
+    "sparsp_placement_permutation", "sparsp_permute_tokens", "sparsp_sharing_histogram",
 ]
 
 
@@ -134,6 +135,29 @@ def sparsp_placement_contiguous(shape: sparsp_shape, n_ranks: int) -> torch.Tens
 
 def sparsp_placement_periodic(shape: sparsp_shape, n_ranks: int) -> torch.Tensor:
     return _placement(lib().sparsp_placement_periodic, shape, n_ranks)
+
+
+def sparsp_placement_permutation(shape: sparsp_shape, n_ranks: int, rank_of_block: torch.Tensor):
+    """-> (block_of_slot int32 [NB], token_offset_of_slot int64 [NB+1], first_slot_of_rank int32 [P+1]), host."""
+    g = sparsp_geometry(shape)
+    rank = rank_of_block.to(torch.int32).cpu().contiguous()
+    bos = torch.empty(g.n_blocks, dtype=torch.int32)
+    off = torch.empty(g.n_blocks + 1, dtype=torch.int64)
+    first = torch.empty(n_ranks + 1, dtype=torch.int32)
+    _check(lib().sparsp_placement_permutation(ctypes.byref(shape), ctypes.c_int32(n_ranks),
+                                              ctypes.c_void_p(rank.data_ptr()), ctypes.c_void_p(bos.data_ptr()),
+                                              ctypes.c_void_p(off.data_ptr()), ctypes.c_void_p(first.data_ptr())))
+    return bos, off, first
+
+
+def sparsp_permute_tokens(shape, X, Y, block_of_slot, token_offset_of_slot, inverse):
+    _check(lib().sparsp_permute_tokens(ctypes.byref(shape), _ptr(X), _ptr(Y), _ptr(block_of_slot),
+                                       _ptr(token_offset_of_slot), ctypes.c_int32(1 if inverse else 0), _stream()))
+
+
+def sparsp_sharing_histogram(shape, mask, rank_of_block, n_ranks, hist):
+    _check(lib().sparsp_sharing_histogram(ctypes.byref(shape), _ptr(mask), _ptr(rank_of_block),
+                                          ctypes.c_int32(n_ranks), _ptr(hist), _stream()))
 
 
 def sparsp_workspace_bytes(shape: sparsp_shape, n_ranks: int) -> int:

@@ -1,4 +1,5 @@
 // extern "C" entry points of the SparSP library: argument checking, workspace carving, launch order.
+#include <algorithm>
 #include <cmath>
 #include <cstring>
 #include <map>
@@ -190,6 +191,68 @@ int sparsp_placement_periodic(const sparsp_shape* shape, int32_t n_ranks, int32_
     rank_of_block[j] = first >= g.n_video ? j % n_ranks : (int32_t)((n_ranks * (first % F)) / F);
   }
   return SPARSP_OK;
+}
+
+int sparsp_placement_permutation(const sparsp_shape* shape, int32_t n_ranks, const int32_t* rank_of_block,
+                                 int32_t* block_of_slot, int64_t* token_offset_of_slot, int32_t* first_slot_of_rank) {
+  Geometry g;
+  SPARSP_TRY(make_geometry(shape, &g));
+  if (n_ranks < 1 || n_ranks > kMaxRanks || !rank_of_block || !block_of_slot || !token_offset_of_slot) {
+    set_error("bad n_ranks or NULL argument");
+    return SPARSP_ERR_INVALID_ARG;
+  }
+  for (int32_t j = 0; j < g.NB; ++j)
+    if (rank_of_block[j] < 0 || rank_of_block[j] >= n_ranks) {
+      set_error("rank_of_block[%d] = %d outside 0..%d", j, rank_of_block[j], n_ranks - 1);
+      return SPARSP_ERR_INVALID_ARG;
+    }
+  int32_t slot = 0;
+  int64_t tok = 0;
+  for (int32_t r = 0; r < n_ranks; ++r) {
+    if (first_slot_of_rank) first_slot_of_rank[r] = slot;
+    for (int32_t j = 0; j < g.NB; ++j)
+      if (rank_of_block[j] == r) {
+        block_of_slot[slot] = j;
+        token_offset_of_slot[slot] = tok;
+        tok += std::min<int64_t>(g.b, g.N - (int64_t)j * g.b);
+        ++slot;
+      }
+  }
+  token_offset_of_slot[g.NB] = tok;
+  if (first_slot_of_rank) first_slot_of_rank[n_ranks] = slot;
+  return SPARSP_OK;
+}
+
+int sparsp_permute_tokens(const sparsp_shape* shape, const void* X, void* Y, const int32_t* block_of_slot,
+                          const int64_t* token_offset_of_slot, int32_t inverse, void* stream) {
+  Geometry g;
+  SPARSP_TRY(make_geometry(shape, &g));
+  SPARSP_TRY(check_supported(g));
+  SPARSP_TRY(check_strides(shape, g));
+  SPARSP_TRY(check_ptr(X, "X"));
+  SPARSP_TRY(check_ptr(Y, "Y"));
+  SPARSP_TRY(check_ptr(block_of_slot, "block_of_slot", 4));
+  SPARSP_TRY(check_ptr(token_offset_of_slot, "token_offset_of_slot", 8));
+  if (X == Y) {
+    set_error("X and Y must be different buffers");
+    return SPARSP_ERR_INVALID_ARG;
+  }
+  return launch_permute_tokens(*shape, g, X, Y, block_of_slot, token_offset_of_slot, inverse != 0,
+                               (cudaStream_t)stream);
+}
+
+int sparsp_sharing_histogram(const sparsp_shape* shape, const uint32_t* mask, const int32_t* rank_of_block,
+                             int32_t n_ranks, int64_t* hist, void* stream) {
+  Geometry g;
+  SPARSP_TRY(make_geometry(shape, &g));
+  if (n_ranks < 1 || n_ranks > kMaxRanks) {
+    set_error("n_ranks %d outside 1..%d", n_ranks, kMaxRanks);
+    return SPARSP_ERR_INVALID_ARG;
+  }
+  SPARSP_TRY(check_ptr(mask, "mask", 4));
+  SPARSP_TRY(check_ptr(rank_of_block, "rank_of_block", 4));
+  SPARSP_TRY(check_ptr(hist, "hist", 8));
+  return launch_sharing(g, mask, rank_of_block, n_ranks, hist, (cudaStream_t)stream);
 }
 
 int sparsp_workspace_bytes(const sparsp_shape* shape, int32_t n_ranks, int64_t* bytes) {

@@ -61,6 +61,11 @@ inline int64_t align_up(int64_t x, int64_t a) { return (x + a - 1) / a * a; }
 // launchers implemented in the kernel files -------------------------------------------------
 int launch_pool(const sparsp_shape& s, const Geometry& g, const void* Q, const void* K, float* pq,
                 float* pk, cudaStream_t st);
+int launch_permute_tokens(const sparsp_shape& s, const Geometry& g, const void* X, void* Y,
+                          const int32_t* block_of_slot, const int64_t* token_offset_of_slot, int inverse,
+                          cudaStream_t st);
+int launch_sharing(const Geometry& g, const uint32_t* mask, const int32_t* rank, int P, int64_t* hist,
+                   cudaStream_t st);
 int launch_score_cdf(const Geometry& g, const float* pq, const float* pk, float* scores, float tau, float scale,
                      uint32_t* mask, int32_t* kv_count, cudaStream_t st);
 int launch_score_topk(const Geometry& g, const float* pq, const float* pk, float* scores, int topk,

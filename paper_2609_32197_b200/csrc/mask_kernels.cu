@@ -337,6 +337,7 @@ int launch_score_cdf(const Geometry& g, const float* pq, const float* pk, float*
     const int64_t n_rows = (int64_t)g.B * g.H * g.NB;
     const size_t smem = (size_t)kTopkWarps * 2 * g.Wd * 32 * 4;
     const float c = scale * 1.4426950408889634f;  // fp32 product, as in the definition above
+    SPARSP_CUDA_OK(ensure_dynamic_smem((const void*)cdf_kernel, (int)smem));
     cdf_kernel<<<(unsigned)((n_rows + kTopkWarps - 1) / kTopkWarps), kTopkWarps * 32, smem, st>>>(
         scores, n_rows, g.NB, g.Wd, g.nb_cand, tau, c, mask, kv_count);
   }

@@ -83,3 +83,22 @@ def test_cdf_mask_full_size(oracle_mod, binding, name, tau):
     units = [(0, 0), (H - 1, NB - 1)] + [(int(rng.integers(H)), int(rng.integers(NB))) for _ in range(10)]
     pu.check_attn_units(oracle_mod, Q, K, V, ref["mask"], b, O, units)
     assert torch.isfinite(O.float()).all()
+
+
+def test_cdf_mask_at_the_largest_block_count(oracle_mod, binding):
+    """NB = 1000 (the limit is 1024): the kernel's per-row scratch is at its largest."""
+    from paper_2609_32197_b200 import synth
+    H, d, b = 1, 64, 64
+    wl = synth.Workload("cdf_big", H, d, (10, 50, 128), 0, b, 4, None, 2, seed=3)   # 64000 tokens = 1000 blocks
+    Q, K, V = synth.make_qkv(wl, "cpu")
+    NB = wl.n_blocks
+    shape = binding.make_shape(H, d, wl.grid, wl.n_text, b)
+    ws = binding.make_workspace(shape, 2)
+    g = binding.sparsp_geometry(shape)
+    mask = torch.zeros(1, H, NB, g.n_words, dtype=torch.int32, device="cuda")
+    cnt = torch.zeros(1, H, NB, dtype=torch.int32, device="cuda")
+    binding.sparsp_block_mask_cdf(shape, Q.cuda(), K.cuda(), 0.9, 0.0, mask, cnt, None, None, ws)
+    torch.cuda.synchronize()
+    ref = oracle_mod.block_mask_cdf(Q, K, b, 0.9, 0)
+    assert np.array_equal(pu.u32(mask[0]), ref["mask"])
+    assert np.array_equal(cnt[0].cpu().numpy(), ref["kv_count"])
