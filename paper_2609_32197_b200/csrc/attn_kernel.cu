@@ -6,7 +6,7 @@
 //                into the Q tile (full-rate M = 128 MMAs); a KV tile is two entries of the UNION of their
 //                kept lists (128 keys, full-rate N = 128); each 64x64 quadrant the mask does not keep is
 //                zeroed in P.
-// The kernel is persistent: one CTA per SM walks items c, c + grid, c + 2 grid, ...; the next item's kept
+// The kernel is persistent: one CTA per SM takes items from a global counter; the next item's kept
 // list, Q tile, first K/V tiles and first Q K^T overlap the current item's last tiles and its epilogue.
 // The scores S = Q K^T and the probabilities P are double-buffered in tensor memory (S: 2 x 128 fp32
 // columns, P: 2 x 64 columns of packed bf16, O: d columns), so that the tensor pipe always has the next
@@ -57,6 +57,7 @@ struct AttnParams {
   __nv_bfloat16* O;
   float* lse;
   int32_t* status;
+  int32_t* work_counter;  // next work item to hand out; zeroed by the preparatory launch
   int64_t N;
   int64_t sB, sH, sT;
   int H, NB, Wd;
@@ -72,6 +73,7 @@ constexpr int kAttnThreads = 512;  // four warpgroups: two of utility warps, sof
 #define SPARSP_REGS_UTILITY2 32
 #define SPARSP_REGS_SOFTMAX 216
 constexpr int kTmemCols = 512;
+constexpr int kWorkCounterWord = 8;  // word of the workspace header that holds the attention work counter
 constexpr float kGrowThreshold = 8.0f;
 constexpr float kSkipMargin = 64.0f;  // 2^64 * (keys of a sequence) * |V| stays far inside fp32
 // Tuning switch (compile-time): how many of the exponentials go to the FMA pipe instead of the
@@ -191,10 +193,10 @@ __global__ void __launch_bounds__(kAttnThreads, 1)
   volatile int* s_abort = reinterpret_cast<volatile int*>(smem + C::kOffMisc + 4);
   int* s_nent = reinterpret_cast<int*>(smem + C::kOffMisc + 8);   // [2]
   int* s_blk = reinterpret_cast<int*>(smem + C::kOffMisc + 16);   // [2][2] the item's query block(s); < 0 = absent
+  int* s_item = reinterpret_cast<int*>(smem + C::kOffMisc + 32);  // [2] the work item of each list buffer; < 0 = no more
   constexpr int kListReaders = 12;  // two producers, two issuers, eight softmax warps
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-  const int G = (int)gridDim.x;
 
   // ---- setup ------------------------------------------------------------------------------
   if (tid == 0) {
@@ -241,10 +243,12 @@ __global__ void __launch_bounds__(kAttnThreads, 1)
     if (warp == 3) {
       // ================================ TMA producer: V =====================================
       if (lane == 0) {
-        int i = 0, vn = 0;  // items seen; V tiles loaded so far
-        for (int it = blockIdx.x; it < p.n_items; it += G, ++i) {
+        int vn = 0;  // V tiles loaded so far
+        for (int i = 0;; ++i) {
           const int buf = i & 1;
           mbar_wait_bounded_inline(list_ready + buf, (i >> 1) & 1, s_abort, 58, p.wait_limit);
+          const int it = s_item[buf];
+          if (it < 0) break;  // (only the list builder decides when to stop, so that all roles stop at the same item)
           const int n_ent = s_nent[buf];
           const int n_tiles = (n_ent + C::kEPT - 1) / C::kEPT;
           if (n_tiles > 0) {
@@ -281,10 +285,12 @@ __global__ void __launch_bounds__(kAttnThreads, 1)
     } else if (warp == 0) {
       // ================================ TMA producer: Q and K ===============================
       if (lane == 0) {
-        int i = 0, kn = 0, qc = 0;  // items seen; K tiles loaded so far; items that had tiles
-        for (int it = blockIdx.x; it < p.n_items; it += G, ++i) {
+        int kn = 0, qc = 0;  // K tiles loaded so far; items that had tiles
+        for (int i = 0;; ++i) {
           const int buf = i & 1;
           mbar_wait_bounded_inline(list_ready + buf, (i >> 1) & 1, s_abort, 51, p.wait_limit);
+          const int it = s_item[buf];
+          if (it < 0) break;  // (only the list builder decides when to stop, so that all roles stop at the same item)
           const int n_ent = s_nent[buf];
           const int n_tiles = (n_ent + C::kEPT - 1) / C::kEPT;
           if (n_tiles > 0) {
@@ -351,10 +357,11 @@ __global__ void __launch_bounds__(kAttnThreads, 1)
         qlo[kk] = (uint32_t)descQ + off;
         klo[kk] = (uint32_t)descK + off;
       }
-      int i = 0, g = 0, qc = 0;
-      for (int it = blockIdx.x; it < p.n_items; it += G, ++i) {
+      int g = 0, qc = 0;
+      for (int i = 0;; ++i) {
         const int buf = i & 1;
         mbar_wait_bounded_inline(list_ready + buf, (i >> 1) & 1, s_abort, 53, p.wait_limit);
+        if (s_item[buf] < 0) break;
         const int n_tiles = (s_nent[buf] + C::kEPT - 1) / C::kEPT;
         if (n_tiles > 0) {
           mbar_wait_bounded_inline(q_full, qc & 1, s_abort, 11, p.wait_limit);
@@ -390,10 +397,11 @@ __global__ void __launch_bounds__(kAttnThreads, 1)
 #pragma unroll
       for (int kk = 0; kk < 8; ++kk) vlo[kk] = (uint32_t)descV + (uint32_t)((kk * 2048) >> 4);
       const uint32_t tO = tmem_base + C::kColO;
-      int i = 0, g = 0;
-      for (int it = blockIdx.x; it < p.n_items; it += G, ++i) {
+      int g = 0;
+      for (int i = 0;; ++i) {
         const int buf = i & 1;
         mbar_wait_bounded_inline(list_ready + buf, (i >> 1) & 1, s_abort, 54, p.wait_limit);
+        if (s_item[buf] < 0) break;
         const int n_tiles = (s_nent[buf] + C::kEPT - 1) / C::kEPT;
         // the previous item's accumulator must have been read out before this item's first P V overwrites it
         if (i > 0) mbar_wait_bounded_inline(o_drained, (i - 1) & 1, s_abort, 55, p.wait_limit);
@@ -422,10 +430,21 @@ __global__ void __launch_bounds__(kAttnThreads, 1)
     if (warp == 4) {
       // union of the item's (up to) two mask rows -> ascending entry list; flag bit q = kept by query
       // block blk[q].  Runs up to two items ahead of the consumers.
-      int i = 0;
-      for (int it = blockIdx.x; it < p.n_items; it += G, ++i) {
+      // Work items are handed out by a global counter (first come, first served), so CTAs whose items are
+      // short simply take more of them; the item number travels to the other roles with the list.
+      for (int i = 0;; ++i) {
         const int buf = i & 1;
         if (i >= 2) mbar_wait_bounded_inline(list_free + buf, ((i - 2) >> 1) & 1, s_abort, 50, p.wait_limit);
+        int it = 0;
+        if (lane == 0) it = atomicAdd(p.work_counter, 1);
+        it = __shfl_sync(0xffffffffu, it, 0);
+        if (it >= p.n_items || *s_abort) {
+          if (lane == 0) {
+            s_item[buf] = -1;
+            mbar_arrive(list_ready + buf);
+          }
+          break;
+        }
         const int bh = it / p.per_bh, x = it - bh * p.per_bh;
         int blk[2];
         if (C::kStacked) {
@@ -502,6 +521,7 @@ __global__ void __launch_bounds__(kAttnThreads, 1)
           }
         }
         if (lane == 0) {
+          s_item[buf] = it;
           s_nent[buf] = running;
           s_blk[buf * 2] = blk[0];
           s_blk[buf * 2 + 1] = blk[1];
@@ -524,11 +544,13 @@ __global__ void __launch_bounds__(kAttnThreads, 1)
     const int bar_mine = 1 + wg * 4 + rgrp;         // I arrive here after my decision
     const int bar_other = 1 + (1 - wg) * 4 + rgrp;  // the row group's other warp arrives here after its decision
 
-    int i = 0, g0 = 0;  // items seen; number of the item's first tile
-    for (int it = blockIdx.x; it < p.n_items; it += G, ++i) {
+    int g0 = 0;  // number of the item's first tile
+    for (int i = 0;; ++i) {
       const int buf = i & 1;
       volatile float* ref = sRef + (i % 3) * 128;
       mbar_wait_bounded_inline(list_ready + buf, (i >> 1) & 1, s_abort, 56, p.wait_limit);
+      const int it = s_item[buf];
+      if (it < 0) break;
       const int n_ent = s_nent[buf];
       const int n_tiles = (n_ent + C::kEPT - 1) / C::kEPT;
       const uint16_t* entJ = sEntJ + buf * kMaxBlocks;
@@ -946,6 +968,7 @@ static int launch_attn_common(const sparsp_shape& s, const Geometry& g, const vo
   p.O = (__nv_bfloat16*)O;
   p.lse = lse;
   p.status = (int32_t*)(ws + L.status);
+  p.work_counter = p.status + kWorkCounterWord;
   p.N = g.N;
   p.sB = s.stride_batch;
   p.sH = s.stride_head;
@@ -1009,8 +1032,10 @@ __global__ void __launch_bounds__(kPairThreads) attn_prep_kernel(const uint32_t*
                                                                  int32_t* __restrict__ pairs, int n_pair,
                                                                  const __nv_bfloat16* __restrict__ K, int64_t sB,
                                                                  int64_t sH, int64_t sT, int H, int b, int64_t N,
-                                                                 int64_t n_units, float* __restrict__ knorm) {
+                                                                 int64_t n_units, float* __restrict__ knorm,
+                                                                 int32_t* __restrict__ work_counter) {
   extern __shared__ __align__(16) unsigned char smem_raw[];
+  if (blockIdx.x == 0 && threadIdx.x == 0) *work_counter = 0;  // the attention kernel's work queue
   if ((int)blockIdx.x < n_pair) {
     pair_body(mask, NB, Wd, 1, pairs, (int)blockIdx.x, smem_raw);
   } else {
@@ -1034,11 +1059,13 @@ int launch_attn(const sparsp_shape& s, const Geometry& g, const void* Q, const v
     if (g.d == 64) {
       SPARSP_CUDA_OK(ensure_dynamic_smem((const void*)attn_prep_kernel<64>, (int)smem));
       attn_prep_kernel<64><<<blocks, kPairThreads, smem, st>>>(mask, g.NB, g.Wd, pairs, n_pair, (const __nv_bfloat16*)K, sB,
-                                                             s.stride_head, s.stride_token, g.H, g.b, g.N, n_units, knorm);
+                                                             s.stride_head, s.stride_token, g.H, g.b, g.N, n_units, knorm,
+                                                             (int32_t*)(ws + L.status) + kWorkCounterWord);
     } else {
       SPARSP_CUDA_OK(ensure_dynamic_smem((const void*)attn_prep_kernel<128>, (int)smem));
       attn_prep_kernel<128><<<blocks, kPairThreads, smem, st>>>(mask, g.NB, g.Wd, pairs, n_pair, (const __nv_bfloat16*)K, sB,
-                                                              s.stride_head, s.stride_token, g.H, g.b, g.N, n_units, knorm);
+                                                              s.stride_head, s.stride_token, g.H, g.b, g.N, n_units, knorm,
+                                                             (int32_t*)(ws + L.status) + kWorkCounterWord);
     }
     count_launch();
   }
@@ -1074,7 +1101,9 @@ __global__ void pair_rank_kernel(const int32_t* __restrict__ rank, int NB, int c
 __global__ void slot_kernel(const uint32_t* __restrict__ U, const int32_t* __restrict__ rank,
                             const int64_t* __restrict__ seg_off, const int64_t* __restrict__ seg_total,
                             const int64_t* __restrict__ dst_base, int B, int H, int NB, int Wd, int P, int consumer,
-                            int64_t tile_bytes, int32_t* __restrict__ slot, int64_t* __restrict__ tile_base) {
+                            int64_t tile_bytes, int32_t* __restrict__ slot, int64_t* __restrict__ tile_base,
+                            int32_t* __restrict__ work_counter) {
+  if (blockIdx.x == 0 && threadIdx.x == 0) *work_counter = 0;  // the attention kernel's work queue
   const int64_t wid = ((int64_t)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
   const int lane = threadIdx.x & 31;
   if (wid < B && lane == 0) {  // first tile of the consumer's buffer for batch item wid
@@ -1141,7 +1170,7 @@ int launch_attn_packed(const sparsp_shape& s, const Geometry& g, const void* Q, 
   const int64_t n_warps = std::max<int64_t>((int64_t)g.B * P * g.H, g.B);
   slot_kernel<<<(unsigned)((n_warps * 32 + 255) / 256), 256, 0, st>>>(U, rank, seg_off, seg_total, dst_base, g.B, g.H,
                                                                     g.NB, g.Wd, P, consumer, tile_bytes, slot,
-                                                                    tile_base);
+                                                                    tile_base, (int32_t*)(ws + L.status) + kWorkCounterWord);
   count_launch(2);
   AttnParams p;
   p.mask = mask;
