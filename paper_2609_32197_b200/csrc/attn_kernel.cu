@@ -31,7 +31,6 @@
 // Every mbarrier wait is bounded; a wait that runs out sets SPARSP_ERR_TIMEOUT in the status word
 // and raises a CTA-wide flag that makes all later waits fall through, so the CTA still drains.
 #include <algorithm>
-#include <cstdlib>
 #include <type_traits>
 
 #include "common.cuh"
@@ -954,8 +953,7 @@ static int launch_attn_t(const sparsp_shape& s, const Geometry& g, const void* Q
   int dev = 0, sms = 0;
   SPARSP_CUDA_OK(cudaGetDevice(&dev));
   SPARSP_CUDA_OK(cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev));
-  static const int ctas_per_sm_x100 = getenv("SPARSP_TUNE_GRID") ? atoi(getenv("SPARSP_TUNE_GRID")) : 100;
-  dim3 grid((unsigned)std::min<long long>(pp.n_items, (long long)sms * ctas_per_sm_x100 / 100));
+  dim3 grid((unsigned)std::min(pp.n_items, sms));
   kern<<<grid, kAttnThreads, smem, st>>>(tq, tk, tv, tp, pp);
   count_launch();
   SPARSP_CUDA_OK(cudaGetLastError());
