@@ -93,8 +93,8 @@ struct AttnCfg {
   static constexpr int kOffK = kOffQ + kQBytes;
   static constexpr int kOffV = kOffK + kStagesK * kTileBytes;
   static constexpr int kOffEntJ = kOffV + kStagesV * kTileBytes;  // uint16 [2][1024] kept / union list
-  static constexpr int kOffEntF = kOffEntJ + 2 * 2 * kMaxBlocks;  // uint8 [2][1024] bit q: kept by query block q
-  static constexpr int kOffSlot = kOffEntF + 2 * kMaxBlocks;      // int32 [2][1024] packed-buffer slot per entry
+  static constexpr int kOffEntV = kOffEntJ + 2 * 2 * kMaxBlocks;  // uint8 [2][1024][2] keys of the entry valid for query block q (0 = not kept)
+  static constexpr int kOffSlot = kOffEntV + 2 * 2 * kMaxBlocks;  // int32 [2][1024] packed-buffer slot per entry
   static constexpr int kOffEntN = kOffSlot + 2 * 4 * kMaxBlocks;  // float [2][1024] largest key norm of the entry's block
   static constexpr int kOffStat = kOffEntN + 2 * 4 * kMaxBlocks;  // float2 [2 items][2 warpgroups][128]
   static constexpr int kOffRef = kOffStat + 2 * 2 * 128 * 8;      // float [3 items][128] reference maximum per row
@@ -166,7 +166,7 @@ __global__ void __launch_bounds__(kAttnThreads, 1)
   unsigned char* sK = smem + C::kOffK;
   unsigned char* sV = smem + C::kOffV;
   uint16_t* sEntJ = reinterpret_cast<uint16_t*>(smem + C::kOffEntJ);  // [2][kMaxBlocks]
-  uint8_t* sEntF = smem + C::kOffEntF;                                // [2][kMaxBlocks]
+  uint8_t* sEntV = smem + C::kOffEntV;                                // [2][kMaxBlocks][2]
   int32_t* sSlot = reinterpret_cast<int32_t*>(smem + C::kOffSlot);    // [2][kMaxBlocks]
   float* sEntN = reinterpret_cast<float*>(smem + C::kOffEntN);        // [2][kMaxBlocks]
   float2* sStat = reinterpret_cast<float2*>(smem + C::kOffStat);      // [2][2][128]
@@ -193,6 +193,7 @@ __global__ void __launch_bounds__(kAttnThreads, 1)
   int* s_nent = reinterpret_cast<int*>(smem + C::kOffMisc + 8);   // [2]
   int* s_blk = reinterpret_cast<int*>(smem + C::kOffMisc + 16);   // [2][2] the item's query block(s); < 0 = absent
   int* s_item = reinterpret_cast<int*>(smem + C::kOffMisc + 32);  // [2] the work item of each list buffer; < 0 = no more
+  int* s_rag = reinterpret_cast<int*>(smem + C::kOffMisc + 40);   // [2] the item's last tile reaches past the end of the sequence
   constexpr int kListReaders = 12;  // two producers, two issuers, eight softmax warps
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
@@ -455,7 +456,7 @@ __global__ void __launch_bounds__(kAttnThreads, 1)
           blk[1] = -1;
         }
         uint16_t* entJ = sEntJ + buf * kMaxBlocks;
-        uint8_t* entF = sEntF + buf * kMaxBlocks;
+        uint8_t* entV = sEntV + buf * kMaxBlocks * 2;
         int32_t* entS = sSlot + buf * kMaxBlocks;
         float* entN = sEntN + buf * kMaxBlocks;
         // NB <= 1024, so a mask row is at most 32 words: one word per lane
@@ -494,7 +495,10 @@ __global__ void __launch_bounds__(kAttnThreads, 1)
             else if (idx < n_mix) pos = n_both + 2 * idx + (c - 1);
             else pos = n_both + n_mix + idx;  // tail of the longer class
             entJ[pos] = (uint16_t)(lane * 32 + t);
-            entF[pos] = (uint8_t)(c == 0 ? 3 : c);
+            const int jb = lane * 32 + t;
+            const int nvalid = (int)min((int64_t)BLK, p.N - (int64_t)jb * BLK);
+            entV[pos * 2] = (uint8_t)(c != 2 ? nvalid : 0);      // keys valid for the first query block's rows
+            entV[pos * 2 + 1] = (uint8_t)(c != 1 ? nvalid : 0);  // ... for the second's
             if (p.slot) entS[pos] = p.slot[(int64_t)bh * p.NB + lane * 32 + t];
             if (p.knorm) entN[pos] = p.knorm[(int64_t)bh * p.NB + lane * 32 + t];
             ++idx;
@@ -503,16 +507,18 @@ __global__ void __launch_bounds__(kAttnThreads, 1)
         __syncwarp();
         // the softmax code lets only the LAST tile reach past the end of the sequence: if the last block of
         // the sequence is ragged and in the list, it trades places with the last entry
+        bool last_ragged = false;
         if ((int64_t)p.NB * BLK > p.N && running > 0) {
           const int lw = (p.NB - 1) >> 5, lb = (p.NB - 1) & 31;
           const uint32_t have = __shfl_sync(0xffffffffu, rb0 | rb1, lw);
           if ((have >> lb) & 1u) {
+            last_ragged = true;
             if (lane == 0) {
               int r = 0;
               while (r < running - 1 && entJ[r] != (uint16_t)(p.NB - 1)) ++r;
               const int e = running - 1;
               const uint16_t tj = entJ[r]; entJ[r] = entJ[e]; entJ[e] = tj;
-              const uint8_t tf = entF[r]; entF[r] = entF[e]; entF[e] = tf;
+              for (int q = 0; q < 2; ++q) { const uint8_t tv = entV[r * 2 + q]; entV[r * 2 + q] = entV[e * 2 + q]; entV[e * 2 + q] = tv; }
               if (p.slot) { const int32_t ts = entS[r]; entS[r] = entS[e]; entS[e] = ts; }
               if (p.knorm) { const float tn = entN[r]; entN[r] = entN[e]; entN[e] = tn; }
             }
@@ -521,6 +527,7 @@ __global__ void __launch_bounds__(kAttnThreads, 1)
         }
         if (lane == 0) {
           s_item[buf] = it;
+          s_rag[buf] = last_ragged ? 1 : 0;
           s_nent[buf] = running;
           s_blk[buf * 2] = blk[0];
           s_blk[buf * 2 + 1] = blk[1];
@@ -552,8 +559,8 @@ __global__ void __launch_bounds__(kAttnThreads, 1)
       if (it < 0) break;
       const int n_ent = s_nent[buf];
       const int n_tiles = (n_ent + C::kEPT - 1) / C::kEPT;
-      const uint16_t* entJ = sEntJ + buf * kMaxBlocks;
-      const uint8_t* entF = sEntF + buf * kMaxBlocks;
+      const uint8_t* entV = sEntV + buf * kMaxBlocks * 2 + (C::kStacked ? rh : 0);  // my query block's column
+      const bool item_ragged = s_rag[buf] != 0;
       const float* entN = sEntN + buf * kMaxBlocks;
       const int bh = it / p.per_bh;
       const int batch = bh / p.H, head = bh % p.H;
@@ -566,17 +573,13 @@ __global__ void __launch_bounds__(kAttnThreads, 1)
       auto do_tile = [&](auto ragged_tag, const int n) {
         constexpr bool kRagged = decltype(ragged_tag)::value;
         const int g = g0 + n;
-        // kept / valid key columns of each 64-column half of the tile (warp-uniform)
+        // kept / valid key columns of each 64-column half of the tile (warp-uniform), as the list builder left them
         int vh[2];
         if (C::kStacked) {
-#pragma unroll
-          for (int h = 0; h < 2; ++h) {
-            const int ent = n * 2 + h;
-            vh[h] = 0;
-            if (ent < n_ent && ((entF[ent] >> rh) & 1)) vh[h] = (int)min((int64_t)64, p.N - (int64_t)entJ[ent] * 64);
-          }
+          vh[0] = entV[(n * 2) * 2];
+          vh[1] = n * 2 + 1 < n_ent ? entV[(n * 2 + 1) * 2] : 0;
         } else {
-          const int nv = (int)min((int64_t)128, p.N - (int64_t)entJ[n] * 128);
+          const int nv = entV[n * 2];
           vh[0] = min(nv, 64);
           vh[1] = max(nv - 64, 0);
         }
@@ -591,7 +594,7 @@ __global__ void __launch_bounds__(kAttnThreads, 1)
           // My first tile of the item: the norm of my query row, read from the Q tile in shared memory (any
           // order of its 16-byte units will do, so the swizzle does not matter).  Q is still there: its last
           // Q K^T cannot have been issued before this warp releases the S buffer below.
-          float ss = 0.0f;
+          float ss[4] = {0.0f, 0.0f, 0.0f, 0.0f};  // four chains, so that the additions do not wait for each other
 #pragma unroll
           for (int c = 0; c < D / 64; ++c) {
 #pragma unroll
@@ -601,12 +604,12 @@ __global__ void __launch_bounds__(kAttnThreads, 1)
 #pragma unroll
               for (int e = 0; e < 4; ++e) {
                 const float lo = __uint_as_float(w[e] << 16), hi = __uint_as_float(w[e] & 0xffff0000u);
-                ss = fmaf(lo, lo, ss);
-                ss = fmaf(hi, hi, ss);
+                ss[e] = fmaf(lo, lo, ss[e]);
+                ss[e] = fmaf(hi, hi, ss[e]);
               }
             }
           }
-          q_bound = sqrtf(ss) * p.scale_log2 * 1.001f;
+          q_bound = sqrtf((ss[0] + ss[1]) + (ss[2] + ss[3])) * p.scale_log2 * 1.001f;
         }
         // S is in registers: the Q K^T of tile g+2 may overwrite the buffer
         tc_fence_before();
@@ -736,7 +739,7 @@ __global__ void __launch_bounds__(kAttnThreads, 1)
       };
       for (int n = (wg - g0) & 1; n < n_tiles; n += 2) {
         // the list builder puts the sequence's last block (the only one that can be ragged) into the last tile
-        const bool ragged = n == n_tiles - 1 && (int64_t)(entJ[n_ent - 1] + 1) * BLK > p.N;
+        const bool ragged = item_ragged && n == n_tiles - 1;
         if (ragged) {
           do_tile(std::true_type{}, n);
         } else {
