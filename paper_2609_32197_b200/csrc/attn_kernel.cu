@@ -784,16 +784,26 @@ __global__ void __launch_bounds__(kAttnThreads, 1)
           mbar_arrive(list_free + buf);
         }
         if (tok < p.N) {
+          // a thread's row segment is 2 HW contiguous bytes but the rows of a warp are sT elements apart, so every
+          // store instruction touches 32 lines: 32-byte stores (when the layout allows) halve their number
+          const bool wide = ((reinterpret_cast<uintptr_t>(orow) | (uintptr_t)(p.sT * 2)) & 31) == 0;
 #pragma unroll
-          for (int v = 0; v < HW / 8; ++v) {
-            uint32_t w[4];
+          for (int v = 0; v < HW / 16; ++v) {
+            uint32_t w[8];
 #pragma unroll
-            for (int e = 0; e < 4; ++e) {
-              const __nv_bfloat162 h2 = __floats2bfloat162_rn(__uint_as_float(o[v * 8 + 2 * e]) * inv_l,
-                                                              __uint_as_float(o[v * 8 + 2 * e + 1]) * inv_l);
+            for (int e = 0; e < 8; ++e) {
+              const __nv_bfloat162 h2 = __floats2bfloat162_rn(__uint_as_float(o[v * 16 + 2 * e]) * inv_l,
+                                                              __uint_as_float(o[v * 16 + 2 * e + 1]) * inv_l);
               w[e] = *reinterpret_cast<const uint32_t*>(&h2);
             }
-            *reinterpret_cast<uint4*>(orow + v * 8) = make_uint4(w[0], w[1], w[2], w[3]);
+            if (wide) {
+              asm volatile("st.global.v8.b32 [%0], {%1, %2, %3, %4, %5, %6, %7, %8};" ::"l"(orow + v * 16), "r"(w[0]),
+                           "r"(w[1]), "r"(w[2]), "r"(w[3]), "r"(w[4]), "r"(w[5]), "r"(w[6]), "r"(w[7])
+                           : "memory");
+            } else {
+              *reinterpret_cast<uint4*>(orow + v * 16) = make_uint4(w[0], w[1], w[2], w[3]);
+              *reinterpret_cast<uint4*>(orow + v * 16 + 8) = make_uint4(w[4], w[5], w[6], w[7]);
+            }
           }
         }
         if (p.lse && wg == 0 && tok < p.N)
