@@ -567,6 +567,8 @@ __global__ void __launch_bounds__(kAttnThreads, 1)
       float q_bound = INFINITY;  // |q_row| * softmax scale * log2(e) (+0.1 %), once known
       float m_ref = -INFINITY;  // the row's reference maximum (log2 domain) as this thread last saw it
       float l_run = 0.0f;       // this thread's partial row sum, relative to m_ref
+      float sv[128];            // my row of the current tile's scores
+      bool have_s = false;      // the loads of my next tile's scores are already in flight (warp-uniform)
 
       // One tile of this warpgroup.  kRagged = the sequence ends inside the tile (possible only for the item's
       // last tile): that variant carries the column masking, the common one stays small.
@@ -584,11 +586,12 @@ __global__ void __launch_bounds__(kAttnThreads, 1)
           vh[1] = max(nv - 64, 0);
         }
 
-        mbar_wait_bounded_inline(s_full + wg, (g >> 1) & 1, s_abort, 30 + wg, p.wait_limit);
-        tc_fence_after();
-        float sv[128];
+        if (!have_s) {
+          mbar_wait_bounded_inline(s_full + wg, (g >> 1) & 1, s_abort, 30 + wg, p.wait_limit);
+          tc_fence_after();
 #pragma unroll
-        for (int c = 0; c < 4; ++c) tmem_ld32(tS + c * 32, reinterpret_cast<uint32_t*>(sv) + c * 32);
+          for (int c = 0; c < 4; ++c) tmem_ld32(tS + c * 32, reinterpret_cast<uint32_t*>(sv) + c * 32);
+        }
         tmem_ld_wait();
         if (p.knorm != nullptr && n < 2 && n_tiles >= n + 3) {
           // My first tile of the item: the norm of my query row, read from the Q tile in shared memory (any
@@ -725,6 +728,16 @@ __global__ void __launch_bounds__(kAttnThreads, 1)
           }
         }
         l_run += lsum2.x + lsum2.y;
+        // The scores are spent, so their registers can already take my next tile's (tile g+2 of the same
+        // item) if its Q K^T has completed, which is the normal case: the load latency then hides behind
+        // the P store below instead of opening the next tile.
+        have_s = false;
+        if (n + 2 < n_tiles && mbar_test_wait(s_full + wg, ((g + 2) >> 1) & 1)) {
+          tc_fence_after();
+#pragma unroll
+          for (int c = 0; c < 4; ++c) tmem_ld32(tS + c * 32, reinterpret_cast<uint32_t*>(sv) + c * 32);
+          have_s = true;
+        }
         // my P buffer was last read by the P V of tile g-2
         if (g >= 2) {
           mbar_wait_bounded_inline(o_full + ((g - 2) & 3), ((g - 2) >> 2) & 1, s_abort, 34 + wg, p.wait_limit);
