@@ -104,7 +104,7 @@ struct AttnCfg {
   static constexpr int kColP = 256;  // P buffers: columns [256, 384)
   static constexpr int kColO = 384;  // accumulator: columns [384, 384 + d)
   static constexpr int kOffMisc = kOffBars + 8 * kNumBars;
-  static constexpr int kTotal = kOffMisc + 64;
+  static constexpr int kTotal = kOffMisc + 80;
   static constexpr int kDynamic = kTotal + 1024;  // slack for the 1024-byte alignment of the base
   static_assert(kDynamic <= 232448, "shared memory budget");
 };
@@ -194,6 +194,8 @@ __global__ void __launch_bounds__(kAttnThreads, 1)
   int* s_blk = reinterpret_cast<int*>(smem + C::kOffMisc + 16);   // [2][2] the item's query block(s); < 0 = absent
   int* s_item = reinterpret_cast<int*>(smem + C::kOffMisc + 32);  // [2] the work item of each list buffer; < 0 = no more
   int* s_rag = reinterpret_cast<int*>(smem + C::kOffMisc + 40);   // [2] the item's last tile reaches past the end of the sequence
+  volatile int* s_frz = reinterpret_cast<volatile int*>(smem + C::kOffMisc + 56);  // [4] per row group: reference frozen
+  float* s_knmax = reinterpret_cast<float*>(smem + C::kOffMisc + 48);  // [2] largest key norm bound among the item's entries
   constexpr int kListReaders = 12;  // two producers, two issuers, eight softmax warps
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
@@ -224,6 +226,7 @@ __global__ void __launch_bounds__(kAttnThreads, 1)
     mbar_init(o_drained, 8);
     mbar_init_fence();
     *s_abort = 0;
+    for (int r = 0; r < 4; ++r) s_frz[r] = 0;
   }
   if (tid < 384) sRef[tid] = -INFINITY;  // 3 x 128 entries
   if (warp == 1) {
@@ -483,6 +486,7 @@ __global__ void __launch_bounds__(kAttnThreads, 1)
         }
         const int n_both = total[0], n_mix = min(total[1], total[2]);
         const int running = total[0] + total[1] + total[2];
+        float kn_max = 0.0f;
 #pragma unroll
         for (int c = 0; c < 3; ++c) {
           uint32_t u = cls[c];
@@ -500,10 +504,16 @@ __global__ void __launch_bounds__(kAttnThreads, 1)
             entV[pos * 2] = (uint8_t)(c != 2 ? nvalid : 0);      // keys valid for the first query block's rows
             entV[pos * 2 + 1] = (uint8_t)(c != 1 ? nvalid : 0);  // ... for the second's
             if (p.slot) entS[pos] = p.slot[(int64_t)bh * p.NB + lane * 32 + t];
-            if (p.knorm) entN[pos] = p.knorm[(int64_t)bh * p.NB + lane * 32 + t];
+            if (p.knorm) {
+              const float kn = p.knorm[(int64_t)bh * p.NB + lane * 32 + t];
+              entN[pos] = kn;
+              kn_max = fmaxf(kn_max, kn);
+            }
             ++idx;
           }
         }
+#pragma unroll
+        for (int s = 16; s > 0; s >>= 1) kn_max = fmaxf(kn_max, __shfl_xor_sync(0xffffffffu, kn_max, s));
         __syncwarp();
         // the softmax code lets only the LAST tile reach past the end of the sequence: if the last block of
         // the sequence is ragged and in the list, it trades places with the last entry
@@ -529,6 +539,7 @@ __global__ void __launch_bounds__(kAttnThreads, 1)
           s_item[buf] = it;
           s_rag[buf] = last_ragged ? 1 : 0;
           s_nent[buf] = running;
+          s_knmax[buf] = kn_max;
           s_blk[buf * 2] = blk[0];
           s_blk[buf * 2 + 1] = blk[1];
         }
@@ -549,6 +560,7 @@ __global__ void __launch_bounds__(kAttnThreads, 1)
     const uint32_t tO = tmem_base + C::kColO + lane_off;
     const int bar_mine = 1 + wg * 4 + rgrp;         // I arrive here after my decision
     const int bar_other = 1 + (1 - wg) * 4 + rgrp;  // the row group's other warp arrives here after its decision
+    volatile int* frz = s_frz + rgrp;               // set by the warp that freezes the reference, cleared by the other
 
     int g0 = 0;  // number of the item's first tile
     for (int i = 0;; ++i) {
@@ -562,13 +574,16 @@ __global__ void __launch_bounds__(kAttnThreads, 1)
       const uint8_t* entV = sEntV + buf * kMaxBlocks * 2 + (C::kStacked ? rh : 0);  // my query block's column
       const bool item_ragged = s_rag[buf] != 0;
       const float* entN = sEntN + buf * kMaxBlocks;
+      const float kn_item = s_knmax[buf];
       const int bh = it / p.per_bh;
       const int batch = bh / p.H, head = bh % p.H;
+      // Once no score of any remaining tile of the item can exceed the row's reference maximum by more than
+      // 2^kSkipMargin (Cauchy-Schwarz with the item's largest key norm), the reference is final: both warps of
+      // the row group stop taking turns and the rest of the item is load -> exponentials -> store.
+      bool frozen = false;
       float q_bound = INFINITY;  // |q_row| * softmax scale * log2(e) (+0.1 %), once known
       float m_ref = -INFINITY;  // the row's reference maximum (log2 domain) as this thread last saw it
       float l_run = 0.0f;       // this thread's partial row sum, relative to m_ref
-      float sv[128];            // my row of the current tile's scores
-      bool have_s = false;      // the loads of my next tile's scores are already in flight (warp-uniform)
 
       // One tile of this warpgroup.  kRagged = the sequence ends inside the tile (possible only for the item's
       // last tile): that variant carries the column masking, the common one stays small.
@@ -586,12 +601,11 @@ __global__ void __launch_bounds__(kAttnThreads, 1)
           vh[1] = max(nv - 64, 0);
         }
 
-        if (!have_s) {
-          mbar_wait_bounded_inline(s_full + wg, (g >> 1) & 1, s_abort, 30 + wg, p.wait_limit);
-          tc_fence_after();
+        mbar_wait_bounded_inline(s_full + wg, (g >> 1) & 1, s_abort, 30 + wg, p.wait_limit);
+        tc_fence_after();
+        float sv[128];
 #pragma unroll
-          for (int c = 0; c < 4; ++c) tmem_ld32(tS + c * 32, reinterpret_cast<uint32_t*>(sv) + c * 32);
-        }
+        for (int c = 0; c < 4; ++c) tmem_ld32(tS + c * 32, reinterpret_cast<uint32_t*>(sv) + c * 32);
         tmem_ld_wait();
         if (p.knorm != nullptr && n < 2 && n_tiles >= n + 3) {
           // My first tile of the item: the norm of my query row, read from the Q tile in shared memory (any
@@ -619,81 +633,101 @@ __global__ void __launch_bounds__(kAttnThreads, 1)
         __syncwarp();
         if (lane == 0) mbar_arrive(s_free + wg);
 
-        // Cauchy-Schwarz: no score of this tile exceeds |q| * max |k| * scale.  If that bound stays within
-        // 2^kSkipMargin of the row's reference maximum (which only grows, so the value this thread saw last
-        // will do) for all 32 rows of the warp, the reference need not move and the row-maximum pass is
-        // skipped: the exponentials stay below 2^kSkipMargin, harmless in fp32 / bf16, and the result does
-        // not depend on the reference.
-        bool skip = false;
-        if (!kRagged && p.knorm != nullptr) {
-          float kn = entN[n * C::kEPT];
-          if (C::kStacked) kn = fmaxf(kn, entN[min(n * 2 + 1, n_ent - 1)]);
-          skip = __all_sync(0xffffffffu, q_bound * kn <= m_ref + kSkipMargin);
-        }
-
-        // one flat instruction stream per 64-key half; a ragged half (the sequence ends inside it) first has
-        // its invalid columns set to -inf, an absent half (not kept by this row's query block) is skipped
-        float mx = -INFINITY;
-        if (!skip)
+        if (kRagged) {
+          // the sequence ends inside this tile: columns past the end count as -inf
 #pragma unroll
-        for (int h = 0; h < 2; ++h) {
-          float* svh = sv + h * 64;
-          if (vh[h] > 0) {
-            if (kRagged && vh[h] < 64) {
+          for (int h = 0; h < 2; ++h) {
+            if (vh[h] > 0 && vh[h] < 64) {
 #pragma unroll
-              for (int e = 0; e < 64; ++e) svh[e] = e < vh[h] ? svh[e] : -INFINITY;
+              for (int e = 0; e < 64; ++e) sv[h * 64 + e] = e < vh[h] ? sv[h * 64 + e] : -INFINITY;
             }
-            float m0 = svh[0], m1 = svh[1], m2 = svh[2], m3 = svh[3];
-#pragma unroll
-            for (int e = 4; e < 64; e += 4) {
-              m0 = fmaxf(m0, svh[e]);
-              m1 = fmaxf(m1, svh[e + 1]);
-              m2 = fmaxf(m2, svh[e + 2]);
-              m3 = fmaxf(m3, svh[e + 3]);
-            }
-            mx = fmaxf(mx, fmaxf(fmaxf(m0, m1), fmaxf(m2, m3)));
           }
         }
-        mx *= p.scale_log2;
+        if (!frozen) {
+          // Cauchy-Schwarz: no score of this tile exceeds |q| * max |k| * scale.  If that bound stays within
+          // 2^kSkipMargin of the row's reference maximum (which only grows, so the value this thread saw last
+          // will do) for all 32 rows of the warp, the reference need not move and the row-maximum pass is
+          // skipped: the exponentials stay below 2^kSkipMargin, harmless in fp32 / bf16, and the result does
+          // not depend on the reference.
+          bool skip = false;
+          if (!kRagged && p.knorm != nullptr) {
+            float kn = entN[n * C::kEPT];
+            if (C::kStacked) kn = fmaxf(kn, entN[min(n * 2 + 1, n_ent - 1)]);
+            skip = __all_sync(0xffffffffu, q_bound * kn <= m_ref + kSkipMargin);
+          }
 
-        // ---- my turn to look at / move the row's reference maximum (strictly in tile order) ----
-        if (n > 0) named_bar_sync(bar_other, 64);
-        {
+          // one flat instruction stream per 64-key half; an absent half (not kept by this row's query block)
+          // is skipped
+          float mx = -INFINITY;
+          if (!skip)
+#pragma unroll
+          for (int h = 0; h < 2; ++h) {
+            const float* svh = sv + h * 64;
+            if (vh[h] > 0) {
+              float m0 = svh[0], m1 = svh[1], m2 = svh[2], m3 = svh[3];
+#pragma unroll
+              for (int e = 4; e < 64; e += 4) {
+                m0 = fmaxf(m0, svh[e]);
+                m1 = fmaxf(m1, svh[e + 1]);
+                m2 = fmaxf(m2, svh[e + 2]);
+                m3 = fmaxf(m3, svh[e + 3]);
+              }
+              mx = fmaxf(mx, fmaxf(fmaxf(m0, m1), fmaxf(m2, m3)));
+            }
+          }
+          mx *= p.scale_log2;
+
+          // ---- my turn to look at / move the row's reference maximum (strictly in tile order) ----
+          if (n > 0) named_bar_sync(bar_other, 64);
           const float m_cur = ref[row];
+          const int told = n > 0 ? *frz : 0;  // the row group's other warp froze the reference in its last turn
           if (m_cur != m_ref) {  // the other thread moved it since my last tile
             l_run *= ex2(m_ref - m_cur);  // m_ref = -inf: l_run is 0 and stays 0
             m_ref = m_cur;
           }
-        }
-        const float m_new = fmaxf(m_ref, mx);
-        const bool grow = m_new > m_ref + kGrowThreshold || (m_ref == -INFINITY && m_new > -INFINITY);
-        if (!skip && __any_sync(0xffffffffu, grow)) {
-          const float alpha = grow ? ex2(m_ref - m_new) : 1.0f;  // m_ref = -inf -> 0
-          if (n > 0) {
-            // every P V of the item issued so far must have landed in O before the row is rescaled; they
-            // complete in order, so the one of tile g-1 suffices
-            mbar_wait_bounded_inline(o_full + ((g - 1) & 3), ((g - 1) >> 2) & 1, s_abort, 38, p.wait_limit);
-            tc_fence_after();
-#pragma unroll 1
-            for (int c = 0; c < D / 16; ++c) {  // the row's accumulator, 16 columns at a time (rare: kept small)
-              uint32_t o[16];
-              tmem_ld16(tO + c * 16, o);
-              tmem_ld_wait();
-#pragma unroll
-              for (int e = 0; e < 16; ++e) o[e] = __float_as_uint(__uint_as_float(o[e]) * alpha);
-              tmem_st16(tO + c * 16, o);
+          if (told) {
+            frozen = true;
+            __syncwarp();
+            if (lane == 0) *frz = 0;  // nobody looks at it again before the next item's turns
+          } else {
+            // the first of the two warps to see the bound hold for the whole item says so, takes its last turn
+            // without moving the reference (no score can make that necessary) and releases the other one more time
+            if (n + 1 < n_tiles && p.knorm != nullptr &&
+                __all_sync(0xffffffffu, q_bound * kn_item <= m_ref + kSkipMargin)) {
+              frozen = true;
+              if (lane == 0) *frz = 1;
             }
-            tmem_st_wait();
-            tc_fence_before();
+            const float m_new = fmaxf(m_ref, mx);
+            const bool grow = !frozen && (m_new > m_ref + kGrowThreshold || (m_ref == -INFINITY && m_new > -INFINITY));
+            if (!skip && __any_sync(0xffffffffu, grow)) {
+              const float alpha = grow ? ex2(m_ref - m_new) : 1.0f;  // m_ref = -inf -> 0
+              if (n > 0) {
+                // every P V of the item issued so far must have landed in O before the row is rescaled; they
+                // complete in order, so the one of tile g-1 suffices
+                mbar_wait_bounded_inline(o_full + ((g - 1) & 3), ((g - 1) >> 2) & 1, s_abort, 38, p.wait_limit);
+                tc_fence_after();
+#pragma unroll 1
+                for (int c = 0; c < D / 16; ++c) {  // the row's accumulator, 16 columns at a time (rare: kept small)
+                  uint32_t o[16];
+                  tmem_ld16(tO + c * 16, o);
+                  tmem_ld_wait();
+#pragma unroll
+                  for (int e = 0; e < 16; ++e) o[e] = __float_as_uint(__uint_as_float(o[e]) * alpha);
+                  tmem_st16(tO + c * 16, o);
+                }
+                tmem_st_wait();
+                tc_fence_before();
+              }
+              l_run *= alpha;
+              if (grow) {
+                m_ref = m_new;
+                ref[row] = m_new;
+              }
+            }
+            if (n + 1 < n_tiles) {
+              asm volatile("bar.arrive %0, %1;" ::"r"(bar_mine), "r"(64) : "memory");
+            }
           }
-          l_run *= alpha;
-          if (grow) {
-            m_ref = m_new;
-            ref[row] = m_new;
-          }
-        }
-        if (n + 1 < n_tiles) {
-          asm volatile("bar.arrive %0, %1;" ::"r"(bar_mine), "r"(64) : "memory");
         }
 
         // exponentials of keys [64h, 64h+64) -> packed bf16 columns [32h, 32h+32) of the P buffer
@@ -728,16 +762,6 @@ __global__ void __launch_bounds__(kAttnThreads, 1)
           }
         }
         l_run += lsum2.x + lsum2.y;
-        // The scores are spent, so their registers can already take my next tile's (tile g+2 of the same
-        // item) if its Q K^T has completed, which is the normal case: the load latency then hides behind
-        // the P store below instead of opening the next tile.
-        have_s = false;
-        if (n + 2 < n_tiles && mbar_test_wait(s_full + wg, ((g + 2) >> 1) & 1)) {
-          tc_fence_after();
-#pragma unroll
-          for (int c = 0; c < 4; ++c) tmem_ld32(tS + c * 32, reinterpret_cast<uint32_t*>(sv) + c * 32);
-          have_s = true;
-        }
         // my P buffer was last read by the P V of tile g-2
         if (g >= 2) {
           mbar_wait_bounded_inline(o_full + ((g - 2) & 3), ((g - 2) >> 2) & 1, s_abort, 34 + wg, p.wait_limit);

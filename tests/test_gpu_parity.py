@@ -226,7 +226,9 @@ def test_batch_of_two(oracle_mod, binding, layout):
     """Batch is an independent outer dimension: each batch item must match the oracle run on it alone."""
     b, d, H, P, k = 64, 64, 2, 3, 4
     wls = [_workload("b0", H, d, (3, 9, 13), 40, b, k, P, seed=31), _workload("b1", H, d, (3, 9, 13), 40, b, k, P, seed=32)]
-    data = [_gen(w) for w in wls]
+    # with only four kept blocks an output row is nearly one V row, |O| passes 4 and bf16 output rounding alone
+    # (up to 0.0156 there) nearly uses up the 2e-2 bound; halving V (exact in bf16) keeps |O| below 2.5
+    data = [(Q, K, (V.float() * 0.5).to(torch.bfloat16)) for (Q, K, V) in (_gen(w) for w in wls)]
     N, NB = wls[0].n_tokens, wls[0].n_blocks
     shape = binding.make_shape(H, d, wls[0].grid, 40, b, batch=2, layout=layout)
     Qd, Kd, Vd = (_stack_batches([x[i] for x in data], layout) for i in range(3))
