@@ -325,3 +325,40 @@ def test_scores_far_above_the_first_tile(oracle_mod, binding, d, b, jump):
     # closed form: the high block dominates by 2^jump, so every row is the mean of V over block 3
     want = V[:, 3 * b:4 * b].float().mean(1)
     assert (O.float().cpu() - want[:, None, :]).abs().max() < 2e-2
+
+
+@pytest.mark.parametrize("d,b", [(128, 128), (64, 128), (128, 64), (64, 64)])
+@pytest.mark.parametrize("outlier", [False, True])
+def test_long_lists_with_final_reference_and_ragged_tail(oracle_mod, binding, d, b, outlier):
+    """Lists long enough (13 kept blocks per row, a different random set per row) that the kernel stops
+    updating a row's reference once the item's largest key norm bounds all remaining scores, with the ragged
+    last block of the sequence in every list.  With `outlier` one block holds keys of 40 times the norm
+    (orthogonal to the queries, so its scores stay ordinary): the item-wide bound then fails while the
+    per-tile bound holds for the other tiles, and the reference keeps being checked tile by tile."""
+    H, NB = 2, 20
+    N = NB * b - 37
+    rng = np.random.default_rng(23 + d + b)
+    Q = torch.tensor(rng.standard_normal((H, N, d))).to(torch.bfloat16)
+    K = torch.tensor(rng.standard_normal((H, N, d))).to(torch.bfloat16)
+    V = torch.tensor(rng.standard_normal((H, N, d)) * 0.5).to(torch.bfloat16)
+    if outlier:
+        Q[:, :, 0] = 0.0
+        K[:, 7 * b:8 * b, 0] = 40.0 * np.sqrt(d)
+    words = np.zeros((H, NB, 1), np.uint32)
+    for h in range(H):
+        for i in range(NB):
+            keep = set(rng.choice(NB - 1, 12, replace=False).tolist()) | {NB - 1}
+            if outlier:
+                keep.add(7)
+            for j in keep:
+                words[h, i, 0] |= np.uint32(1 << j)
+    shape = binding.make_shape(H, d, (1, 1, N), 0, b)
+    ws = binding.make_workspace(shape, 2)
+    Qd, Kd, Vd = Q.cuda(), K.cuda(), V.cuda()
+    O = torch.zeros_like(Qd)
+    lse = torch.zeros(1, H, N, dtype=torch.float32, device="cuda")
+    binding.sparsp_sparse_attn_fwd(shape, Qd, Kd, Vd, torch.as_tensor(words.view(np.int32)).cuda(), 0.0, O, lse, ws)
+    torch.cuda.synchronize()
+    assert binding.sparsp_status(ws) == binding.SPARSP_OK
+    units = [(h, i) for h in range(H) for i in range(NB)]
+    pu.check_attn_units(oracle_mod, Q, K, V, words, b, O, units, lse_gpu=lse[0])
