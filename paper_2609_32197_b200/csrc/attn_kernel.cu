@@ -867,6 +867,55 @@ __global__ void __launch_bounds__(kAttnThreads, 1)
 constexpr int kPairThreads = 256;
 constexpr int kPairSample = 4;
 
+// Sorts n keys (n a power of two, <= 1024) in shared memory into descending order; all kPairThreads threads call it.
+__device__ __forceinline__ void sort_keys_descending(uint32_t* keys, int n) {
+  for (int k = 2; k <= n; k <<= 1) {
+    for (int j = k >> 1; j > 0; j >>= 1) {
+      for (int t = threadIdx.x; t < n; t += kPairThreads) {
+        const int u = t ^ j;
+        if (u > t) {
+          const uint32_t a = keys[t], b = keys[u];
+          if (((t & k) == 0) ? a < b : a > b) {
+            keys[t] = b;
+            keys[u] = a;
+          }
+        }
+      }
+      __syncthreads();
+    }
+  }
+}
+
+// Work items of one (batch, head) are handed out longest list first: the items still running when the queue
+// runs dry are then the short ones, which matters when list lengths vary (threshold selection, unions of two
+// stacked blocks).  Key = (list length << 10) | (1023 - index): equal lengths keep their index order.
+__device__ __forceinline__ int next_pow2(int n) {
+  int v = 1;
+  while (v < n) v <<= 1;
+  return v;
+}
+
+// block 128: order[x] = the query block that item x of this (batch, head) handles
+__device__ __forceinline__ void order_body(const uint32_t* __restrict__ mask, int NB, int Wd,
+                                           int32_t* __restrict__ pairs, int bh) {
+  __shared__ uint32_t s_keys[1024];
+  const int n2 = next_pow2(NB);
+  const uint32_t* rows = mask + (int64_t)bh * NB * Wd;
+  for (int i = threadIdx.x; i < n2; i += kPairThreads) {
+    uint32_t key = 0;
+    if (i < NB) {
+      int len = 0;
+      for (int w = 0; w < Wd; ++w) len += __popc(rows[(int64_t)i * Wd + w]);
+      key = ((uint32_t)len << 10) | (uint32_t)(1023 - i);
+    }
+    s_keys[i] = key;
+  }
+  __syncthreads();
+  sort_keys_descending(s_keys, n2);
+  int32_t* out = pairs + (int64_t)bh * ((NB + 1) / 2) * 2;
+  for (int x = threadIdx.x; x < NB; x += kPairThreads) out[x] = 1023 - (int)(s_keys[x] & 1023u);
+}
+
 __device__ __forceinline__ void pair_body(const uint32_t* __restrict__ mask, int NB, int Wd, int search,
                                           int32_t* __restrict__ pairs, int bh, unsigned char* smem_raw) {
   uint32_t* m = reinterpret_cast<uint32_t*>(smem_raw);  // [NB][Wd]
@@ -907,6 +956,43 @@ __device__ __forceinline__ void pair_body(const uint32_t* __restrict__ mask, int
         out[2 * c] = i;
         out[2 * c + 1] = (k + 1 < n_left) ? i + 1 : -1;
       }
+    }
+  }
+  // longest union first
+  __shared__ uint32_t s_keys[512];
+  const int n_pairs = (NB + 1) / 2, n2 = next_pow2(n_pairs);
+  const uint32_t* rows = mask + (int64_t)bh * NB * Wd;
+  __syncthreads();  // the pairs written above are visible to the whole block
+  for (int c = threadIdx.x; c < n2; c += kPairThreads) {
+    uint32_t key = 0;
+    if (c < n_pairs) {
+      const int a = out[2 * c], b = out[2 * c + 1];
+      int len = 0;
+      for (int w = 0; w < Wd; ++w)
+        len += __popc(rows[(int64_t)a * Wd + w] | (b >= 0 ? rows[(int64_t)b * Wd + w] : 0u));
+      key = ((uint32_t)len << 10) | (uint32_t)(1023 - c);
+    }
+    s_keys[c] = key;
+  }
+  __syncthreads();
+  sort_keys_descending(s_keys, n2);
+  int pa[2], pb[2];  // at most 512 pairs for 256 threads
+#pragma unroll
+  for (int r = 0; r < 2; ++r) {
+    const int x = threadIdx.x + r * kPairThreads;
+    if (x < n_pairs) {
+      const int c = 1023 - (int)(s_keys[x] & 1023u);
+      pa[r] = out[2 * c];
+      pb[r] = out[2 * c + 1];
+    }
+  }
+  __syncthreads();
+#pragma unroll
+  for (int r = 0; r < 2; ++r) {
+    const int x = threadIdx.x + r * kPairThreads;
+    if (x < n_pairs) {
+      out[2 * x] = pa[r];
+      out[2 * x + 1] = pb[r];
     }
   }
 }
@@ -1072,7 +1158,8 @@ __device__ __forceinline__ void knorm_body(const __nv_bfloat16* __restrict__ K, 
 }
 
 // One launch for the two passes that precede the attention kernel and do not depend on each other: blocks
-// [0, n_pair) choose the query-block pairs of one (batch, head) each (block 64 only), the rest take the largest
+// [0, n_pair) fix the work items of one (batch, head) each (block 64: which query blocks are stacked; both block
+// sizes: longest list first), the rest take the largest
 // key norm of every KV block (times 1.001), fp32 [B*H][NB], one warp per block and d/8 lanes per token: with the
 // norm of a query row it bounds the scores of a tile.
 template <int D>
@@ -1085,7 +1172,8 @@ __global__ void __launch_bounds__(kPairThreads) attn_prep_kernel(const uint32_t*
   extern __shared__ __align__(16) unsigned char smem_raw[];
   if (blockIdx.x == 0 && threadIdx.x == 0) *work_counter = 0;  // the attention kernel's work queue
   if ((int)blockIdx.x < n_pair) {
-    pair_body(mask, NB, Wd, 1, pairs, (int)blockIdx.x, smem_raw);
+    if (b == 64) pair_body(mask, NB, Wd, 1, pairs, (int)blockIdx.x, smem_raw);
+    else order_body(mask, NB, Wd, pairs, (int)blockIdx.x);
   } else {
     const int64_t unit = ((int64_t)(blockIdx.x - n_pair) * kPairThreads + threadIdx.x) >> 5;
     knorm_body<D>(K, sB, sH, sT, H, NB, b, N, n_units, knorm, unit);
@@ -1095,12 +1183,11 @@ __global__ void __launch_bounds__(kPairThreads) attn_prep_kernel(const uint32_t*
 int launch_attn(const sparsp_shape& s, const Geometry& g, const void* Q, const void* K, const void* V,
                 const uint32_t* mask, float scale, void* O, float* lse, char* ws, const WsLayout& L,
                 cudaStream_t st) {
-  int32_t* pairs = nullptr;  // block 128: item x handles query block x
+  int32_t* pairs = (int32_t*)(ws + L.pairs);  // block 64: the two stacked blocks of each item; block 128: its block
   float* knorm = (float*)(ws + L.knorm);
   {
-    const int n_pair = g.b == 64 ? g.B * g.H : 0;
-    if (n_pair) pairs = (int32_t*)(ws + L.pairs);
-    const size_t smem = n_pair ? (size_t)g.NB * g.Wd * 4 : 0;
+    const int n_pair = g.B * g.H;
+    const size_t smem = g.b == 64 ? (size_t)g.NB * g.Wd * 4 : 0;
     const int64_t n_units = (int64_t)g.B * g.H * g.NB;
     const unsigned blocks = (unsigned)(n_pair + (n_units * 32 + kPairThreads - 1) / kPairThreads);
     const int64_t sB = s.stride_batch > 0 ? s.stride_batch : 0;
