@@ -362,3 +362,29 @@ def test_long_lists_with_final_reference_and_ragged_tail(oracle_mod, binding, d,
     assert binding.sparsp_status(ws) == binding.SPARSP_OK
     units = [(h, i) for h in range(H) for i in range(NB)]
     pu.check_attn_units(oracle_mod, Q, K, V, words, b, O, units, lse_gpu=lse[0])
+
+
+@pytest.mark.parametrize("b,tokens_grid", [(64, (10, 50, 128)), (128, (10, 100, 128))])
+def test_attention_near_the_largest_block_count(oracle_mod, binding, b, tokens_grid):
+    """NB = 1000 (the limit is 1024): mask rows of 32 words, the list buffers and the sort of a head's work items
+    at their largest.  Sampled query blocks against the oracle; every other row finite and written."""
+    from paper_2609_32197_b200 import synth
+    H, d, k = 1, 64, 9
+    wl = synth.Workload("big_nb", H, d, tokens_grid, 0, b, k, None, 2, seed=5)
+    assert wl.n_blocks == 1000
+    Qd, Kd, Vd = synth.make_qkv(wl, "cuda")
+    Q, K, V = Qd.cpu(), Kd.cpu(), Vd.cpu()
+    shape = binding.make_shape(H, d, wl.grid, 0, b)
+    ws = binding.make_workspace(shape, 2)
+    got = pu.gpu_block_mask(binding, shape, Qd, Kd, k, ws)
+    ref = oracle_mod.block_mask(Q, K, b, k, 0)
+    assert np.array_equal(pu.u32(got["mask"][0]), ref["mask"])
+    Od = torch.zeros_like(Qd)
+    lse = torch.zeros(1, H, wl.n_tokens, dtype=torch.float32, device="cuda")
+    binding.sparsp_sparse_attn_fwd(shape, Qd, Kd, Vd, got["mask"], 0.0, Od, lse, ws)
+    torch.cuda.synchronize()
+    assert binding.sparsp_status(ws) == binding.SPARSP_OK, binding.sparsp_last_error()
+    units = [(0, i) for i in (0, 1, 31, 32, 499, 500, 767, 998, 999)]
+    pu.check_attn_units(oracle_mod, Q, K, V, ref["mask"], b, Od, units, lse_gpu=lse[0])
+    assert bool(torch.isfinite(Od.float()).all())
+    assert bool((Od.float().abs().amax(dim=-1) > 0).all())
