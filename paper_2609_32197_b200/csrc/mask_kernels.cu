@@ -167,7 +167,7 @@ __global__ void __launch_bounds__(kScoreThreads) score_kernel(const float* __res
 
 // ------------------------------------------------------------------------------------------------
 // top-k: one warp per (batch, head, query block) row.  The row's scores become order-preserving
-// uint32 keys in shared memory; the warp finds the k-th largest key by a 32-step radix search with
+// uint32 keys in registers (lane l holds blocks l, l + 32, ...); the warp finds the k-th largest key by a 32-step radix search with
 // ballots/popcounts, breaks ties towards the lower index, forces the text blocks on, and emits the
 // mask words and the ascending kept list by ballot-prefix compaction.
 // ------------------------------------------------------------------------------------------------
@@ -179,23 +179,24 @@ __device__ __forceinline__ uint32_t score_key(float s) {
   return (u & 0x80000000u) ? ~u : (u | 0x80000000u);
 }
 
+template <int WMAX>  // mask words per row this instance can hold (keys live in registers: WMAX per lane)
 __global__ void __launch_bounds__(kTopkWarps * 32) topk_kernel(const float* __restrict__ scores, int64_t n_rows,
                                                                int NB, int Wd, int nb_cand, int topk,
                                                                int kept_cap, uint32_t* __restrict__ mask,
                                                                int32_t* __restrict__ kv_list,
                                                                int32_t* __restrict__ kv_count) {
-  extern __shared__ __align__(16) unsigned char smem_raw[];
-  const int NBpad = Wd * 32;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  uint32_t* keys = reinterpret_cast<uint32_t*>(smem_raw) + warp * NBpad;
   const int64_t row = (int64_t)blockIdx.x * kTopkWarps + warp;  // (batch*H + head) * NB + i
   if (row >= n_rows) return;
   const float* srow = scores + row * NB;
-  for (int t = 0; t < Wd; ++t) {
+  // lane l holds the keys of blocks l, l + 32, ...; a block that is not a candidate (text, padding) holds 0,
+  // which no trial threshold (>= 1) counts
+  uint32_t key[WMAX];
+#pragma unroll
+  for (int t = 0; t < WMAX; ++t) {
     const int j = t * 32 + lane;
-    keys[j] = j < NB ? score_key(__ldcs(srow + j)) : 0u;
+    key[t] = (t < Wd && j < nb_cand) ? score_key(__ldcs(srow + j)) : 0u;
   }
-  __syncwarp();
 
   const uint32_t lt_mask = (1u << lane) - 1u;
   // largest T with |{ candidates : key >= T }| >= topk  ==> T is the topk-th largest key
@@ -203,37 +204,35 @@ __global__ void __launch_bounds__(kTopkWarps * 32) topk_kernel(const float* __re
   for (int bit = 31; bit >= 0; --bit) {
     const uint32_t trial = T | (1u << bit);
     int c = 0;
-    for (int t = 0; t < Wd; ++t) {
-      const int j = t * 32 + lane;
-      c += (j < nb_cand && keys[j] >= trial) ? 1 : 0;
-    }
+#pragma unroll
+    for (int t = 0; t < WMAX; ++t) c += key[t] >= trial ? 1 : 0;
     c = __reduce_add_sync(0xffffffffu, c);
     if (c >= topk) T = trial;
   }
   int gt = 0;
-  for (int t = 0; t < Wd; ++t) {
-    const int j = t * 32 + lane;
-    gt += (j < nb_cand && keys[j] > T) ? 1 : 0;
-  }
+#pragma unroll
+  for (int t = 0; t < WMAX; ++t) gt += key[t] > T ? 1 : 0;
   gt = __reduce_add_sync(0xffffffffu, gt);
   const int need_eq = topk - gt;  // ties at T taken in ascending index order
   int eq_seen = 0, out_pos = 0;
-  for (int t = 0; t < Wd; ++t) {
-    const int j = t * 32 + lane;
-    const bool cand = j < nb_cand;
-    const uint32_t key = keys[j];
-    const bool is_eq = cand && key == T;
-    const uint32_t eq_ballot = __ballot_sync(0xffffffffu, is_eq);
-    const bool take_eq = is_eq && (eq_seen + __popc(eq_ballot & lt_mask) < need_eq);
-    eq_seen += __popc(eq_ballot);
-    const bool keep = (cand && key > T) || take_eq || (j >= nb_cand && j < NB);
-    const uint32_t word = __ballot_sync(0xffffffffu, keep);
-    if (lane == 0) mask[row * Wd + t] = word;
-    if (kv_list && keep) {
-      const int pos = out_pos + __popc(word & lt_mask);
-      if (pos < kept_cap) kv_list[row * kept_cap + pos] = j;
+#pragma unroll
+  for (int t = 0; t < WMAX; ++t) {
+    if (t < Wd) {
+      const int j = t * 32 + lane;
+      const bool cand = j < nb_cand;
+      const bool is_eq = cand && key[t] == T;
+      const uint32_t eq_ballot = __ballot_sync(0xffffffffu, is_eq);
+      const bool take_eq = is_eq && (eq_seen + __popc(eq_ballot & lt_mask) < need_eq);
+      eq_seen += __popc(eq_ballot);
+      const bool keep = (cand && key[t] > T) || take_eq || (j >= nb_cand && j < NB);
+      const uint32_t word = __ballot_sync(0xffffffffu, keep);
+      if (lane == 0) mask[row * Wd + t] = word;
+      if (kv_list && keep) {
+        const int pos = out_pos + __popc(word & lt_mask);
+        if (pos < kept_cap) kv_list[row * kept_cap + pos] = j;
+      }
+      out_pos += __popc(word);
     }
-    out_pos += __popc(word);
   }
   if (kv_count && lane == 0) kv_count[row] = out_pos;
 }
@@ -268,37 +267,41 @@ __device__ __forceinline__ float butterfly_sum(float v) {
   return v;
 }
 
+template <int WMAX>  // mask words per row this instance can hold (keys and terms live in registers)
 __global__ void __launch_bounds__(kTopkWarps * 32) cdf_kernel(const float* __restrict__ scores, int64_t n_rows, int NB,
                                                               int Wd, int nb_cand, float tau, float c,
                                                               uint32_t* __restrict__ mask,
                                                               int32_t* __restrict__ kv_count) {
-  extern __shared__ __align__(16) unsigned char smem_raw[];
-  const int NBpad = Wd * 32;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  uint32_t* keys = reinterpret_cast<uint32_t*>(smem_raw) + (size_t)warp * 2 * NBpad;
-  float* e = reinterpret_cast<float*>(keys + NBpad);
   const int64_t row = (int64_t)blockIdx.x * kTopkWarps + warp;  // (batch*H + head) * NB + i
   if (row >= n_rows) return;
   const float* srow = scores + row * NB;
+  // lane l holds blocks l, l + 32, ... in ascending order: exactly the terms of its partial sums.  A block that
+  // is not a candidate holds key 0 (no trial threshold, all >= 1, selects it) and the term 0.
+  uint32_t key[WMAX];
+  float e[WMAX];
   float mx = -INFINITY;
-  for (int t = 0; t < Wd; ++t) {
+#pragma unroll
+  for (int t = 0; t < WMAX; ++t) {
     const int j = t * 32 + lane;
-    const float s = j < nb_cand ? __ldcs(srow + j) : -INFINITY;
-    e[j] = s;
-    keys[j] = j < nb_cand ? score_key(s) : 0u;
+    const bool cand = t < Wd && j < nb_cand;
+    const float s = cand ? __ldcs(srow + j) : -INFINITY;
+    e[t] = s;
+    key[t] = cand ? score_key(s) : 0u;
     mx = fmaxf(mx, s);
   }
 #pragma unroll
   for (int s = 16; s >= 1; s >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, s));
   float acc = 0.0f;
-  for (int t = 0; t < Wd; ++t) {
+#pragma unroll
+  for (int t = 0; t < WMAX; ++t) {
     const int j = t * 32 + lane;
     float pj = 0.0f;
-    if (j < nb_cand) {
-      pj = exp2c(__fmul_rn(__fsub_rn(e[j], mx), c));
+    if (t < Wd && j < nb_cand) {
+      pj = exp2c(__fmul_rn(__fsub_rn(e[t], mx), c));
       acc = __fadd_rn(acc, pj);
     }
-    e[j] = pj;
+    e[t] = pj;
   }
   const float theta = __fmul_rn(tau, butterfly_sum(acc));
   // largest T with mass{ key >= T } >= theta
@@ -306,19 +309,20 @@ __global__ void __launch_bounds__(kTopkWarps * 32) cdf_kernel(const float* __res
   for (int bit = 31; bit >= 0; --bit) {
     const uint32_t trial = T | (1u << bit);
     float m = 0.0f;
-    for (int t = 0; t < Wd; ++t) {
-      const int j = t * 32 + lane;
-      if (j < nb_cand && keys[j] >= trial) m = __fadd_rn(m, e[j]);
-    }
+#pragma unroll
+    for (int t = 0; t < WMAX; ++t) m = key[t] >= trial ? __fadd_rn(m, e[t]) : m;
     if (butterfly_sum(m) >= theta) T = trial;
   }
   int cnt = 0;
-  for (int t = 0; t < Wd; ++t) {
-    const int j = t * 32 + lane;
-    const bool keep = (j < nb_cand && keys[j] >= T) || (j >= nb_cand && j < NB);
-    const uint32_t word = __ballot_sync(0xffffffffu, keep);
-    if (lane == 0) mask[row * Wd + t] = word;
-    cnt += __popc(word);
+#pragma unroll
+  for (int t = 0; t < WMAX; ++t) {
+    if (t < Wd) {
+      const int j = t * 32 + lane;
+      const bool keep = (j < nb_cand && key[t] >= T) || (j >= nb_cand && j < NB);
+      const uint32_t word = __ballot_sync(0xffffffffu, keep);
+      if (lane == 0) mask[row * Wd + t] = word;
+      cnt += __popc(word);
+    }
   }
   if (kv_count && lane == 0) kv_count[row] = cnt;
 }
@@ -335,11 +339,10 @@ int launch_score_cdf(const Geometry& g, const float* pq, const float* pk, float*
   }
   {
     const int64_t n_rows = (int64_t)g.B * g.H * g.NB;
-    const size_t smem = (size_t)kTopkWarps * 2 * g.Wd * 32 * 4;
     const float c = scale * 1.4426950408889634f;  // fp32 product, as in the definition above
-    SPARSP_CUDA_OK(ensure_dynamic_smem((const void*)cdf_kernel, (int)smem));
-    cdf_kernel<<<(unsigned)((n_rows + kTopkWarps - 1) / kTopkWarps), kTopkWarps * 32, smem, st>>>(
-        scores, n_rows, g.NB, g.Wd, g.nb_cand, tau, c, mask, kv_count);
+    const unsigned grid = (unsigned)((n_rows + kTopkWarps - 1) / kTopkWarps);
+    auto kern = g.Wd <= 4 ? cdf_kernel<4> : g.Wd <= 8 ? cdf_kernel<8> : g.Wd <= 16 ? cdf_kernel<16> : cdf_kernel<32>;
+    kern<<<grid, kTopkWarps * 32, 0, st>>>(scores, n_rows, g.NB, g.Wd, g.nb_cand, tau, c, mask, kv_count);
   }
   count_launch(2);
   SPARSP_CUDA_OK(cudaGetLastError());
@@ -359,9 +362,9 @@ int launch_score_topk(const Geometry& g, const float* pq, const float* pk, float
   }
   {
     const int64_t n_rows = (int64_t)g.B * g.H * g.NB;
-    const size_t smem = (size_t)kTopkWarps * g.Wd * 32 * 4;
-    topk_kernel<<<(unsigned)((n_rows + kTopkWarps - 1) / kTopkWarps), kTopkWarps * 32, smem, st>>>(
-        scores, n_rows, g.NB, g.Wd, g.nb_cand, topk, kept_cap, mask, kv_list, kv_count);
+    const unsigned grid = (unsigned)((n_rows + kTopkWarps - 1) / kTopkWarps);
+    auto kern = g.Wd <= 4 ? topk_kernel<4> : g.Wd <= 8 ? topk_kernel<8> : g.Wd <= 16 ? topk_kernel<16> : topk_kernel<32>;
+    kern<<<grid, kTopkWarps * 32, 0, st>>>(scores, n_rows, g.NB, g.Wd, g.nb_cand, topk, kept_cap, mask, kv_list, kv_count);
   }
   count_launch(2);
   SPARSP_CUDA_OK(cudaGetLastError());
