@@ -23,21 +23,37 @@ __global__ void own_kernel(const int32_t* __restrict__ rank, int NB, int Wd, int
   own[idx] = bits;
 }
 
-// U[b][r][h][w] = OR over the query blocks i of rank r of M[b][h][i][w].  One thread per output word.
-__global__ void union_kernel(const uint32_t* __restrict__ mask, const int32_t* __restrict__ rank,
-                             int B, int H, int NB, int Wd, int P, uint32_t* __restrict__ U) {
-  const int64_t idx = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
-  const int64_t total = (int64_t)B * P * H * Wd;
-  if (idx >= total) return;
-  const int w = (int)(idx % Wd);
-  const int h = (int)((idx / Wd) % H);
-  const int r = (int)((idx / ((int64_t)Wd * H)) % P);
-  const int bb = (int)(idx / ((int64_t)Wd * H * P));
-  const uint32_t* m = mask + ((int64_t)(bb * H + h) * NB) * Wd + w;
-  uint32_t acc = 0;
-  for (int i = 0; i < NB; ++i)
-    if (rank[i] == r) acc |= m[(int64_t)i * Wd];
-  U[idx] = acc;
+// U[b][r][h][w] = OR over the query blocks i of rank r of M[b][h][i][w].  One CTA per (batch, head): the head's
+// mask rows are read once, coalesced, and OR-ed into a [P][Wd] table in shared memory (at most 64 ranks x 32
+// words = 8 KiB); OR does not depend on the order, so the bits are well defined.  A rank value outside [0, P)
+// is ignored.
+constexpr int kUnionThreads = 256;
+static_assert(kMaxRanks * (kMaxBlocks / 32) * 4 <= 48 * 1024, "union table must fit static-size dynamic shared memory");
+
+__global__ void __launch_bounds__(kUnionThreads) union_kernel(const uint32_t* __restrict__ mask,
+                                                                   const int32_t* __restrict__ rank, int H, int NB,
+                                                                   int Wd, int P, uint32_t* __restrict__ U) {
+  extern __shared__ uint32_t u_s[];  // [P][Wd]
+  const int bh = blockIdx.x, bb = bh / H, h = bh % H;
+  for (int idx = threadIdx.x; idx < P * Wd; idx += kUnionThreads) u_s[idx] = 0u;
+  __syncthreads();
+  const uint32_t* m = mask + (int64_t)bh * NB * Wd;
+  for (int idx = threadIdx.x; idx < NB * Wd; idx += kUnionThreads) {
+    const int i = idx / Wd, w = idx - i * Wd;
+    const uint32_t v = m[idx];
+    const int r = rank[i];
+    if (v != 0u && (unsigned)r < (unsigned)P) atomicOr(&u_s[r * Wd + w], v);
+  }
+  __syncthreads();
+  for (int idx = threadIdx.x; idx < P * Wd; idx += kUnionThreads) {
+    const int r = idx / Wd, w = idx - r * Wd;
+    U[((int64_t)(bb * P + r) * H + h) * Wd + w] = u_s[idx];
+  }
+}
+
+static void launch_union(const uint32_t* mask, const int32_t* rank, const Geometry& g, int P, uint32_t* U,
+                         cudaStream_t st) {
+  union_kernel<<<g.B * g.H, kUnionThreads, (size_t)P * g.Wd * 4, st>>>(mask, rank, g.H, g.NB, g.Wd, P, U);
 }
 
 // cnt[b][r][p][h] = popcount(U[b][r][h] & own[p]).  One thread per output.
@@ -158,8 +174,7 @@ int launch_demand(const Geometry& g, const uint32_t* mask, const int32_t* rank_o
     return SPARSP_ERR_UNSUPPORTED;
   }
   own_kernel<<<(P * g.Wd + 127) / 128, 128, 0, st>>>(rank_of_block, g.NB, g.Wd, P, own);
-  const int64_t n_u = (int64_t)g.B * P * g.H * g.Wd;
-  union_kernel<<<(int)((n_u + 127) / 128), 128, 0, st>>>(mask, rank_of_block, g.B, g.H, g.NB, g.Wd, P, U);
+  launch_union(mask, rank_of_block, g, P, U, st);
   const int64_t n_c = (int64_t)g.B * P * P * g.H;
   count_kernel<<<(int)((n_c + 127) / 128), 128, 0, st>>>(U, own, g.B, g.H, g.Wd, P, cnt);
   scan_kernel<<<1, 1024, 0, st>>>(cnt, g.B, g.H, P, include_local, entry_bytes, seg_off, seg_total,
@@ -506,8 +521,7 @@ extern "C" SPARSP_API int sparsp_demand_plan_noalloc(const sparsp_shape* shape, 
   const int64_t entry_bytes = 2LL * g.b * g.d * 2;
   cudaStream_t st = (cudaStream_t)stream;
   own_kernel<<<(P * g.Wd + 127) / 128, 128, 0, st>>>(rank_of_block, g.NB, g.Wd, P, own);
-  const int64_t n_u = (int64_t)g.B * P * g.H * g.Wd;
-  union_kernel<<<(int)((n_u + 127) / 128), 128, 0, st>>>(mask, rank_of_block, g.B, g.H, g.NB, g.Wd, P, union_mask);
+  launch_union(mask, rank_of_block, g, P, union_mask, st);
   const int64_t n_c = (int64_t)g.B * P * P * g.H;
   count_kernel<<<(int)((n_c + 127) / 128), 128, 0, st>>>(union_mask, own, g.B, g.H, g.Wd, P, cnt);
   scan_kernel<<<1, 1024, 0, st>>>(cnt, g.B, g.H, P, include_local, entry_bytes, seg_offset, seg_total,

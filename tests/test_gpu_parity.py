@@ -388,3 +388,26 @@ def test_attention_near_the_largest_block_count(oracle_mod, binding, b, tokens_g
     pu.check_attn_units(oracle_mod, Q, K, V, ref["mask"], b, Od, units, lse_gpu=lse[0])
     assert bool(torch.isfinite(Od.float()).all())
     assert bool((Od.float().abs().amax(dim=-1) > 0).all())
+
+
+def test_demand_plan_with_the_most_ranks_and_blocks(oracle_mod, binding):
+    """64 virtual ranks (the limit) over 1000 blocks, scattered placement with one rank that owns nothing: the
+    per-head union table is at its largest; plan only, every integer against the oracle."""
+    H, NB, b, d, P = 2, 1000, 64, 64, 64
+    rng = np.random.default_rng(3)
+    M = rng.random((H, NB, NB)) < 0.004
+    M[:, np.arange(NB), np.arange(NB)] = True
+    bits = np.zeros((H, NB, 32 * 32), bool)
+    bits[:, :, :NB] = M
+    words = (bits.reshape(H, NB, 32, 32) * (1 << np.arange(32, dtype=np.uint64))).sum(-1).astype(np.uint32)
+    rank = rng.integers(0, P - 1, NB).astype(np.int32)  # rank P-1 owns no block
+    shape = binding.make_shape(H, d, (1, 1, NB * b), 0, b)
+    ws = binding.make_workspace(shape, P)
+    outs = binding.alloc_demand_outputs(shape, P)
+    mask_d = torch.as_tensor(words.view(np.int32)).cuda()[None]
+    binding.sparsp_demand_pack(shape, mask_d, torch.as_tensor(rank).cuda(), P, binding.SPARSP_PLAN_ONLY, None, None,
+                               outs["union_mask"], outs["cnt"], outs["seg_offset"], outs["seg_total"],
+                               outs["volume_bytes"], None, 0, None, ws)
+    torch.cuda.synchronize()
+    assert binding.sparsp_status(ws) == binding.SPARSP_OK
+    pu.check_demand(oracle_mod, binding, shape, words, rank, P, False, outs)
