@@ -9,33 +9,37 @@
 
 namespace sparsp {
 
-// own[p][w]: bit j set iff rank_of_block[j] == p.  One thread per (p, w).
-__global__ void own_kernel(const int32_t* __restrict__ rank, int NB, int Wd, int P,
-                           uint32_t* __restrict__ own) {
-  const int idx = blockIdx.x * blockDim.x + threadIdx.x;
-  if (idx >= P * Wd) return;
-  const int p = idx / Wd, w = idx % Wd;
-  uint32_t bits = 0;
-  for (int t = 0; t < 32; ++t) {
-    const int j = w * 32 + t;
-    if (j < NB && rank[j] == p) bits |= 1u << t;
-  }
-  own[idx] = bits;
-}
-
-// U[b][r][h][w] = OR over the query blocks i of rank r of M[b][h][i][w].  One CTA per (batch, head): the head's
-// mask rows are read once, coalesced, and OR-ed into a [P][Wd] table in shared memory (at most 64 ranks x 32
-// words = 8 KiB); OR does not depend on the order, so the bits are well defined.  A rank value outside [0, P)
-// is ignored.
+// One CTA per (batch, head) computes, for that head,
+//   own[p][w]     : bit j set iff rank_of_block[j] == p                      (CTA 0 also writes it out)
+//   U[b][r][h][w] = OR over the query blocks i of rank r of M[b][h][i][w]
+//   cnt[b][r][p][h] = popcount(U[b][r][h] & own[p])
+// The head's mask rows are read once, coalesced, and OR-ed into a [P][Wd] table in shared memory (at most
+// 64 ranks x 32 words = 8 KiB; OR does not depend on the order, so the bits are well defined); the ownership
+// words are rebuilt per CTA from the rank table (a few thousand compares) rather than fetched from an earlier
+// launch.  A rank value outside [0, P) is ignored.
 constexpr int kUnionThreads = 256;
-static_assert(kMaxRanks * (kMaxBlocks / 32) * 4 <= 48 * 1024, "union table must fit static-size dynamic shared memory");
+static_assert(2 * kMaxRanks * (kMaxBlocks / 32) * 4 <= 48 * 1024, "union and ownership tables must fit shared memory");
 
-__global__ void __launch_bounds__(kUnionThreads) union_kernel(const uint32_t* __restrict__ mask,
-                                                                   const int32_t* __restrict__ rank, int H, int NB,
-                                                                   int Wd, int P, uint32_t* __restrict__ U) {
-  extern __shared__ uint32_t u_s[];  // [P][Wd]
+__global__ void __launch_bounds__(kUnionThreads) union_count_kernel(const uint32_t* __restrict__ mask,
+                                                                    const int32_t* __restrict__ rank, int H, int NB,
+                                                                    int Wd, int P, uint32_t* __restrict__ own,
+                                                                    uint32_t* __restrict__ U,
+                                                                    int32_t* __restrict__ cnt) {
+  extern __shared__ uint32_t tab[];
+  uint32_t* u_s = tab;             // [P][Wd]
+  uint32_t* own_s = tab + P * Wd;  // [P][Wd]
   const int bh = blockIdx.x, bb = bh / H, h = bh % H;
-  for (int idx = threadIdx.x; idx < P * Wd; idx += kUnionThreads) u_s[idx] = 0u;
+  for (int idx = threadIdx.x; idx < P * Wd; idx += kUnionThreads) {
+    const int p = idx / Wd, w = idx - p * Wd;
+    uint32_t bits = 0;
+    for (int t = 0; t < 32; ++t) {
+      const int j = w * 32 + t;
+      if (j < NB && rank[j] == p) bits |= 1u << t;
+    }
+    own_s[idx] = bits;
+    u_s[idx] = 0u;
+    if (bh == 0) own[idx] = bits;
+  }
   __syncthreads();
   const uint32_t* m = mask + (int64_t)bh * NB * Wd;
   for (int idx = threadIdx.x; idx < NB * Wd; idx += kUnionThreads) {
@@ -49,28 +53,18 @@ __global__ void __launch_bounds__(kUnionThreads) union_kernel(const uint32_t* __
     const int r = idx / Wd, w = idx - r * Wd;
     U[((int64_t)(bb * P + r) * H + h) * Wd + w] = u_s[idx];
   }
+  for (int idx = threadIdx.x; idx < P * P; idx += kUnionThreads) {
+    const int r = idx / P, p = idx - r * P;
+    int c = 0;
+    for (int w = 0; w < Wd; ++w) c += __popc(u_s[r * Wd + w] & own_s[p * Wd + w]);
+    cnt[((int64_t)(bb * P + r) * P + p) * H + h] = c;
+  }
 }
 
-static void launch_union(const uint32_t* mask, const int32_t* rank, const Geometry& g, int P, uint32_t* U,
-                         cudaStream_t st) {
-  union_kernel<<<g.B * g.H, kUnionThreads, (size_t)P * g.Wd * 4, st>>>(mask, rank, g.H, g.NB, g.Wd, P, U);
-}
-
-// cnt[b][r][p][h] = popcount(U[b][r][h] & own[p]).  One thread per output.
-__global__ void count_kernel(const uint32_t* __restrict__ U, const uint32_t* __restrict__ own, int B,
-                             int H, int Wd, int P, int32_t* __restrict__ cnt) {
-  const int64_t idx = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
-  const int64_t total = (int64_t)B * P * P * H;
-  if (idx >= total) return;
-  const int h = (int)(idx % H);
-  const int p = (int)((idx / H) % P);
-  const int r = (int)((idx / ((int64_t)H * P)) % P);
-  const int bb = (int)(idx / ((int64_t)H * P * P));
-  const uint32_t* u = U + ((int64_t)(bb * P + r) * H + h) * Wd;
-  const uint32_t* o = own + (int64_t)p * Wd;
-  int c = 0;
-  for (int w = 0; w < Wd; ++w) c += __popc(u[w] & o[w]);
-  cnt[idx] = c;
+static void launch_union_count(const uint32_t* mask, const int32_t* rank, const Geometry& g, int P, uint32_t* own,
+                               uint32_t* U, int32_t* cnt, cudaStream_t st) {
+  union_count_kernel<<<g.B * g.H, kUnionThreads, (size_t)2 * P * g.Wd * 4, st>>>(mask, rank, g.H, g.NB, g.Wd, P, own,
+                                                                                 U, cnt);
 }
 
 // One thread per (b, r): exclusive scan of cnt over (p, h) in pack order, totals and volume; then
@@ -173,17 +167,15 @@ int launch_demand(const Geometry& g, const uint32_t* mask, const int32_t* rank_o
     set_error("batch * n_ranks = %d exceeds 1024", g.B * P);
     return SPARSP_ERR_UNSUPPORTED;
   }
-  own_kernel<<<(P * g.Wd + 127) / 128, 128, 0, st>>>(rank_of_block, g.NB, g.Wd, P, own);
-  launch_union(mask, rank_of_block, g, P, U, st);
+  launch_union_count(mask, rank_of_block, g, P, own, U, cnt, st);
   const int64_t n_c = (int64_t)g.B * P * P * g.H;
-  count_kernel<<<(int)((n_c + 127) / 128), 128, 0, st>>>(U, own, g.B, g.H, g.Wd, P, cnt);
   scan_kernel<<<1, 1024, 0, st>>>(cnt, g.B, g.H, P, include_local, entry_bytes, seg_off, seg_total,
                                   volume, ent_base, n_entries);
   entries_kernel<<<(int)((n_c * 32 + 255) / 256), 256, 0, st>>>(U, own, g.B, g.H, g.Wd, P,
                                                                include_local, entry_bytes, seg_off,
                                                                ent_base, dst_base, capacity, entries,
                                                                status);
-  count_launch(5);
+  count_launch(3);
   SPARSP_CUDA_OK(cudaGetLastError());
   return SPARSP_OK;
 }
@@ -520,13 +512,10 @@ extern "C" SPARSP_API int sparsp_demand_plan_noalloc(const sparsp_shape* shape, 
   const int include_local = (flags & SPARSP_INCLUDE_LOCAL) ? 1 : 0;
   const int64_t entry_bytes = 2LL * g.b * g.d * 2;
   cudaStream_t st = (cudaStream_t)stream;
-  own_kernel<<<(P * g.Wd + 127) / 128, 128, 0, st>>>(rank_of_block, g.NB, g.Wd, P, own);
-  launch_union(mask, rank_of_block, g, P, union_mask, st);
-  const int64_t n_c = (int64_t)g.B * P * P * g.H;
-  count_kernel<<<(int)((n_c + 127) / 128), 128, 0, st>>>(union_mask, own, g.B, g.H, g.Wd, P, cnt);
+  launch_union_count(mask, rank_of_block, g, P, own, union_mask, cnt, st);
   scan_kernel<<<1, 1024, 0, st>>>(cnt, g.B, g.H, P, include_local, entry_bytes, seg_offset, seg_total,
                                   volume_bytes, ent_base, n_entries);
-  count_launch(4);
+  count_launch(2);
   SPARSP_CUDA_OK(cudaGetLastError());
   return SPARSP_OK;
 }
