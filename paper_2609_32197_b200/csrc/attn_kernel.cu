@@ -865,7 +865,7 @@ __global__ void __launch_bounds__(kAttnThreads, 1)
 // is masked away.  Without `search`, D = 1 (neighbours).  One CTA per (batch, head).
 // ------------------------------------------------------------------------------------------------
 constexpr int kPairThreads = 256;
-constexpr int kPairSample = 4;
+constexpr int kPairSample = 8;
 
 // Sorts n keys (n a power of two, <= 1024) in shared memory into descending order; all kPairThreads threads call it.
 __device__ __forceinline__ void sort_keys_descending(uint32_t* keys, int n) {
