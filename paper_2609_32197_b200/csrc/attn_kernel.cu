@@ -195,6 +195,7 @@ __global__ void __launch_bounds__(kAttnThreads, 1)
   int* s_item = reinterpret_cast<int*>(smem + C::kOffMisc + 32);  // [2] the work item of each list buffer; < 0 = no more
   int* s_rag = reinterpret_cast<int*>(smem + C::kOffMisc + 40);   // [2] the item's last tile reaches past the end of the sequence
   volatile int* s_frz = reinterpret_cast<volatile int*>(smem + C::kOffMisc + 56);  // [4] per row group: reference frozen
+  volatile int* s_pv_items = reinterpret_cast<volatile int*>(smem + C::kOffMisc + 72);  // items whose P V are all issued
   float* s_knmax = reinterpret_cast<float*>(smem + C::kOffMisc + 48);  // [2] largest key norm bound among the item's entries
   constexpr int kListReaders = 12;  // two producers, two issuers, eight softmax warps
 
@@ -226,6 +227,7 @@ __global__ void __launch_bounds__(kAttnThreads, 1)
     mbar_init(o_drained, 8);
     mbar_init_fence();
     *s_abort = 0;
+    *s_pv_items = 0;
     for (int r = 0; r < 4; ++r) s_frz[r] = 0;
   }
   if (tid < 384) sRef[tid] = -INFINITY;  // 3 x 128 entries
@@ -367,6 +369,20 @@ __global__ void __launch_bounds__(kAttnThreads, 1)
         if (s_item[buf] < 0) break;
         const int n_tiles = (s_nent[buf] + C::kEPT - 1) / C::kEPT;
         if (n_tiles > 0) {
+          // The tensor pipe works in issue order.  The first Q K^T of an item could be issued a tile or two
+          // before the previous item ends, ahead of that item's last P V, and the epilogue (which waits for
+          // that P V) would start ~1000 cycles later for nothing: the scores are not needed before the
+          // epilogue is over.  So they wait until the previous item's P V are all issued.
+          if (i > 0) {
+            const long long t0 = clock64();
+            while (*s_pv_items < i) {
+              if (*s_abort) break;
+              if (clock64() - t0 > p.wait_limit) {
+                *s_abort = 14;
+                break;
+              }
+            }
+          }
           mbar_wait_bounded_inline(q_full, qc & 1, s_abort, 11, p.wait_limit);
           ++qc;
           for (int n = 0; n < n_tiles; ++n, ++g) {
@@ -423,7 +439,10 @@ __global__ void __launch_bounds__(kAttnThreads, 1)
           }
           __syncwarp();
         }
-        if (lane == 0) mbar_arrive(list_free + buf);
+        if (lane == 0) {
+          *s_pv_items = i + 1;
+          mbar_arrive(list_free + buf);
+        }
         __syncwarp();
       }
     }
