@@ -33,7 +33,7 @@ NOMINAL = {"hbm_gbs": 8000.0, "bf16_tflops": 2250.0}
 # dram__bytes_read.sum + dram__bytes_write.sum per launch of the attention kernel, from the ncu
 # captures summarised under profiles/ (None = not captured for that workload).
 ATTN_DRAM_TRAFFIC = {
-    ("mid", 58): 590.3e6,            # profiles/attn_fwd_kernel_mid_and_hunyuan4.md, full workload
+    ("mid", 58): 591.0e6,            # profiles/attn_fwd_kernel_mid_and_hunyuan4.md, full workload
     ("hunyuan", 93): 6 * 710.0e6,     # same file: 4-head capture scaled by heads (24 / 4)
 }
 
