@@ -411,3 +411,39 @@ def test_demand_plan_with_the_most_ranks_and_blocks(oracle_mod, binding):
     torch.cuda.synchronize()
     assert binding.sparsp_status(ws) == binding.SPARSP_OK
     pu.check_demand(oracle_mod, binding, shape, words, rank, P, False, outs)
+
+
+@pytest.mark.parametrize("seed", [1, 2, 3, 4, 5, 6])
+def test_random_norm_profiles(oracle_mod, binding, seed):
+    """Random shapes with key blocks and query rows scaled by random factors (0.1 ... 20): tiles whose norm
+    bound holds, tiles where it fails, references that become final early, late or never, all in one launch."""
+    rng = np.random.default_rng(100 + seed)
+    d = int(rng.choice([64, 128]))
+    b = int(rng.choice([64, 128]))
+    H = 2
+    NB = int(rng.integers(18, 30))
+    N = NB * b - int(rng.integers(0, b - 1))
+    keep_n = int(rng.integers(6, 16))
+    Qf = rng.standard_normal((H, N, d)) * np.exp(rng.uniform(np.log(0.1), np.log(4.0), (H, N, 1)))
+    Kf = rng.standard_normal((H, N, d))
+    for j in range(NB):
+        Kf[:, j * b:(j + 1) * b] *= np.exp(rng.uniform(np.log(0.1), np.log(20.0 if j % 5 == 0 else 2.0)))
+    Q = torch.tensor(Qf).to(torch.bfloat16)
+    K = torch.tensor(Kf).to(torch.bfloat16)
+    V = torch.tensor(rng.standard_normal((H, N, d)) * 0.5).to(torch.bfloat16)
+    Wd = (NB + 31) // 32
+    words = np.zeros((H, NB, Wd), np.uint32)
+    for h in range(H):
+        for i in range(NB):
+            for j in rng.choice(NB, keep_n, replace=False):
+                words[h, i, j >> 5] |= np.uint32(1 << (int(j) & 31))
+    shape = binding.make_shape(H, d, (1, 1, N), 0, b)
+    ws = binding.make_workspace(shape, 2)
+    Qd, Kd, Vd = Q.cuda(), K.cuda(), V.cuda()
+    O = torch.zeros_like(Qd)
+    lse = torch.zeros(1, H, N, dtype=torch.float32, device="cuda")
+    binding.sparsp_sparse_attn_fwd(shape, Qd, Kd, Vd, torch.as_tensor(words.view(np.int32)).cuda(), 0.0, O, lse, ws)
+    torch.cuda.synchronize()
+    assert binding.sparsp_status(ws) == binding.SPARSP_OK
+    units = [(h, i) for h in range(H) for i in range(NB)]
+    pu.check_attn_units(oracle_mod, Q, K, V, words, b, O, units, lse_gpu=lse[0])
