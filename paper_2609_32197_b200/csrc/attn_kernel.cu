@@ -28,6 +28,12 @@
 // Online softmax is base-2 in fp32; O is rescaled lazily, only when a row's maximum has grown by more
 // than 2^8 since the reference last moved -- the thread that decides so first waits for every P V
 // issued so far, then rescales the row of O.
+// Norm bounds shorten most tiles: |q_row| * (largest key norm of a block) * scale bounds the block's scores, so
+// a tile whose bound stays within 2^64 of the row's reference skips its row-maximum pass, and once the bound
+// with the item's largest key norm holds, the reference is final and the two warps of a row group stop taking
+// turns for the rest of the item (load scores -> exponentials -> store P).
+// The block-64 pairing and the order of a head's items (longest list first) come from attn_prep_kernel,
+// which also takes the key norms.
 // Every mbarrier wait is bounded; a wait that runs out sets SPARSP_ERR_TIMEOUT in the status word
 // and raises a CTA-wide flag that makes all later waits fall through, so the CTA still drains.
 #include <algorithm>
@@ -42,8 +48,8 @@ using namespace ptx;
 
 struct AttnParams {
   const uint32_t* mask;
-  // block 64: [B*H][ceil(NB/2)][2] query blocks of each item (second may be -1); block 128: NULL (item x
-  // handles block x) or [B*H][2*ceil(NB/2)] query block of each item (-1 = none)
+  // block 64: [B*H][ceil(NB/2)][2] query blocks of each item (second may be -1); block 128:
+  // [B*H][2*ceil(NB/2)] query block of each item (-1 = none), or NULL (item x handles block x)
   const int32_t* pairs;
   // packed-source mode (NULL = every tile comes from K / V): slot[bh][j] = entry index of KV block j in
   // the consumer's packed buffer, or -1 if the consumer owns the block; tile_base = index of the
