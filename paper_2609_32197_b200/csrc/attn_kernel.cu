@@ -7,7 +7,7 @@
 //                kept lists (128 keys, full-rate N = 128); each 64x64 quadrant the mask does not keep is
 //                zeroed in P.
 // The kernel is persistent: one CTA per SM takes items from a global counter; the next item's kept
-// list, Q tile, first K/V tiles and first Q K^T overlap the current item's last tiles and its epilogue.
+// list, Q tile and first K/V tiles overlap the current item's last tiles, its first Q K^T the epilogue.
 // The scores S = Q K^T and the probabilities P are double-buffered in tensor memory (S: 2 x 128 fp32
 // columns, P: 2 x 64 columns of packed bf16, O: d columns), so that the tensor pipe always has the next
 // tiles' MMAs queued while the softmax of the current tile runs: Q K^T of tile g+2 starts as soon as the
