@@ -490,11 +490,13 @@ __global__ void __launch_bounds__(kAttnThreads, 1)
         // NB <= 1024, so a mask row is at most 32 words: one word per lane
         const uint32_t rb0 = (lane < p.Wd && blk[0] >= 0) ? p.mask[((int64_t)bh * p.NB + blk[0]) * p.Wd + lane] : 0u;
         const uint32_t rb1 = (lane < p.Wd && blk[1] >= 0) ? p.mask[((int64_t)bh * p.NB + blk[1]) * p.Wd + lane] : 0u;
-        // Entry order (any order gives the same attention): first the blocks BOTH query blocks keep, then the
-        // blocks only the first keeps alternating with the blocks only the second keeps, then what is left of
-        // the longer of those two lists.  A tile is two consecutive entries, so a tile of the middle part costs
-        // every softmax row one 64-key half instead of costing half of the rows two.  With a single query
-        // block this is plain ascending order.
+        // Entry order (any order gives the same attention).  Blocks BOTH query blocks keep make full tiles; a
+        // block only the first keeps is put next to a block only the second keeps, so that such a tile costs
+        // every softmax row one 64-key half instead of costing half of the rows two.  A full tile is bound by
+        // the softmax warps, a half-work tile by the tensor pipe (its MMAs cost the same), so the two kinds
+        // alternate in groups of two tiles (one of each per softmax warpgroup) while both last; then the rest
+        // of the full tiles, the rest of the paired one-sided blocks and what is left of the longer one-sided
+        // list.  With a single query block this is plain ascending order.
         uint32_t cls[3] = {rb0 & rb1, rb0 & ~rb1, rb1 & ~rb0};
         int before[3], total[3];
 #pragma unroll
@@ -510,6 +512,8 @@ __global__ void __launch_bounds__(kAttnThreads, 1)
           total[c] = __shfl_sync(0xffffffffu, incl, 31);
         }
         const int n_both = total[0], n_mix = min(total[1], total[2]);
+        // two full tiles (four blocks both keep), then two half-work tiles (two one-sided pairs), and so on
+        const int n_grp = min(n_both >> 2, n_mix >> 1);
         const int running = total[0] + total[1] + total[2];
         float kn_max = 0.0f;
 #pragma unroll
@@ -520,7 +524,8 @@ __global__ void __launch_bounds__(kAttnThreads, 1)
             const int t = __ffs(u) - 1;
             u &= u - 1;
             int pos;
-            if (c == 0) pos = idx;
+            if (c == 0) pos = idx < 4 * n_grp ? 8 * (idx >> 2) + (idx & 3) : 4 * n_grp + idx;
+            else if (idx < 2 * n_grp) pos = 8 * (idx >> 1) + 4 + 2 * (idx & 1) + (c - 1);
             else if (idx < n_mix) pos = n_both + 2 * idx + (c - 1);
             else pos = n_both + n_mix + idx;  // tail of the longer class
             entJ[pos] = (uint16_t)(lane * 32 + t);
