@@ -86,6 +86,11 @@ constexpr float kSkipMargin = 64.0f;  // 2^64 * (keys of a sequence) * |V| stays
 #ifndef SPARSP_TUNE_POLY
 #define SPARSP_TUNE_POLY 4
 #endif
+// ... at d = 64, where the row sum is taken by the tensor pipe and the FMA pipe has more room (measured: every
+// 3rd pair is 3 % faster than every 4th there, every 2nd 4 % slower)
+#ifndef SPARSP_TUNE_POLY_D64
+#define SPARSP_TUNE_POLY_D64 3
+#endif
 
 template <int D, int BLK>
 struct AttnCfg {
@@ -98,7 +103,14 @@ struct AttnCfg {
   static constexpr int kOffQ = 0;
   static constexpr int kOffK = kOffQ + kQBytes;
   static constexpr int kOffV = kOffK + kStagesK * kTileBytes;
-  static constexpr int kOffEntJ = kOffV + kStagesV * kTileBytes;  // uint16 [2][1024] kept / union list
+  // d = 64 leaves room in tensor memory for 16 more accumulator columns: P V then runs with N = 80, its B
+  // operand continuing, 64 columns on, into a constant [128 keys][column 64 = 1, the rest 0] block in shared
+  // memory, so that accumulator column 64 is the row sum of P -- taken by the tensor pipe from the very
+  // bf16 values it multiplies with V, instead of one more packed add per pair of scores in the softmax warps
+  static constexpr bool kOnes = (D == 64);
+  static constexpr int kAccCols = D + (kOnes ? 16 : 0);
+  static constexpr int kOffOnes = kOffV + kStagesV * kTileBytes;  // bf16 [128][64], 128-byte swizzle like a V box
+  static constexpr int kOffEntJ = kOffOnes + (kOnes ? 128 * 128 : 0);  // uint16 [2][1024] kept / union list
   static constexpr int kOffEntV = kOffEntJ + 2 * 2 * kMaxBlocks;  // uint8 [2][1024][2] keys of the entry valid for query block q (0 = not kept)
   static constexpr int kOffSlot = kOffEntV + 2 * 2 * kMaxBlocks;  // int32 [2][1024] packed-buffer slot per entry
   static constexpr int kOffEntN = kOffSlot + 2 * 4 * kMaxBlocks;  // float [2][1024] largest key norm of the entry's block
@@ -237,6 +249,15 @@ __global__ void __launch_bounds__(kAttnThreads, 1)
     for (int r = 0; r < 4; ++r) s_frz[r] = 0;
   }
   if (tid < 384) sRef[tid] = -INFINITY;  // 3 x 128 entries
+  if (C::kOnes) {
+    // key row r holds column 64 + c at byte r*128 + ((c/8 ^ (r & 7)) << 4) + (c%8)*2 (the swizzle of a TMA box)
+    uint4* ones = reinterpret_cast<uint4*>(smem + C::kOffOnes);
+    for (int idx = tid; idx < 128 * 8; idx += kAttnThreads) {
+      const int r = idx >> 3, chunk = idx & 7;
+      ones[idx] = make_uint4(chunk == (r & 7) ? 0x3F80u : 0u, 0u, 0u, 0u);  // bf16 1.0 in element 0 of logical chunk 0
+    }
+    fence_proxy_async_smem();  // read by the tensor pipe
+  }
   if (warp == 1) {
     tmem_alloc(s_tmem, kTmemCols);
     tmem_relinquish();
@@ -415,8 +436,10 @@ __global__ void __launch_bounds__(kAttnThreads, 1)
     } else {
       // ================================ P V issuer ==========================================
       const bool leader = elect_one();
-      constexpr uint32_t kIdescPV = make_idesc_bf16(128, D, 0, 1);
-      const uint64_t descV = make_smem_desc(smem_u32(sV), 16384, 1024);
+      constexpr uint32_t kIdescPV = make_idesc_bf16(128, C::kAccCols, 0, 1);
+      // second 64-column group of the B operand: the other half of a d = 128 tile, or the block of ones, which
+      // lies kOffOnes - kOffV behind the FIRST stage (the stage offset is taken off again below)
+      const uint64_t descV = make_smem_desc(smem_u32(sV), C::kOnes ? (uint32_t)(C::kOffOnes - C::kOffV) : 16384u, 1024);
       const uint32_t hiV = (uint32_t)(descV >> 32);
       uint32_t vlo[8];
 #pragma unroll
@@ -434,7 +457,8 @@ __global__ void __launch_bounds__(kAttnThreads, 1)
           mbar_wait_bounded_inline(p_full + (g & 1), (g >> 1) & 1, s_abort, 20, p.wait_limit);
           mbar_wait_bounded_inline(v_full + g % SV, (g / SV) & 1, s_abort, 22, p.wait_limit);
           tc_fence_after();
-          const uint32_t stage_off = (uint32_t)(((g % SV) * C::kTileBytes) >> 4);
+          uint32_t stage_off = (uint32_t)(((g % SV) * C::kTileBytes) >> 4);
+          if (C::kOnes) stage_off -= stage_off << 16;  // start address up, distance to the ones block down
           const uint32_t tP = tmem_base + C::kColP + (g & 1) * 64;
           if (leader) {
 #pragma unroll
@@ -737,7 +761,7 @@ __global__ void __launch_bounds__(kAttnThreads, 1)
                 mbar_wait_bounded_inline(o_full + ((g - 1) & 3), ((g - 1) >> 2) & 1, s_abort, 38, p.wait_limit);
                 tc_fence_after();
 #pragma unroll 1
-                for (int c = 0; c < D / 16; ++c) {  // the row's accumulator, 16 columns at a time (rare: kept small)
+                for (int c = 0; c < C::kAccCols / 16; ++c) {  // the row's accumulator, 16 columns at a time (rare: kept small)
                   uint32_t o[16];
                   tmem_ld16(tO + c * 16, o);
                   tmem_ld_wait();
@@ -773,10 +797,11 @@ __global__ void __launch_bounds__(kAttnThreads, 1)
 #pragma unroll
             for (int e = 0; e < 32; ++e) {
               const float2 x = ffma2(make_float2(svh[2 * e], svh[2 * e + 1]), sc2, nm2);
-              const float2 pp = (SPARSP_TUNE_POLY > 0 && (e % (SPARSP_TUNE_POLY > 0 ? SPARSP_TUNE_POLY : 1)) == 1)
+              constexpr int kPoly = C::kOnes ? SPARSP_TUNE_POLY_D64 : SPARSP_TUNE_POLY;
+              const float2 pp = (kPoly > 0 && (e % (kPoly > 0 ? kPoly : 1)) == 1)
                                     ? exp2_poly2(x)
                                     : make_float2(ex2(x.x), ex2(x.y));
-              lsum2 = fadd2(lsum2, pp);
+              if (!C::kOnes) lsum2 = fadd2(lsum2, pp);
               const __nv_bfloat162 h2 = __floats2bfloat162_rn(pp.x, pp.y);
               pkh[e] = *reinterpret_cast<const uint32_t*>(&h2);
             }
@@ -829,7 +854,16 @@ __global__ void __launch_bounds__(kAttnThreads, 1)
         // this reference buffer serves the item after next: no warp can be there before every warp has passed
         // the barrier above, and the item before this one (its last user) is finished for all of them
         sRef[((i + 2) % 3) * 128 + row] = -INFINITY;
-        const float l = (st0.y > 0.0f ? st0.y * ex2(st0.x - m_fin) : 0.0f) + (st1.y > 0.0f ? st1.y * ex2(st1.x - m_fin) : 0.0f);
+        float l = (st0.y > 0.0f ? st0.y * ex2(st0.x - m_fin) : 0.0f) + (st1.y > 0.0f ? st1.y * ex2(st1.x - m_fin) : 0.0f);
+        if (C::kOnes) {  // the row sum is accumulator column d (CTA-uniform branch: the load is warp-collective)
+          l = 0.0f;
+          if (n_tiles > 0) {
+            uint32_t sums[16];
+            tmem_ld16(tO + D, sums);
+            tmem_ld_wait();
+            l = __uint_as_float(sums[0]);
+          }
+        }
         const float inv_l = l > 0.0f ? 1.0f / l : 0.0f;
         const int qb = C::kStacked ? s_blk[buf * 2 + rh] : s_blk[buf * 2];
         const int64_t tok = qb >= 0 ? (int64_t)qb * BLK + (C::kStacked ? (row & 63) : row) : p.N;
