@@ -294,6 +294,41 @@ def pack(K, V, U: np.ndarray, rank_of_block: np.ndarray, b: int, P: int, total: 
     return out
 
 
+def exchange_plan(cnt: np.ndarray, seg_off: np.ndarray, b: int, d: int, steady_chunks: int = 1,
+                  tail_chunks: int = 1, w_bytes: int = 2):
+    """The transfer list of the demand-routed exchange for one batch item, written out from the paper's
+    description (plain loops; cnt and seg_off as returned by demand() without include_local):
+      * Section 5.1: in round k = 0 .. P-2 every consumer r receives from the producer at ring distance k+1,
+        p = (r - (k+1)) mod P, exactly the blocks it selected from that producer;
+      * Section 5.2 / 6: the blocks of one (consumer, producer) pair are one contiguous run of the consumer's
+        buffer, heads ascending, so both ends derive every byte range from the demand counts alone;
+      * Section 7.1: a hop is cut into chunks of contiguous heads, `steady_chunks` of them in every round but
+        the last, `tail_chunks` in the last (never more chunks than heads; chunk c starts at head c*H // C);
+      * Section 7.2: the chunks of a hop go in descending order of their number of kept blocks (ties: lower
+        head first), so that the sparsest chunk, whose attention is the shortest, comes last.
+    -> list of dicts (consumer, producer, round, order, head_begin, head_end, entry_begin, n_entries,
+       byte_offset, n_bytes), sorted by consumer, round, order; offsets relative to the consumer's buffer."""
+    P, _, H = cnt.shape
+    entry = 2 * b * d * w_bytes
+    out = []
+    for r in range(P):
+        for k in range(P - 1):
+            p = (r - (k + 1)) % P
+            C = tail_chunks if k == P - 2 else steady_chunks
+            C = max(1, min(C, H))
+            chunks = []
+            for c in range(C):
+                h0, h1 = (c * H) // C, ((c + 1) * H) // C
+                n = int(sum(int(cnt[r, p, h]) for h in range(h0, h1)))
+                chunks.append((h0, h1, n))
+            chunks.sort(key=lambda t: (-t[2], t[0]))
+            for order, (h0, h1, n) in enumerate(chunks):
+                e0 = int(seg_off[r, p, h0])
+                out.append(dict(consumer=r, producer=p, round=k, order=order, head_begin=h0, head_end=h1,
+                                entry_begin=e0, n_entries=n, byte_offset=e0 * entry, n_bytes=n * entry))
+    return out
+
+
 # ---------------------------------------------------------------------------------------------
 # step 3
 # ---------------------------------------------------------------------------------------------
