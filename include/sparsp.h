@@ -241,6 +241,32 @@ SPARSP_API int sparsp_hop_mask(const sparsp_shape* shape, const uint32_t* mask, 
 SPARSP_API int sparsp_attn_merge(const sparsp_shape* shape, const void* O_a, const float* lse_a, const void* O_b,
                                  const float* lse_b, void* O, float* lse, void* stream);
 
+/* The transfer list of the demand-routed exchange, derived from the demand counts alone (host arithmetic, no
+ * GPU work).  Section 5.1: in round k = 0 .. P-2 consumer r receives from the producer at ring distance
+ * k+1, p = (r - (k+1)) mod P, exactly the blocks it selected there.  Sections 5.2 / 6: those blocks are one
+ * contiguous run of the consumer's buffer (heads ascending), so producer and consumer compute the same byte
+ * ranges without exchanging any descriptor.  Section 7.1: a hop is cut into chunks of contiguous heads,
+ * `steady_chunks` in every round but the last and `tail_chunks` in the last (never more than heads; chunk c
+ * of C starts at head c*H/C).  Section 7.2: the chunks of a hop are listed in descending order of their
+ * number of kept blocks (ties: lower head first), the sparsest last.
+ *   cnt, seg_offset   in   HOST copies of sparsp_demand_pack's outputs (made WITHOUT SPARSP_INCLUDE_LOCAL),
+ *                          int32 / int64 [B][P][P][H]
+ *   transfers         out  HOST [capacity]; sorted by batch, consumer, round, order; a chunk without blocks is
+ *                          listed with n_bytes = 0.  Offsets are relative to the consumer's buffer.
+ *   n_transfers       out  B * P * sum over rounds of that round's chunk count (written even if the list does
+ *                          not fit, in which case the call returns SPARSP_ERR_CAPACITY and writes nothing else) */
+typedef struct sparsp_transfer {
+  int32_t batch, consumer, producer, round; /* round = ring distance - 1 */
+  int32_t order;                            /* position inside its hop */
+  int32_t head_begin, head_end;             /* heads [head_begin, head_end) */
+  int32_t reserved;
+  int64_t entry_begin, n_entries;           /* entries (K tile + V tile of one block) of the consumer's buffer */
+  int64_t byte_offset, n_bytes;             /* the same run in bytes */
+} sparsp_transfer;
+SPARSP_API int sparsp_exchange_plan(const sparsp_shape* shape, int32_t n_ranks, const int32_t* cnt,
+                                    const int64_t* seg_offset, int32_t steady_chunks, int32_t tail_chunks,
+                                    sparsp_transfer* transfers, int64_t capacity, int64_t* n_transfers);
+
 /* Planning without any allocation.  (No counterpart in the paper: an engineering variant of the
  * planning half of sparsp_demand_pack.)
  * For callers that are not allowed to allocate device memory -- for example a plug-in running inside a

@@ -30,7 +30,7 @@ EXPORTS = [
     "sparsp_workspace_bytes", "sparsp_block_mask", "sparsp_demand_pack", "sparsp_sparse_attn_fwd",
     "sparsp_status", "sparsp_last_error", "sparsp_launch_count", "sparsp_demand_plan_noalloc",
     "sparsp_hop_mask", "sparsp_attn_merge", "sparsp_sparse_attn_fwd_packed", "sparsp_block_mask_cdf",
-    "sparsp_placement_permutation", "sparsp_permute_tokens", "sparsp_sharing_histogram",
+    "sparsp_placement_permutation", "sparsp_permute_tokens", "sparsp_sharing_histogram", "sparsp_exchange_plan",
 ]
 
 
@@ -148,6 +148,29 @@ def sparsp_placement_permutation(shape: sparsp_shape, n_ranks: int, rank_of_bloc
                                               ctypes.c_void_p(rank.data_ptr()), ctypes.c_void_p(bos.data_ptr()),
                                               ctypes.c_void_p(off.data_ptr()), ctypes.c_void_p(first.data_ptr())))
     return bos, off, first
+
+
+class sparsp_transfer(ctypes.Structure):
+    _fields_ = [("batch", ctypes.c_int32), ("consumer", ctypes.c_int32), ("producer", ctypes.c_int32),
+                ("round", ctypes.c_int32), ("order", ctypes.c_int32), ("head_begin", ctypes.c_int32),
+                ("head_end", ctypes.c_int32), ("reserved", ctypes.c_int32), ("entry_begin", ctypes.c_int64),
+                ("n_entries", ctypes.c_int64), ("byte_offset", ctypes.c_int64), ("n_bytes", ctypes.c_int64)]
+
+
+def sparsp_exchange_plan(shape: sparsp_shape, n_ranks: int, cnt: torch.Tensor, seg_offset: torch.Tensor,
+                         steady_chunks: int = 1, tail_chunks: int = 1):
+    """-> list of sparsp_transfer (host).  cnt / seg_offset: sparsp_demand_pack's outputs (any device)."""
+    c = cnt.to(torch.int32).cpu().contiguous()
+    o = seg_offset.to(torch.int64).cpu().contiguous()
+    n = ctypes.c_int64(0)
+    args = (ctypes.byref(shape), ctypes.c_int32(n_ranks), ctypes.c_void_p(c.data_ptr()),
+            ctypes.c_void_p(o.data_ptr()), ctypes.c_int32(steady_chunks), ctypes.c_int32(tail_chunks))
+    rc = lib().sparsp_exchange_plan(*args, None, ctypes.c_int64(0), ctypes.byref(n))
+    if rc not in (SPARSP_OK, SPARSP_ERR_CAPACITY):
+        _check(rc)
+    buf = (sparsp_transfer * max(n.value, 1))()
+    _check(lib().sparsp_exchange_plan(*args, buf, ctypes.c_int64(n.value), ctypes.byref(n)))
+    return list(buf[:n.value])
 
 
 def sparsp_permute_tokens(shape, X, Y, block_of_slot, token_offset_of_slot, inverse):

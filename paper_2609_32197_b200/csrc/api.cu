@@ -255,6 +255,52 @@ int sparsp_sharing_histogram(const sparsp_shape* shape, const uint32_t* mask, co
   return launch_sharing(g, mask, rank_of_block, n_ranks, hist, (cudaStream_t)stream);
 }
 
+int sparsp_exchange_plan(const sparsp_shape* shape, int32_t n_ranks, const int32_t* cnt, const int64_t* seg_offset,
+                         int32_t steady_chunks, int32_t tail_chunks, sparsp_transfer* transfers, int64_t capacity,
+                         int64_t* n_transfers) {
+  Geometry g;
+  SPARSP_TRY(make_geometry(shape, &g));
+  if (n_ranks < 1 || n_ranks > kMaxRanks || !cnt || !seg_offset || !n_transfers || capacity < 0 ||
+      (capacity > 0 && !transfers) || steady_chunks < 1 || tail_chunks < 1) {
+    set_error("bad n_ranks, chunk count, capacity or NULL argument");
+    return SPARSP_ERR_INVALID_ARG;
+  }
+  const int P = n_ranks, H = g.H;
+  const int c_steady = std::min(steady_chunks, H), c_tail = std::min(tail_chunks, H);
+  const int64_t per_consumer = P > 1 ? (int64_t)(P - 2) * c_steady + c_tail : 0;
+  *n_transfers = (int64_t)g.B * P * per_consumer;
+  if (*n_transfers > capacity) {
+    set_error("transfer list needs %lld records, capacity %lld", (long long)*n_transfers, (long long)capacity);
+    return SPARSP_ERR_CAPACITY;
+  }
+  const int64_t entry_bytes = 2LL * g.b * g.d * 2;
+  sparsp_transfer* out = transfers;
+  for (int bb = 0; bb < g.B; ++bb)
+    for (int r = 0; r < P; ++r)
+      for (int k = 0; k + 1 < P; ++k) {
+        const int p = ((r - (k + 1)) % P + P) % P;
+        const int C = k == P - 2 ? c_tail : c_steady;
+        const int32_t* c_row = cnt + (((int64_t)bb * P + r) * P + p) * H;
+        const int64_t* o_row = seg_offset + (((int64_t)bb * P + r) * P + p) * H;
+        sparsp_transfer* hop = out;
+        for (int c = 0; c < C; ++c) {
+          const int h0 = (int)(((int64_t)c * H) / C), h1 = (int)(((int64_t)(c + 1) * H) / C);
+          int64_t n = 0;
+          for (int h = h0; h < h1; ++h) n += c_row[h];
+          sparsp_transfer t;
+          t.batch = bb; t.consumer = r; t.producer = p; t.round = k; t.order = 0;
+          t.head_begin = h0; t.head_end = h1; t.reserved = 0;
+          t.entry_begin = o_row[h0]; t.n_entries = n;
+          t.byte_offset = t.entry_begin * entry_bytes; t.n_bytes = n * entry_bytes;
+          *out++ = t;
+        }
+        // most blocks first, lower head first among equals (the chunks were produced in head order)
+        std::stable_sort(hop, out, [](const sparsp_transfer& a, const sparsp_transfer& b) { return a.n_entries > b.n_entries; });
+        for (int c = 0; c < C; ++c) hop[c].order = c;
+      }
+  return SPARSP_OK;
+}
+
 int sparsp_workspace_bytes(const sparsp_shape* shape, int32_t n_ranks, int64_t* bytes) {
   Geometry g;
   SPARSP_TRY(make_geometry(shape, &g));

@@ -190,3 +190,75 @@ def test_packed_attention_rejects_bad_arguments(binding):
         with pytest.raises(RuntimeError):
             binding.sparsp_sparse_attn_fwd_packed(shape, z, z, z, z, z, 2, consumer, z, z, z, z, cap, None, 0.0, z,
                                                   None, ws)
+
+
+@pytest.mark.parametrize("d,b,steady,tail", [(128, 128, 1, 1), (64, 64, 2, 3), (128, 64, 3, 2)])
+def test_exchange_plan_executed_with_virtual_ranks(oracle_mod, binding, d, b, steady, tail):
+    """The whole consumer-side pipeline on one device, driven by sparsp_exchange_plan: every virtual rank starts
+    from its own blocks, then, round by round and chunk by chunk in the plan's order, "fetches" exactly the plan's
+    byte ranges of its packed buffer into a receive buffer that is NaN everywhere else (a device-to-device copy
+    stands in for the peer copy of Section 6), runs the packed-source attention on that hop and merges.  K and V
+    of blocks the rank does not own are NaN throughout.  The result must be the rank's rows of one-shot attention."""
+    from paper_2609_32197_b200 import synth
+    H, P = 4, 4
+    wl = synth.Workload("xchg", H, d, (5, 11, 13), 70, b, 5 if b == 128 else 9, None, P, seed=71)
+    Q, K, V = synth.make_qkv(wl, "cpu")
+    V = (V.float() * 0.5).to(torch.bfloat16)   # keeps |O| below 2.5 (see the packed-buffer test above)
+    N, NB = wl.n_tokens, wl.n_blocks
+    shape = binding.make_shape(H, d, wl.grid, wl.n_text, b)
+    Qd, Kd, Vd = Q.cuda(), K.cuda(), V.cuda()
+    ws = binding.make_workspace(shape, P)
+    ref = oracle_mod.block_mask(Q, K, b, wl.topk_abs, wl.n_text)
+    mo = pu.gpu_block_mask(binding, shape, Qd, Kd, wl.topk_abs, ws)
+    rank = np.array([(j * 3 + j // 4) % P for j in range(NB)], np.int32)
+    rank_d = torch.as_tensor(rank).cuda()
+    dg = pu.gpu_demand_pack(binding, shape, mo["mask"], rank_d, P, 0, Kd, Vd, ws)
+    plan = binding.sparsp_exchange_plan(shape, P, dg["cnt"], dg["seg_offset"], steady, tail)
+    entry = 2 * b * d * 2
+    totals = dg["seg_total"][0].cpu().numpy()
+    base = np.concatenate([[0], np.cumsum(totals)[:-1]]) * entry      # dense consumer bases of the packed buffer
+    assert sum(t.n_bytes for t in plan) == int(dg["volume_bytes"].sum().item())
+    o_ref, lse_ref = oracle_mod.attn_all(Q, K, V, ref["mask"], b)
+    blk_of_tok = np.arange(N) // b
+    hop = torch.empty_like(mo["mask"])
+    nan_byte = 0xFF  # 0xFFFF is a bf16 NaN
+    for r in range(P):
+        foreign = torch.as_tensor(rank[blk_of_tok] != r)
+        Kp, Vp = K.clone(), V.clone()
+        Kp[:, foreign] = float("nan")
+        Vp[:, foreign] = float("nan")
+        Kpd, Vpd = Kp.cuda(), Vp.cuda()
+        recv = torch.full_like(dg["packed"], nan_byte)
+        acc = torch.zeros_like(Qd)
+        acc_lse = torch.full((1, H, N), float("-inf"), dtype=torch.float32, device="cuda")
+        binding.sparsp_hop_mask(shape, mo["mask"], rank_d, P, r, r, hop)          # local blocks first
+        binding.sparsp_sparse_attn_fwd(shape, Qd, Kpd, Vpd, hop, 0.0, acc, acc_lse, ws)
+        mine = [t for t in plan if t.consumer == r]
+        for k in range(P - 1):
+            chunks = [t for t in mine if t.round == k]
+            assert [t.order for t in chunks] == list(range(len(chunks)))
+            p = chunks[0].producer
+            assert p == (r - (k + 1)) % P
+            for t in chunks:  # Fetch: exactly the planned byte range, nothing else
+                lo = int(base[r]) + t.byte_offset
+                recv[lo:lo + t.n_bytes].copy_(dg["packed"][lo:lo + t.n_bytes])
+            binding.sparsp_hop_mask(shape, mo["mask"], rank_d, P, r, p, hop)
+            part = torch.zeros_like(Qd)
+            part_lse = torch.zeros(1, H, N, dtype=torch.float32, device="cuda")
+            binding.sparsp_sparse_attn_fwd_packed(shape, Qd, Kpd, Vpd, hop, rank_d, P, r, dg["union_mask"],
+                                                  dg["seg_offset"], dg["seg_total"], recv, recv.numel() - 64, None,
+                                                  0.0, part, part_lse, ws)
+            rows_t = torch.as_tensor(np.repeat(rank == r, b)[:N]).cuda()
+            part[:, ~rows_t] = 0                          # rows of other ranks are left unwritten by the call
+            part_lse[0][:, ~rows_t] = float("-inf")
+            binding.sparsp_attn_merge(shape, acc, acc_lse, part, part_lse, acc, acc_lse)
+        torch.cuda.synchronize()
+        assert binding.sparsp_status(ws) == binding.SPARSP_OK, binding.sparsp_last_error()
+        rows = np.repeat(rank == r, b)[:N]
+        got = acc.float().cpu().numpy()[:, rows]
+        assert np.isfinite(got).all()
+        err = np.abs(got - o_ref[:, rows])
+        tol_max = pu.ATTN_MAX_ABS + P * 2.0 ** -9 * np.abs(o_ref[:, rows]).max()
+        tol_mean = pu.ATTN_MEAN_ABS + P * 2.0 ** -10 * np.abs(o_ref[:, rows]).mean()
+        assert err.max() <= tol_max and err.mean() <= tol_mean, (r, err.max(), err.mean())
+        assert np.abs(acc_lse[0].cpu().numpy()[:, rows] - lse_ref[:, rows]).max() < 2e-2

@@ -82,3 +82,33 @@ def test_synthetic_inputs_are_seeded_and_shaped():
     r = synth.shuffled_placement(37, 4, seed=1)
     assert torch.equal(r, synth.shuffled_placement(37, 4, seed=1))
     assert sorted(torch.bincount(r.long(), minlength=4).tolist()) == [9, 9, 9, 10]
+
+
+def test_exchange_plan_matches_the_oracle(binding, oracle_mod):
+    """sparsp_exchange_plan is host arithmetic: checked record by record against the oracle's transfer list,
+    for several rank counts and chunkings, on demand counts the oracle computed from random masks."""
+    import numpy as np
+    import torch
+    rng = np.random.default_rng(2)
+    for (H, NB, P, steady, tail) in [(5, 40, 4, 1, 1), (8, 33, 3, 2, 4), (3, 20, 2, 2, 9), (6, 50, 7, 3, 2), (4, 12, 1, 1, 1)]:
+        b, d = 64, 128
+        M = rng.random((H, NB, NB)) < 0.1
+        words = np.zeros((H, NB, (NB + 31) // 32), np.uint32)
+        for h, i, j in zip(*np.nonzero(M)):
+            words[h, i, j >> 5] |= np.uint32(1 << (int(j) & 31))
+        rank = rng.integers(0, P, NB).astype(np.int32)
+        dem = oracle_mod.demand(words, rank, P, b, d)
+        want = oracle_mod.exchange_plan(dem["cnt"], dem["seg_off"], b, d, steady, tail)
+        shape = binding.make_shape(H, d, (1, 1, NB * b), 0, b)
+        got = binding.sparsp_exchange_plan(shape, P, torch.as_tensor(dem["cnt"])[None], torch.as_tensor(dem["seg_off"])[None],
+                                           steady, tail)
+        assert len(got) == len(want)
+        for g, w in zip(got, want):
+            assert g.batch == 0
+            assert (g.consumer, g.producer, g.round, g.order, g.head_begin, g.head_end, g.entry_begin, g.n_entries,
+                    g.byte_offset, g.n_bytes) == tuple(w[k] for k in (
+                        "consumer", "producer", "round", "order", "head_begin", "head_end", "entry_begin",
+                        "n_entries", "byte_offset", "n_bytes"))
+    with pytest.raises(binding.SparspError):
+        binding.sparsp_exchange_plan(shape, 1, torch.zeros(1, 1, 1, 4, dtype=torch.int32),
+                                     torch.zeros(1, 1, 1, 4, dtype=torch.int64), 0, 1)

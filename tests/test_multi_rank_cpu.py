@@ -48,3 +48,50 @@ def test_single_process_passthrough():
     from paper_2609_32197_b200 import dist_util
     t, s = dist_util.reduce_over_ranks({"a": 1.5}, {"b": 2})
     assert t == {"a": 1.5} and s == {"b": 2}
+
+
+def _exchange_worker(rank, world, port, out):
+    """Each rank knows only the mask rows of its own query blocks (Section 5.2: it computes its demand for every
+    peer, the ranks swap those, and from then on both ends of a transfer derive the same byte ranges)."""
+    import numpy as np
+    os.environ["MASTER_ADDR"] = "127.0.0.1"
+    os.environ["MASTER_PORT"] = str(port)
+    dist.init_process_group("gloo", rank=rank, world_size=world)
+    import oracle
+    from paper_2609_32197_b200 import binding
+    H, NB, b, d = 4, 24, 64, 64
+    rng = np.random.default_rng(5)  # same inputs on both ranks; each then forgets the other's rows
+    M = rng.random((H, NB, NB)) < 0.15
+    words = np.zeros((H, NB, 1), np.uint32)
+    for h, i, j in zip(*np.nonzero(M)):
+        words[h, i, 0] |= np.uint32(1 << int(j))
+    placement = oracle.placement_contiguous(NB, world)
+    mine = words.copy()
+    mine[:, placement != rank] = 0
+    dem = oracle.demand(mine, placement, world, b, d)          # only row `rank` of the consumer axis is non-zero
+    assert not dem["cnt"][np.arange(world) != rank].any()
+    rows_c = [torch.zeros(world, H, dtype=torch.int32) for _ in range(world)]
+    rows_o = [torch.zeros(world, H, dtype=torch.int64) for _ in range(world)]
+    dist.all_gather(rows_c, torch.as_tensor(dem["cnt"][rank]))
+    dist.all_gather(rows_o, torch.as_tensor(dem["seg_off"][rank]))
+    cnt, off = torch.stack(rows_c), torch.stack(rows_o)
+    shape = binding.make_shape(H, d, (1, 1, NB * b), 0, b)
+    plan = binding.sparsp_exchange_plan(shape, world, cnt[None], off[None], 2, 3)
+    recs = [(t.consumer, t.producer, t.round, t.order, t.head_begin, t.head_end, t.byte_offset, t.n_bytes) for t in plan]
+    full = oracle.demand(words, placement, world, b, d)
+    ref = [(t["consumer"], t["producer"], t["round"], t["order"], t["head_begin"], t["head_end"], t["byte_offset"],
+            t["n_bytes"]) for t in oracle.exchange_plan(full["cnt"], full["seg_off"], b, d, 2, 3)]
+    out[rank] = (recs, recs == ref, int(full["volume"][rank]))
+    dist.barrier()
+    dist.destroy_process_group()
+
+
+def test_two_ranks_derive_the_same_transfer_list():
+    world, port = 2, _free_port()
+    with mp.Manager() as mgr:
+        out = mgr.dict()
+        mp.spawn(_exchange_worker, args=(world, port, out), nprocs=world, join=True)
+        res = dict(out)
+    assert res[0][0] == res[1][0] and res[0][1] and res[1][1]   # producer's and consumer's view agree, and with the oracle
+    for r in range(world):
+        assert sum(t[7] for t in res[r][0] if t[0] == r) == res[r][2]   # what rank r receives is its exchange volume
