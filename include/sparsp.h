@@ -238,6 +238,11 @@ SPARSP_API int sparsp_sparse_attn_fwd_packed(const sparsp_shape* shape, const vo
 SPARSP_API int sparsp_hop_mask(const sparsp_shape* shape, const uint32_t* mask, const int32_t* rank_of_block,
                                int32_t n_ranks, int32_t consumer, int32_t producer, uint32_t* hop_mask,
                                void* stream);
+/* One chunk of a hop (Section 7.1: a hop is cut into chunks of heads so that attention on a chunk can start as
+ * soon as it has arrived): sparsp_hop_mask with the rows of heads outside [head_begin, head_end) zeroed as well. */
+SPARSP_API int sparsp_hop_chunk_mask(const sparsp_shape* shape, const uint32_t* mask, const int32_t* rank_of_block,
+                                     int32_t n_ranks, int32_t consumer, int32_t producer, int32_t head_begin,
+                                     int32_t head_end, uint32_t* hop_mask, void* stream);
 SPARSP_API int sparsp_attn_merge(const sparsp_shape* shape, const void* O_a, const float* lse_a, const void* O_b,
                                  const float* lse_b, void* O, float* lse, void* stream);
 

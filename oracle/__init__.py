@@ -376,11 +376,14 @@ def attn_dense_masked(Q, K, V, mask: np.ndarray, b: int, scale: float | None = N
 # ---------------------------------------------------------------------------------------------
 # consumer-side pipeline ("next" rows): per-hop masks and log-sum-exp merging of partial results
 # ---------------------------------------------------------------------------------------------
-def hop_mask(mask: np.ndarray, rank_of_block: np.ndarray, consumer: int, producer: int) -> np.ndarray:
+def hop_mask(mask: np.ndarray, rank_of_block: np.ndarray, consumer: int, producer: int,
+             head_begin: int = 0, head_end: int | None = None) -> np.ndarray:
     """Rows of the consumer rank's query blocks, restricted to the KV blocks the producer owns
-    (the blocks that travel in one hop of the demand-routed exchange, Section 5.1); all else zero."""
+    (the blocks that travel in one hop of the demand-routed exchange, Section 5.1); all else zero.
+    With a head range: one chunk of that hop (Section 7.1), i.e. the other heads are zero as well."""
     mask = np.ascontiguousarray(mask, dtype=np.uint32)
     H, NB, Wd = mask.shape
+    head_end = H if head_end is None else head_end
     own = np.zeros(Wd, dtype=np.uint32)
     for j in range(NB):
         if rank_of_block[j] == producer:
@@ -388,7 +391,8 @@ def hop_mask(mask: np.ndarray, rank_of_block: np.ndarray, consumer: int, produce
     out = np.zeros_like(mask)
     for i in range(NB):
         if rank_of_block[i] == consumer:
-            out[:, i, :] = mask[:, i, :] & own
+            for h in range(head_begin, head_end):
+                out[h, i, :] = mask[h, i, :] & own
     return out
 
 

@@ -31,6 +31,7 @@ EXPORTS = [
     "sparsp_status", "sparsp_last_error", "sparsp_launch_count", "sparsp_demand_plan_noalloc",
     "sparsp_hop_mask", "sparsp_attn_merge", "sparsp_sparse_attn_fwd_packed", "sparsp_block_mask_cdf",
     "sparsp_placement_permutation", "sparsp_permute_tokens", "sparsp_sharing_histogram", "sparsp_exchange_plan",
+    "sparsp_hop_chunk_mask",
 ]
 
 
@@ -247,6 +248,12 @@ def sparsp_sparse_attn_fwd_packed(shape, Q, K, V, mask, rank_of_block, n_ranks, 
 def sparsp_hop_mask(shape, mask, rank_of_block, n_ranks, consumer, producer, hop_mask):
     _check(lib().sparsp_hop_mask(ctypes.byref(shape), _ptr(mask), _ptr(rank_of_block), ctypes.c_int32(n_ranks),
                                  ctypes.c_int32(consumer), ctypes.c_int32(producer), _ptr(hop_mask), _stream()))
+
+
+def sparsp_hop_chunk_mask(shape, mask, rank_of_block, n_ranks, consumer, producer, head_begin, head_end, hop_mask):
+    _check(lib().sparsp_hop_chunk_mask(ctypes.byref(shape), _ptr(mask), _ptr(rank_of_block), ctypes.c_int32(n_ranks),
+                                       ctypes.c_int32(consumer), ctypes.c_int32(producer), ctypes.c_int32(head_begin),
+                                       ctypes.c_int32(head_end), _ptr(hop_mask), _stream()))
 
 
 def sparsp_attn_merge(shape, O_a, lse_a, O_b, lse_b, O, lse):

@@ -485,8 +485,9 @@ int sparsp_sparse_attn_fwd_packed(const sparsp_shape* shape, const void* Q, cons
                             (char*)workspace, L, (cudaStream_t)stream);
 }
 
-int sparsp_hop_mask(const sparsp_shape* shape, const uint32_t* mask, const int32_t* rank_of_block, int32_t n_ranks,
-                    int32_t consumer, int32_t producer, uint32_t* hop_mask, void* stream) {
+int sparsp_hop_chunk_mask(const sparsp_shape* shape, const uint32_t* mask, const int32_t* rank_of_block,
+                          int32_t n_ranks, int32_t consumer, int32_t producer, int32_t head_begin, int32_t head_end,
+                          uint32_t* hop_mask, void* stream) {
   Geometry g;
   SPARSP_TRY(make_geometry(shape, &g));
   if (n_ranks < 1 || n_ranks > kMaxRanks || consumer < 0 || consumer >= n_ranks || producer < 0 ||
@@ -494,10 +495,22 @@ int sparsp_hop_mask(const sparsp_shape* shape, const uint32_t* mask, const int32
     set_error("consumer/producer %d/%d outside 0..%d", consumer, producer, n_ranks - 1);
     return SPARSP_ERR_INVALID_ARG;
   }
+  if (head_begin < 0 || head_end > g.H || head_begin > head_end) {
+    set_error("head range [%d, %d) outside [0, %d)", head_begin, head_end, g.H);
+    return SPARSP_ERR_INVALID_ARG;
+  }
   SPARSP_TRY(check_ptr(mask, "mask", 4));
   SPARSP_TRY(check_ptr(rank_of_block, "rank_of_block", 4));
   SPARSP_TRY(check_ptr(hop_mask, "hop_mask", 4));
-  return launch_hop_mask(g, mask, rank_of_block, consumer, producer, hop_mask, (cudaStream_t)stream);
+  return launch_hop_mask(g, mask, rank_of_block, consumer, producer, head_begin, head_end, hop_mask,
+                         (cudaStream_t)stream);
+}
+
+int sparsp_hop_mask(const sparsp_shape* shape, const uint32_t* mask, const int32_t* rank_of_block, int32_t n_ranks,
+                    int32_t consumer, int32_t producer, uint32_t* hop_mask, void* stream) {
+  if (!shape) return sparsp_hop_chunk_mask(shape, mask, rank_of_block, n_ranks, consumer, producer, 0, 0, hop_mask, stream);
+  return sparsp_hop_chunk_mask(shape, mask, rank_of_block, n_ranks, consumer, producer, 0, shape->heads, hop_mask,
+                               stream);
 }
 
 int sparsp_attn_merge(const sparsp_shape* shape, const void* O_a, const float* lse_a, const void* O_b,

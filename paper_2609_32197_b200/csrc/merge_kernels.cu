@@ -5,16 +5,18 @@
 
 namespace sparsp {
 
-// hop[b][h][i][w] = rank[i] == consumer ? mask[b][h][i][w] & own_producer[w] : 0.  Thread per word.
-__global__ void hop_mask_kernel(const uint32_t* __restrict__ mask, const int32_t* __restrict__ rank, int NB,
-                                int Wd, int64_t n_words, int consumer, int producer,
+// hop[b][h][i][w] = (rank[i] == consumer and head_begin <= h < head_end) ? mask[b][h][i][w] & own_producer[w] : 0.
+// Thread per word.
+__global__ void hop_mask_kernel(const uint32_t* __restrict__ mask, const int32_t* __restrict__ rank, int H, int NB,
+                                int Wd, int64_t n_words, int consumer, int producer, int head_begin, int head_end,
                                 uint32_t* __restrict__ hop) {
   const int64_t idx = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
   if (idx >= n_words) return;
   const int w = (int)(idx % Wd);
   const int i = (int)((idx / Wd) % NB);
+  const int h = (int)((idx / ((int64_t)Wd * NB)) % H);
   uint32_t out = 0;
-  if (rank[i] == consumer) {
+  if (rank[i] == consumer && h >= head_begin && h < head_end) {
     uint32_t own = 0;
     for (int t = 0; t < 32; ++t) {
       const int j = w * 32 + t;
@@ -64,10 +66,10 @@ __global__ void attn_merge_kernel(const __nv_bfloat16* __restrict__ Oa, const fl
 }
 
 int launch_hop_mask(const Geometry& g, const uint32_t* mask, const int32_t* rank, int consumer, int producer,
-                    uint32_t* hop, cudaStream_t st) {
+                    int head_begin, int head_end, uint32_t* hop, cudaStream_t st) {
   const int64_t n_words = (int64_t)g.B * g.H * g.NB * g.Wd;
-  hop_mask_kernel<<<(unsigned)((n_words + 255) / 256), 256, 0, st>>>(mask, rank, g.NB, g.Wd, n_words, consumer,
-                                                                     producer, hop);
+  hop_mask_kernel<<<(unsigned)((n_words + 255) / 256), 256, 0, st>>>(mask, rank, g.H, g.NB, g.Wd, n_words, consumer,
+                                                                     producer, head_begin, head_end, hop);
   count_launch();
   SPARSP_CUDA_OK(cudaGetLastError());
   return SPARSP_OK;

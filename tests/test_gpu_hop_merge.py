@@ -239,19 +239,23 @@ def test_exchange_plan_executed_with_virtual_ranks(oracle_mod, binding, d, b, st
             assert [t.order for t in chunks] == list(range(len(chunks)))
             p = chunks[0].producer
             assert p == (r - (k + 1)) % P
-            for t in chunks:  # Fetch: exactly the planned byte range, nothing else
+            rows_t = torch.as_tensor(np.repeat(rank == r, b)[:N]).cuda()
+            for t in chunks:
+                # Fetch: exactly the planned byte range, nothing else ...
                 lo = int(base[r]) + t.byte_offset
                 recv[lo:lo + t.n_bytes].copy_(dg["packed"][lo:lo + t.n_bytes])
-            binding.sparsp_hop_mask(shape, mo["mask"], rank_d, P, r, p, hop)
-            part = torch.zeros_like(Qd)
-            part_lse = torch.zeros(1, H, N, dtype=torch.float32, device="cuda")
-            binding.sparsp_sparse_attn_fwd_packed(shape, Qd, Kpd, Vpd, hop, rank_d, P, r, dg["union_mask"],
-                                                  dg["seg_offset"], dg["seg_total"], recv, recv.numel() - 64, None,
-                                                  0.0, part, part_lse, ws)
-            rows_t = torch.as_tensor(np.repeat(rank == r, b)[:N]).cuda()
-            part[:, ~rows_t] = 0                          # rows of other ranks are left unwritten by the call
-            part_lse[0][:, ~rows_t] = float("-inf")
-            binding.sparsp_attn_merge(shape, acc, acc_lse, part, part_lse, acc, acc_lse)
+                # ... and attention on the chunk as soon as it is there (Section 7.1), before the next one arrives
+                binding.sparsp_hop_chunk_mask(shape, mo["mask"], rank_d, P, r, p, t.head_begin, t.head_end, hop)
+                assert np.array_equal(pu.u32(hop[0]),
+                                      oracle_mod.hop_mask(ref["mask"], rank, r, p, t.head_begin, t.head_end))
+                part = torch.zeros_like(Qd)
+                part_lse = torch.zeros(1, H, N, dtype=torch.float32, device="cuda")
+                binding.sparsp_sparse_attn_fwd_packed(shape, Qd, Kpd, Vpd, hop, rank_d, P, r, dg["union_mask"],
+                                                      dg["seg_offset"], dg["seg_total"], recv, recv.numel() - 64,
+                                                      None, 0.0, part, part_lse, ws)
+                part[:, ~rows_t] = 0                      # rows of other ranks are left unwritten by the call
+                part_lse[0][:, ~rows_t] = float("-inf")
+                binding.sparsp_attn_merge(shape, acc, acc_lse, part, part_lse, acc, acc_lse)
         torch.cuda.synchronize()
         assert binding.sparsp_status(ws) == binding.SPARSP_OK, binding.sparsp_last_error()
         rows = np.repeat(rank == r, b)[:N]

@@ -136,6 +136,10 @@ def test_hop_partials_merge_to_full_attention(oracle_mod):
                     for j in range(NB):
                         bit = (int(hm[h, i, j >> 5]) >> (j & 31)) & 1
                         assert bit == int(M[h, i, j] and rank[i] == r and rank[j] == p)
+            # the chunks of a hop (head ranges) are disjoint and add up to the hop
+            parts = [oracle_mod.hop_mask(words, rank, r, p, h0, h0 + 1) for h0 in range(H)]
+            assert all(not pc[np.arange(H) != h0].any() for h0, pc in enumerate(parts))
+            assert np.array_equal(np.bitwise_or.reduce(np.stack(parts)), hm)
             part, part_lse = oracle_mod.attn_all(Q, K, V, hm, b)
             acc, acc_lse = oracle_mod.attn_merge(acc, acc_lse, part, part_lse)
         rows = np.repeat(rank == r, b)[:N]
