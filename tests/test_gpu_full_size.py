@@ -84,21 +84,21 @@ def _full_size(oracle, binding, name, n_attn_random):
 
 
 def test_mid_full_size(oracle_mod, binding):
-    _full_size(oracle_mod, binding, "mid", 24)
+    _full_size(oracle_mod, binding, "mid", 40)
 
 
 def test_cog_like_full_size_text_blocks_and_shuffled_placement(oracle_mod, binding):
-    _full_size(oracle_mod, binding, "cog", 24)
+    _full_size(oracle_mod, binding, "cog", 40)
 
 
 def test_wan_like_full_size_two_placements(oracle_mod, binding):
-    rep = _full_size(oracle_mod, binding, "wan", 8)
+    rep = _full_size(oracle_mod, binding, "wan", 32)
     vols = {p: v for (k, p), v in rep.items() if p in ("contiguous", "periodic")}
     assert set(vols) == {"contiguous", "periodic"}
 
 
 def test_hunyuan_like_full_size_topk_sweep(oracle_mod, binding):
-    rep = _full_size(oracle_mod, binding, "hunyuan", 4)
+    rep = _full_size(oracle_mod, binding, "hunyuan", 28)
     vols = sorted((k, v) for (k, p), v in rep.items() if p == "contiguous")
     assert [k for k, _ in vols] == [47, 93, 233]
     assert vols[0][1] < vols[1][1] < vols[2][1]  # more kept blocks, more demanded bytes
