@@ -801,9 +801,16 @@ __global__ void __launch_bounds__(kAttnThreads, 1)
               const float2 pp = (kPoly > 0 && (e % (kPoly > 0 ? kPoly : 1)) == 1)
                                     ? exp2_poly2(x)
                                     : make_float2(ex2(x.x), ex2(x.y));
-              if (!C::kOnes) lsum2 = fadd2(lsum2, pp);
               const __nv_bfloat162 h2 = __floats2bfloat162_rn(pp.x, pp.y);
               pkh[e] = *reinterpret_cast<const uint32_t*>(&h2);
+              if (!C::kOnes) {
+                // the row sum adds the bf16 values that P V multiplies, not the unrounded exponentials: with a
+                // reference that is not the row's maximum the largest term is an arbitrary 2^x, and a sum of
+                // unrounded terms would differ from the numerator's weights by up to 2^-9 of a peaked row
+                asm("{\n\t.reg .b16 lo, hi;\n\tmov.b32 {lo, hi}, %2;\n\tadd.rn.f32.bf16 %0, lo, %0;\n\tadd.rn.f32.bf16 %1, hi, %1;\n\t}"
+                    : "+f"(lsum2.x), "+f"(lsum2.y)
+                    : "r"(pkh[e]));
+              }
             }
             if (kRagged && vh[h] < 64) {
               // columns past the end of the sequence: exactly zero in P (the polynomial path returns

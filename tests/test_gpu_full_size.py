@@ -4,8 +4,10 @@ Inputs are generated on the device with the shared seeded generator and copied t
 sides see the same bits.  Masks, unions, counts, offsets and volumes are compared in full with the
 oracle; the packed buffer is compared in full, in device memory, against a library gather driven by
 the ORACLE's entry list; attention is compared on a seeded sample of (head, query block) units the
-oracle computes one by one (first block, last ragged block, one block per virtual rank, the
-video/text boundary, random ones)."""
+oracle computes one by one: for EVERY head the first block, the last (ragged) block, the first block of
+every virtual rank, the video/text boundary blocks and random ones (12 to 20 blocks per head), and with
+64-token blocks two heads in full (both members of every stacked pair); the tolerance is asserted over the
+pooled sample and per head, for every sparsity level of the workload."""
 import numpy as np
 import pytest
 import torch
@@ -73,32 +75,39 @@ def _full_size(oracle, binding, name, n_attn_random):
         torch.cuda.synchronize()
         assert binding.sparsp_status(ws) == binding.SPARSP_OK, binding.sparsp_last_error()
         extra = [wl.nb_video - 1, wl.nb_video] if wl.n_text else []
-        units = pu.sample_units(H, NB, _placement(oracle, synth, wl, wl.placements[0]), n_attn_random, 17, extra)
-        mx, mean = pu.check_attn_units(oracle, Q, K, V, mask_ref, b, Od, units)
+        full_heads = (0, H - 1) if b == 64 else ()
+        units = pu.sample_units_per_head(H, NB, _placement(oracle, synth, wl, wl.placements[0]), n_attn_random,
+                                         17 + k, extra, full_heads)
+        assert {h for h, _ in units} == set(range(H)) and min(sum(1 for u in units if u[0] == h) for h in range(H)) >= 8
+        rep = {}
+        pu.check_attn_units(oracle, Q, K, V, mask_ref, b, Od, units, report=rep)
         # rows the sample does not cover: finite, and not left at the zero fill
         assert bool(torch.isfinite(Od.float()).all())
         assert bool((Od.float().abs().amax(dim=-1) > 0).all())
-        report[(k, "attn")] = (len(units), mx, mean)
-    print(name, report)
+        report[(k, "attn")] = rep
+        print(f"{name} k={k}: attention on {rep['units']} units (every head): max |err| {rep['max_abs']:.5f} at reference "
+              f"value {rep['ref_at_max']:.4f} (bf16 rounding of that value alone {rep['bf16_rounding_of_ref_at_max']:.5f}), "
+              f"mean |err| {rep['mean_abs']:.6f}, worst head mean {rep['worst_head_mean']:.6f}")
+    print(name, {k_: v for k_, v in report.items() if k_[1] != "attn"})
     return report
 
 
 def test_mid_full_size(oracle_mod, binding):
-    _full_size(oracle_mod, binding, "mid", 40)
+    _full_size(oracle_mod, binding, "mid", 6)
 
 
 def test_cog_like_full_size_text_blocks_and_shuffled_placement(oracle_mod, binding):
-    _full_size(oracle_mod, binding, "cog", 40)
+    _full_size(oracle_mod, binding, "cog", 4)
 
 
 def test_wan_like_full_size_two_placements(oracle_mod, binding):
-    rep = _full_size(oracle_mod, binding, "wan", 32)
+    rep = _full_size(oracle_mod, binding, "wan", 8)
     vols = {p: v for (k, p), v in rep.items() if p in ("contiguous", "periodic")}
     assert set(vols) == {"contiguous", "periodic"}
 
 
 def test_hunyuan_like_full_size_topk_sweep(oracle_mod, binding):
-    rep = _full_size(oracle_mod, binding, "hunyuan", 28)
+    rep = _full_size(oracle_mod, binding, "hunyuan", 10)
     vols = sorted((k, v) for (k, p), v in rep.items() if p == "contiguous")
     assert [k for k, _ in vols] == [47, 93, 233]
     assert vols[0][1] < vols[1][1] < vols[2][1]  # more kept blocks, more demanded bytes

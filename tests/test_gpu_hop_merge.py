@@ -92,7 +92,8 @@ def test_merge_kernel_matches_oracle_elementwise(oracle_mod, binding):
 
 
 @pytest.mark.parametrize("d,b,layout", [(128, 128, "HND"), (64, 64, "HND"), (128, 64, "NHD"), (64, 128, "HND")])
-def test_attention_reading_remote_blocks_from_the_packed_buffer(oracle_mod, binding, d, b, layout):
+@pytest.mark.parametrize("v_scale", [1.0, 0.5])
+def test_attention_reading_remote_blocks_from_the_packed_buffer(oracle_mod, binding, d, b, layout, v_scale):
     """The consumer-side attention must produce the consumer's rows from its own K/V blocks plus its
     packed buffer alone: the K/V handed to it have every block the consumer does NOT own overwritten
     with NaN, and the oracle computes the expected rows from the same restricted view."""
@@ -100,9 +101,7 @@ def test_attention_reading_remote_blocks_from_the_packed_buffer(oracle_mod, bind
     H, P = 3, 3
     wl = synth.Workload("packed", H, d, (5, 11, 13), 70, b, 5 if b == 128 else 9, None, P, seed=61)
     Q, K, V = synth.make_qkv(wl, "cpu")
-    # with this few kept blocks some outputs of the stock recipe pass 4, where half a bf16 ulp (0.0156) of
-    # output rounding alone nearly uses up the 2e-2 bound; halving V (exact in bf16) keeps |O| below 2.5
-    V = (V.float() * 0.5).to(torch.bfloat16)
+    V = (V.float() * v_scale).to(torch.bfloat16)  # 1: the generator's own V ~ N(0,1); 0.5: an extra case
     N, NB = wl.n_tokens, wl.n_blocks
     shape = binding.make_shape(H, d, wl.grid, wl.n_text, b, layout=layout)
     Qd, Kd, Vd = (pu.to_layout(x.cuda(), layout) for x in (Q, K, V))
@@ -193,7 +192,8 @@ def test_packed_attention_rejects_bad_arguments(binding):
 
 
 @pytest.mark.parametrize("d,b,steady,tail", [(128, 128, 1, 1), (64, 64, 2, 3), (128, 64, 3, 2)])
-def test_exchange_plan_executed_with_virtual_ranks(oracle_mod, binding, d, b, steady, tail):
+@pytest.mark.parametrize("v_scale", [1.0, 0.5])
+def test_exchange_plan_executed_with_virtual_ranks(oracle_mod, binding, d, b, steady, tail, v_scale):
     """The whole consumer-side pipeline on one device, driven by sparsp_exchange_plan: every virtual rank starts
     from its own blocks, then, round by round and chunk by chunk in the plan's order, "fetches" exactly the plan's
     byte ranges of its packed buffer into a receive buffer that is NaN everywhere else (a device-to-device copy
@@ -203,7 +203,7 @@ def test_exchange_plan_executed_with_virtual_ranks(oracle_mod, binding, d, b, st
     H, P = 4, 4
     wl = synth.Workload("xchg", H, d, (5, 11, 13), 70, b, 5 if b == 128 else 9, None, P, seed=71)
     Q, K, V = synth.make_qkv(wl, "cpu")
-    V = (V.float() * 0.5).to(torch.bfloat16)   # keeps |O| below 2.5 (see the packed-buffer test above)
+    V = (V.float() * v_scale).to(torch.bfloat16)  # 1: the generator's own V ~ N(0,1); 0.5: an extra case
     N, NB = wl.n_tokens, wl.n_blocks
     shape = binding.make_shape(H, d, wl.grid, wl.n_text, b)
     Qd, Kd, Vd = Q.cuda(), K.cuda(), V.cuda()
