@@ -7,12 +7,16 @@ Prints ONE JSON line (rank 0).  `value` = kept-block attention FLOPs of all rank
 effective TFLOP/s of the whole layer; the per-kernel figures (attention TFLOP/s against the bf16
 tensor peak, pack GB/s against the HBM copy peak, ms per stage) ride along in the same line.
 
-    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload mid|cog|wan|hunyuan|tiny]
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload hunyuan|wan|cog|mid|tiny]
                     [--pct P] [--placement contiguous|periodic|shuffle] [--impl ours|reference]
+                    [--shard replicas|heads] [--no-per-config] [--sustained-s S]
 
+The headline configuration is the largest single-GPU one (Hunyuan-like, 118 800 tokens, top-k 10 %); at
+N = 1 the same line carries `per_config` (all eight configurations of the contract measured the same way)
+and `sustained` (the attention call alone, back to back for a couple of seconds, with the clocks sampled).
 With N > 1 launch under torch.distributed.run; every rank runs its own replica of the workload
-(different seed) -- the path has no exchange step on one node, so scaling is weak and there is no
-data-path collective.
+(different seed; weak scaling) or, with --shard heads, its share of the heads of ONE layer (strong
+scaling) -- either way the path has no exchange step, so there is no data-path collective.
 """
 from __future__ import annotations
 
@@ -30,12 +34,11 @@ sys.path.insert(0, ROOT)
 METRIC = "sparse-attn effective TFLOP/s + %bf16 peak; pack GB/s + %HBM; ms/layer"
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
 NOMINAL = {"hbm_gbs": 8000.0, "bf16_tflops": 2250.0}
-# dram__bytes_read.sum + dram__bytes_write.sum per launch of the attention kernel, from the ncu
-# captures summarised under profiles/ (None = not captured for that workload).
-ATTN_DRAM_TRAFFIC = {
-    ("mid", 58): 591.0e6,            # profiles/attn_fwd_kernel_mid_and_hunyuan4.md, full workload
-    ("hunyuan", 93): 6 * 710.0e6,     # same file: 4-head capture scaled by heads (24 / 4)
-}
+L2_BYTES = 126 << 20
+# the configurations of the per_config list: (workload, top-k percent or None, placement)
+PER_CONFIG = [("tiny", None, "contiguous"), ("mid", 15, "contiguous"), ("cog", 20, "shuffle"),
+              ("wan", 10, "contiguous"), ("wan", 10, "periodic"),
+              ("hunyuan", 5, "contiguous"), ("hunyuan", 10, "contiguous"), ("hunyuan", 25, "contiguous")]
 
 
 def load_peaks():
@@ -45,6 +48,29 @@ def load_peaks():
             p = json.load(f)
         return {k: float(p[k]) for k in FALLBACK_PEAKS if k in p} | {"source": "measured"}
     return dict(FALLBACK_PEAKS) | {"source": "fallback"}
+
+
+def load_attn_traffic():
+    """DRAM bytes per launch of the attention kernel from the ncu captures summarised under profiles/
+    (dram__bytes_read.sum + dram__bytes_write.sum).  The table is a text file: one line per capture,
+    `workload topk_blocks heads_captured bytes source`; a capture of fewer heads than the workload has is
+    scaled by the head ratio (traffic grows in proportion to the heads: every head has its own Q, K, V, O).
+    Returns {(workload, topk): (bytes_per_full_launch, note)}."""
+    table = {}
+    path = os.path.join(ROOT, "profiles", "attn_dram_traffic.txt")
+    if not os.path.exists(path):
+        return table
+    from paper_2609_32197_b200 import synth
+    with open(path) as f:
+        for line in f:
+            line = line.split("#", 1)[0].strip()
+            if not line:
+                continue
+            name, k, heads, nbytes, source = line.split(None, 4)
+            full = synth.WORKLOADS[name].heads
+            table[(name, int(k))] = (float(nbytes) * full / int(heads),
+                                     "ncu capture of %s of %d heads (%s), not measured in this run" % (heads, full, source))
+    return table
 
 
 class ClockSampler(threading.Thread):
@@ -92,9 +118,10 @@ class ClockSampler(threading.Thread):
         if self.is_alive():
             self.join(timeout=2)
         if not self.samples:
-            return {"sm_mhz": None, "sm_max_mhz": self.max_mhz, "reasons": sorted(self.reasons)}
+            return {"sm_mhz": None, "sm_max_mhz": self.max_mhz, "reasons": sorted(self.reasons), "samples": 0}
         s = sorted(self.samples)
-        return {"sm_mhz": s[len(s) // 2], "sm_max_mhz": self.max_mhz, "reasons": sorted(self.reasons)}
+        return {"sm_mhz": s[len(s) // 2], "sm_max_mhz": self.max_mhz, "reasons": sorted(self.reasons),
+                "samples": len(s)}
 
 
 def physical_gpu_index(local_index: int) -> int:
@@ -122,21 +149,322 @@ def kept_flops_and_counts(mask_i32, N, b, d):
     import torch
     B, H, NB, Wd = mask_i32.shape
     bits = torch.arange(32, device=mask_i32.device, dtype=torch.int32)
-    m = ((mask_i32.unsqueeze(-1) >> bits) & 1).reshape(B, H, NB, Wd * 32)[..., :NB].to(torch.float64)
     sizes = torch.full((NB,), float(b), dtype=torch.float64, device=mask_i32.device)
     sizes[-1] = float(N - (NB - 1) * b)
-    pairs = torch.einsum("i,bhij,j->", sizes, m, sizes).item()
-    return 4.0 * d * pairs, int(m.sum().item())
+    pairs, kept = 0.0, 0
+    for h in range(H):  # head by head: the unpacked mask of a whole layer would be gigabytes
+        m = ((mask_i32[:, h].unsqueeze(-1) >> bits) & 1).reshape(B, NB, Wd * 32)[..., :NB].to(torch.float64)
+        pairs += torch.einsum("i,bij,j->", sizes, m, sizes).item()
+        kept += int(m.sum().item())
+    return 4.0 * d * pairs, kept
 
 
 # ------------------------------------------------------------------------------------------------
 # our arm
 # ------------------------------------------------------------------------------------------------
+class Config:
+    """One workload resident on the device with its buffers and the three calls of a step."""
+
+    def __init__(self, wl, placement, pct, tau, dev, head_range=None):
+        import torch
+
+        from paper_2609_32197_b200 import binding, synth
+        self.binding, self.wl, self.placement, self.tau, self.dev = binding, wl, placement, tau, dev
+        h0, h1 = head_range if head_range else (0, wl.heads)
+        self.H, self.d, self.b, self.P = h1 - h0, wl.head_dim, wl.block, wl.ranks
+        self.shape = binding.make_shape(self.H, self.d, wl.grid, wl.n_text, self.b)
+        g = binding.sparsp_geometry(self.shape)
+        self.N, self.NB = g.n_tokens, g.n_blocks
+        self.k = wl.topk_abs if pct is None else binding.sparsp_resolve_topk(pct, g.n_video_blocks)
+        self.Q, self.K, self.V = synth.make_qkv(wl, dev, heads=self.H, head_begin=h0)
+        if placement == "contiguous":
+            self.rank_of_block = binding.sparsp_placement_contiguous(self.shape, self.P)
+        elif placement == "periodic":
+            self.rank_of_block = binding.sparsp_placement_periodic(self.shape, self.P)
+        else:
+            self.rank_of_block = synth.shuffled_placement(self.NB, self.P, seed=1)
+        self.rank_d = self.rank_of_block.to(dev)
+        self.ws = binding.make_workspace(self.shape, self.P, dev)
+        self.mo = binding.alloc_mask_outputs(self.shape, self.k, dev, with_list=True)
+        self.do = binding.alloc_demand_outputs(self.shape, self.P, dev)
+        self.O = torch.empty_like(self.Q)
+        self.entry = 2 * self.b * self.d * 2
+        # size the packed buffer once (the mask is a function of the inputs, which do not change)
+        self.step_mask()
+        self.step_plan()
+        torch.cuda.synchronize()
+        total_entries = int(self.do["seg_total"].sum().item())
+        self.packed = torch.empty(max(total_entries * self.entry, 16), dtype=torch.uint8, device=dev)
+        self.volume = int(self.do["volume_bytes"].sum().item())
+        self.flops, self.kept_pairs = kept_flops_and_counts(self.mo["mask"], self.N, self.b, self.d)
+        self.input_bytes = 3 * self.Q.numel() * 2
+        # a working set that fits L2 would turn "HBM GB/s" into an L2 figure: flush L2 between iterations
+        self.flush = torch.empty(2 * L2_BYTES, dtype=torch.uint8, device=dev) if self.input_bytes < 2 * L2_BYTES else None
+
+    def step_mask(self):
+        b, mo = self.binding, self.mo
+        if self.tau > 0:  # CDF-threshold selection instead of top-k (rows keep different numbers of blocks)
+            b.sparsp_block_mask_cdf(self.shape, self.Q, self.K, self.tau, 0.0, mo["mask"], mo["kv_count"], None, None, self.ws)
+        else:
+            b.sparsp_block_mask(self.shape, self.Q, self.K, self.k, mo["mask"], mo["kv_list"], mo["kv_count"], None, None,
+                                self.ws)
+
+    def step_plan(self):
+        b, do = self.binding, self.do
+        b.sparsp_demand_pack(self.shape, self.mo["mask"], self.rank_d, self.P, b.SPARSP_PLAN_ONLY, None, None,
+                             do["union_mask"], do["cnt"], do["seg_offset"], do["seg_total"], do["volume_bytes"], None, 0,
+                             None, self.ws)
+
+    def step_pack(self):
+        b, do = self.binding, self.do
+        b.sparsp_demand_pack(self.shape, self.mo["mask"], self.rank_d, self.P, 0, self.K, self.V, do["union_mask"],
+                             do["cnt"], do["seg_offset"], do["seg_total"], do["volume_bytes"], self.packed,
+                             self.packed.numel(), None, self.ws)
+
+    def step_attn(self):
+        self.binding.sparsp_sparse_attn_fwd(self.shape, self.Q, self.K, self.V, self.mo["mask"], 0.0, self.O, None, self.ws)
+
+    def step(self):
+        self.step_mask()
+        self.step_pack()
+        self.step_attn()
+
+    def check_status(self):
+        assert self.binding.sparsp_status(self.ws) == self.binding.SPARSP_OK, self.binding.sparsp_last_error()
+
+    def l2_policy(self):
+        if self.flush is None:
+            return "inputs larger than L2 (Q+K+V = %.0f MB)" % (self.input_bytes / 1e6)
+        return "L2 flushed between iterations (a %d MB buffer is overwritten; Q+K+V = %.1f MB)" % (
+            self.flush.numel() >> 20, self.input_bytes / 1e6)
+
+    def describe(self):
+        wl = self.wl
+        return {"workload": wl.name, "heads": self.H, "head_dim": self.d, "grid": list(wl.grid), "n_text": wl.n_text,
+                "tokens": self.N, "block": self.b, "n_blocks": self.NB,
+                "topk_blocks": (self.k if self.tau <= 0 else None),
+                "selection": ("top-k" if self.tau <= 0 else "cdf tau=%g" % self.tau), "kept_pairs": self.kept_pairs,
+                "virtual_ranks": self.P, "placement": self.placement, "layout": "[H][N][d]",
+                "l2_policy": self.l2_policy()}
+
+
+def time_steps(cfg, steps, warmup, barrier, local_gpu):
+    """W warm-up steps, then `steps` timed steps bracketed by `barrier`; per-stage CUDA events on the launching
+    stream.  Returns the device times (ms), the launch count and the clocks sampled during the timed region."""
+    import torch
+    binding = cfg.binding
+    stream = torch.cuda.current_stream()
+    for _ in range(warmup):
+        cfg.step()
+    barrier()
+    cfg.check_status()
+    sampler = ClockSampler(physical_gpu_index(local_gpu))
+    sampler.start()
+    launches0 = binding.sparsp_launch_count()
+    ev = [[torch.cuda.Event(enable_timing=True) for _ in range(4)] for _ in range(steps)]
+    barrier()
+    for s in range(steps):
+        if cfg.flush is not None:
+            cfg.flush.fill_(s & 0xFF)
+        ev[s][0].record(stream)
+        cfg.step_mask()
+        ev[s][1].record(stream)
+        cfg.step_pack()
+        ev[s][2].record(stream)
+        cfg.step_attn()
+        ev[s][3].record(stream)
+    end = torch.cuda.Event(enable_timing=True)
+    end.record(stream)
+    barrier()
+    launches = binding.sparsp_launch_count() - launches0
+    clocks = sampler.finish()
+    cfg.check_status()
+
+    def avg(i):
+        return sum(ev[s][i].elapsed_time(ev[s][i + 1]) for s in range(steps)) / steps
+
+    mask_ms, dpack_ms, attn_ms = avg(0), avg(1), avg(2)
+    # one step = the three calls; with an L2 flush between steps the flush itself is outside the step
+    step_ms = ev[0][0].elapsed_time(end) / steps if cfg.flush is None else mask_ms + dpack_ms + attn_ms
+    # demand bookkeeping alone (plan-only call), to separate the gather kernel's time
+    pe = [torch.cuda.Event(enable_timing=True) for _ in range(2)]
+    cfg.step_plan()
+    torch.cuda.synchronize()
+    pe[0].record(stream)
+    for _ in range(steps):
+        cfg.step_plan()
+    pe[1].record(stream)
+    torch.cuda.synchronize()
+    plan_ms = pe[0].elapsed_time(pe[1]) / steps
+    return {"step": step_ms, "mask": mask_ms, "plan": plan_ms, "pack": max(dpack_ms - plan_ms, 1e-6), "attn": attn_ms,
+            "launches": launches, "clocks": clocks}
+
+
+def figures(cfg, t, peaks, traffic_table):
+    """The per-kernel figures of one measured configuration."""
+    attn_tflops = cfg.flops / (t["attn"] * 1e-3) / 1e12
+    pack_bytes = 2.0 * cfg.volume
+    pack_gbs = pack_bytes / (t["pack"] * 1e-3) / 1e9 if cfg.volume else 0.0
+    traffic = traffic_table.get((cfg.wl.name, cfg.k)) if cfg.tau <= 0 and cfg.H == cfg.wl.heads else None
+    return {
+        "ms_per_layer": t["step"],
+        "stage_ms": {"block_mask": t["mask"], "demand_plan": t["plan"], "pack": t["pack"], "sparse_attn": t["attn"]},
+        "attn_tflops": attn_tflops,
+        "attn_pct_bf16_peak": {"of_measured_burst": attn_tflops / peaks["bf16_tflops"],
+                               "of_measured_sustained": attn_tflops / peaks["bf16_tflops_sustained"],
+                               "of_nominal": attn_tflops / NOMINAL["bf16_tflops"]},
+        "pack_gbs": pack_gbs,
+        "pack_pct_hbm": {"of_measured": pack_gbs / peaks["hbm_gbs"], "of_nominal": pack_gbs / NOMINAL["hbm_gbs"]},
+        "volume_bytes_total": cfg.volume,
+        "kept_flops": cfg.flops,
+        "roofline": {"bound": "tensor", "kernel": "attn_fwd_kernel (+ attn_prep_kernel, timed together)",
+                     "achieved": attn_tflops, "peak": peaks["bf16_tflops"], "peak_source": peaks["source"] + " burst",
+                     "unit": "TFLOP/s", "frac": attn_tflops / peaks["bf16_tflops"],
+                     "traffic": traffic[0] if traffic else None,
+                     "traffic_source": traffic[1] if traffic else "no ncu capture of this configuration"},
+        "roofline_pack": {"bound": "hbm", "kernel": "pack_bulk_kernel", "achieved": pack_gbs, "peak": peaks["hbm_gbs"],
+                          "peak_source": peaks["source"], "unit": "GB/s", "frac": pack_gbs / peaks["hbm_gbs"],
+                          "algorithmic_bytes": pack_bytes},
+    }
+
+
+def sustained_attention(cfg, seconds, local_gpu, peaks):
+    """The attention call alone, back to back for `seconds`: long enough for the power cap to settle and for
+    NVML's clock samples to see it; reported against the sustained tensor peak."""
+    import torch
+    stream = torch.cuda.current_stream()
+    e = [torch.cuda.Event(enable_timing=True) for _ in range(2)]
+    cfg.step_attn()
+    torch.cuda.synchronize()
+    e[0].record(stream)
+    cfg.step_attn()
+    e[1].record(stream)
+    torch.cuda.synchronize()
+    n = max(3, int(seconds * 1e3 / max(e[0].elapsed_time(e[1]), 1e-3)))
+    sampler = ClockSampler(physical_gpu_index(local_gpu))
+    sampler.start()
+    e[0].record(stream)
+    for _ in range(n):
+        cfg.step_attn()
+    e[1].record(stream)
+    torch.cuda.synchronize()
+    clocks = sampler.finish()
+    ms = e[0].elapsed_time(e[1]) / n
+    tf = cfg.flops / (ms * 1e-3) / 1e12
+    return {"calls": n, "seconds": ms * n * 1e-3, "attn_ms": ms, "attn_tflops": tf,
+            "peak": peaks["bf16_tflops_sustained"], "peak_source": peaks["source"] + " sustained",
+            "frac": tf / peaks["bf16_tflops_sustained"], "clocks": clocks}
+
+
+def end_to_end(cfg, args, barrier):
+    """End to end through the public API from pinned host buffers, result read back to the host.  The path is
+    independent per head, so the heads go through in a few chunks on three streams (copy in, compute, copy
+    out): a chunk's kernels run while the next chunk's inputs arrive and the previous chunk's output leaves."""
+    import torch
+    binding, wl, dev = cfg.binding, cfg.wl, cfg.dev
+    Q, K, V, O, H, P, k = cfg.Q, cfg.K, cfg.V, cfg.O, cfg.H, cfg.P, cfg.k
+    stream = torch.cuda.current_stream()
+    h2d = 3 * Q.numel() * 2
+    d2h = O.numel() * 2 + cfg.do["volume_bytes"].numel() * 8
+    hQ, hK, hV = (torch.empty(x.shape, dtype=x.dtype, pin_memory=True) for x in (Q, K, V))
+    hQ.copy_(Q); hK.copy_(K); hV.copy_(V)
+    hO = torch.empty(O.shape, dtype=O.dtype, pin_memory=True)
+    n_chunks = min(4, H) if h2d >= (32 << 20) else 1  # a small workload gains nothing from more launches
+    bounds = [(c * H // n_chunks, (c + 1) * H // n_chunks) for c in range(n_chunks)]
+    chunks = []
+    for (h0, h1) in bounds:
+        sh = binding.make_shape(h1 - h0, cfg.d, wl.grid, wl.n_text, cfg.b)
+        c = {"h": (h0, h1), "shape": sh, "ws": binding.make_workspace(sh, P, dev),
+             "mo": binding.alloc_mask_outputs(sh, k, dev, with_list=True),
+             "do": binding.alloc_demand_outputs(sh, P, dev)}
+        c["hVol"] = torch.empty(c["do"]["volume_bytes"].shape, dtype=torch.int64, pin_memory=True)
+        chunks.append(c)
+
+    def chunk_mask(c):
+        h0, h1 = c["h"]
+        if args.tau > 0:
+            binding.sparsp_block_mask_cdf(c["shape"], Q[h0:h1], K[h0:h1], args.tau, 0.0, c["mo"]["mask"],
+                                          c["mo"]["kv_count"], None, None, c["ws"])
+        else:
+            binding.sparsp_block_mask(c["shape"], Q[h0:h1], K[h0:h1], k, c["mo"]["mask"], c["mo"]["kv_list"],
+                                      c["mo"]["kv_count"], None, None, c["ws"])
+
+    def chunk_pack(c, plan_only):
+        h0, h1 = c["h"]
+        o = c["do"]
+        binding.sparsp_demand_pack(c["shape"], c["mo"]["mask"], cfg.rank_d, P,
+                                   binding.SPARSP_PLAN_ONLY if plan_only else 0,
+                                   None if plan_only else K[h0:h1], None if plan_only else V[h0:h1],
+                                   o["union_mask"], o["cnt"], o["seg_offset"], o["seg_total"], o["volume_bytes"],
+                                   None if plan_only else c["packed"], 0 if plan_only else c["packed"].numel(),
+                                   None, c["ws"])
+
+    for c in chunks:  # size each chunk's packed buffer once (the masks are a function of the inputs)
+        chunk_mask(c)
+        chunk_pack(c, True)
+        torch.cuda.synchronize()
+        c["packed"] = torch.empty(max(int(c["do"]["seg_total"].sum().item()) * cfg.entry, 16), dtype=torch.uint8,
+                                  device=dev)
+    s_in, s_comp, s_out = torch.cuda.Stream(dev), torch.cuda.Stream(dev), torch.cuda.Stream(dev)
+    ev_in = [torch.cuda.Event() for _ in chunks]
+    ev_comp = [torch.cuda.Event() for _ in chunks]
+    ev_out = [torch.cuda.Event() for _ in chunks]
+
+    def e2e_step():
+        for i, c in enumerate(chunks):
+            h0, h1 = c["h"]
+            with torch.cuda.stream(s_in):
+                s_in.wait_event(ev_comp[i])  # the previous step's kernels have read this slice
+                Q[h0:h1].copy_(hQ[h0:h1], non_blocking=True)
+                K[h0:h1].copy_(hK[h0:h1], non_blocking=True)
+                V[h0:h1].copy_(hV[h0:h1], non_blocking=True)
+                ev_in[i].record(s_in)
+            with torch.cuda.stream(s_comp):
+                s_comp.wait_event(ev_in[i])
+                s_comp.wait_event(ev_out[i])  # the previous step's output slice has left
+                chunk_mask(c)
+                chunk_pack(c, False)
+                binding.sparsp_sparse_attn_fwd(c["shape"], Q[h0:h1], K[h0:h1], V[h0:h1], c["mo"]["mask"], 0.0,
+                                               O[h0:h1], None, c["ws"])
+                ev_comp[i].record(s_comp)
+            with torch.cuda.stream(s_out):
+                s_out.wait_event(ev_comp[i])
+                hO[h0:h1].copy_(O[h0:h1], non_blocking=True)
+                c["hVol"].copy_(c["do"]["volume_bytes"], non_blocking=True)
+                ev_out[i].record(s_out)
+
+    def join():
+        for st_ in (s_in, s_comp, s_out):
+            stream.wait_stream(st_)
+
+    e2e_steps = max(1, min(args.steps, 5))
+    for st_ in (s_in, s_comp, s_out):
+        st_.wait_stream(stream)
+    e2e_step()
+    join()
+    barrier()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record(stream)
+    for st_ in (s_in, s_comp, s_out):
+        st_.wait_stream(stream)
+    for _ in range(e2e_steps):
+        e2e_step()
+    join()
+    e1.record(stream)
+    barrier()
+    e2e_ms = e0.elapsed_time(e1) / e2e_steps
+    assert all(binding.sparsp_status(c["ws"]) == binding.SPARSP_OK for c in chunks)
+    assert int(sum(int(c["hVol"].sum().item()) for c in chunks)) == int(cfg.volume)
+    return e2e_ms, n_chunks, h2d, d2h
+
+
 def run_ours(args):
+    import gc
+
     import torch
     import torch.distributed as dist
 
-    from paper_2609_32197_b200 import binding, dist_util, synth
+    from paper_2609_32197_b200 import binding, dist_util
 
     rank = int(os.environ.get("RANK", 0))
     world = int(os.environ.get("WORLD_SIZE", 1))
@@ -146,65 +474,8 @@ def run_ours(args):
     if world > 1:
         dist.init_process_group("nccl", device_id=dev)
     binding.lib()
-
-    wl, placement = resolve_workload(args)
-    wl = dist_util.replica_workload(wl, rank)  # every rank its own replica of the workload
-    H, d, b, P = wl.heads, wl.head_dim, wl.block, wl.ranks
-    shape = binding.make_shape(H, d, wl.grid, wl.n_text, b)
-    g = binding.sparsp_geometry(shape)
-    N, NB = g.n_tokens, g.n_blocks
-    pct = args.pct if args.pct else (wl.topk_pct[0] if wl.topk_pct else None)
-    k = wl.topk_abs if pct is None else binding.sparsp_resolve_topk(pct, g.n_video_blocks)
-
-    Q, K, V = synth.make_qkv(wl, dev)
-    if placement == "contiguous":
-        rank_of_block = binding.sparsp_placement_contiguous(shape, P)
-    elif placement == "periodic":
-        rank_of_block = binding.sparsp_placement_periodic(shape, P)
-    else:
-        rank_of_block = synth.shuffled_placement(NB, P, seed=1)
-    rank_d = rank_of_block.to(dev)
-
-    ws = binding.make_workspace(shape, P, dev)
-    mo = binding.alloc_mask_outputs(shape, k, dev, with_list=True)
-    do = binding.alloc_demand_outputs(shape, P, dev)
-    O = torch.empty_like(Q)
-    entry = 2 * b * d * 2
-
-    def step_mask():
-        if args.tau > 0:  # CDF-threshold selection instead of top-k (rows keep different numbers of blocks)
-            binding.sparsp_block_mask_cdf(shape, Q, K, args.tau, 0.0, mo["mask"], mo["kv_count"], None, None, ws)
-        else:
-            binding.sparsp_block_mask(shape, Q, K, k, mo["mask"], mo["kv_list"], mo["kv_count"], None, None, ws)
-
-    def step_plan():
-        binding.sparsp_demand_pack(shape, mo["mask"], rank_d, P, binding.SPARSP_PLAN_ONLY, None, None,
-                                   do["union_mask"], do["cnt"], do["seg_offset"], do["seg_total"],
-                                   do["volume_bytes"], None, 0, None, ws)
-
-    # size the packed buffer once (the mask is a function of the inputs, which do not change)
-    step_mask()
-    step_plan()
-    torch.cuda.synchronize()
-    total_entries = int(do["seg_total"].sum().item())
-    packed = torch.empty(max(total_entries * entry, 16), dtype=torch.uint8, device=dev)
-    volume = do["volume_bytes"].sum().item()
-
-    def step_pack():
-        binding.sparsp_demand_pack(shape, mo["mask"], rank_d, P, 0, K, V, do["union_mask"], do["cnt"],
-                                   do["seg_offset"], do["seg_total"], do["volume_bytes"], packed,
-                                   packed.numel(), None, ws)
-
-    def step_attn():
-        binding.sparsp_sparse_attn_fwd(shape, Q, K, V, mo["mask"], 0.0, O, None, ws)
-
-    def step():
-        step_mask()
-        step_pack()
-        step_attn()
-
-    flops, kept_pairs = kept_flops_and_counts(mo["mask"], N, b, d)
-    stream = torch.cuda.current_stream()
+    peaks = load_peaks()
+    traffic_table = load_attn_traffic()
 
     def barrier():
         torch.cuda.synchronize()
@@ -212,162 +483,38 @@ def run_ours(args):
             dist.barrier()
         torch.cuda.synchronize()
 
-    for _ in range(args.warmup):
-        step()
-    barrier()
-    assert binding.sparsp_status(ws) == binding.SPARSP_OK, binding.sparsp_last_error()
+    wl, placement = resolve_workload(args)
+    pct = args.pct if args.pct else (wl.topk_pct[0] if wl.topk_pct else None)
+    if args.shard == "heads" and world > 1:
+        # strong scaling: ONE layer, rank r takes heads [r*H/N, (r+1)*H/N) of all three calls (every step of the
+        # path is independent per head, so nothing is exchanged)
+        head_range = dist_util.head_shard(wl.heads, rank, world)
+        scaling = "strong"
+    else:
+        # weak scaling: every rank its own replica of the workload (own seed)
+        wl = dist_util.replica_workload(wl, rank)
+        head_range = None
+        scaling = "weak"
+    cfg = Config(wl, placement, pct, args.tau, dev, head_range)
+    t = time_steps(cfg, args.steps, args.warmup, barrier, local)
+    fig = figures(cfg, t, peaks, traffic_table)
 
-    sampler = ClockSampler(physical_gpu_index(local))
-    sampler.start()
-    launches0 = binding.sparsp_launch_count()
-    ev = [[torch.cuda.Event(enable_timing=True) for _ in range(4)] for _ in range(args.steps)]
-    barrier()
-    for s in range(args.steps):
-        ev[s][0].record(stream)
-        step_mask()
-        ev[s][1].record(stream)
-        step_pack()
-        ev[s][2].record(stream)
-        step_attn()
-        ev[s][3].record(stream)
-    end = torch.cuda.Event(enable_timing=True)
-    end.record(stream)
-    barrier()
-    launches = binding.sparsp_launch_count() - launches0
-    total_ms = ev[0][0].elapsed_time(end)
-    clocks = sampler.finish()
-    assert binding.sparsp_status(ws) == binding.SPARSP_OK, binding.sparsp_last_error()
-
-    def avg(i):
-        return sum(ev[s][i].elapsed_time(ev[s][i + 1]) for s in range(args.steps)) / args.steps
-
-    mask_ms, dpack_ms, attn_ms = avg(0), avg(1), avg(2)
-
-    # demand bookkeeping alone (plan-only call), to separate the gather kernel's time
-    pe = [torch.cuda.Event(enable_timing=True) for _ in range(2)]
-    step_plan()
-    torch.cuda.synchronize()
-    pe[0].record(stream)
-    for _ in range(args.steps):
-        step_plan()
-    pe[1].record(stream)
-    torch.cuda.synchronize()
-    plan_ms = pe[0].elapsed_time(pe[1]) / args.steps
-    pack_ms = max(dpack_ms - plan_ms, 1e-6)
-
-    # End to end through the public API from pinned host buffers, result read back to the host.  The path is
-    # independent per head, so the heads go through in a few chunks on three streams (copy in, compute, copy
-    # out): a chunk's kernels run while the next chunk's inputs arrive and the previous chunk's output leaves.
-    h2d = 3 * Q.numel() * 2
-    d2h = O.numel() * 2 + do["volume_bytes"].numel() * 8
-    e2e_ms = float("nan")
-    e2e_chunks = 0
+    e2e_ms, e2e_chunks, h2d, d2h = float("nan"), 0, 3 * cfg.Q.numel() * 2, cfg.O.numel() * 2 + cfg.do["volume_bytes"].numel() * 8
     if not args.no_e2e:
-        hQ, hK, hV = (torch.empty(x.shape, dtype=x.dtype, pin_memory=True) for x in (Q, K, V))
-        hQ.copy_(Q); hK.copy_(K); hV.copy_(V)
-        hO = torch.empty(O.shape, dtype=O.dtype, pin_memory=True)
-        n_chunks = min(4, H) if h2d >= (32 << 20) else 1  # a small workload gains nothing from more launches
-        e2e_chunks = n_chunks
-        bounds = [(c * H // n_chunks, (c + 1) * H // n_chunks) for c in range(n_chunks)]
-        chunks = []
-        for (h0, h1) in bounds:
-            sh = binding.make_shape(h1 - h0, d, wl.grid, wl.n_text, b)
-            c = {"h": (h0, h1), "shape": sh, "ws": binding.make_workspace(sh, P, dev),
-                 "mo": binding.alloc_mask_outputs(sh, k, dev, with_list=True),
-                 "do": binding.alloc_demand_outputs(sh, P, dev)}
-            c["hVol"] = torch.empty(c["do"]["volume_bytes"].shape, dtype=torch.int64, pin_memory=True)
-            chunks.append(c)
-
-        def chunk_mask(c):
-            h0, h1 = c["h"]
-            if args.tau > 0:
-                binding.sparsp_block_mask_cdf(c["shape"], Q[h0:h1], K[h0:h1], args.tau, 0.0, c["mo"]["mask"],
-                                              c["mo"]["kv_count"], None, None, c["ws"])
-            else:
-                binding.sparsp_block_mask(c["shape"], Q[h0:h1], K[h0:h1], k, c["mo"]["mask"], c["mo"]["kv_list"],
-                                          c["mo"]["kv_count"], None, None, c["ws"])
-
-        def chunk_pack(c, plan_only):
-            h0, h1 = c["h"]
-            o = c["do"]
-            binding.sparsp_demand_pack(c["shape"], c["mo"]["mask"], rank_d, P,
-                                       binding.SPARSP_PLAN_ONLY if plan_only else 0,
-                                       None if plan_only else K[h0:h1], None if plan_only else V[h0:h1],
-                                       o["union_mask"], o["cnt"], o["seg_offset"], o["seg_total"], o["volume_bytes"],
-                                       None if plan_only else c["packed"], 0 if plan_only else c["packed"].numel(),
-                                       None, c["ws"])
-
-        for c in chunks:  # size each chunk's packed buffer once (the masks are a function of the inputs)
-            chunk_mask(c)
-            chunk_pack(c, True)
-            torch.cuda.synchronize()
-            c["packed"] = torch.empty(max(int(c["do"]["seg_total"].sum().item()) * entry, 16), dtype=torch.uint8,
-                                      device=dev)
-        s_in, s_comp, s_out = torch.cuda.Stream(dev), torch.cuda.Stream(dev), torch.cuda.Stream(dev)
-        ev_in = [torch.cuda.Event() for _ in chunks]
-        ev_comp = [torch.cuda.Event() for _ in chunks]
-        ev_out = [torch.cuda.Event() for _ in chunks]
-
-        def e2e_step():
-            for i, c in enumerate(chunks):
-                h0, h1 = c["h"]
-                with torch.cuda.stream(s_in):
-                    s_in.wait_event(ev_comp[i])  # the previous step's kernels have read this slice
-                    Q[h0:h1].copy_(hQ[h0:h1], non_blocking=True)
-                    K[h0:h1].copy_(hK[h0:h1], non_blocking=True)
-                    V[h0:h1].copy_(hV[h0:h1], non_blocking=True)
-                    ev_in[i].record(s_in)
-                with torch.cuda.stream(s_comp):
-                    s_comp.wait_event(ev_in[i])
-                    s_comp.wait_event(ev_out[i])  # the previous step's output slice has left
-                    chunk_mask(c)
-                    chunk_pack(c, False)
-                    binding.sparsp_sparse_attn_fwd(c["shape"], Q[h0:h1], K[h0:h1], V[h0:h1], c["mo"]["mask"], 0.0,
-                                                   O[h0:h1], None, c["ws"])
-                    ev_comp[i].record(s_comp)
-                with torch.cuda.stream(s_out):
-                    s_out.wait_event(ev_comp[i])
-                    hO[h0:h1].copy_(O[h0:h1], non_blocking=True)
-                    c["hVol"].copy_(c["do"]["volume_bytes"], non_blocking=True)
-                    ev_out[i].record(s_out)
-
-        def join():
-            for st_ in (s_in, s_comp, s_out):
-                stream.wait_stream(st_)
-
-        e2e_steps = max(1, min(args.steps, 5))
-        for st_ in (s_in, s_comp, s_out):
-            st_.wait_stream(stream)
-        e2e_step()
-        join()
-        barrier()
-        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-        e0.record(stream)
-        for st_ in (s_in, s_comp, s_out):
-            st_.wait_stream(stream)
-        for _ in range(e2e_steps):
-            e2e_step()
-        join()
-        e1.record(stream)
-        barrier()
-        e2e_ms = e0.elapsed_time(e1) / e2e_steps
-        assert all(binding.sparsp_status(c["ws"]) == binding.SPARSP_OK for c in chunks)
-        assert int(sum(int(c["hVol"].sum().item()) for c in chunks)) == int(volume)
+        e2e_ms, e2e_chunks, h2d, d2h = end_to_end(cfg, args, barrier)
+    sustained = None
+    if world == 1 and args.sustained_s > 0:
+        sustained = sustained_attention(cfg, args.sustained_s, local, peaks)
 
     # max over ranks (device-timed), whole-job totals
     tm, tot = dist_util.reduce_over_ranks(
-        {"total": total_ms, "e2e": e2e_ms if e2e_ms == e2e_ms else 0.0, "attn": attn_ms, "pack": pack_ms, "mask": mask_ms},
-        {"flops": flops, "launches": float(launches)}, dev)
-    total_ms, attn_ms, pack_ms, mask_ms = tm["total"], tm["attn"], tm["pack"], tm["mask"]
+        {"step": t["step"], "e2e": e2e_ms if e2e_ms == e2e_ms else 0.0},
+        {"flops": cfg.flops, "launches": float(t["launches"]), "h2d": float(h2d), "d2h": float(d2h)}, dev)
+    ms_per_step = tm["step"]
     if e2e_ms == e2e_ms:
         e2e_ms = tm["e2e"]
-    flops_all, launches_all = tot["flops"], tot["launches"]
-    ms_per_step = total_ms / args.steps
+    flops_all = tot["flops"]
 
-    peaks = load_peaks()
-    attn_tflops = flops / (attn_ms * 1e-3) / 1e12
-    pack_bytes = 2.0 * volume
-    pack_gbs = pack_bytes / (pack_ms * 1e-3) / 1e9 if volume else 0.0
     result = {
         "metric": METRIC,
         "value": flops_all / (ms_per_step * 1e-3) / 1e12,
@@ -377,41 +524,44 @@ def run_ours(args):
         "warmup": args.warmup,
         "ms_per_step": ms_per_step,
         "higher_is_better": True,
-        "scaling": "weak",
+        "scaling": scaling,
         "vs_baseline": None,
         "dtype": "bf16",
         "data": "synthetic",
-        "config": {
-            "workload": wl.name, "heads": H, "head_dim": d, "grid": list(wl.grid), "n_text": wl.n_text,
-            "tokens": N, "block": b, "n_blocks": NB, "topk_blocks": (k if args.tau <= 0 else None),
-            "selection": ("top-k" if args.tau <= 0 else "cdf tau=%g" % args.tau), "kept_pairs": kept_pairs,
-            "virtual_ranks": P, "placement": placement, "layout": "[H][N][d]",
-            "l2_policy": "inputs larger than L2 (Q+K+V = %.0f MB)" % (3 * Q.numel() * 2 / 1e6),
-        },
-        "ms_per_layer": ms_per_step,
-        "stage_ms": {"block_mask": mask_ms, "demand_plan": plan_ms, "pack": pack_ms, "sparse_attn": attn_ms},
-        "attn_tflops": attn_tflops,
-        "attn_pct_bf16_peak": {"of_measured_burst": attn_tflops / peaks["bf16_tflops"],
-                               "of_measured_sustained": attn_tflops / peaks["bf16_tflops_sustained"],
-                               "of_nominal": attn_tflops / NOMINAL["bf16_tflops"]},
-        "pack_gbs": pack_gbs,
-        "pack_pct_hbm": {"of_measured": pack_gbs / peaks["hbm_gbs"], "of_nominal": pack_gbs / NOMINAL["hbm_gbs"]},
-        "volume_bytes_total": volume,
-        "roofline": {"bound": "tensor", "kernel": "attn_fwd_kernel (+ attn_prep_kernel, timed together)", "achieved": attn_tflops,
-                     "peak": peaks["bf16_tflops"], "peak_source": peaks["source"] + " burst", "unit": "TFLOP/s",
-                     "frac": attn_tflops / peaks["bf16_tflops"],
-                     "traffic": ATTN_DRAM_TRAFFIC.get((wl.name, k)) if args.tau <= 0 else None},
-        "roofline_pack": {"bound": "hbm", "kernel": "pack_bulk_kernel", "achieved": pack_gbs, "peak": peaks["hbm_gbs"],
-                          "peak_source": peaks["source"], "unit": "GB/s", "frac": pack_gbs / peaks["hbm_gbs"],
-                          "algorithmic_bytes": pack_bytes},
-        "e2e": {"value": None if e2e_ms != e2e_ms else flops_all / (e2e_ms * 1e-3) / 1e12, "unit": "TFLOP/s",
-                "ms_per_step": None if e2e_ms != e2e_ms else e2e_ms, "head_chunks": e2e_chunks,
-                "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h},
-        "gpu_launches": int(launches_all),
-        "clocks": clocks,
+        "config": cfg.describe() | ({"sharding": "heads %d-%d of %d on rank 0" % (head_range[0], head_range[1] - 1, wl.heads)}
+                                    if head_range else {}),
     }
+    result.update(fig)
+    result["ms_per_layer"] = ms_per_step
+    result["e2e"] = {"value": None if e2e_ms != e2e_ms else flops_all / (e2e_ms * 1e-3) / 1e12, "unit": "TFLOP/s",
+                     "ms_per_step": None if e2e_ms != e2e_ms else e2e_ms, "head_chunks": e2e_chunks,
+                     "h2d_bytes_per_step": int(tot["h2d"]), "d2h_bytes_per_step": int(tot["d2h"])}
+    result["gpu_launches"] = int(tot["launches"])
+    result["clocks"] = t["clocks"]
+    if sustained:
+        result["sustained"] = sustained
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
-        result["cpu_baseline"] = cpu_baseline(wl, k, placement, rank_of_block.numpy(), Q, K, V, flops, budget_s=15.0)
+        result["cpu_baseline"] = cpu_baseline(cfg.wl, cfg.k, placement, cfg.rank_of_block.numpy(), cfg.Q, cfg.K, cfg.V,
+                                              cfg.flops, budget_s=15.0)
+    if world == 1 and not args.no_per_config and args.tau <= 0 and not args.heads:
+        # every configuration of the contract, measured the same way in this run (>= 10 timed iterations each)
+        headline = (cfg.wl.name, cfg.k, placement)
+        rows = []
+        del cfg
+        for (name, p_, plc) in PER_CONFIG:
+            gc.collect()
+            torch.cuda.empty_cache()
+            from paper_2609_32197_b200 import synth
+            c = Config(synth.WORKLOADS[name], plc, p_, 0.0, dev)
+            tt = time_steps(c, max(10, min(args.steps, 20)), 3, barrier, local)
+            row = {"config": c.describe()}
+            row.update(figures(c, tt, peaks, traffic_table))
+            row["clocks"] = tt["clocks"]
+            row["gpu_launches"] = tt["launches"]
+            row["is_headline_config"] = (name, c.k, plc) == headline
+            rows.append(row)
+            del c
+        result["per_config"] = rows
     if rank == 0:
         print(json.dumps(result))
     if world > 1:
@@ -546,13 +696,19 @@ def main():
     ap.add_argument("--steps", type=int, default=10)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--workload", default="mid", choices=["tiny", "mid", "cog", "wan", "hunyuan"])
+    ap.add_argument("--workload", default="hunyuan", choices=["tiny", "mid", "cog", "wan", "hunyuan"],
+                    help="headline configuration (default: the largest single-GPU one, Hunyuan-like at 10 %%)")
     ap.add_argument("--pct", type=int, default=0, help="top-k as a percentage of the video blocks")
     ap.add_argument("--tau", type=float, default=0.0, help="CDF-threshold selection with this mass instead of top-k (ours only)")
     ap.add_argument("--placement", default=None, choices=[None, "contiguous", "periodic", "shuffle"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true", help="skip the host-buffer end-to-end leg")
     ap.add_argument("--heads", type=int, default=0, help="override the head count (small profiling cases)")
+    ap.add_argument("--no-per-config", action="store_true", help="skip the per_config list (all eight configurations)")
+    ap.add_argument("--sustained-s", type=float, default=2.0,
+                    help="seconds of back-to-back attention calls for the sustained figure (0 = skip)")
+    ap.add_argument("--shard", default="replicas", choices=["replicas", "heads"],
+                    help="with N > 1: independent replicas (weak scaling) or the heads of ONE layer split over the ranks (strong)")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
     if args.impl == "reference":

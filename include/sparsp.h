@@ -297,6 +297,14 @@ SPARSP_API int sparsp_demand_plan_noalloc(const sparsp_shape* shape, const uint3
  * reported a problem since the last reset), then resets it. */
 SPARSP_API int sparsp_status(void* workspace, void* stream, int32_t* code);
 
+/* Diagnostic (no counterpart in the paper): launches one tiny kernel whose only wait is on a barrier nobody
+ * arrives on, bounded by `limit_cycles` SM clock cycles (1 .. 1e8) -- the same bounded wait every kernel of the
+ * library uses.  The wait runs out, the kernel writes SPARSP_ERR_TIMEOUT and the detail words (where = 99, CTA 0)
+ * to the workspace's status words and returns normally; the next sparsp_status() reports it (and resets it), and
+ * the context stays usable.  Nothing else is in flight in that kernel (no copy, no MMA).  For testing the
+ * error path of bounded waits without any kernel actually being stuck; any workspace of >= 256 bytes will do. */
+SPARSP_API int sparsp_selftest_wait_timeout(void* workspace, int64_t limit_cycles, void* stream);
+
 /* Text of the calling thread's most recent error ("" if none). */
 SPARSP_API const char* sparsp_last_error(void);
 

@@ -31,7 +31,7 @@ EXPORTS = [
     "sparsp_status", "sparsp_last_error", "sparsp_launch_count", "sparsp_demand_plan_noalloc",
     "sparsp_hop_mask", "sparsp_attn_merge", "sparsp_sparse_attn_fwd_packed", "sparsp_block_mask_cdf",
     "sparsp_placement_permutation", "sparsp_permute_tokens", "sparsp_sharing_histogram", "sparsp_exchange_plan",
-    "sparsp_hop_chunk_mask",
+    "sparsp_hop_chunk_mask", "sparsp_selftest_wait_timeout",
 ]
 
 
@@ -265,6 +265,10 @@ def sparsp_status(workspace) -> int:
     code = ctypes.c_int32()
     _check(lib().sparsp_status(_ptr(workspace), _stream(), ctypes.byref(code)))
     return code.value
+
+
+def sparsp_selftest_wait_timeout(workspace, limit_cycles: int):
+    _check(lib().sparsp_selftest_wait_timeout(_ptr(workspace), ctypes.c_int64(limit_cycles), _stream()))
 
 
 def sparsp_last_error() -> str:

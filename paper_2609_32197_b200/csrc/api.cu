@@ -528,6 +528,17 @@ int sparsp_attn_merge(const sparsp_shape* shape, const void* O_a, const float* l
   return launch_attn_merge(*shape, g, O_a, lse_a, O_b, lse_b, O, lse, (cudaStream_t)stream);
 }
 
+int sparsp_selftest_wait_timeout(void* workspace, int64_t limit_cycles, void* stream) {
+  SPARSP_TRY(check_ptr(workspace, "workspace", 256));
+  if (limit_cycles < 1 || limit_cycles > 100000000LL) {
+    set_error("limit_cycles %lld outside 1..1e8", (long long)limit_cycles);
+    return SPARSP_ERR_INVALID_ARG;
+  }
+  WsLayout L;
+  L.status = 0;  // the status words open the workspace whatever the shape
+  return launch_wait_timeout((char*)workspace, L, limit_cycles, (cudaStream_t)stream);
+}
+
 int sparsp_status(void* workspace, void* stream, int32_t* code) {
   SPARSP_TRY(check_ptr(workspace, "workspace", 256));
   if (!code) {

@@ -87,6 +87,7 @@ int launch_attn_packed(const sparsp_shape& s, const Geometry& g, const void* Q, 
                        cudaStream_t st);
 int launch_hop_mask(const Geometry& g, const uint32_t* mask, const int32_t* rank, int consumer, int producer,
                     int head_begin, int head_end, uint32_t* hop, cudaStream_t st);
+int launch_wait_timeout(char* ws, const WsLayout& L, long long limit_cycles, cudaStream_t st);
 int launch_attn_merge(const sparsp_shape& s, const Geometry& g, const void* Oa, const float* la, const void* Ob,
                       const float* lb, void* O, float* lse, cudaStream_t st);
 

@@ -27,29 +27,38 @@ __global__ void hop_mask_kernel(const uint32_t* __restrict__ mask, const int32_t
   hop[idx] = out;
 }
 
-// Thread per (row, 8 columns).  O_a, O_b, O: bf16 with the shape's strides; lse: fp32 [B][H][N].
+// Thread per (row, 8 columns).  O_a, O_b, O: bf16 with the shape's strides; lse: fp32 [B][H][N].  O may be O_a or
+// O_b and lse may be lse_a or lse_b (no pointer is declared restrict): a thread reads the 16 bytes it later
+// writes, and only the row's first thread touches the log-sum-exp values -- it reads both inputs, computes the
+// weights and hands them to the row's other threads by shuffle (the D/8 threads of a row are consecutive lanes of
+// one warp) before it writes the merged value.
 template <int D>
-__global__ void attn_merge_kernel(const __nv_bfloat16* __restrict__ Oa, const float* __restrict__ la,
-                                  const __nv_bfloat16* __restrict__ Ob, const float* __restrict__ lb,
-                                  __nv_bfloat16* __restrict__ O, float* __restrict__ lse, int H, int64_t N,
-                                  int64_t sB, int64_t sH, int64_t sT, int64_t n_rows) {
+__global__ void attn_merge_kernel(const __nv_bfloat16* Oa, const float* la, const __nv_bfloat16* Ob, const float* lb,
+                                  __nv_bfloat16* O, float* lse, int H, int64_t N, int64_t sB, int64_t sH, int64_t sT,
+                                  int64_t n_rows) {
   constexpr int VPR = D / 8;
   const int64_t idx = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
   const int64_t row = idx / VPR;
   const int col = (int)(idx % VPR);
-  if (row >= n_rows) return;
+  const bool live = row < n_rows;
+  float wa = 0.0f, wb = 0.0f, out_lse = -INFINITY;
+  if (live && col == 0) {
+    const float a = la[row], b = lb[row];
+    const float m = fmaxf(a, b);
+    if (m > -INFINITY) {
+      const float ea = __expf(a - m), eb = __expf(b - m);
+      const float tot = ea + eb;
+      wa = ea / tot;
+      wb = eb / tot;
+      out_lse = m + __logf(tot);
+    }
+  }
+  const int leader = (threadIdx.x & 31) & ~(VPR - 1);  // lane of the row's first thread
+  wa = __shfl_sync(0xffffffffu, wa, leader);
+  wb = __shfl_sync(0xffffffffu, wb, leader);
+  if (!live) return;
   const int64_t tok = row % N, bh = row / N;
   const int64_t off = (bh / H) * sB + (bh % H) * sH + tok * sT + col * 8;
-  const float a = la[row], b = lb[row];
-  const float m = fmaxf(a, b);
-  float wa = 0.0f, wb = 0.0f, out_lse = -INFINITY;
-  if (m > -INFINITY) {
-    const float ea = __expf(a - m), eb = __expf(b - m);
-    const float tot = ea + eb;
-    wa = ea / tot;
-    wb = eb / tot;
-    out_lse = m + __logf(tot);
-  }
   const uint4 va = *reinterpret_cast<const uint4*>(Oa + off);
   const uint4 vb = *reinterpret_cast<const uint4*>(Ob + off);
   const uint32_t xa[4] = {va.x, va.y, va.z, va.w}, xb[4] = {vb.x, vb.y, vb.z, vb.w};

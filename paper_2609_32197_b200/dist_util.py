@@ -16,6 +16,12 @@ def replica_workload(wl: synth.Workload, rank: int) -> synth.Workload:
                           wl.topk_pct, wl.ranks, wl.placements, seed=wl.seed + rank)
 
 
+def head_shard(heads: int, rank: int, world: int):
+    """Heads [begin, end) of ONE layer that rank `rank` of `world` takes (strong scaling by heads: every step of
+    the path is independent per head, so the shards need no exchange and their outputs concatenate)."""
+    return (rank * heads) // world, ((rank + 1) * heads) // world
+
+
 def reduce_over_ranks(times_ms: dict, totals: dict, device="cpu"):
     """Device-timed milliseconds -> MAX over ranks; work totals (flops, launches) -> SUM over ranks.
     With a single process (no process group) the inputs come back unchanged."""

@@ -94,8 +94,9 @@ def features(wl: Workload, device="cpu") -> torch.Tensor:
     return f
 
 
-def make_qkv(wl: Workload, device="cpu", heads: int | None = None):
-    """-> Q, K, V bf16 tensors of shape [H][N][d] on ``device`` (H = wl.heads unless overridden).
+def make_qkv(wl: Workload, device="cpu", heads: int | None = None, head_begin: int = 0):
+    """-> Q, K, V bf16 tensors of shape [H][N][d] on ``device`` (H = wl.heads unless overridden); output head
+    h holds the workload's head ``head_begin + h`` (a shard of the heads draws the same values as the whole).
 
     Random draws are made by a CPU generator per (seed, head, tensor) when device is the CPU and by
     the device's generator otherwise; values for a given device type are reproducible."""
@@ -108,7 +109,7 @@ def make_qkv(wl: Workload, device="cpu", heads: int | None = None):
     dev = torch.device(device)
     for h in range(H):
         g = torch.Generator(device=dev.type if dev.type == "cpu" else dev)
-        g.manual_seed(wl.seed * 1000003 + h * 101 + 1)
+        g.manual_seed(wl.seed * 1000003 + (head_begin + h) * 101 + 1)
         W = torch.randn(d, N_FEAT, generator=g, dtype=torch.float32, device=device) / math.sqrt(N_FEAT)
         base = 2.0 * (f @ W.t())
         Q[h] = (base + 0.5 * torch.randn(N, d, generator=g, dtype=torch.float32, device=device)).to(torch.bfloat16)

@@ -91,6 +91,33 @@ def test_merge_kernel_matches_oracle_elementwise(oracle_mod, binding):
     assert np.array_equal(np.isneginf(lse.cpu().numpy()), np.isneginf(rl))
 
 
+@pytest.mark.parametrize("d", [64, 128])
+@pytest.mark.parametrize("alias", ["a", "b"])
+def test_merge_in_place_equals_out_of_place(binding, d, alias):
+    """O / lse may alias either input: the result must be bit for bit the out-of-place one."""
+    rng = np.random.default_rng(9 + d)
+    H, N = 3, 333
+    shape = binding.make_shape(H, d, (1, 9, 37), 0, 64)
+    oa = torch.tensor(rng.standard_normal((1, H, N, d)), dtype=torch.float32).to(torch.bfloat16).cuda()
+    ob = torch.tensor(rng.standard_normal((1, H, N, d)), dtype=torch.float32).to(torch.bfloat16).cuda()
+    la = torch.tensor(rng.standard_normal((1, H, N)) * 3, dtype=torch.float32).cuda()
+    lb = torch.tensor(rng.standard_normal((1, H, N)) * 3, dtype=torch.float32).cuda()
+    la[0, 0, :7] = float("-inf")
+    lb[0, 0, 3:11] = float("-inf")
+    out, lse = torch.empty_like(oa), torch.empty_like(la)
+    binding.sparsp_attn_merge(shape, oa, la, ob, lb, out, lse)
+    xa, xla, xb, xlb = oa.clone(), la.clone(), ob.clone(), lb.clone()
+    if alias == "a":
+        binding.sparsp_attn_merge(shape, xa, xla, xb, xlb, xa, xla)
+        got, got_l = xa, xla
+    else:
+        binding.sparsp_attn_merge(shape, xa, xla, xb, xlb, xb, xlb)
+        got, got_l = xb, xlb
+    torch.cuda.synchronize()
+    assert torch.equal(got.view(torch.int16), out.view(torch.int16))
+    assert torch.equal(got_l.view(torch.int32), lse.view(torch.int32))
+
+
 @pytest.mark.parametrize("d,b,layout", [(128, 128, "HND"), (64, 64, "HND"), (128, 64, "NHD"), (64, 128, "HND")])
 @pytest.mark.parametrize("v_scale", [1.0, 0.5])
 def test_attention_reading_remote_blocks_from_the_packed_buffer(oracle_mod, binding, d, b, layout, v_scale):

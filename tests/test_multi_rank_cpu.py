@@ -95,3 +95,50 @@ def test_two_ranks_derive_the_same_transfer_list():
     assert res[0][0] == res[1][0] and res[0][1] and res[1][1]   # producer's and consumer's view agree, and with the oracle
     for r in range(world):
         assert sum(t[7] for t in res[r][0] if t[0] == r) == res[r][2]   # what rank r receives is its exchange volume
+
+
+def _head_shard_worker(rank, world, port, out):
+    """Strong scaling by heads: rank r takes heads [r*H/N, (r+1)*H/N) of ONE layer through all three steps."""
+    import numpy as np
+    os.environ["MASTER_ADDR"] = "127.0.0.1"
+    os.environ["MASTER_PORT"] = str(port)
+    dist.init_process_group("gloo", rank=rank, world_size=world)
+    import oracle
+    from paper_2609_32197_b200 import dist_util, synth
+    wl = synth.Workload("shard", 5, 64, (3, 8, 16), 20, 64, 3, None, 3, seed=77)  # 5 heads over 2 ranks: 2 + 3
+    h0, h1 = dist_util.head_shard(wl.heads, rank, world)
+    Q, K, V = synth.make_qkv(wl, "cpu", heads=h1 - h0, head_begin=h0)
+    placement = oracle.placement_contiguous(wl.n_blocks, wl.ranks)
+    m = oracle.block_mask(Q, K, wl.block, wl.topk_abs, wl.n_text)
+    dem = oracle.demand(m["mask"], placement, wl.ranks, wl.block, wl.head_dim)
+    o, lse = oracle.attn_all(Q, K, V, m["mask"], wl.block)
+    # the only thing that crosses ranks is the reduction of the per-rank volumes (SUM) for the report
+    _, tot = dist_util.reduce_over_ranks({"step": 1.0}, {"volume": float(dem["volume"].sum())})
+    out[rank] = (h0, h1, m["mask"], dem["U"], dem["cnt"], dem["volume"], o, tot["volume"])
+    dist.barrier()
+    dist.destroy_process_group()
+
+
+def test_head_shards_concatenate_to_the_single_rank_result():
+    import numpy as np
+
+    import oracle
+    from paper_2609_32197_b200 import synth
+    world, port = 2, _free_port()
+    with mp.Manager() as mgr:
+        out = mgr.dict()
+        mp.spawn(_head_shard_worker, args=(world, port, out), nprocs=world, join=True)
+        res = dict(out)
+    assert (res[0][0], res[0][1], res[1][0], res[1][1]) == (0, 2, 2, 5)      # the shards tile the heads
+    wl = synth.Workload("shard", 5, 64, (3, 8, 16), 20, 64, 3, None, 3, seed=77)
+    Q, K, V = synth.make_qkv(wl, "cpu")
+    placement = oracle.placement_contiguous(wl.n_blocks, wl.ranks)
+    m = oracle.block_mask(Q, K, wl.block, wl.topk_abs, wl.n_text)
+    dem = oracle.demand(m["mask"], placement, wl.ranks, wl.block, wl.head_dim)
+    o, _ = oracle.attn_all(Q, K, V, m["mask"], wl.block)
+    assert np.array_equal(np.concatenate([res[0][2], res[1][2]], axis=0), m["mask"])          # masks [H][NB][Wd]
+    assert np.array_equal(np.concatenate([res[0][3], res[1][3]], axis=1), dem["U"])           # unions [P][H][Wd]
+    assert np.array_equal(np.concatenate([res[0][4], res[1][4]], axis=2), dem["cnt"])         # counts [P][P][H]
+    assert np.array_equal(res[0][5] + res[1][5], dem["volume"])                               # volumes add up per rank
+    assert np.array_equal(np.concatenate([res[0][6], res[1][6]], axis=0), o)                  # outputs [H][N][d]
+    assert res[0][7] == res[1][7] == float(dem["volume"].sum())
