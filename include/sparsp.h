@@ -73,7 +73,7 @@ SPARSP_API int sparsp_geometry(const sparsp_shape* shape, int64_t* n_tokens, int
 /* "top-k = pct % of the blocks": ceil(pct * n_video_blocks / 100) clamped to [1, n_video_blocks]. */
 SPARSP_API int32_t sparsp_resolve_topk(int32_t pct, int32_t n_video_blocks);
 
-/* Naive contiguous partition of the sequence (Section 3.1): rank(j) = floor(j * n_ranks / NB).
+/* Naive contiguous partition of the sequence (Section 3.2): rank(j) = floor(j * n_ranks / NB).
  * rank_of_block: HOST array of NB int32. */
 SPARSP_API int sparsp_placement_contiguous(const sparsp_shape* shape, int32_t n_ranks, int32_t* rank_of_block);
 
@@ -102,7 +102,7 @@ SPARSP_API int sparsp_placement_permutation(const sparsp_shape* shape, int32_t n
 SPARSP_API int sparsp_permute_tokens(const sparsp_shape* shape, const void* X, void* Y, const int32_t* block_of_slot,
                           const int64_t* token_offset_of_slot, int32_t inverse, void* stream);
 
-/* How widely received K blocks are shared (Section 3.1): for every remote KV block j that consumer r
+/* How widely received K blocks are shared (Section 3.2): for every remote KV block j that consumer r
  * receives for head h (some query block of r keeps it), the fraction of r's query blocks that keep it.
  *   hist  out  DEVICE int64 [B][n_ranks][101]: hist[b][r][q] = number of such (h, j) pairs whose fraction,
  *              in whole percent rounded down, is q
@@ -153,7 +153,7 @@ SPARSP_API int sparsp_block_mask_cdf(const sparsp_shape* shape, const void* Q, c
                           float score_scale, uint32_t* mask, int32_t* kv_count, float* pooled_q,
                           float* pooled_k, void* workspace, void* stream);
 
-/* Step 2 -- demand and packing for n_ranks virtual ranks (Section 4.2, Eq. "receiver-demand" and
+/* Step 2 -- demand and packing for n_ranks virtual ranks (Section 4.1, Eq. "receiver-demand" and
  * Eq. "sparse-exchange-volume"; Section 5.2: head-preserving demand, row-major packing with
  * locally derived offsets; Section 6: one slot per (producer, consumer) pair).
  *   Q_r = { i : rank_of_block[i] = r },  P(j) = rank_of_block[j]

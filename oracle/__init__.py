@@ -152,7 +152,7 @@ def permute_tokens(X, block_of_slot, token_offset_of_slot, b: int, inverse: bool
 
 
 def sharing_histogram(mask: np.ndarray, rank_of_block: np.ndarray, P: int) -> np.ndarray:
-    """Section 3.1: for each remote K block a rank receives (per head), the fraction of that rank's local Q
+    """Section 3.2: for each remote K block a rank receives (per head), the fraction of that rank's local Q
     blocks that access it.  hist[r][q], q = 0..100, counts the (head, remote block) pairs of consumer r whose
     fraction, in whole percent rounded down, is q (a received block is accessed by at least one local Q block,
     so a fraction below 1 % lands in bin 0)."""

@@ -7,12 +7,12 @@
  *
  * What each function follows:
  *   oracle_pool           mean-pooled query / key tiles ("masks materialised from pooled query and
- *                         key tiles", Section 4.2 Design Overview); fp32, ascending-token sum.
+ *                         key tiles", Section 4.2, Sparse KV Selection); fp32, ascending-token sum.
  *   oracle_scores         pooled-Q x pooled-K^T per head; fp32 fused-multiply-add chain.
  *   oracle_scores_f64     the same contraction in fp64 (near-tie audit only).
- *   oracle_topk_mask      block mask M[h,i,j] (Section 4.2), selection = top-k per query block
+ *   oracle_topk_mask      block mask M[h,i,j] (Section 4.1, Design Overview), selection = top-k per query block
  *                         with lowest-index tie-break; text blocks always kept.
- *   oracle_demand         receiver demand D[r,h,p] (Eq. "receiver-demand"), exchange volume V_r
+ *   oracle_demand         receiver demand D[r,h,p] (Section 4.1, Eq. "receiver-demand"), exchange volume V_r
  *                         (Eq. "sparse-exchange-volume"), head-preserving Boolean demand
  *                         (Section 5.2), locally derived per-head offsets (Section 5.2).
  *   oracle_pack           row-major (head, block) packing, one contiguous segment per

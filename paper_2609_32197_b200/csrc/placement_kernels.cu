@@ -1,5 +1,5 @@
 // Placement tools (Section 4.3: the layout is applied as a deterministic permutation of whole KV blocks,
-// undone by the inverse permutation; Section 3.1: how widely a received K block is shared by the
+// undone by the inverse permutation; Section 3.2: how widely a received K block is shared by the
 // receiving rank's query blocks).  permute_tokens_kernel is an HBM-bound copy of block-sized runs of
 // token rows; sharing_kernel counts bits of mask columns.
 #include "common.cuh"

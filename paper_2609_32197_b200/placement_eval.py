@@ -1,5 +1,5 @@
 """Compares block placements on a workload: exchange volume (Eq. "sparse-exchange-volume") and how widely
-received K blocks are shared by the receiving rank's queries (Section 3.1), for contiguous, interval-periodic
+received K blocks are shared by the receiving rank's queries (Section 3.2), for contiguous, interval-periodic
 (Eq. "periodic-placement") and shuffled layouts, across virtual rank counts and sparsity levels; also times
 the token permutation that applies a layout.  Everything runs through the C-ABI calls on the GPU.
 

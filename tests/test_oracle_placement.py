@@ -1,5 +1,5 @@
 """Pins for the oracle's placement tools: the block permutation (Section 4.3), the token permutation and
-its inverse, and the remote-K sharing statistic (Section 3.1) against the band-mask closed form."""
+its inverse, and the remote-K sharing statistic (Section 3.2) against the band-mask closed form."""
 import numpy as np
 import torch
 
