@@ -458,6 +458,43 @@ def end_to_end(cfg, args, barrier):
     return e2e_ms, n_chunks, h2d, d2h
 
 
+def exchange_leg(cfg, args, rank, world):
+    """The consumer-side pipeline over the transfer runtime (Export / Publish / Fetch / Release / Fence): with one
+    GPU its P virtual ranks are host threads on this device, with N > 1 every process is one rank on its own GPU.
+    Timed twice: pipelined (a chunk is fetched while attention runs on the previous one) and serial."""
+    import torch
+
+    from paper_2609_32197_b200 import exchange_driver
+    out = {"virtual_ranks_on_one_device": world == 1, "window": args.exchange_window,
+           "steady_chunks": args.exchange_chunks[0], "tail_chunks": args.exchange_chunks[1]}
+    Q4, K4, V4 = cfg.Q[None], cfg.K[None], cfg.V[None]
+    for mode, pipelined in (("pipelined", True), ("serial", False)):
+        if world == 1:
+            res = exchange_driver.run_exchange(cfg.shape, cfg.P, cfg.rank_of_block, Q4, [K4] * cfg.P, [V4] * cfg.P,
+                                               cfg.mo["mask"], window=args.exchange_window,
+                                               steady_chunks=args.exchange_chunks[0], tail_chunks=args.exchange_chunks[1],
+                                               pipelined=pipelined, calls=3)
+        else:
+            res = exchange_driver.run_exchange_multi_gpu(cfg.shape, cfg.rank_of_block, Q4, K4, V4, cfg.mo["mask"],
+                                                         window=args.exchange_window,
+                                                         steady_chunks=args.exchange_chunks[0],
+                                                         tail_chunks=args.exchange_chunks[1], pipelined=pipelined,
+                                                         calls=3)
+        if res.errors:
+            out[mode] = {"error": "; ".join("rank %d: %s" % (r_, e) for r_, e in res.errors)}
+            continue
+        st = list(res.stats.values())
+        out[mode] = {"ms": res.ms, "bytes_fetched_per_call": res.bytes_moved,
+                     "fetches": sum(s_["fetches"] for s_ in st) // 3,
+                     "acquires_that_waited": sum(s_["acquires_that_waited"] for s_ in st),
+                     "ms_waiting_for_publish": sum(s_["us_waiting_for_publish"] for s_ in st) / 1e3,
+                     "ms_waiting_for_release": sum(s_["us_waiting_for_release"] for s_ in st) / 1e3}
+        out["slot_bytes"] = res.slot_bytes
+        del res
+        torch.cuda.empty_cache()
+    return out
+
+
 def run_ours(args):
     import gc
 
@@ -502,6 +539,11 @@ def run_ours(args):
     e2e_ms, e2e_chunks, h2d, d2h = float("nan"), 0, 3 * cfg.Q.numel() * 2, cfg.O.numel() * 2 + cfg.do["volume_bytes"].numel() * 8
     if not args.no_e2e:
         e2e_ms, e2e_chunks, h2d, d2h = end_to_end(cfg, args, barrier)
+    exchange = None
+    if args.exchange:
+        if world > 1 and cfg.P != world:
+            raise SystemExit("--exchange with N > 1 needs a workload whose rank count equals N (got %d ranks)" % cfg.P)
+        exchange = exchange_leg(cfg, args, rank, world)
     sustained = None
     if world == 1 and args.sustained_s > 0:
         sustained = sustained_attention(cfg, args.sustained_s, local, peaks)
@@ -540,6 +582,8 @@ def run_ours(args):
     result["clocks"] = t["clocks"]
     if sustained:
         result["sustained"] = sustained
+    if exchange:
+        result["exchange"] = exchange
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
         result["cpu_baseline"] = cpu_baseline(cfg.wl, cfg.k, placement, cfg.rank_of_block.numpy(), cfg.Q, cfg.K, cfg.V,
                                               cfg.flops, budget_s=15.0)
@@ -707,6 +751,10 @@ def main():
     ap.add_argument("--no-per-config", action="store_true", help="skip the per_config list (all eight configurations)")
     ap.add_argument("--sustained-s", type=float, default=2.0,
                     help="seconds of back-to-back attention calls for the sustained figure (0 = skip)")
+    ap.add_argument("--exchange", action="store_true",
+                    help="also run the demand-routed exchange over the transfer runtime (pipelined vs serial)")
+    ap.add_argument("--exchange-window", type=int, default=2, help="slots per rank")
+    ap.add_argument("--exchange-chunks", type=int, nargs=2, default=(2, 4), help="chunks per hop: steady rounds, last round")
     ap.add_argument("--shard", default="replicas", choices=["replicas", "heads"],
                     help="with N > 1: independent replicas (weak scaling) or the heads of ONE layer split over the ranks (strong)")
     args = ap.parse_args()

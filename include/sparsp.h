@@ -245,6 +245,13 @@ SPARSP_API int sparsp_hop_chunk_mask(const sparsp_shape* shape, const uint32_t* 
                                      int32_t head_end, uint32_t* hop_mask, void* stream);
 SPARSP_API int sparsp_attn_merge(const sparsp_shape* shape, const void* O_a, const float* lse_a, const void* O_b,
                                  const float* lse_b, void* O, float* lse, void* stream);
+/* The same merge restricted to what one chunk of one hop produced (Section 7.1): only the rows of the query blocks
+ * of `consumer` in heads [head_begin, head_end) are merged; every other row of O / lse is left untouched.
+ *   rank_of_block  DEVICE int32 [NB] */
+SPARSP_API int sparsp_attn_merge_rows(const sparsp_shape* shape, const void* O_a, const float* lse_a, const void* O_b,
+                                      const float* lse_b, void* O, float* lse, const int32_t* rank_of_block,
+                                      int32_t n_ranks, int32_t consumer, int32_t head_begin, int32_t head_end,
+                                      void* stream);
 
 /* The transfer list of the demand-routed exchange, derived from the demand counts alone (host arithmetic, no
  * GPU work).  Section 5.1: in round k = 0 .. P-2 consumer r receives from the producer at ring distance
@@ -271,6 +278,78 @@ typedef struct sparsp_transfer {
 SPARSP_API int sparsp_exchange_plan(const sparsp_shape* shape, int32_t n_ranks, const int32_t* cnt,
                                     const int64_t* seg_offset, int32_t steady_chunks, int32_t tail_chunks,
                                     sparsp_transfer* transfers, int64_t capacity, int64_t* n_transfers);
+
+/* Transfer runtime of the demand-routed exchange (Section 6.1: the five primitives Export, Publish, Fetch,
+ * Release, Fence; Section 6.2: raw asynchronous peer copies of receiver-derived byte ranges; Section 6.3: a
+ * bounded window of reusable slots whose dependencies are Publish and Release alone).
+ *
+ * One endpoint (`sparsp_xchg`) per rank.  A rank is a GPU of the node or, on one device, a virtual rank driven by
+ * its own host thread with its own streams.  In round k = 0 .. P-2 rank p packs what consumer (p + k + 1) mod P
+ * selected from it into slot (k mod window) of its own window (`use` = k below), and consumer r fetches from
+ * producer (r - (k + 1)) mod P.  A slot holds the whole payload of one (consumer, producer) pair, laid out like that
+ * pair's run of the consumer's buffer (heads ascending, blocks ascending), so a consumer derives any chunk's byte
+ * range inside the slot from the demand counts: chunk.byte_offset - seg_offset[r][p][0] * entry bytes.
+ *
+ * Flags: 4-byte sequence numbers, one (publish, release) pair per (rank, slot), in a page of
+ * sparsp_xchg_flag_bytes() bytes of HOST memory that every rank can read and write (pinned memory for the ranks of
+ * one process, inter-process shared memory for one process per GPU); zero-filled by whoever creates it.  Publish and
+ * Release store them from a host function enqueued on the given stream, i.e. in stream order after the pack
+ * (Publish) or after the copies (Release); no kernel is launched and no kernel ever waits for another rank.  Every
+ * wait -- sparsp_xchg_acquire for the release of the slot's previous content, sparsp_xchg_fetch for the
+ * publication -- polls on the host for at most `wait_limit_us` and then fails with SPARSP_ERR_TIMEOUT (text in
+ * sparsp_last_error()); the endpoint stays usable.
+ *
+ *   sparsp_xchg_export   Export: registers this rank's window (`slots`: `window` slots of `slot_bytes` each, DEVICE
+ *                        memory the caller owns, 16-byte aligned) and the shared flag page; *out is the endpoint.
+ *                        flags: 0, or SPARSP_XCHG_HOST_MEMORY -- slots and destinations are HOST memory, copies
+ *                        are memcpy and flag stores happen at once (for multi-process tests of the protocol on
+ *                        machines without a GPU; never chosen by the library itself).
+ *   sparsp_xchg_connect  address under which this rank reaches `peer`'s window (the same pointer on one device; a
+ *                        peer mapping of the other GPU's window on a node).
+ *   sparsp_xchg_fence    Fence: call once per attention call on every rank, AFTER the caller's barrier across
+ *                        ranks (and after this rank's copies of the previous call have completed).  Moves the
+ *                        endpoint to the next epoch: flags of the previous call no longer satisfy any wait.
+ *   sparsp_xchg_acquire  producer: slot of packing number `use` (use mod window) and its address; for use >= window
+ *                        waits until the consumer of packing use - window has released it.
+ *   sparsp_xchg_publish  producer: marks packing `use` as ready once the work enqueued on `stream` so far is done.
+ *   sparsp_xchg_fetch    consumer: waits for producer's packing `use`, then enqueues ONE asynchronous copy of
+ *                        [src_offset, src_offset + n_bytes) of that slot to `dst` (device memory of this rank) on
+ *                        `copy_stream` (copy engines; no SM).  n_bytes = 0 only waits.
+ *   sparsp_xchg_release  consumer: returns producer's slot of packing `use` once the copies enqueued on
+ *                        `copy_stream` so far are done.
+ *   sparsp_xchg_stats    out[8] (HOST): publications, fetches, releases, acquisitions that found the slot still in
+ *                        use, bytes fetched, microseconds waited for releases, for publications, timeouts.
+ *   sparsp_xchg_destroy  frees the endpoint (not the slots or the flag page).
+ * `use` is 0 .. 65534.  Calls on one endpoint come from one host thread. */
+#define SPARSP_XCHG_HOST_MEMORY 1
+typedef struct sparsp_xchg sparsp_xchg;
+SPARSP_API int sparsp_xchg_flag_bytes(int32_t n_ranks, int32_t window, int64_t* bytes);
+SPARSP_API int sparsp_xchg_export(int32_t n_ranks, int32_t rank, int32_t window, int64_t slot_bytes, void* slots,
+                                  void* flag_page, int64_t wait_limit_us, int32_t flags, sparsp_xchg** out);
+SPARSP_API int sparsp_xchg_connect(sparsp_xchg* x, int32_t peer, void* peer_slots);
+SPARSP_API int sparsp_xchg_fence(sparsp_xchg* x);
+SPARSP_API int sparsp_xchg_acquire(sparsp_xchg* x, int64_t use, int32_t* slot, void** slot_ptr);
+SPARSP_API int sparsp_xchg_publish(sparsp_xchg* x, int64_t use, void* stream);
+SPARSP_API int sparsp_xchg_fetch(sparsp_xchg* x, int32_t producer, int64_t use, int64_t src_offset, void* dst,
+                                 int64_t n_bytes, void* copy_stream);
+SPARSP_API int sparsp_xchg_release(sparsp_xchg* x, int32_t producer, int64_t use, void* copy_stream);
+SPARSP_API int sparsp_xchg_stats(sparsp_xchg* x, int64_t* out);
+SPARSP_API int sparsp_xchg_destroy(sparsp_xchg* x);
+
+/* The producer's pack of ONE hop (Section 6.1: for each producer-consumer pair the producer packs the payload into
+ * the slot designated for it).  Writes, starting at `dst`, the K and V tiles of every block that `consumer` selected
+ * from `producer` -- the entries seg_offset[consumer][producer][0] .. of the consumer's buffer, in that order (heads
+ * ascending, blocks ascending; entry = K tile then V tile; rows at or beyond N are zero).  Only blocks `producer`
+ * owns are read from K / V.  An entry that would end beyond dst_capacity_bytes is not written and the status word
+ * becomes SPARSP_ERR_CAPACITY.  One batch item.
+ *   union_mask, cnt, seg_offset   outputs of sparsp_demand_pack / sparsp_demand_plan_noalloc made WITHOUT
+ *                                 SPARSP_INCLUDE_LOCAL (DEVICE)
+ *   dst                           DEVICE, 16-byte aligned (a slot of the producer's window)
+ *   workspace                     this rank's own (the call rewrites the workspace's entry table) */
+SPARSP_API int sparsp_pack_segment(const sparsp_shape* shape, const uint32_t* union_mask, const int32_t* rank_of_block,
+                                   int32_t n_ranks, int32_t consumer, int32_t producer, const int32_t* cnt,
+                                   const int64_t* seg_offset, const void* K, const void* V, void* dst,
+                                   int64_t dst_capacity_bytes, void* workspace, void* stream);
 
 /* Planning without any allocation.  (No counterpart in the paper: an engineering variant of the
  * planning half of sparsp_demand_pack.)

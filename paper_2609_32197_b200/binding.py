@@ -31,8 +31,11 @@ EXPORTS = [
     "sparsp_status", "sparsp_last_error", "sparsp_launch_count", "sparsp_demand_plan_noalloc",
     "sparsp_hop_mask", "sparsp_attn_merge", "sparsp_sparse_attn_fwd_packed", "sparsp_block_mask_cdf",
     "sparsp_placement_permutation", "sparsp_permute_tokens", "sparsp_sharing_histogram", "sparsp_exchange_plan",
-    "sparsp_hop_chunk_mask", "sparsp_selftest_wait_timeout",
+    "sparsp_hop_chunk_mask", "sparsp_selftest_wait_timeout", "sparsp_attn_merge_rows", "sparsp_pack_segment",
+    "sparsp_xchg_flag_bytes", "sparsp_xchg_export", "sparsp_xchg_connect", "sparsp_xchg_fence", "sparsp_xchg_acquire",
+    "sparsp_xchg_publish", "sparsp_xchg_fetch", "sparsp_xchg_release", "sparsp_xchg_stats", "sparsp_xchg_destroy",
 ]
+SPARSP_XCHG_HOST_MEMORY = 1
 
 
 class SparspError(RuntimeError):
@@ -259,6 +262,96 @@ def sparsp_hop_chunk_mask(shape, mask, rank_of_block, n_ranks, consumer, produce
 def sparsp_attn_merge(shape, O_a, lse_a, O_b, lse_b, O, lse):
     _check(lib().sparsp_attn_merge(ctypes.byref(shape), _ptr(O_a), _ptr(lse_a), _ptr(O_b), _ptr(lse_b), _ptr(O),
                                    _ptr(lse), _stream()))
+
+
+def sparsp_attn_merge_rows(shape, O_a, lse_a, O_b, lse_b, O, lse, rank_of_block, n_ranks, consumer, head_begin,
+                           head_end):
+    _check(lib().sparsp_attn_merge_rows(ctypes.byref(shape), _ptr(O_a), _ptr(lse_a), _ptr(O_b), _ptr(lse_b), _ptr(O),
+                                        _ptr(lse), _ptr(rank_of_block), ctypes.c_int32(n_ranks),
+                                        ctypes.c_int32(consumer), ctypes.c_int32(head_begin), ctypes.c_int32(head_end),
+                                        _stream()))
+
+
+def _addr(x):
+    """Raw address: an int, a torch tensor (its data pointer) or None."""
+    if x is None:
+        return ctypes.c_void_p(0)
+    if isinstance(x, int):
+        return ctypes.c_void_p(x)
+    return ctypes.c_void_p(x.data_ptr())
+
+
+def _stream_of(stream):
+    """cudaStream_t of a torch stream (None: the current stream; 0: no stream, host-memory endpoints)."""
+    if stream is None:
+        return _stream()
+    if isinstance(stream, int):
+        return ctypes.c_void_p(stream)
+    return ctypes.c_void_p(stream.cuda_stream)
+
+
+def sparsp_pack_segment(shape, union_mask, rank_of_block, n_ranks, consumer, producer, cnt, seg_offset, K, V, dst,
+                        dst_capacity_bytes, workspace):
+    """dst: a tensor or a raw device address (a slot of the producer's window)."""
+    _check(lib().sparsp_pack_segment(ctypes.byref(shape), _ptr(union_mask), _ptr(rank_of_block),
+                                     ctypes.c_int32(n_ranks), ctypes.c_int32(consumer), ctypes.c_int32(producer),
+                                     _ptr(cnt), _ptr(seg_offset), _ptr(K), _ptr(V), _addr(dst),
+                                     ctypes.c_int64(dst_capacity_bytes), _ptr(workspace), _stream()))
+
+
+def sparsp_xchg_flag_bytes(n_ranks: int, window: int) -> int:
+    out = ctypes.c_int64()
+    _check(lib().sparsp_xchg_flag_bytes(ctypes.c_int32(n_ranks), ctypes.c_int32(window), ctypes.byref(out)))
+    return out.value
+
+
+def sparsp_xchg_export(n_ranks, rank, window, slot_bytes, slots, flag_page, wait_limit_us, flags=0):
+    """-> endpoint handle.  slots / flag_page: tensors or raw addresses."""
+    h = ctypes.c_void_p()
+    _check(lib().sparsp_xchg_export(ctypes.c_int32(n_ranks), ctypes.c_int32(rank), ctypes.c_int32(window),
+                                    ctypes.c_int64(slot_bytes), _addr(slots), _addr(flag_page),
+                                    ctypes.c_int64(wait_limit_us), ctypes.c_int32(flags), ctypes.byref(h)))
+    return h
+
+
+def sparsp_xchg_connect(x, peer, peer_slots):
+    _check(lib().sparsp_xchg_connect(x, ctypes.c_int32(peer), _addr(peer_slots)))
+
+
+def sparsp_xchg_fence(x):
+    _check(lib().sparsp_xchg_fence(x))
+
+
+def sparsp_xchg_acquire(x, use):
+    """-> (slot index, slot address)"""
+    slot, ptr = ctypes.c_int32(), ctypes.c_void_p()
+    _check(lib().sparsp_xchg_acquire(x, ctypes.c_int64(use), ctypes.byref(slot), ctypes.byref(ptr)))
+    return slot.value, ptr.value
+
+
+def sparsp_xchg_publish(x, use, stream=None):
+    _check(lib().sparsp_xchg_publish(x, ctypes.c_int64(use), _stream_of(stream)))
+
+
+def sparsp_xchg_fetch(x, producer, use, src_offset, dst, n_bytes, copy_stream=None):
+    _check(lib().sparsp_xchg_fetch(x, ctypes.c_int32(producer), ctypes.c_int64(use), ctypes.c_int64(src_offset),
+                                   _addr(dst), ctypes.c_int64(n_bytes), _stream_of(copy_stream)))
+
+
+def sparsp_xchg_release(x, producer, use, copy_stream=None):
+    _check(lib().sparsp_xchg_release(x, ctypes.c_int32(producer), ctypes.c_int64(use), _stream_of(copy_stream)))
+
+
+def sparsp_xchg_stats(x) -> dict:
+    out = (ctypes.c_int64 * 8)()
+    _check(lib().sparsp_xchg_stats(x, out))
+    names = ("publications", "fetches", "releases", "acquires_that_waited", "bytes_fetched", "us_waiting_for_release",
+             "us_waiting_for_publish", "timeouts")
+    return dict(zip(names, [int(v) for v in out]))
+
+
+def sparsp_xchg_destroy(x):
+    _check(lib().sparsp_xchg_destroy(x))
 
 
 def sparsp_status(workspace) -> int:

@@ -10,7 +10,7 @@ HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libsparsp.so")
 SOURCES = ["api.cu", "mask_kernels.cu", "demand_kernels.cu", "attn_kernel.cu", "merge_kernels.cu",
-           "placement_kernels.cu", "diag_kernels.cu"]
+           "placement_kernels.cu", "diag_kernels.cu", "exchange.cu"]
 HEADERS = ["common.cuh", "sm100_ptx.cuh", os.path.join("..", "..", "include", "sparsp.h")]
 NVCC_FLAGS = ["-O3", "-std=c++17", "-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo",
               "-Xcompiler", "-fPIC", "-Xcompiler", "-fvisibility=hidden"]

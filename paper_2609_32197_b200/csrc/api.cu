@@ -421,6 +421,40 @@ int sparsp_demand_pack(const sparsp_shape* shape, const uint32_t* mask, const in
   return SPARSP_OK;
 }
 
+int sparsp_pack_segment(const sparsp_shape* shape, const uint32_t* union_mask, const int32_t* rank_of_block,
+                        int32_t n_ranks, int32_t consumer, int32_t producer, const int32_t* cnt,
+                        const int64_t* seg_offset, const void* K, const void* V, void* dst, int64_t dst_capacity_bytes,
+                        void* workspace, void* stream) {
+  Geometry g;
+  SPARSP_TRY(make_geometry(shape, &g));
+  SPARSP_TRY(check_supported(g));
+  SPARSP_TRY(check_strides(shape, g));
+  if (g.B != 1) {
+    set_error("sparsp_pack_segment handles one batch item per call (batch = %d)", g.B);
+    return SPARSP_ERR_UNSUPPORTED;
+  }
+  if (n_ranks < 1 || n_ranks > kMaxRanks || consumer < 0 || consumer >= n_ranks || producer < 0 ||
+      producer >= n_ranks || consumer == producer) {
+    set_error("consumer / producer %d / %d must be two different ranks of 0..%d", consumer, producer, n_ranks - 1);
+    return SPARSP_ERR_INVALID_ARG;
+  }
+  SPARSP_TRY(check_ptr(union_mask, "union_mask", 4));
+  SPARSP_TRY(check_ptr(rank_of_block, "rank_of_block", 4));
+  SPARSP_TRY(check_ptr(cnt, "cnt", 4));
+  SPARSP_TRY(check_ptr(seg_offset, "seg_offset", 8));
+  SPARSP_TRY(check_ptr(K, "K"));
+  SPARSP_TRY(check_ptr(V, "V"));
+  SPARSP_TRY(check_ptr(dst, "dst"));
+  SPARSP_TRY(check_ptr(workspace, "workspace", 256));
+  if (dst_capacity_bytes < 0) {
+    set_error("negative dst_capacity_bytes");
+    return SPARSP_ERR_INVALID_ARG;
+  }
+  const WsLayout L = make_layout(g, n_ranks);
+  return launch_pack_segment(*shape, g, union_mask, rank_of_block, n_ranks, consumer, producer, seg_offset, cnt, K, V,
+                             dst, dst_capacity_bytes, (char*)workspace, L, (cudaStream_t)stream);
+}
+
 int sparsp_sparse_attn_fwd(const sparsp_shape* shape, const void* Q, const void* K, const void* V,
                            const uint32_t* mask, float softmax_scale, void* O, float* lse,
                            void* workspace, void* stream) {
@@ -525,7 +559,31 @@ int sparsp_attn_merge(const sparsp_shape* shape, const void* O_a, const float* l
   SPARSP_TRY(check_ptr(lse_a, "lse_a", 4));
   SPARSP_TRY(check_ptr(lse_b, "lse_b", 4));
   SPARSP_TRY(check_ptr(lse, "lse", 4));
-  return launch_attn_merge(*shape, g, O_a, lse_a, O_b, lse_b, O, lse, (cudaStream_t)stream);
+  return launch_attn_merge(*shape, g, O_a, lse_a, O_b, lse_b, O, lse, nullptr, 0, 0, g.H, (cudaStream_t)stream);
+}
+
+int sparsp_attn_merge_rows(const sparsp_shape* shape, const void* O_a, const float* lse_a, const void* O_b,
+                           const float* lse_b, void* O, float* lse, const int32_t* rank_of_block, int32_t n_ranks,
+                           int32_t consumer, int32_t head_begin, int32_t head_end, void* stream) {
+  Geometry g;
+  SPARSP_TRY(make_geometry(shape, &g));
+  SPARSP_TRY(check_supported(g));
+  SPARSP_TRY(check_strides(shape, g));
+  SPARSP_TRY(check_ptr(O_a, "O_a"));
+  SPARSP_TRY(check_ptr(O_b, "O_b"));
+  SPARSP_TRY(check_ptr(O, "O"));
+  SPARSP_TRY(check_ptr(lse_a, "lse_a", 4));
+  SPARSP_TRY(check_ptr(lse_b, "lse_b", 4));
+  SPARSP_TRY(check_ptr(lse, "lse", 4));
+  SPARSP_TRY(check_ptr(rank_of_block, "rank_of_block", 4));
+  if (n_ranks < 1 || n_ranks > kMaxRanks || consumer < 0 || consumer >= n_ranks || head_begin < 0 ||
+      head_end > g.H || head_begin > head_end) {
+    set_error("consumer %d outside 0..%d or head range [%d, %d) outside [0, %d)", consumer, n_ranks - 1, head_begin,
+              head_end, g.H);
+    return SPARSP_ERR_INVALID_ARG;
+  }
+  return launch_attn_merge(*shape, g, O_a, lse_a, O_b, lse_b, O, lse, rank_of_block, consumer, head_begin, head_end,
+                           (cudaStream_t)stream);
 }
 
 int sparsp_selftest_wait_timeout(void* workspace, int64_t limit_cycles, void* stream) {

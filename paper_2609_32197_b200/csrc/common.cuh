@@ -76,6 +76,9 @@ int launch_demand(const Geometry& g, const uint32_t* mask, const int32_t* rank_o
                   const WsLayout& L, cudaStream_t st);
 int launch_pack(const sparsp_shape& s, const Geometry& g, const void* K, const void* V, void* packed,
                 int64_t capacity, int P, char* ws, const WsLayout& L, cudaStream_t st);
+int launch_pack_segment(const sparsp_shape& s, const Geometry& g, const uint32_t* U, const int32_t* rank, int P,
+                        int consumer, int producer, const int64_t* seg_off, const int32_t* cnt, const void* K,
+                        const void* V, void* dst, int64_t capacity, char* ws, const WsLayout& L, cudaStream_t st);
 int launch_attn(const sparsp_shape& s, const Geometry& g, const void* Q, const void* K, const void* V,
                 const uint32_t* mask, float scale, void* O, float* lse, char* ws, const WsLayout& L,
                 cudaStream_t st);
@@ -89,6 +92,7 @@ int launch_hop_mask(const Geometry& g, const uint32_t* mask, const int32_t* rank
                     int head_begin, int head_end, uint32_t* hop, cudaStream_t st);
 int launch_wait_timeout(char* ws, const WsLayout& L, long long limit_cycles, cudaStream_t st);
 int launch_attn_merge(const sparsp_shape& s, const Geometry& g, const void* Oa, const float* la, const void* Ob,
-                      const float* lb, void* O, float* lse, cudaStream_t st);
+                      const float* lb, void* O, float* lse, const int32_t* rank, int consumer, int head_begin,
+                      int head_end, cudaStream_t st);
 
 }  // namespace sparsp

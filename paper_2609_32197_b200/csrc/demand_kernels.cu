@@ -438,6 +438,78 @@ int launch_pack(const sparsp_shape& s, const Geometry& g, const void* K, const v
 }
 
 // ------------------------------------------------------------------------------------------------
+// Pack of ONE (consumer, producer) segment (Section 6.1: the producer packs the payload of one consumer into
+// the slot designated for that pair).  The entry table holds that segment alone, with destinations relative
+// to the start of the slot: entry (h, j) sits where it sits inside the consumer's buffer, minus the segment's
+// first entry, so that consumer and producer derive the same byte ranges from the demand counts.
+// One warp per head enumerates U[consumer][h] & own[producer] in ascending block order.
+// ------------------------------------------------------------------------------------------------
+__global__ void segment_entries_kernel(const uint32_t* __restrict__ U, const int32_t* __restrict__ rank, int H, int NB,
+                                       int Wd, int P, int consumer, int producer,
+                                       const int64_t* __restrict__ seg_off, const int32_t* __restrict__ cnt,
+                                       int64_t entry_bytes, int64_t capacity, PackEntry* __restrict__ entries,
+                                       int64_t* __restrict__ n_entries, int32_t* __restrict__ status) {
+  const int h = (int)(((int64_t)blockIdx.x * blockDim.x + threadIdx.x) >> 5);
+  const int lane = threadIdx.x & 31;
+  if (h >= H) return;
+  const int64_t seg0 = ((int64_t)consumer * P + producer) * H;  // batch item 0
+  const int64_t first_of_segment = seg_off[seg0];
+  if (h == 0 && lane == 0) *n_entries = seg_off[seg0 + H - 1] + cnt[seg0 + H - 1] - first_of_segment;
+  const uint32_t* u = U + ((int64_t)consumer * H + h) * Wd;
+  const int64_t first = seg_off[seg0 + h] - first_of_segment;
+  int running = 0;
+  for (int w0 = 0; w0 < Wd; w0 += 32) {
+    const int w = w0 + lane;
+    uint32_t bits = 0;
+    if (w < Wd) {
+      uint32_t own = 0;
+      for (int t = 0; t < 32; ++t) {
+        const int j = w * 32 + t;
+        if (j < NB && rank[j] == producer) own |= 1u << t;
+      }
+      bits = u[w] & own;
+    }
+    const int mine = __popc(bits);
+    int incl = mine;
+#pragma unroll
+    for (int s = 1; s < 32; s <<= 1) {
+      const int v = __shfl_up_sync(0xffffffffu, incl, s);
+      if (lane >= s) incl += v;
+    }
+    int pos = running + incl - mine;
+    while (bits) {
+      const int t = __ffs(bits) - 1;
+      bits &= bits - 1;
+      PackEntry e;
+      e.dst_byte = (first + pos) * entry_bytes;
+      e.bh = h;
+      e.j = w * 32 + t;
+      if (e.dst_byte + entry_bytes > capacity) {
+        e.j = -1;  // would not fit the slot: skipped by the gather
+        atomicExch(status, SPARSP_ERR_CAPACITY);
+      }
+      entries[first + pos] = e;
+      ++pos;
+    }
+    running += __shfl_sync(0xffffffffu, incl, 31);
+  }
+}
+
+int launch_pack_segment(const sparsp_shape& s, const Geometry& g, const uint32_t* U, const int32_t* rank, int P,
+                        int consumer, int producer, const int64_t* seg_off, const int32_t* cnt, const void* K,
+                        const void* V, void* dst, int64_t capacity, char* ws, const WsLayout& L, cudaStream_t st) {
+  PackEntry* entries = (PackEntry*)(ws + L.entries);
+  int64_t* n_entries = (int64_t*)(ws + L.n_entries);
+  int32_t* status = (int32_t*)(ws + L.status);
+  const int64_t entry_bytes = 2LL * g.b * g.d * 2;
+  segment_entries_kernel<<<(g.H * 32 + 255) / 256, 256, 0, st>>>(U, rank, g.H, g.NB, g.Wd, P, consumer, producer, seg_off,
+                                                                cnt, entry_bytes, capacity, entries, n_entries, status);
+  count_launch();
+  SPARSP_CUDA_OK(cudaGetLastError());
+  return launch_pack(s, g, K, V, dst, capacity, P, ws, L, st);
+}
+
+// ------------------------------------------------------------------------------------------------
 // Allocation-free planning call.  Its scratch (the per-rank ownership bit words and the per-consumer
 // table bases) lives in one file-scope device array instead of a caller-provided workspace, so a
 // caller that cannot allocate device memory at all can still obtain unions, counts, offsets and

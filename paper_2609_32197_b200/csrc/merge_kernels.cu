@@ -32,15 +32,22 @@ __global__ void hop_mask_kernel(const uint32_t* __restrict__ mask, const int32_t
 // writes, and only the row's first thread touches the log-sum-exp values -- it reads both inputs, computes the
 // weights and hands them to the row's other threads by shuffle (the D/8 threads of a row are consecutive lanes of
 // one warp) before it writes the merged value.
+// With `rank` given, only the rows of the query blocks of `consumer` in heads [head_begin, head_end) are merged;
+// all other rows are left untouched (one chunk of one hop of one rank).
 template <int D>
 __global__ void attn_merge_kernel(const __nv_bfloat16* Oa, const float* la, const __nv_bfloat16* Ob, const float* lb,
                                   __nv_bfloat16* O, float* lse, int H, int64_t N, int64_t sB, int64_t sH, int64_t sT,
-                                  int64_t n_rows) {
+                                  int64_t n_rows, const int32_t* __restrict__ rank, int consumer, int b,
+                                  int head_begin, int head_end) {
   constexpr int VPR = D / 8;
   const int64_t idx = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
   const int64_t row = idx / VPR;
   const int col = (int)(idx % VPR);
-  const bool live = row < n_rows;
+  bool live = row < n_rows;
+  if (live && rank != nullptr) {
+    const int head = (int)((row / N) % H);
+    live = head >= head_begin && head < head_end && rank[(row % N) / b] == consumer;
+  }
   float wa = 0.0f, wb = 0.0f, out_lse = -INFINITY;
   if (live && col == 0) {
     const float a = la[row], b = lb[row];
@@ -85,7 +92,8 @@ int launch_hop_mask(const Geometry& g, const uint32_t* mask, const int32_t* rank
 }
 
 int launch_attn_merge(const sparsp_shape& s, const Geometry& g, const void* Oa, const float* la, const void* Ob,
-                      const float* lb, void* O, float* lse, cudaStream_t st) {
+                      const float* lb, void* O, float* lse, const int32_t* rank, int consumer, int head_begin,
+                      int head_end, cudaStream_t st) {
   const int64_t n_rows = (int64_t)g.B * g.H * g.N;
   const int64_t threads = n_rows * (g.d / 8);
   const unsigned grid = (unsigned)((threads + 255) / 256);
@@ -94,10 +102,10 @@ int launch_attn_merge(const sparsp_shape& s, const Geometry& g, const void* Oa, 
   auto o = (__nv_bfloat16*)O;
   if (g.d == 64)
     attn_merge_kernel<64><<<grid, 256, 0, st>>>(a, la, b, lb, o, lse, g.H, g.N, s.stride_batch, s.stride_head,
-                                                s.stride_token, n_rows);
+                                                s.stride_token, n_rows, rank, consumer, g.b, head_begin, head_end);
   else
     attn_merge_kernel<128><<<grid, 256, 0, st>>>(a, la, b, lb, o, lse, g.H, g.N, s.stride_batch, s.stride_head,
-                                                 s.stride_token, n_rows);
+                                                 s.stride_token, n_rows, rank, consumer, g.b, head_begin, head_end);
   count_launch();
   SPARSP_CUDA_OK(cudaGetLastError());
   return SPARSP_OK;

@@ -142,3 +142,124 @@ def test_head_shards_concatenate_to_the_single_rank_result():
     assert np.array_equal(res[0][5] + res[1][5], dem["volume"])                               # volumes add up per rank
     assert np.array_equal(np.concatenate([res[0][6], res[1][6]], axis=0), o)                  # outputs [H][N][d]
     assert res[0][7] == res[1][7] == float(dem["volume"].sum())
+
+
+def _shm_addr(shm):
+    import ctypes
+    return ctypes.addressof(ctypes.c_char.from_buffer(shm.buf))
+
+
+def _slot_protocol_worker(rank, world, port, names, out, stall_from):
+    """Two processes, one exchange endpoint each, slots and flag page in inter-process shared memory (host-memory
+    endpoints: copies are memcpy, so the protocol runs without a GPU).  Each rank packs `n_uses` payloads for its peer
+    into a window of 2 slots and consumes the peer's; the consumer sleeps before every fetch, so a producer that
+    did not wait for Release would overwrite a slot that is still unread.  With `stall_from` >= 0 rank 1 stops
+    releasing from that use on: rank 0's bounded wait for the slot must end in SPARSP_ERR_TIMEOUT."""
+    import time
+    from multiprocessing import shared_memory
+
+    import numpy as np
+    os.environ["MASTER_ADDR"] = "127.0.0.1"
+    os.environ["MASTER_PORT"] = str(port)
+    dist.init_process_group("gloo", rank=rank, world_size=world)
+    from paper_2609_32197_b200 import binding as b
+    W, slot_bytes, n_uses = 2, 1 << 16, 6
+    shm_flags = shared_memory.SharedMemory(name=names["flags"])
+    shm_slots = [shared_memory.SharedMemory(name=names["slots%d" % r]) for r in range(world)]
+    x = b.sparsp_xchg_export(world, rank, W, slot_bytes, _shm_addr(shm_slots[rank]), _shm_addr(shm_flags), 300_000,
+                             b.SPARSP_XCHG_HOST_MEMORY)
+    peer = 1 - rank
+    b.sparsp_xchg_connect(x, peer, _shm_addr(shm_slots[peer]))
+    dist.barrier()            # Fence: the barrier across ranks, then the next epoch
+    b.sparsp_xchg_fence(x)
+    mine = np.ndarray((W, slot_bytes), np.uint8, buffer=shm_slots[rank].buf)
+    recv = np.zeros(slot_bytes, np.uint8)
+    import ctypes
+    log = {"acquired": [], "bad_payload": 0, "timeout": None, "consumed": 0}
+
+    def produce(u):
+        slot, _ = b.sparsp_xchg_acquire(x, u)
+        mine[slot, :] = (17 * rank + u) % 251      # the "pack"
+        b.sparsp_xchg_publish(x, u, 0)
+        log["acquired"].append((u, slot))
+
+    def consume(u):
+        time.sleep(0.02)                            # a slow consumer
+        b.sparsp_xchg_fetch(x, peer, u, 0, recv.ctypes.data, slot_bytes, 0)
+        if not (recv == (17 * peer + u) % 251).all():
+            log["bad_payload"] += 1
+        log["consumed"] += 1
+        if not (rank == 1 and 0 <= stall_from <= u):
+            b.sparsp_xchg_release(x, peer, u, 0)
+
+    try:
+        for u in range(min(W, n_uses)):
+            produce(u)
+        for u in range(n_uses):
+            consume(u)
+            if u + W < n_uses:
+                produce(u + W)
+    except b.SparspError as exc:
+        log["timeout"] = (exc.code, str(exc))
+    log["stats"] = b.sparsp_xchg_stats(x)
+    out[rank] = log
+    b.sparsp_xchg_destroy(x)
+    del mine
+    for s_ in [shm_flags] + shm_slots:
+        s_.close()
+    try:
+        dist.barrier()
+    except Exception:  # noqa: BLE001  (the peer may have left after its timeout)
+        pass
+    dist.destroy_process_group()
+
+
+def _run_slot_protocol(stall_from):
+    from multiprocessing import shared_memory
+
+    from paper_2609_32197_b200 import binding as b
+    world, W, slot_bytes = 2, 2, 1 << 16
+    shms = {"flags": shared_memory.SharedMemory(create=True, size=max(b.sparsp_xchg_flag_bytes(world, W), 64))}
+    for r in range(world):
+        shms["slots%d" % r] = shared_memory.SharedMemory(create=True, size=W * slot_bytes)
+    for s_ in shms.values():
+        s_.buf[:] = bytes(len(s_.buf))
+    try:
+        with mp.Manager() as mgr:
+            out = mgr.dict()
+            names = {k: v.name for k, v in shms.items()}
+            mp.spawn(_slot_protocol_worker, args=(world, _free_port(), names, out, stall_from), nprocs=world, join=True)
+            return dict(out)
+    finally:
+        for s_ in shms.values():
+            s_.close()
+            s_.unlink()
+
+
+def test_slot_window_protocol_between_two_processes():
+    res = _run_slot_protocol(stall_from=-1)
+    for r in (0, 1):
+        log = res[r]
+        assert log["timeout"] is None and log["bad_payload"] == 0 and log["consumed"] == 6
+        assert log["acquired"] == [(u, u % 2) for u in range(6)]            # six payloads through two slots
+        st = log["stats"]
+        assert st["publications"] == 6 and st["fetches"] == 6 and st["releases"] == 6 and st["timeouts"] == 0
+        assert st["bytes_fetched"] == 6 * (1 << 16)
+        assert st["acquires_that_waited"] >= 1                               # Release did gate a later pack
+
+
+def test_a_consumer_that_stops_releasing_times_the_producer_out():
+    res = _run_slot_protocol(stall_from=1)
+    from paper_2609_32197_b200 import binding as b
+    # rank 1 consumed everything rank 0 could publish (uses 0..2: slot 1 is never returned after use 1, so use 3
+    # cannot be packed) and saw only intact payloads; rank 0's wait for the slot of use 3 ran out
+    assert res[0]["timeout"] is not None and res[0]["timeout"][0] == b.SPARSP_ERR_TIMEOUT
+    assert "release" in res[0]["timeout"][1]
+    assert [u for u, _ in res[0]["acquired"]] == [0, 1, 2]
+    assert res[0]["stats"]["timeouts"] == 1
+    assert res[0]["bad_payload"] == 0 and res[1]["bad_payload"] == 0
+    # rank 1 in turn loses its consumer (rank 0 has left before reading use 2): the slot of its use 4 is never
+    # returned and its own bounded wait gives up as well
+    assert res[1]["timeout"] is not None and res[1]["timeout"][0] == b.SPARSP_ERR_TIMEOUT
+    assert "release" in res[1]["timeout"][1] and res[1]["consumed"] == 3
+    assert [u for u, _ in res[1]["acquired"]] == [0, 1, 2, 3]
