@@ -144,6 +144,20 @@ def resolve_workload(args):
     return wl, placement
 
 
+def describe_config(wl, heads, k, tau, kept_pairs, placement):
+    """The `config` object of a result line (the same keys and values in both arms)."""
+    input_bytes = 3 * heads * wl.n_tokens * wl.head_dim * 2
+    if input_bytes >= 2 * L2_BYTES:
+        l2 = "inputs larger than L2 (Q+K+V = %.0f MB)" % (input_bytes / 1e6)
+    else:
+        l2 = "L2 flushed between iterations (a %d MB buffer is overwritten; Q+K+V = %.1f MB)" % (
+            (2 * L2_BYTES) >> 20, input_bytes / 1e6)
+    return {"workload": wl.name, "heads": heads, "head_dim": wl.head_dim, "grid": list(wl.grid), "n_text": wl.n_text,
+            "tokens": wl.n_tokens, "block": wl.block, "n_blocks": wl.n_blocks, "topk_blocks": (k if tau <= 0 else None),
+            "selection": ("top-k" if tau <= 0 else "cdf tau=%g" % tau), "kept_pairs": kept_pairs,
+            "virtual_ranks": wl.ranks, "placement": placement, "layout": "[H][N][d]", "l2_policy": l2}
+
+
 def kept_flops_and_counts(mask_i32, N, b, d):
     """4*d*sum over kept (h,i,j) of rows_i*cols_j, from the device mask (library tensor ops)."""
     import torch
@@ -232,20 +246,8 @@ class Config:
     def check_status(self):
         assert self.binding.sparsp_status(self.ws) == self.binding.SPARSP_OK, self.binding.sparsp_last_error()
 
-    def l2_policy(self):
-        if self.flush is None:
-            return "inputs larger than L2 (Q+K+V = %.0f MB)" % (self.input_bytes / 1e6)
-        return "L2 flushed between iterations (a %d MB buffer is overwritten; Q+K+V = %.1f MB)" % (
-            self.flush.numel() >> 20, self.input_bytes / 1e6)
-
     def describe(self):
-        wl = self.wl
-        return {"workload": wl.name, "heads": self.H, "head_dim": self.d, "grid": list(wl.grid), "n_text": wl.n_text,
-                "tokens": self.N, "block": self.b, "n_blocks": self.NB,
-                "topk_blocks": (self.k if self.tau <= 0 else None),
-                "selection": ("top-k" if self.tau <= 0 else "cdf tau=%g" % self.tau), "kept_pairs": self.kept_pairs,
-                "virtual_ranks": self.P, "placement": self.placement, "layout": "[H][N][d]",
-                "l2_policy": self.l2_policy()}
+        return describe_config(self.wl, self.H, self.k, self.tau, self.kept_pairs, self.placement)
 
 
 def time_steps(cfg, steps, warmup, barrier, local_gpu):
@@ -721,9 +723,8 @@ def run_reference(args):
         "impl": "reference", "metric": METRIC, "value": value, "unit": "TFLOP/s", "n_gpus": world,
         "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms, "higher_is_better": True,
         "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
-        "config": {"workload": wl.name, "heads": H, "head_dim": d, "grid": list(wl.grid), "n_text": wl.n_text,
-                   "tokens": wl.n_tokens, "block": b, "n_blocks": NB, "topk_blocks": k, "virtual_ranks": P,
-                   "placement": placement, "layout": "[H][N][d]"},
+        # every row keeps k video blocks and all text blocks: the kept pairs of the layer follow from the shape
+        "config": describe_config(wl, H, k, 0.0, H * NB * (k + (NB - wl.nb_video)), placement),
         "cpu_baseline": {"value": value, "unit": "TFLOP/s", "cores": oracle.num_threads(), "kind": "oracle",
                          "sample": "each step: steps 1-2 on 1 head, step 3 on %d query blocks of that head; "
                                    "throughput = sampled kept flops / (sample's share of steps 1-2 + step 3 time)"
