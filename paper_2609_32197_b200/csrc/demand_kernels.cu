@@ -17,7 +17,7 @@ namespace sparsp {
 // 64 ranks x 32 words = 8 KiB; OR does not depend on the order, so the bits are well defined); the ownership
 // words are rebuilt per CTA from the rank table (a few thousand compares) rather than fetched from an earlier
 // launch.  A rank value outside [0, P) is ignored.
-constexpr int kUnionThreads = 256;
+constexpr int kUnionThreads = 1024;
 static_assert(2 * kMaxRanks * (kMaxBlocks / 32) * 4 <= 48 * 1024, "union and ownership tables must fit shared memory");
 
 __global__ void __launch_bounds__(kUnionThreads) union_count_kernel(const uint32_t* __restrict__ mask,
