@@ -169,3 +169,69 @@ def test_a_consumer_that_never_fetches_times_the_producer_out(binding):
     assert e.value.code == binding.SPARSP_ERR_TIMEOUT and "publish" in str(e.value)
     binding.sparsp_xchg_destroy(x)
     binding.sparsp_xchg_destroy(y)
+
+
+def _process_rank(rank, world, port, d, b, out):
+    """One PROCESS per rank (as on a node with a GPU each), both on device 0 here: slot windows are opened through
+    CUDA inter-process handles, the flag page is shared host memory, the Fence's barrier a gloo barrier.  No kernel
+    of one process waits for the other: every cross-rank wait is the endpoint's bounded host-side poll."""
+    import os
+    import torch.distributed as dist
+    os.environ["MASTER_ADDR"] = "127.0.0.1"
+    os.environ["MASTER_PORT"] = str(port)
+    torch.cuda.set_device(0)
+    dist.init_process_group("gloo", rank=rank, world_size=world)
+    try:
+        import oracle
+        from paper_2609_32197_b200 import binding, exchange_driver, synth
+        oracle.build()
+        H, P, k = 3, world, 5 if b == 128 else 9
+        wl = synth.Workload("xproc", H, d, (5, 11, 13), 70, b, k, None, P, seed=91)
+        Q, K, V = synth.make_qkv(wl, "cpu")
+        N, NB = wl.n_tokens, wl.n_blocks
+        shape = binding.make_shape(H, d, wl.grid, wl.n_text, b)
+        Qd = Q.cuda()[None].contiguous()
+        ws = binding.make_workspace(shape, P)
+        mo = pu.gpu_block_mask(binding, shape, Qd, K.cuda(), k, ws)
+        ref = oracle.block_mask(Q, K, b, k, wl.n_text)
+        assert np.array_equal(pu.u32(mo["mask"][0]), ref["mask"])
+        rank_np = np.array([(j * 3 + j // 4) % P for j in range(NB)], np.int32)
+        foreign = torch.as_tensor(rank_np[np.arange(N) // b] != rank)
+        Kp, Vp = K.clone(), V.clone()
+        Kp[:, foreign] = float("nan")      # this rank's view: everything it does not own is NaN
+        Vp[:, foreign] = float("nan")
+        res = exchange_driver.run_exchange_multi_gpu(shape, rank_np, Qd, Kp.cuda()[None].contiguous(),
+                                                     Vp.cuda()[None].contiguous(), mo["mask"], window=1,
+                                                     steady_chunks=2, tail_chunks=3, calls=2, wait_limit_us=30_000_000)
+        if res.errors:
+            out[rank] = ("error", repr(res.errors))
+            return
+        o_ref, lse_ref = oracle.attn_all(Q, K, V, ref["mask"], b)
+        rows = np.repeat(rank_np == rank, b)[:N]
+        got = res.O[rank][0].float().cpu().numpy()[:, rows]
+        err = np.abs(got - o_ref[:, rows])
+        out[rank] = ("ok", bool(np.isfinite(got).all()), float(err.max()), float(err.mean()),
+                     float(np.abs(o_ref[:, rows]).max()), res.stats[rank])
+    finally:
+        dist.destroy_process_group()
+
+
+@pytest.mark.parametrize("d,b", [(128, 128), (64, 64)])
+def test_one_process_per_rank_through_interprocess_windows(binding, d, b):
+    import socket
+
+    import torch.multiprocessing as mp
+    with socket.socket() as s_:
+        s_.bind(("127.0.0.1", 0))
+        port = s_.getsockname()[1]
+    world = 2
+    with mp.Manager() as mgr:
+        out = mgr.dict()
+        mp.spawn(_process_rank, args=(world, port, d, b, out), nprocs=world, join=True)
+        res = dict(out)
+    for r in range(world):
+        assert res[r][0] == "ok", res[r]
+        _, finite, mx, mean, omax, st = res[r]
+        assert finite, f"rank {r}: a byte that never travelled reached the result"
+        assert mx <= pu.ATTN_MAX_ABS + world * 2.0 ** -9 * omax and mean <= pu.ATTN_MEAN_ABS + world * 2.0 ** -10 * omax
+        assert st["publications"] == 2 and st["releases"] == 2 and st["timeouts"] == 0   # one hop per call, two calls
