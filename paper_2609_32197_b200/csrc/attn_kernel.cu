@@ -63,6 +63,9 @@ struct AttnParams {
   float* lse;
   int32_t* status;
   int32_t* work_counter;  // next work item to hand out; zeroed by the preparatory launch
+  // packed-source mode: number of work items per (batch, head) that can have rows at all (the consumer's query
+  // blocks come first in the pairs table), a device scalar; NULL = all per_bh items
+  const int32_t* active_per_bh;
   int64_t N;
   int64_t sB, sH, sT;
   int H, NB, Wd;
@@ -490,14 +493,17 @@ __global__ void __launch_bounds__(kAttnThreads, 1)
         int it = 0;
         if (lane == 0) it = atomicAdd(p.work_counter, 1);
         it = __shfl_sync(0xffffffffu, it, 0);
-        if (it >= p.n_items || *s_abort) {
+        // one consumer's call walks only the items of its own query blocks (the first `active` of every head)
+        const int active = p.active_per_bh ? *p.active_per_bh : p.per_bh;
+        if (it >= active * (p.n_items / p.per_bh) || *s_abort) {
           if (lane == 0) {
             s_item[buf] = -1;
             mbar_arrive(list_ready + buf);
           }
           break;
         }
-        const int bh = it / p.per_bh, x = it - bh * p.per_bh;
+        const int bh = it / active, x = it - bh * active;
+        it = bh * p.per_bh + x;  // the item's number in the full table, which the other roles derive the head from
         int blk[2];
         if (C::kStacked) {
           const int32_t* pr = p.pairs + ((int64_t)bh * p.per_bh + x) * 2;
@@ -1280,6 +1286,7 @@ int launch_attn(const sparsp_shape& s, const Geometry& g, const void* Q, const v
   p.pairs = pairs;
   p.slot = nullptr;
   p.tile_base = nullptr;
+  p.active_per_bh = nullptr;
   p.knorm = knorm;
   return launch_attn_common(s, g, Q, K, V, nullptr, 0, p, scale, O, lse, ws, L, st);
 }
@@ -1289,7 +1296,9 @@ int launch_attn(const sparsp_shape& s, const Geometry& g, const void* Q, const v
 // blocks, and every kept KV block the consumer does not own is read from the consumer's packed buffer.
 // ------------------------------------------------------------------------------------------------
 // pairs of the consumer's blocks (ascending, neighbours in that order); the rest of the table is (-1, -1)
-__global__ void pair_rank_kernel(const int32_t* __restrict__ rank, int NB, int consumer, int32_t* __restrict__ pairs) {
+// Also leaves the number of work items per (batch, head) that hold any of the consumer's blocks.
+__global__ void pair_rank_kernel(const int32_t* __restrict__ rank, int NB, int consumer, int stacked,
+                                 int32_t* __restrict__ pairs, int32_t* __restrict__ active_per_bh) {
   const int n_pairs = (NB + 1) / 2;
   int32_t* out = pairs + (int64_t)blockIdx.x * n_pairs * 2;
   for (int i = threadIdx.x; i < 2 * n_pairs; i += blockDim.x) out[i] = -1;
@@ -1298,6 +1307,7 @@ __global__ void pair_rank_kernel(const int32_t* __restrict__ rank, int NB, int c
     int k = 0;
     for (int i = 0; i < NB; ++i)
       if (rank[i] == consumer) out[k++] = i;  // pair c = entries 2c and 2c+1
+    if (blockIdx.x == 0) *active_per_bh = stacked ? (k + 1) / 2 : k;
   }
 }
 
@@ -1372,7 +1382,8 @@ int launch_attn_packed(const sparsp_shape& s, const Geometry& g, const void* Q, 
   int64_t* tile_base = (int64_t*)(ws + L.tile_base);
   const int64_t tile_bytes = (int64_t)g.b * g.d * 2;
   SPARSP_CUDA_OK(cudaMemsetAsync(slot, 0xFF, (size_t)g.B * g.H * g.NB * 4, st));
-  pair_rank_kernel<<<g.B * g.H, 128, 0, st>>>(rank, g.NB, consumer, pairs);
+  int32_t* active = (int32_t*)(ws + L.status) + kWorkCounterWord + 1;
+  pair_rank_kernel<<<g.B * g.H, 128, 0, st>>>(rank, g.NB, consumer, g.b == 64 ? 1 : 0, pairs, active);
   const int64_t n_warps = std::max<int64_t>((int64_t)g.B * P * g.H, g.B);
   slot_kernel<<<(unsigned)((n_warps * 32 + 255) / 256), 256, 0, st>>>(U, rank, seg_off, seg_total, dst_base, g.B, g.H,
                                                                     g.NB, g.Wd, P, consumer, tile_bytes, slot,
@@ -1383,6 +1394,7 @@ int launch_attn_packed(const sparsp_shape& s, const Geometry& g, const void* Q, 
   p.pairs = pairs;
   p.slot = slot;
   p.tile_base = tile_base;
+  p.active_per_bh = active;
   p.knorm = nullptr;  // remote keys live in the packed buffer: every tile takes its row maximum
   return launch_attn_common(s, g, Q, K, V, packed, capacity, p, scale, O, lse, ws, L, st);
 }
