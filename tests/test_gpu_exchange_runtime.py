@@ -99,8 +99,8 @@ def test_serial_order_gives_the_same_result(oracle_mod, binding):
 
 
 def test_pack_segment_equals_the_segment_of_the_packed_buffer(oracle_mod, binding):
-    """A slot's content is exactly the (consumer, producer) run of the consumer's packed buffer; too small a slot
-    writes nothing beyond its capacity and reports SPARSP_ERR_CAPACITY."""
+    """A slot's content is exactly the (consumer, producer) run of the consumer's packed buffer as the ORACLE packs
+    it; too small a slot writes nothing beyond its capacity and reports SPARSP_ERR_CAPACITY."""
     H, P, d, b = 3, 3, 64, 64
     wl, shape, Qd, Ks, Vs, mask, rank, _, _ = _case(oracle_mod, binding, d, b, H, P, 85, 7)
     from paper_2609_32197_b200 import synth
@@ -109,11 +109,14 @@ def test_pack_segment_equals_the_segment_of_the_packed_buffer(oracle_mod, bindin
     ws = binding.make_workspace(shape, P)
     rank_d = torch.as_tensor(rank).cuda()
     dg = pu.gpu_demand_pack(binding, shape, mask, rank_d, P, 0, Kd, Vd, ws)
+    # expected bytes: the ORACLE's packed buffer, cut at the oracle's offsets
+    ref = oracle_mod.block_mask(Q, K, b, 7, wl.n_text)
+    dref = oracle_mod.demand(ref["mask"], rank, P, b, d)
+    packed_ref = torch.as_tensor(oracle_mod.pack(K, V, dref["U"], rank, b, P, dref["total"])).cuda()
     entry = 2 * b * d * 2
-    tot = dg["seg_total"][0].cpu().numpy()
-    base = np.concatenate([[0], np.cumsum(tot)[:-1]]) * entry
-    seg = dg["seg_offset"][0].cpu().numpy()
-    cnt = dg["cnt"][0].cpu().numpy()
+    base = np.concatenate([[0], np.cumsum(dref["total"])[:-1]]) * entry
+    seg, cnt = dref["seg_off"], dref["cnt"]
+    assert np.array_equal(dg["cnt"][0].cpu().numpy(), cnt) and np.array_equal(dg["seg_offset"][0].cpu().numpy(), seg)
     for r in range(P):
         for p in range(P):
             if p == r:
@@ -126,7 +129,7 @@ def test_pack_segment_equals_the_segment_of_the_packed_buffer(oracle_mod, bindin
                                         Vs[p], slot, n * entry, ws)
             torch.cuda.synchronize()
             assert binding.sparsp_status(ws) == binding.SPARSP_OK
-            assert torch.equal(slot[:n * entry], dg["packed"][lo:lo + n * entry]), (r, p)
+            assert torch.equal(slot[:n * entry], packed_ref[lo:lo + n * entry]), (r, p)
             assert bool((slot[n * entry:] == 0xAB).all())
             if n >= 2:
                 small = torch.full((n * entry,), 0xAB, dtype=torch.uint8, device="cuda")
@@ -134,8 +137,37 @@ def test_pack_segment_equals_the_segment_of_the_packed_buffer(oracle_mod, bindin
                                             Ks[p], Vs[p], small, (n - 1) * entry, ws)
                 torch.cuda.synchronize()
                 assert binding.sparsp_status(ws) == binding.SPARSP_ERR_CAPACITY
-                assert torch.equal(small[:(n - 1) * entry], dg["packed"][lo:lo + (n - 1) * entry])
+                assert torch.equal(small[:(n - 1) * entry], packed_ref[lo:lo + (n - 1) * entry])
                 assert bool((small[(n - 1) * entry:] == 0xAB).all())
+
+
+def test_merge_of_one_chunks_rows_matches_the_oracle_and_touches_nothing_else(oracle_mod, binding):
+    """sparsp_attn_merge_rows merges only the rows of the consumer's blocks in the given heads (against the oracle's
+    merge of the same rows); every other row keeps its bytes."""
+    rng = np.random.default_rng(5)
+    H, d, b, P = 4, 64, 64, 3
+    shape = binding.make_shape(H, d, (1, 9, 37), 0, b)       # 333 tokens: 6 blocks, the last one ragged
+    N, NB = 333, 6
+    rank = np.array([0, 2, 1, 2, 0, 2], np.int32)
+    oa = torch.tensor(rng.standard_normal((1, H, N, d)), dtype=torch.float32).to(torch.bfloat16).cuda()
+    ob = torch.tensor(rng.standard_normal((1, H, N, d)), dtype=torch.float32).to(torch.bfloat16).cuda()
+    la = torch.tensor(rng.standard_normal((1, H, N)) * 3, dtype=torch.float32).cuda()
+    lb = torch.tensor(rng.standard_normal((1, H, N)) * 3, dtype=torch.float32).cuda()
+    lb[0, 1, 70:80] = float("-inf")
+    ro, rl = oracle_mod.attn_merge(oa.float().cpu().numpy(), la.cpu().numpy(), ob.float().cpu().numpy(), lb.cpu().numpy())
+    for consumer, (h0, h1) in [(2, (1, 3)), (0, (0, 4)), (1, (3, 4))]:
+        acc, acc_l = oa.clone(), la.clone()
+        binding.sparsp_attn_merge_rows(shape, acc, acc_l, ob, lb, acc, acc_l, torch.as_tensor(rank).cuda(), P, consumer,
+                                       h0, h1)
+        torch.cuda.synchronize()
+        rows = np.repeat(rank == consumer, b)[:N]
+        sel = np.zeros((H, N), bool)
+        sel[h0:h1, :] = rows
+        got, got_l = acc[0].float().cpu().numpy(), acc_l[0].cpu().numpy()
+        assert np.abs(got[sel] - ro[0][sel]).max() <= 2e-2          # bf16 rounding of the merged rows
+        assert np.abs(got_l[sel] - rl[0][sel]).max() < 1e-4
+        assert np.array_equal(got[~sel], oa[0].float().cpu().numpy()[~sel])   # untouched elsewhere
+        assert np.array_equal(got_l[~sel], la[0].cpu().numpy()[~sel])
 
 
 def test_a_consumer_that_never_fetches_times_the_producer_out(binding):
