@@ -136,13 +136,14 @@ SPARSP_API int sparsp_block_mask(const sparsp_shape* shape, const void* Q, const
  *   p_j = exp(score_scale * (S_j - max S)),  Z = sum_j p_j,
  *   keep the smallest set { j : S_j >= v } (v one of the row's scores) whose mass reaches tau * Z --
  *   blocks with equal scores (-0 == +0) are kept or dropped together -- then every text block.
- * The arithmetic is fixed (all fp32): x_j = (S_j - max S) * (score_scale * log2 e), one subtraction and
- * one multiplication; p_j = 2^x_j by clamping x at -125, splitting off the nearest integer (ties to
+ * The arithmetic is fixed: x_j = (S_j - max S) * (score_scale * log2 e) in fp32, one subtraction and
+ * one multiplication; p_j = 2^x_j in fp32 by clamping x at -125, splitting off the nearest integer (ties to
  * even) and a degree-5 Horner polynomial of the remainder with fused multiply-adds (coefficients
  * 0.0013400432653725147, 0.009676037356257439, 0.05550327152013779, 0.2402210682630539,
- * 0.6931471824645996, 1.0000001192092896), the integer part added into the exponent field; every sum
- * is 32 partial sums (partial l adds the terms with j = l mod 32 in ascending order, from 0) combined
- * by a butterfly (s = 16, 8, 4, 2, 1: partial[l] += partial[l xor s]); theta = tau * Z.
+ * 0.6931471824645996, 1.0000001192092896), the integer part added into the exponent field.  The mass is
+ * counted in integers, so that no order of additions is part of the definition: w_j = floor(p_j * 2^31),
+ * Z = sum_j w_j, and a set reaches the threshold when its sum of w_j is >= ceil(tau * Z), that product
+ * taken once in fp64.
  *   tau          in   (0, 1]
  *   score_scale  in   0 means 1/sqrt(d)
  *   mask         out  uint32 [B][H][NB][Wd]   (rows keep different numbers of blocks)

@@ -163,13 +163,16 @@ void oracle_topk_mask(const float* scores, const uint8_t* is_text, int64_t H, in
  * cumulative attention mass reaches the threshold tau).  Per (h, i), over the candidate KV blocks
  * (is_text[j] == 0):   p_j = exp(scale * (S_j - max S)),  Z = sum p_j,  keep the smallest set
  * { j : S_j >= v } (v one of the row's scores) whose mass reaches tau * Z; blocks with equal scores
- * are kept or dropped together; every text block is kept.  The arithmetic is fixed so that the kept
- * set is a well-defined integer result (all fp32):
- *   x_j  = (S_j - max S) * (scale * log2 e)        one subtraction, one multiplication
- *   p_j  = exp2c(x_j)                              below
- *   sums = 32 partial sums (partial l adds the terms with j = l mod 32, j ascending, from 0),
- *          combined by a butterfly: for s = 16, 8, 4, 2, 1: partial[l] += partial[l xor s]
- *   theta = tau * Z;  mass(v) = the same sum over { j : S_j >= v }
+ * are kept or dropped together; every text block is kept.  A floating-point sum would make the kept
+ * set depend on the order of its additions, so the mass is counted in integers, where any order gives
+ * the same sum:
+ *   x_j  = (S_j - max S) * (scale * log2 e)        fp32: one subtraction, one multiplication
+ *   p_j  = exp2c(x_j)                              fp32, below
+ *   w_j  = floor(p_j * 2^31)                       an integer <= 2^31 + 256 (the scaling is exact)
+ *   Z    = sum w_j,  mass(v) = sum of w_j over { j : S_j >= v }      exact integer sums
+ *   kept: the largest v with  mass(v) >= ceil(tau * Z),  the product taken once in fp64 (Z < 2^42 is exact
+ *   there, tau is the caller's fp32 value)
+ * Dropping what lies below 2^-31 of a term changes the mass by less than NB * 2^-31 < 5e-7.
  * exp2c(x): x clamped below at -125; i = nearest integer (ties to even); f = x - i; degree-5 Horner
  * polynomial in f with fused multiply-adds; i added into the exponent field.
  * ---------------------------------------------------------------------------------------------- */
@@ -194,21 +197,12 @@ void oracle_exp2c_array(const float* x, int64_t n, float* y) {
   for (int64_t t = 0; t < n; ++t) y[t] = oracle_exp2c(x[t]);
 }
 
-/* sum of e[j] over the candidates j with take[j] != 0, in the fixed order described above */
-static float tree_sum32(const float* e, const uint8_t* take, int64_t n) {
-  float part[32];
-  for (int l = 0; l < 32; ++l) {
-    float acc = 0.0f;
-    for (int64_t j = l; j < n; j += 32)
-      if (take[j]) acc = acc + e[j];
-    part[l] = acc;
-  }
-  for (int s = 16; s >= 1; s >>= 1) {
-    float nxt[32];
-    for (int l = 0; l < 32; ++l) nxt[l] = part[l] + part[l ^ s];
-    memcpy(part, nxt, sizeof part);
-  }
-  return part[0];
+/* sum of w[j] over the candidates j with take[j] != 0 */
+static uint64_t mass_of(const uint32_t* w, const uint8_t* take, int64_t n) {
+  uint64_t acc = 0;
+  for (int64_t j = 0; j < n; ++j)
+    if (take[j]) acc += w[j];
+  return acc;
 }
 
 void oracle_cdf_mask(const float* scores, const uint8_t* is_text, int64_t H, int64_t NB, float tau,
@@ -219,7 +213,7 @@ void oracle_cdf_mask(const float* scores, const uint8_t* is_text, int64_t H, int
   for (int64_t h = 0; h < H; ++h) {
     for (int64_t i = 0; i < NB; ++i) {
       const float* srow = scores + (h * NB + i) * NB;
-      float* e = (float*)malloc((size_t)NB * sizeof(float));
+      uint32_t* w = (uint32_t*)malloc((size_t)NB * sizeof(uint32_t));
       uint8_t* take = (uint8_t*)malloc((size_t)NB);
       cand_t* cand = (cand_t*)malloc((size_t)NB * sizeof(cand_t));
       int64_t nc = 0;
@@ -227,17 +221,17 @@ void oracle_cdf_mask(const float* scores, const uint8_t* is_text, int64_t H, int
       for (int64_t j = 0; j < NB; ++j)
         if (!is_text[j] && srow[j] > mx) mx = srow[j];
       for (int64_t j = 0; j < NB; ++j) {
-        e[j] = 0.0f;
+        w[j] = 0u;
         take[j] = 0;
         if (!is_text[j]) {
-          e[j] = oracle_exp2c((srow[j] - mx) * c);
+          w[j] = (uint32_t)(oracle_exp2c((srow[j] - mx) * c) * 2147483648.0f);
           take[j] = 1;
           cand[nc].s = srow[j];
           cand[nc].j = (int32_t)j;
           ++nc;
         }
       }
-      const float theta = tau * tree_sum32(e, take, NB);
+      const uint64_t theta = (uint64_t)ceil((double)tau * (double)mass_of(w, take, NB));
       qsort(cand, (size_t)nc, sizeof(cand_t), cand_cmp);
       /* grow the set one group of equal scores at a time, highest first */
       for (int64_t j = 0; j < NB; ++j) take[j] = 0;
@@ -245,7 +239,7 @@ void oracle_cdf_mask(const float* scores, const uint8_t* is_text, int64_t H, int
       while (t < nc) {
         const float v = cand[t].s;
         while (t < nc && cand[t].s == v) take[cand[t++].j] = 1;
-        if (tree_sum32(e, take, NB) >= theta) break;
+        if (mass_of(w, take, NB) >= theta) break;
       }
       uint32_t* row = mask + (h * NB + i) * Wd;
       for (int64_t w = 0; w < Wd; ++w) row[w] = 0u;
@@ -257,7 +251,7 @@ void oracle_cdf_mask(const float* scores, const uint8_t* is_text, int64_t H, int
         }
       }
       if (kv_count) kv_count[h * NB + i] = (int32_t)cnt;
-      free(e);
+      free(w);
       free(take);
       free(cand);
     }

@@ -239,14 +239,14 @@ __global__ void __launch_bounds__(kTopkWarps * 32) topk_kernel(const float* __re
 
 // ------------------------------------------------------------------------------------------------
 // CDF-threshold selection (Section 8.1): per row, softmax over the candidate scores, keep the smallest
-// top set by score (whole groups of equal scores) whose mass reaches tau.  Fixed fp32 arithmetic so that
-// the kept set is a well-defined integer result:
-//   x_j = (S_j - max S) * (scale * log2 e);  p_j = exp2c(x_j)  (clamp at -125, nearest-integer split,
-//   degree-5 Horner polynomial with fused multiply-adds, integer part added into the exponent field);
-//   every sum = 32 partial sums (lane l adds its terms j = l mod 32 in ascending order, from 0) combined
-//   by a butterfly (s = 16, 8, 4, 2, 1: partial[l] += partial[l xor s]);  theta = tau * Z.
-// One warp per row; the threshold is found by a 32-step search over the order-preserving key space,
-// which is valid because the mass of { key >= t } (nonnegative terms, fixed order) never grows with t.
+// top set by score (whole groups of equal scores) whose mass reaches tau.  The mass is counted in integers, so
+// that the kept set does not depend on the order of the additions:
+//   x_j = (S_j - max S) * (scale * log2 e)  (fp32);  p_j = exp2c(x_j)  (fp32: clamp at -125, nearest-integer
+//   split, degree-5 Horner polynomial with fused multiply-adds, integer part added into the exponent field);
+//   w_j = floor(p_j * 2^31);  Z = sum w_j;  kept = { key >= T } for the largest T with
+//   mass{ key >= T } >= ceil(tau * Z), the product taken once in fp64.
+// One warp per row; T is found by a 32-step search over the order-preserving key space, which is valid
+// because the mass of { key >= t } never grows with t.
 // ------------------------------------------------------------------------------------------------
 __device__ __forceinline__ float exp2c(float x) {
   x = fmaxf(x, -125.0f);
@@ -261,9 +261,9 @@ __device__ __forceinline__ float exp2c(float x) {
   return __int_as_float(__float_as_int(p) + (int)fi * (1 << 23));
 }
 
-__device__ __forceinline__ float butterfly_sum(float v) {
+__device__ __forceinline__ unsigned long long warp_sum(unsigned long long v) {
 #pragma unroll
-  for (int s = 16; s >= 1; s >>= 1) v = __fadd_rn(v, __shfl_xor_sync(0xffffffffu, v, s));
+  for (int s = 16; s >= 1; s >>= 1) v += __shfl_xor_sync(0xffffffffu, v, s);
   return v;
 }
 
@@ -276,42 +276,43 @@ __global__ void __launch_bounds__(kTopkWarps * 32) cdf_kernel(const float* __res
   const int64_t row = (int64_t)blockIdx.x * kTopkWarps + warp;  // (batch*H + head) * NB + i
   if (row >= n_rows) return;
   const float* srow = scores + row * NB;
-  // lane l holds blocks l, l + 32, ... in ascending order: exactly the terms of its partial sums.  A block that
-  // is not a candidate holds key 0 (no trial threshold, all >= 1, selects it) and the term 0.
+  // lane l holds blocks l, l + 32, ...  A block that is not a candidate holds key 0 (no trial threshold, all
+  // >= 1, selects it) and the weight 0.
   uint32_t key[WMAX];
-  float e[WMAX];
+  uint32_t w[WMAX];
   float mx = -INFINITY;
 #pragma unroll
   for (int t = 0; t < WMAX; ++t) {
     const int j = t * 32 + lane;
     const bool cand = t < Wd && j < nb_cand;
     const float s = cand ? __ldcs(srow + j) : -INFINITY;
-    e[t] = s;
+    w[t] = __float_as_uint(s);
     key[t] = cand ? score_key(s) : 0u;
     mx = fmaxf(mx, s);
   }
 #pragma unroll
   for (int s = 16; s >= 1; s >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, s));
-  float acc = 0.0f;
+  unsigned long long acc = 0;
 #pragma unroll
   for (int t = 0; t < WMAX; ++t) {
     const int j = t * 32 + lane;
-    float pj = 0.0f;
+    uint32_t wj = 0u;
     if (t < Wd && j < nb_cand) {
-      pj = exp2c(__fmul_rn(__fsub_rn(e[t], mx), c));
-      acc = __fadd_rn(acc, pj);
+      // p <= 1.0000002, so p * 2^31 (exact) fits in 32 bits; the conversion truncates
+      wj = __float2uint_rz(__fmul_rn(exp2c(__fmul_rn(__fsub_rn(__uint_as_float(w[t]), mx), c)), 2147483648.0f));
+      acc += wj;
     }
-    e[t] = pj;
+    w[t] = wj;
   }
-  const float theta = __fmul_rn(tau, butterfly_sum(acc));
+  const unsigned long long theta = (unsigned long long)ceil(__dmul_rn((double)tau, (double)warp_sum(acc)));
   // largest T with mass{ key >= T } >= theta
   uint32_t T = 0;
   for (int bit = 31; bit >= 0; --bit) {
     const uint32_t trial = T | (1u << bit);
-    float m = 0.0f;
+    unsigned long long m = 0;
 #pragma unroll
-    for (int t = 0; t < WMAX; ++t) m = key[t] >= trial ? __fadd_rn(m, e[t]) : m;
-    if (butterfly_sum(m) >= theta) T = trial;
+    for (int t = 0; t < WMAX; ++t) m += key[t] >= trial ? w[t] : 0u;
+    if (warp_sum(m) >= theta) T = trial;
   }
   int cnt = 0;
 #pragma unroll

@@ -108,3 +108,20 @@ def test_scale_and_text_blocks(oracle_mod):
     m_big, c_big = oracle_mod.cdf_mask(sc, is_text, 0.9, 10.0)      # peaked distribution: few blocks
     assert c_small.mean() > c_big.mean() + 5
     assert np.all(c_big >= 4)                     # at least one candidate + the three text blocks
+
+
+def test_kept_set_does_not_depend_on_block_order(oracle_mod):
+    """The mass is an integer sum, so renumbering the key blocks renumbers the kept set and changes nothing else
+    (a floating-point sum taken in index order would not guarantee that)."""
+    rng = np.random.default_rng(11)
+    NB = 75
+    sc = (rng.standard_normal((2, NB, NB)) * 2.0).astype(np.float32)
+    is_text = np.zeros(NB, np.uint8)
+    for tau in (0.5, 0.9, 0.99):
+        mask, cnt = oracle_mod.cdf_mask(sc, is_text, tau, 0.5)
+        perm = rng.permutation(NB)
+        mask_p, cnt_p = oracle_mod.cdf_mask(np.ascontiguousarray(sc[:, :, perm]), is_text, tau, 0.5)
+        assert np.array_equal(cnt, cnt_p)
+        for h in range(2):
+            for i in range(NB):
+                assert {int(perm[j]) for j in _bits(mask_p[h, i], NB)} == _bits(mask[h, i], NB)
