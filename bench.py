@@ -9,11 +9,12 @@ tensor peak, pack GB/s against the HBM copy peak, ms per stage) ride along in th
 
     python bench.py [--gpus N] [--steps K] [--warmup W] [--workload hunyuan|wan|cog|mid|tiny]
                     [--pct P] [--placement contiguous|periodic|shuffle] [--impl ours|reference]
-                    [--shard replicas|heads] [--no-per-config] [--sustained-s S]
+                    [--shard replicas|heads] [--no-per-config] [--sustained-s S] [--no-graph]
 
 The headline configuration is the largest single-GPU one (Hunyuan-like, 118 800 tokens, top-k 10 %); at
 N = 1 the same line carries `per_config` (all eight configurations of the contract measured the same way)
-and `sustained` (the attention call alone, back to back for a couple of seconds, with the clocks sampled).
+and `sustained` (the attention call alone, back to back for a couple of seconds, with the clocks sampled);
+`graph_ms_per_step` is the same step captured once in a CUDA graph and replayed (the headline stays plain launches).
 With N > 1 launch under torch.distributed.run; every rank runs its own replica of the workload
 (different seed; weak scaling) or, with --shard heads, its share of the heads of ONE layer (strong
 scaling) -- either way the path has no exchange step, so there is no data-path collective.
@@ -302,6 +303,33 @@ def time_steps(cfg, steps, warmup, barrier, local_gpu):
             "launches": launches, "clocks": clocks}
 
 
+def graph_replay(cfg, steps):
+    """The same step captured ONCE in a CUDA graph (the three calls, nine launches) and replayed: what the launch
+    gaps between the library's kernels cost.  Per-replay CUDA events; the L2 flush (small workloads) stays outside
+    the timed pairs.  Returns ms per step."""
+    import torch
+    torch.cuda.synchronize()
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(graph):
+        cfg.step()
+    stream = torch.cuda.current_stream()
+    for _ in range(3):
+        graph.replay()
+    torch.cuda.synchronize()
+    cfg.check_status()
+    ev = [[torch.cuda.Event(enable_timing=True) for _ in range(2)] for _ in range(steps)]
+    for s in range(steps):
+        if cfg.flush is not None:
+            cfg.flush.fill_(s & 0xFF)
+        ev[s][0].record(stream)
+        graph.replay()
+        ev[s][1].record(stream)
+    torch.cuda.synchronize()
+    cfg.check_status()
+    del graph
+    return sum(e[0].elapsed_time(e[1]) for e in ev) / steps
+
+
 def figures(cfg, t, peaks, traffic_table):
     """The per-kernel figures of one measured configuration."""
     attn_tflops = cfg.flops / (t["attn"] * 1e-3) / 1e12
@@ -582,6 +610,8 @@ def run_ours(args):
                      "h2d_bytes_per_step": int(tot["h2d"]), "d2h_bytes_per_step": int(tot["d2h"])}
     result["gpu_launches"] = int(tot["launches"])
     result["clocks"] = t["clocks"]
+    if world == 1 and not args.no_graph:
+        result["graph_ms_per_step"] = graph_replay(cfg, args.steps)
     if sustained:
         result["sustained"] = sustained
     if exchange:
@@ -604,6 +634,8 @@ def run_ours(args):
             row.update(figures(c, tt, peaks, traffic_table))
             row["clocks"] = tt["clocks"]
             row["gpu_launches"] = tt["launches"]
+            if not args.no_graph:
+                row["graph_ms_per_step"] = graph_replay(c, max(10, min(args.steps, 20)))
             row["is_headline_config"] = (name, c.k, plc) == headline
             rows.append(row)
             del c
@@ -750,6 +782,7 @@ def main():
     ap.add_argument("--no-e2e", action="store_true", help="skip the host-buffer end-to-end leg")
     ap.add_argument("--heads", type=int, default=0, help="override the head count (small profiling cases)")
     ap.add_argument("--no-per-config", action="store_true", help="skip the per_config list (all eight configurations)")
+    ap.add_argument("--no-graph", action="store_true", help="skip the CUDA-graph replay of the step (graph_ms_per_step)")
     ap.add_argument("--sustained-s", type=float, default=2.0,
                     help="seconds of back-to-back attention calls for the sustained figure (0 = skip)")
     ap.add_argument("--exchange", action="store_true",
