@@ -152,8 +152,8 @@ def _shm_addr(shm):
 def _slot_protocol_worker(rank, world, port, names, out, stall_from):
     """Two processes, one exchange endpoint each, slots and flag page in inter-process shared memory (host-memory
     endpoints: copies are memcpy, so the protocol runs without a GPU).  Each rank packs `n_uses` payloads for its peer
-    into a window of 2 slots and consumes the peer's; the consumer sleeps before every fetch, so a producer that
-    did not wait for Release would overwrite a slot that is still unread.  With `stall_from` >= 0 rank 1 stops
+    into a window of 2 slots and consumes the peer's; rank 1 sleeps before every fetch, so rank 0, which does not,
+    must wait for Release before it re-packs a slot (and would overwrite an unread slot if it did not).  With `stall_from` >= 0 rank 1 stops
     releasing from that use on: rank 0's bounded wait for the slot must end in SPARSP_ERR_TIMEOUT."""
     import time
     from multiprocessing import shared_memory
@@ -184,7 +184,8 @@ def _slot_protocol_worker(rank, world, port, names, out, stall_from):
         log["acquired"].append((u, slot))
 
     def consume(u):
-        time.sleep(0.02)                            # a slow consumer
+        if rank == 1:
+            time.sleep(0.03)                        # a slow consumer
         b.sparsp_xchg_fetch(x, peer, u, 0, recv.ctypes.data, slot_bytes, 0)
         if not (recv == (17 * peer + u) % 251).all():
             log["bad_payload"] += 1
@@ -245,7 +246,7 @@ def test_slot_window_protocol_between_two_processes():
         st = log["stats"]
         assert st["publications"] == 6 and st["fetches"] == 6 and st["releases"] == 6 and st["timeouts"] == 0
         assert st["bytes_fetched"] == 6 * (1 << 16)
-        assert st["acquires_that_waited"] >= 1                               # Release did gate a later pack
+    assert res[0]["stats"]["acquires_that_waited"] >= 1                      # Release did gate the fast rank's later packs
 
 
 def test_a_consumer_that_stops_releasing_times_the_producer_out():
