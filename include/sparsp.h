@@ -141,7 +141,7 @@ SPARSP_API int sparsp_block_mask(const sparsp_shape* shape, const void* Q, const
  * even) and a degree-5 Horner polynomial of the remainder with fused multiply-adds (coefficients
  * 0.0013400432653725147, 0.009676037356257439, 0.05550327152013779, 0.2402210682630539,
  * 0.6931471824645996, 1.0000001192092896), the integer part added into the exponent field.  The mass is
- * counted in integers, so that no order of additions is part of the definition: w_j = floor(p_j * 2^31),
+ * counted in integers, so that no order of additions is part of the definition: w_j = floor(p_j * 2^26),
  * Z = sum_j w_j, and a set reaches the threshold when its sum of w_j is >= ceil(tau * Z), that product
  * taken once in fp64.
  *   tau          in   (0, 1]

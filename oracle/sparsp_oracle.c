@@ -168,11 +168,12 @@ void oracle_topk_mask(const float* scores, const uint8_t* is_text, int64_t H, in
  * the same sum:
  *   x_j  = (S_j - max S) * (scale * log2 e)        fp32: one subtraction, one multiplication
  *   p_j  = exp2c(x_j)                              fp32, below
- *   w_j  = floor(p_j * 2^31)                       an integer <= 2^31 + 256 (the scaling is exact)
+ *   w_j  = floor(p_j * 2^26)                       an integer <= 2^26 + 8 (the scaling is exact)
  *   Z    = sum w_j,  mass(v) = sum of w_j over { j : S_j >= v }      exact integer sums
- *   kept: the largest v with  mass(v) >= ceil(tau * Z),  the product taken once in fp64 (Z < 2^42 is exact
+ *   kept: the largest v with  mass(v) >= ceil(tau * Z),  the product taken once in fp64 (Z < 2^37 is exact
  *   there, tau is the caller's fp32 value)
- * Dropping what lies below 2^-31 of a term changes the mass by less than NB * 2^-31 < 5e-7.
+ * Dropping what lies below 2^-26 of a term changes the mass (>= 1: the largest term is 1) by less than
+ * NB * 2^-26 <= 1.6e-5, the size of the rounding error of an fp32 sum of as many terms.
  * exp2c(x): x clamped below at -125; i = nearest integer (ties to even); f = x - i; degree-5 Horner
  * polynomial in f with fused multiply-adds; i added into the exponent field.
  * ---------------------------------------------------------------------------------------------- */
@@ -224,7 +225,7 @@ void oracle_cdf_mask(const float* scores, const uint8_t* is_text, int64_t H, int
         w[j] = 0u;
         take[j] = 0;
         if (!is_text[j]) {
-          w[j] = (uint32_t)(oracle_exp2c((srow[j] - mx) * c) * 2147483648.0f);
+          w[j] = (uint32_t)(oracle_exp2c((srow[j] - mx) * c) * 67108864.0f);
           take[j] = 1;
           cand[nc].s = srow[j];
           cand[nc].j = (int32_t)j;

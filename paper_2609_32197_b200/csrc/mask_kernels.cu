@@ -243,7 +243,7 @@ __global__ void __launch_bounds__(kTopkWarps * 32) topk_kernel(const float* __re
 // that the kept set does not depend on the order of the additions:
 //   x_j = (S_j - max S) * (scale * log2 e)  (fp32);  p_j = exp2c(x_j)  (fp32: clamp at -125, nearest-integer
 //   split, degree-5 Horner polynomial with fused multiply-adds, integer part added into the exponent field);
-//   w_j = floor(p_j * 2^31);  Z = sum w_j;  kept = { key >= T } for the largest T with
+//   w_j = floor(p_j * 2^26);  Z = sum w_j;  kept = { key >= T } for the largest T with
 //   mass{ key >= T } >= ceil(tau * Z), the product taken once in fp64.
 // One warp per row; T is found by a 32-step search over the order-preserving key space, which is valid
 // because the mass of { key >= t } never grows with t.
@@ -261,10 +261,11 @@ __device__ __forceinline__ float exp2c(float x) {
   return __int_as_float(__float_as_int(p) + (int)fi * (1 << 23));
 }
 
-__device__ __forceinline__ unsigned long long warp_sum(unsigned long long v) {
-#pragma unroll
-  for (int s = 16; s >= 1; s >>= 1) v += __shfl_xor_sync(0xffffffffu, v, s);
-  return v;
+// Sum over the warp of one 32-bit partial sum per lane (each < 2^32, the total needs up to 37 bits): the halves of
+// the partial sums are added by the warp-reduction instruction and put together again.
+__device__ __forceinline__ unsigned long long warp_sum(uint32_t v) {
+  const uint32_t lo = __reduce_add_sync(0xffffffffu, v & 0xffffu), hi = __reduce_add_sync(0xffffffffu, v >> 16);
+  return ((unsigned long long)hi << 16) + lo;
 }
 
 template <int WMAX>  // mask words per row this instance can hold (keys and terms live in registers)
@@ -292,14 +293,14 @@ __global__ void __launch_bounds__(kTopkWarps * 32) cdf_kernel(const float* __res
   }
 #pragma unroll
   for (int s = 16; s >= 1; s >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, s));
-  unsigned long long acc = 0;
+  uint32_t acc = 0;  // at most 32 terms of at most 2^26 + 8 each
 #pragma unroll
   for (int t = 0; t < WMAX; ++t) {
     const int j = t * 32 + lane;
     uint32_t wj = 0u;
     if (t < Wd && j < nb_cand) {
-      // p <= 1.0000002, so p * 2^31 (exact) fits in 32 bits; the conversion truncates
-      wj = __float2uint_rz(__fmul_rn(exp2c(__fmul_rn(__fsub_rn(__uint_as_float(w[t]), mx), c)), 2147483648.0f));
+      // the scaling is exact, the conversion truncates
+      wj = __float2uint_rz(__fmul_rn(exp2c(__fmul_rn(__fsub_rn(__uint_as_float(w[t]), mx), c)), 67108864.0f));
       acc += wj;
     }
     w[t] = wj;
@@ -309,7 +310,7 @@ __global__ void __launch_bounds__(kTopkWarps * 32) cdf_kernel(const float* __res
   uint32_t T = 0;
   for (int bit = 31; bit >= 0; --bit) {
     const uint32_t trial = T | (1u << bit);
-    unsigned long long m = 0;
+    uint32_t m = 0;
 #pragma unroll
     for (int t = 0; t < WMAX; ++t) m += key[t] >= trial ? w[t] : 0u;
     if (warp_sum(m) >= theta) T = trial;
