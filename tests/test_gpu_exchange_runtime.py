@@ -267,3 +267,47 @@ def test_one_process_per_rank_through_interprocess_windows(binding, d, b):
         assert finite, f"rank {r}: a byte that never travelled reached the result"
         assert mx <= pu.ATTN_MAX_ABS + world * 2.0 ** -9 * omax and mean <= pu.ATTN_MEAN_ABS + world * 2.0 ** -10 * omax
         assert st["publications"] == 2 and st["releases"] == 2 and st["timeouts"] == 0   # one hop per call, two calls
+
+
+@pytest.mark.parametrize("case", range(16))
+def test_random_exchange_configurations(oracle_mod, binding, case):
+    """Shapes, rank counts (1-6, some owning nothing), random placements, windows, chunk counts, serial / pipelined and
+    one or two calls drawn per case: every rank's rows equal the oracle's one-shot attention, every byte of the
+    exchange volume came through Fetch, no wait ran out."""
+    from paper_2609_32197_b200 import exchange_driver, synth
+    rng = np.random.default_rng(4200 + case)
+    while True:
+        d, b = int(rng.choice([64, 128])), int(rng.choice([64, 128]))
+        H, P = int(rng.integers(1, 6)), int(rng.integers(1, 7))
+        grid = (int(rng.integers(1, 6)), int(rng.integers(4, 16)), int(rng.integers(4, 20)))
+        n_text = int(rng.choice([0, int(rng.integers(1, 200))]))
+        wl = synth.Workload("xsweep", H, d, grid, n_text, b, 1, None, P, seed=int(rng.integers(0, 1 << 30)))
+        if wl.nb_video >= 1:
+            break
+    N, NB = wl.n_tokens, wl.n_blocks
+    k = int(rng.integers(1, wl.nb_video + 1))
+    window, steady, tail = int(rng.integers(1, 4)), int(rng.integers(1, 5)), int(rng.integers(1, 5))
+    pipelined, calls = bool(rng.integers(0, 2)), int(rng.integers(1, 3))
+    Q, K, V = synth.make_qkv(wl, "cpu")
+    shape = binding.make_shape(H, d, grid, n_text, b)
+    Qd, Kd = Q.cuda()[None].contiguous(), K.cuda()
+    ws = binding.make_workspace(shape, P)
+    ref = oracle_mod.block_mask(Q, K, b, k, n_text)
+    mo = pu.gpu_block_mask(binding, shape, Qd, Kd, k, ws)
+    assert np.array_equal(pu.u32(mo["mask"][0]), ref["mask"])
+    rank = rng.integers(0, P, NB).astype(np.int32)
+    blk_of_tok = np.arange(N) // b
+    Ks, Vs = [], []
+    for r in range(P):   # rank r's view: everything it does not own is NaN
+        foreign = torch.as_tensor(rank[blk_of_tok] != r)
+        Kp, Vp = K.clone(), V.clone()
+        Kp[:, foreign] = float("nan")
+        Vp[:, foreign] = float("nan")
+        Ks.append(Kp.cuda()[None].contiguous())
+        Vs.append(Vp.cuda()[None].contiguous())
+    o_ref, lse_ref = oracle_mod.attn_all(Q, K, V, ref["mask"], b)
+    res = exchange_driver.run_exchange(shape, P, rank, Qd, Ks, Vs, mo["mask"], window=window, steady_chunks=steady,
+                                       tail_chunks=tail, pipelined=pipelined, calls=calls, wait_limit_us=5_000_000)
+    _check_result(res, P, rank, b, N, o_ref, lse_ref)
+    assert sum(res.stats[r]["bytes_fetched"] for r in range(P)) == calls * res.bytes_moved
+    assert all(res.stats[r]["timeouts"] == 0 for r in range(P))
