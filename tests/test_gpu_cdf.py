@@ -102,3 +102,31 @@ def test_cdf_mask_at_the_largest_block_count(oracle_mod, binding):
     ref = oracle_mod.block_mask_cdf(Q, K, b, 0.9, 0)
     assert np.array_equal(pu.u32(mask[0]), ref["mask"])
     assert np.array_equal(cnt[0].cpu().numpy(), ref["kv_count"])
+
+
+def test_cdf_rows_of_maximum_length(oracle_mod, binding):
+    """1024 blocks (the largest supported row).  With all scores equal every term is the largest weight and every lane of
+    the selection warp adds 32 of them (the 32-bit partial sums come closest to their range); one tie group, so every
+    row keeps everything.  With random scores: masks and counts against the oracle, tau up to 1."""
+    from paper_2609_32197_b200 import synth
+    wl = synth.Workload("cdfmax", 1, 64, (16, 64, 64), 0, 64, 1, None, 2)
+    assert wl.n_blocks == 1024
+    shape = binding.make_shape(1, 64, wl.grid, 0, 64)
+    ws = binding.make_workspace(shape, 2)
+    g = binding.sparsp_geometry(shape)
+    gen = torch.Generator().manual_seed(5)
+    cases = [(torch.zeros(1, wl.n_tokens, 64), torch.ones(1, wl.n_tokens, 64), 0.5, True),
+             (torch.randn(1, wl.n_tokens, 64, generator=gen) * 3, torch.randn(1, wl.n_tokens, 64, generator=gen), 0.9, False),
+             (torch.randn(1, wl.n_tokens, 64, generator=gen) * 0.1, torch.randn(1, wl.n_tokens, 64, generator=gen), 1.0, False)]
+    for Qf, Kf, tau, all_kept in cases:
+        Q, K = Qf.to(torch.bfloat16), Kf.to(torch.bfloat16)
+        mask = torch.zeros(1, 1, 1024, g.n_words, dtype=torch.int32, device="cuda")
+        cnt = torch.zeros(1, 1, 1024, dtype=torch.int32, device="cuda")
+        binding.sparsp_block_mask_cdf(shape, Q.cuda()[None].contiguous(), K.cuda()[None].contiguous(), tau, 0.0, mask, cnt,
+                                      None, None, ws)
+        torch.cuda.synchronize()
+        ref = oracle_mod.block_mask_cdf(Q, K, 64, tau, 0, 0.0)
+        assert np.array_equal(pu.u32(mask[0]), ref["mask"])
+        assert np.array_equal(cnt[0].cpu().numpy(), ref["kv_count"])
+        if all_kept:
+            assert int(ref["kv_count"].min()) == 1024
