@@ -32,6 +32,9 @@
 // a tile whose bound stays within 2^64 of the row's reference skips its row-maximum pass, and once the bound
 // with the item's largest key norm holds, the reference is final and the two warps of a row group stop taking
 // turns for the rest of the item (load scores -> exponentials -> store P).
+// And if that bound is at most 2^80 in absolute terms -- ordinary inputs -- the item needs no reference at all: every
+// softmax thread takes its row's norm from the Q tile while the first Q K^T runs, and an item whose bounds hold runs
+// on the fixed reference 0 from its first tile on.
 // The block-64 pairing and the order of a head's items (longest list first) come from attn_prep_kernel,
 // which also takes the key norms.
 // Every mbarrier wait is bounded; a wait that runs out sets SPARSP_ERR_TIMEOUT in the status word
@@ -84,6 +87,11 @@ constexpr int kTmemCols = 512;
 constexpr int kWorkCounterWord = 8;  // word of the workspace header that holds the attention work counter
 constexpr float kGrowThreshold = 8.0f;
 constexpr float kSkipMargin = 64.0f;  // 2^64 * (keys of a sequence) * |V| stays far inside fp32
+// If |q_row| * (largest key norm of the item) * scale * log2(e) <= kStaticBound for all rows of a warp, every score of
+// the item lies in [-kStaticBound, kStaticBound] (log2 domain) and the fixed reference 0 serves the whole item:
+// exponentials between 2^-80 and 2^80 are normal numbers in fp32 and bf16 with full relative precision, and
+// 2^80 * (keys of a sequence) * |V| stays inside fp32.
+constexpr float kStaticBound = 80.0f;
 // Tuning switch (compile-time): how many of the exponentials go to the FMA pipe instead of the
 // special-function unit (every n-th pair; 0 = none).
 #ifndef SPARSP_TUNE_POLY
@@ -623,6 +631,7 @@ __global__ void __launch_bounds__(kAttnThreads, 1)
     volatile int* frz = s_frz + rgrp;               // set by the warp that freezes the reference, cleared by the other
 
     int g0 = 0;  // number of the item's first tile
+    int qn = 0;  // items that had tiles (the phase of the Q barrier)
     for (int i = 0;; ++i) {
       const int buf = i & 1;
       volatile float* ref = sRef + (i % 3) * 128;
@@ -644,6 +653,40 @@ __global__ void __launch_bounds__(kAttnThreads, 1)
       float q_bound = INFINITY;  // |q_row| * softmax scale * log2(e) (+0.1 %), once known
       float m_ref = -INFINITY;  // the row's reference maximum (log2 domain) as this thread last saw it
       float l_run = 0.0f;       // this thread's partial row sum, relative to m_ref
+      if (n_tiles > 0) {
+        if (p.knorm != nullptr && n_tiles >= 4) {
+          // The norm of my query row, read from the Q tile in shared memory while the item's first Q K^T runs (any
+          // order of its 16-byte units will do, so the swizzle does not matter).  Q stays there until the item's
+          // last Q K^T has completed; with four or more tiles that one cannot be issued before both warpgroups
+          // have released a score buffer, which they do after this.
+          mbar_wait_bounded_inline(q_full, qn & 1, s_abort, 42, p.wait_limit);
+          float ss[4] = {0.0f, 0.0f, 0.0f, 0.0f};  // four chains, so that the additions do not wait for each other
+#pragma unroll
+          for (int c = 0; c < D / 64; ++c) {
+#pragma unroll
+            for (int k = 0; k < 8; ++k) {
+              const uint4 v = *reinterpret_cast<const uint4*>(sQ + c * 16384 + row * 128 + (((k + lane) & 7) << 4));
+              const uint32_t w[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+              for (int e = 0; e < 4; ++e) {
+                const float lo = __uint_as_float(w[e] << 16), hi = __uint_as_float(w[e] & 0xffff0000u);
+                ss[e] = fmaf(lo, lo, ss[e]);
+                ss[e] = fmaf(hi, hi, ss[e]);
+              }
+            }
+          }
+          q_bound = sqrtf((ss[0] + ss[1]) + (ss[2] + ss[3])) * p.scale_log2 * 1.001f;
+          // Both threads of a row compute the same bound from the same data, so both warps of a row group take this
+          // decision alike without talking to each other: the item runs on the fixed reference 0 from its first
+          // tile on -- no row maximum, no turns, no named barrier (neither warp arrives, neither waits).
+          if (__all_sync(0xffffffffu, q_bound * kn_item <= kStaticBound)) {
+            frozen = true;
+            m_ref = 0.0f;
+            ref[row] = 0.0f;  // (both threads of the row write the same value; the epilogue reads it)
+          }
+        }
+        ++qn;
+      }
 
       // One tile of this warpgroup.  kRagged = the sequence ends inside the tile (possible only for the item's
       // last tile): that variant carries the column masking, the common one stays small.
@@ -667,27 +710,6 @@ __global__ void __launch_bounds__(kAttnThreads, 1)
 #pragma unroll
         for (int c = 0; c < 4; ++c) tmem_ld32(tS + c * 32, reinterpret_cast<uint32_t*>(sv) + c * 32);
         tmem_ld_wait();
-        if (p.knorm != nullptr && n < 2 && n_tiles >= n + 3) {
-          // My first tile of the item: the norm of my query row, read from the Q tile in shared memory (any
-          // order of its 16-byte units will do, so the swizzle does not matter).  Q is still there: its last
-          // Q K^T cannot have been issued before this warp releases the S buffer below.
-          float ss[4] = {0.0f, 0.0f, 0.0f, 0.0f};  // four chains, so that the additions do not wait for each other
-#pragma unroll
-          for (int c = 0; c < D / 64; ++c) {
-#pragma unroll
-            for (int k = 0; k < 8; ++k) {
-              const uint4 v = *reinterpret_cast<const uint4*>(sQ + c * 16384 + row * 128 + (((k + lane) & 7) << 4));
-              const uint32_t w[4] = {v.x, v.y, v.z, v.w};
-#pragma unroll
-              for (int e = 0; e < 4; ++e) {
-                const float lo = __uint_as_float(w[e] << 16), hi = __uint_as_float(w[e] & 0xffff0000u);
-                ss[e] = fmaf(lo, lo, ss[e]);
-                ss[e] = fmaf(hi, hi, ss[e]);
-              }
-            }
-          }
-          q_bound = sqrtf((ss[0] + ss[1]) + (ss[2] + ss[3])) * p.scale_log2 * 1.001f;
-        }
         // S is in registers: the Q K^T of tile g+2 may overwrite the buffer
         tc_fence_before();
         __syncwarp();
