@@ -137,7 +137,7 @@ __device__ __forceinline__ void tc_fence_after() {
 __device__ __forceinline__ void prefetch_tmap(const CUtensorMap* m) {
   asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(m)) : "memory");
 }
-// 4-D tile load global -> shared, completion counted on an mbarrier (no multicast).
+// 4-D tile load global -> shared, completion counted on an mbarrier.
 __device__ __forceinline__ void tma_load_4d(void* smem_dst, const CUtensorMap* m, uint64_t* bar, int c0,
                                             int c1, int c2, int c3) {
   asm volatile(
