@@ -449,3 +449,57 @@ def test_random_norm_profiles(oracle_mod, binding, seed, v_sigma):
     assert binding.sparsp_status(ws) == binding.SPARSP_OK
     units = [(h, i) for h in range(H) for i in range(NB)]
     pu.check_attn_units(oracle_mod, Q, K, V, words, b, O, units, lse_gpu=lse[0])
+
+
+@pytest.mark.parametrize("d,b", [(128, 128), (64, 64), (128, 64), (64, 128)])
+@pytest.mark.parametrize("level", [30.0, 74.0])
+def test_fixed_reference_at_the_edge_of_its_bound(oracle_mod, binding, d, b, level):
+    """An item whose norm bound |q| |k| scale log2(e) stays under 2^80 runs on the fixed reference 0.  Here every score
+    is about +level or -level (log2 units; 74 is just inside the bound): query blocks that keep only the low-scoring
+    blocks work with exponentials around 2^-74 throughout, blocks that keep only the high ones with 2^+74, the rest
+    with both at once.  All must give the oracle's rows (and log-sum-exp), which for the one-sided blocks are close
+    to the mean of V over the kept keys."""
+    H, NB = 2, 12
+    N = NB * b - 7                                    # ragged last block
+    rng = np.random.default_rng(29)
+    scale_log2 = 1.4426950408889634 / np.sqrt(d)
+    a = float(np.sqrt(level / scale_log2))            # |q| = |k| = a: a * a * scale * log2(e) = level
+    Q = torch.zeros(H, N, d, dtype=torch.float32)
+    K = torch.zeros(H, N, d, dtype=torch.float32)
+    Q[:, :, 0] = a
+    K[:, :, 0] = a
+    for j in range(1, NB, 2):
+        K[:, j * b:(j + 1) * b, 0] = -a               # odd key blocks score -level, even ones +level
+    Q[:, :, 1:] = torch.tensor(rng.standard_normal((H, N, d - 1)) * 0.02)
+    K[:, :, 1:] = torch.tensor(rng.standard_normal((H, N, d - 1)) * 0.02)
+    Q, K = Q.to(torch.bfloat16), K.to(torch.bfloat16)
+    V = torch.tensor(rng.standard_normal((H, N, d))).to(torch.bfloat16)
+    M = np.zeros((H, NB, NB), bool)
+    for i in range(NB):
+        if i % 3 == 0:
+            M[:, i, 1::2] = True                      # low blocks only (six kept blocks: enough tiles for the fixed reference)
+        elif i % 3 == 1:
+            M[:, i, 0::2] = True                      # high blocks only
+        else:
+            M[:, i, :] = True                         # both
+    words = np.zeros((H, NB, 1), np.uint32)
+    for h in range(H):
+        for i in range(NB):
+            for j in range(NB):
+                if M[h, i, j]:
+                    words[h, i, 0] |= np.uint32(1 << j)
+    shape = binding.make_shape(H, d, (1, 1, N), 0, b)
+    ws = binding.make_workspace(shape, 2)
+    Qd, Kd, Vd = Q.cuda(), K.cuda(), V.cuda()
+    mask_d = torch.as_tensor(words.view(np.int32)).cuda()
+    O = torch.zeros_like(Qd)
+    lse = torch.zeros(1, H, N, dtype=torch.float32, device="cuda")
+    binding.sparsp_sparse_attn_fwd(shape, Qd, Kd, Vd, mask_d, 0.0, O, lse, ws)
+    torch.cuda.synchronize()
+    assert binding.sparsp_status(ws) == binding.SPARSP_OK
+    units = [(h, i) for h in range(H) for i in range(NB)]
+    pu.check_attn_units(oracle_mod, Q, K, V, words, b, O, units, lse_gpu=lse[0])
+    got_lse = lse[0].cpu().numpy()
+    ln2 = 0.6931471805599453
+    assert got_lse[:, :b].max() < -(level - 12) * ln2          # low-only rows: every term is tiny, none was lost
+    assert got_lse[:, b:2 * b].min() > (level - 12) * ln2      # high-only rows
