@@ -80,9 +80,11 @@ struct AttnParams {
 
 constexpr int kAttnThreads = 512;  // four warpgroups: two of utility warps, softmax of the even tiles, softmax of the odd tiles
 // register budget per thread after the warpgroups re-balance (128*48 + 128*32 + 256*216 = 512*128)
+#ifndef SPARSP_REGS_UTILITY
 #define SPARSP_REGS_UTILITY 48
 #define SPARSP_REGS_UTILITY2 32
 #define SPARSP_REGS_SOFTMAX 216
+#endif
 constexpr int kTmemCols = 512;
 constexpr int kWorkCounterWord = 8;  // word of the workspace header that holds the attention work counter
 constexpr float kGrowThreshold = 8.0f;
