@@ -8,8 +8,8 @@
 //                zeroed in P.
 // The kernel is persistent: one CTA per SM takes items from a global counter; the next item's kept
 // list, Q tile and first K/V tiles overlap the current item's last tiles, its first Q K^T the epilogue.
-// The scores S = Q K^T and the probabilities P are double-buffered in tensor memory (S: 2 x 128 fp32
-// columns, P: 2 x 64 columns of packed bf16, O: d columns), so that the tensor pipe always has the next
+// The scores S = Q K^T are double-buffered in tensor memory (S: 2 x 128 fp32 columns; P: 64 columns of packed bf16,
+// two buffers at d = 64, one at d = 128 where 16 columns hold the row sums instead; O: d columns), so that the tensor pipe always has the next
 // tiles' MMAs queued while the softmax of the current tile runs: Q K^T of tile g+2 starts as soon as the
 // scores of tile g have been READ, and P V of tile g is issued as soon as P_g is written.  Tiles are
 // numbered g = 0, 1, 2, ... across the CTA's items; every ring, buffer and barrier phase follows g.
@@ -101,6 +101,11 @@ constexpr float kStaticBound = 80.0f;
 #endif
 // ... at d = 64, where the row sum is taken by the tensor pipe and the FMA pipe has more room (measured: every
 // 3rd pair is 3 % faster than every 4th there, every 2nd 4 % slower)
+// d = 128: take the row sum on the tensor pipe as well (an extra N = 16 MMA per 16 keys against a small block of
+// ones), at the price of the second P buffer, whose tensor-memory columns the 16 sum columns need (1 = on)
+#ifndef SPARSP_SUM_MMA_128
+#define SPARSP_SUM_MMA_128 1
+#endif
 #ifndef SPARSP_TUNE_POLY_D64
 #define SPARSP_TUNE_POLY_D64 3
 #endif
@@ -122,8 +127,14 @@ struct AttnCfg {
   // bf16 values it multiplies with V, instead of one more packed add per pair of scores in the softmax warps
   static constexpr bool kOnes = (D == 64);
   static constexpr int kAccCols = D + (kOnes ? 16 : 0);
+  // d = 128: the row sum also comes from the tensor pipe, through a separate N = 16 MMA per 16
+  // keys against a [16 keys][column 0 = 1] block (2 KB, 128-byte swizzle like a V box), into 16 tensor-memory columns
+  // of its own -- which exist only if P keeps ONE buffer instead of two (tensor memory is full otherwise)
+  static constexpr bool kSum128 = (D == 128 && SPARSP_SUM_MMA_128 != 0);
+  static constexpr bool kSumMma = kOnes || kSum128;  // the softmax warps keep no row sums
+  static constexpr int kNumP = kSum128 ? 1 : 2;
   static constexpr int kOffOnes = kOffV + kStagesV * kTileBytes;  // bf16 [128][64], 128-byte swizzle like a V box
-  static constexpr int kOffEntJ = kOffOnes + (kOnes ? 128 * 128 : 0);  // uint16 [2][1024] kept / union list
+  static constexpr int kOffEntJ = kOffOnes + (kOnes ? 128 * 128 : (kSum128 ? 2048 : 0));  // uint16 [2][1024] kept / union list
   static constexpr int kOffEntV = kOffEntJ + 2 * 2 * kMaxBlocks;  // uint8 [2][1024][2] keys of the entry valid for query block q (0 = not kept)
   static constexpr int kOffSlot = kOffEntV + 2 * 2 * kMaxBlocks;  // int32 [2][1024] packed-buffer slot per entry
   static constexpr int kOffEntN = kOffSlot + 2 * 4 * kMaxBlocks;  // float [2][1024] largest key norm of the entry's block
@@ -134,6 +145,7 @@ struct AttnCfg {
   static constexpr int kColS = 0;    // S buffers: columns [0, 256)
   static constexpr int kColP = 256;  // P buffers: columns [256, 384)
   static constexpr int kColO = 384;  // accumulator: columns [384, 384 + d)
+  static constexpr int kColL = kOnes ? kColO + D : 320;  // row sums (column 0 of 16), where the tensor pipe takes them
   static constexpr int kOffMisc = kOffBars + 8 * kNumBars;
   static constexpr int kTotal = kOffMisc + 80;
   static constexpr int kDynamic = kTotal + 1024;  // slack for the 1024-byte alignment of the base
@@ -262,10 +274,11 @@ __global__ void __launch_bounds__(kAttnThreads, 1)
     for (int r = 0; r < 4; ++r) s_frz[r] = 0;
   }
   if (tid < 384) sRef[tid] = -INFINITY;  // 3 x 128 entries
-  if (C::kOnes) {
-    // key row r holds column 64 + c at byte r*128 + ((c/8 ^ (r & 7)) << 4) + (c%8)*2 (the swizzle of a TMA box)
+  if (C::kSumMma) {
+    // key row r holds column 64 + c at byte r*128 + ((c/8 ^ (r & 7)) << 4) + (c%8)*2 (the swizzle of a TMA box);
+    // 128 key rows at d = 64 (one block for a whole tile), 16 at d = 128 (every group of 16 keys uses the same)
     uint4* ones = reinterpret_cast<uint4*>(smem + C::kOffOnes);
-    for (int idx = tid; idx < 128 * 8; idx += kAttnThreads) {
+    for (int idx = tid; idx < (C::kOnes ? 128 : 16) * 8; idx += kAttnThreads) {
       const int r = idx >> 3, chunk = idx & 7;
       ones[idx] = make_uint4(chunk == (r & 7) ? 0x3F80u : 0u, 0u, 0u, 0u);  // bf16 1.0 in element 0 of logical chunk 0
     }
@@ -458,6 +471,9 @@ __global__ void __launch_bounds__(kAttnThreads, 1)
 #pragma unroll
       for (int kk = 0; kk < 8; ++kk) vlo[kk] = (uint32_t)descV + (uint32_t)((kk * 2048) >> 4);
       const uint32_t tO = tmem_base + C::kColO;
+      constexpr uint32_t kIdescSum = make_idesc_bf16(128, 16, 0, 1);
+      const uint64_t descOnes = make_smem_desc(smem_u32(smem + C::kOffOnes), 16384u, 1024);
+      const uint32_t tL = tmem_base + C::kColL;
       int g = 0;
       for (int i = 0;; ++i) {
         const int buf = i & 1;
@@ -472,11 +488,15 @@ __global__ void __launch_bounds__(kAttnThreads, 1)
           tc_fence_after();
           uint32_t stage_off = (uint32_t)(((g % SV) * C::kTileBytes) >> 4);
           if (C::kOnes) stage_off -= stage_off << 16;  // start address up, distance to the ones block down
-          const uint32_t tP = tmem_base + C::kColP + (g & 1) * 64;
+          const uint32_t tP = tmem_base + C::kColP + (C::kNumP == 2 ? (g & 1) * 64 : 0);
           if (leader) {
 #pragma unroll
-            for (int kk = 0; kk < 8; ++kk)
+            for (int kk = 0; kk < 8; ++kk) {
               mma_ts_lohi(tO, tP + kk * 8, vlo[kk] + stage_off, hiV, kIdescPV, (kk > 0 || n > 0) ? 1u : 0u);
+              if (C::kSum128)
+                mma_ts_lohi(tL, tP + kk * 8, (uint32_t)descOnes, (uint32_t)(descOnes >> 32), kIdescSum,
+                            (kk > 0 || n > 0) ? 1u : 0u);
+            }
             mma_commit(o_full + (g & 3));
             mma_commit(v_empty + g % SV);
           }
@@ -626,7 +646,7 @@ __global__ void __launch_bounds__(kAttnThreads, 1)
     const int rh = row >> 6;         // which query block of a stacked Q tile the row belongs to
     const uint32_t lane_off = (uint32_t)(rgrp * 32) << 16;
     const uint32_t tS = tmem_base + C::kColS + wg * 128 + lane_off;
-    const uint32_t tP = tmem_base + C::kColP + wg * 64 + lane_off;
+    const uint32_t tP = tmem_base + C::kColP + (C::kNumP == 2 ? wg * 64 : 0) + lane_off;
     const uint32_t tO = tmem_base + C::kColO + lane_off;
     const int bar_mine = 1 + wg * 4 + rgrp;         // I arrive here after my decision
     const int bar_other = 1 + (1 - wg) * 4 + rgrp;  // the row group's other warp arrives here after its decision
@@ -799,6 +819,14 @@ __global__ void __launch_bounds__(kAttnThreads, 1)
                   for (int e = 0; e < 16; ++e) o[e] = __float_as_uint(__uint_as_float(o[e]) * alpha);
                   tmem_st16(tO + c * 16, o);
                 }
+                if (C::kSum128) {  // the row sums live in columns of their own
+                  uint32_t o[16];
+                  tmem_ld16(tmem_base + C::kColL + lane_off, o);
+                  tmem_ld_wait();
+#pragma unroll
+                  for (int e = 0; e < 16; ++e) o[e] = __float_as_uint(__uint_as_float(o[e]) * alpha);
+                  tmem_st16(tmem_base + C::kColL + lane_off, o);
+                }
                 tmem_st_wait();
                 tc_fence_before();
               }
@@ -833,7 +861,7 @@ __global__ void __launch_bounds__(kAttnThreads, 1)
                                     : make_float2(ex2(x.x), ex2(x.y));
               const __nv_bfloat162 h2 = __floats2bfloat162_rn(pp.x, pp.y);
               pkh[e] = *reinterpret_cast<const uint32_t*>(&h2);
-              if (!C::kOnes) {
+              if (!C::kSumMma) {
                 // the row sum adds the bf16 values that P V multiplies, not the unrounded exponentials: with a
                 // reference that is not the row's maximum the largest term is an arbitrary 2^x, and a sum of
                 // unrounded terms would differ from the numerator's weights by up to 2^-9 of a peaked row
@@ -854,9 +882,10 @@ __global__ void __launch_bounds__(kAttnThreads, 1)
           }
         }
         l_run += lsum2.x + lsum2.y;
-        // my P buffer was last read by the P V of tile g-2
-        if (g >= 2) {
-          mbar_wait_bounded_inline(o_full + ((g - 2) & 3), ((g - 2) >> 2) & 1, s_abort, 34 + wg, p.wait_limit);
+        // my P buffer was last read by the P V of tile g-2; a single P buffer by that of tile g-1
+        constexpr int kBack = C::kNumP == 2 ? 2 : 1;
+        if (g >= kBack) {
+          mbar_wait_bounded_inline(o_full + ((g - kBack) & 3), ((g - kBack) >> 2) & 1, s_abort, 34 + wg, p.wait_limit);
           tc_fence_after();
         }
 #pragma unroll
@@ -892,11 +921,11 @@ __global__ void __launch_bounds__(kAttnThreads, 1)
         // the barrier above, and the item before this one (its last user) is finished for all of them
         sRef[((i + 2) % 3) * 128 + row] = -INFINITY;
         float l = (st0.y > 0.0f ? st0.y * ex2(st0.x - m_fin) : 0.0f) + (st1.y > 0.0f ? st1.y * ex2(st1.x - m_fin) : 0.0f);
-        if (C::kOnes) {  // the row sum is accumulator column d (CTA-uniform branch: the load is warp-collective)
+        if (C::kSumMma) {  // the row sum is a tensor-memory column (CTA-uniform branch: the load is warp-collective)
           l = 0.0f;
           if (n_tiles > 0) {
             uint32_t sums[16];
-            tmem_ld16(tO + D, sums);
+            tmem_ld16(tmem_base + C::kColL + lane_off, sums);
             tmem_ld_wait();
             l = __uint_as_float(sums[0]);
           }
