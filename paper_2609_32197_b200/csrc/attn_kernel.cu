@@ -97,15 +97,15 @@ constexpr float kStaticBound = 80.0f;
 // Tuning switch (compile-time): how many of the exponentials go to the FMA pipe instead of the
 // special-function unit (every n-th pair; 0 = none).
 #ifndef SPARSP_TUNE_POLY
-#define SPARSP_TUNE_POLY 4
+#define SPARSP_TUNE_POLY 3
 #endif
-// ... at d = 64, where the row sum is taken by the tensor pipe and the FMA pipe has more room (measured: every
-// 3rd pair is 3 % faster than every 4th there, every 2nd 4 % slower)
 // d = 128: take the row sum on the tensor pipe as well (an extra N = 16 MMA per 16 keys against a small block of
 // ones), at the price of the second P buffer, whose tensor-memory columns the 16 sum columns need (1 = on)
 #ifndef SPARSP_SUM_MMA_128
 #define SPARSP_SUM_MMA_128 1
 #endif
+// ... at d = 64 (measured there: every 3rd pair is 3 % faster than every 4th, every 2nd 4 % slower; at d = 128, with the
+// row sum on the tensor pipe, every 3rd is 1-2 % faster than every 4th and every 2nd 2 % slower)
 #ifndef SPARSP_TUNE_POLY_D64
 #define SPARSP_TUNE_POLY_D64 3
 #endif
