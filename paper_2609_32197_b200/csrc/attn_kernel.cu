@@ -143,7 +143,7 @@ struct AttnCfg {
   static constexpr int kOffBars = kOffRef + 3 * 128 * 4;
   static constexpr int kNumBars = 2 + 2 * (kStagesK + kStagesV) + 10 + 1 + 4;
   static constexpr int kColS = 0;    // S buffers: columns [0, 256)
-  static constexpr int kColP = 256;  // P buffers: columns [256, 384)
+  static constexpr int kColP = 256;  // P: two buffers in columns [256, 384), or one in [256, 320) with the row sums in [320, 336)
   static constexpr int kColO = 384;  // accumulator: columns [384, 384 + d)
   static constexpr int kColL = kOnes ? kColO + D : 320;  // row sums (column 0 of 16), where the tensor pipe takes them
   static constexpr int kOffMisc = kOffBars + 8 * kNumBars;
@@ -223,7 +223,7 @@ __global__ void __launch_bounds__(kAttnThreads, 1)
   uint64_t* v_empty = v_full + SV;
   uint64_t* s_full = v_empty + SV;  // [2] S buffer written by a Q K^T
   uint64_t* s_free = s_full + 2;    // [2] S buffer read into registers by its 4 softmax warps
-  uint64_t* p_full = s_free + 2;    // [2] P buffer written by its 4 softmax warps
+  uint64_t* p_full = s_free + 2;    // [2] P of an even / odd tile written by its 4 softmax warps
   // [4] the P V of tile g arrives on o_full[g % 4].  Four barriers, because a parity wait can only tell the
   // phase a barrier is in from the one before: a softmax thread that wants P V g-1 or g-2 has itself seen
   // P V g-4 complete, and P V g+2 cannot complete before that thread has stored P_g.
@@ -640,7 +640,7 @@ __global__ void __launch_bounds__(kAttnThreads, 1)
   } else {
     asm volatile("setmaxnreg.inc.sync.aligned.u32 %0;" ::"n"(SPARSP_REGS_SOFTMAX));
     // ================================ softmax warpgroups ==================================
-    const int wg = (warp >> 2) - 2;  // 0: even tiles g, 1: odd tiles; also the S / P buffer this warpgroup uses
+    const int wg = (warp >> 2) - 2;  // 0: even tiles g, 1: odd tiles; also the S (and, where there are two, P) buffer this warpgroup uses
     const int rgrp = warp & 3;       // tensor-memory lane group this warp may access
     const int row = rgrp * 32 + lane;
     const int rh = row >> 6;         // which query block of a stacked Q tile the row belongs to
